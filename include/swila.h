@@ -1,0 +1,146 @@
+/*
+ * swila.h -- C ABI of the B200 (sm_100a) Switching Linear Attention recurrence.
+ *
+ * The library evaluates, for every (batch b, head h), the token recurrence of the SwiLA
+ * layer (Sec. 3.2): the state is J linear regressors W[j] in R^{Dv x Dk} (rows = output
+ * dimensions, columns = key dimensions, App. B.4).  Per token t, for all (j, d):
+ *
+ *   delta = v_td - w_{t-1,jd} . k_t                               (text below Eq. 3.3)
+ *   r     = softmax over j of ( log prior_jd - delta^2 / 2 )       (E-step, Eq. 3.4)
+ *   w_tjd = w_{t-1,jd} + beta_tjd r delta k_t                      (M-step, Eq. 3.3)
+ *   o_td  = sum_j prior^q_jd  w_tjd . q_t                          (readout, Eq. 3.5, updated state)
+ *
+ * beta = sigmoid(beta_logit); prior = softmax over j of pik_logit, prior^q = softmax over
+ * j of piq_logit (App. B.2) -- the activations are fused into the kernels, the linear
+ * projections that produce the logits are not part of this library.
+ *
+ * Conventions
+ *  - Every pointer is a DEVICE pointer owned by the caller unless a function says HOST.
+ *    The library allocates no device memory and keeps no per-call state.
+ *  - All tensors are contiguous, last index fastest.  Base addresses must be 16-byte
+ *    aligned.  Dv must be a multiple of 8.
+ *  - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default
+ *    stream).  Inputs are never written.
+ *  - Every function returning int returns SWILA_OK (0) or a negative swila_status code;
+ *    nothing throws, aborts or prints.  Arguments are validated on the host before any
+ *    launch.
+ */
+#ifndef SWILA_H_
+#define SWILA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum swila_status {
+  SWILA_OK = 0,
+  SWILA_ERR_NULL = -1,        /* a required pointer is NULL */
+  SWILA_ERR_SHAPE = -2,       /* non-positive dimension, or Dv not a multiple of 8 */
+  SWILA_ERR_UNSUPPORTED = -3, /* Dk / J / dtype / flag combination not compiled */
+  SWILA_ERR_ALIGN = -4,       /* a pointer is not 16-byte aligned */
+  SWILA_ERR_ALIAS = -5,       /* the output o overlaps an input */
+  SWILA_ERR_CUDA = -6,        /* a CUDA runtime call failed; see swila_last_cuda_error() */
+  SWILA_ERR_SIZE = -7         /* a problem exceeds a stated size limit of the entry point */
+};
+
+enum { SWILA_IO_FP32 = 0, SWILA_IO_BF16 = 1 };
+
+/* flags */
+enum {
+  SWILA_TEMPORAL = 1,   /* Temporal SwiLA (Sec. 3.3, App. B.3) */
+  SWILA_GATED = 2,      /* Gated SwiLA, pre-decay form (Eq. 3.8) unless POST_DECAY */
+  SWILA_POST_DECAY = 4  /* with GATED: post-decay form (Eq. 3.7) */
+};
+
+/* gate_granularity (App. B.4): which indices the decay alpha depends on */
+enum {
+  SWILA_GATE_NONE = 0,
+  SWILA_GATE_PER_KEY = 1, /* alpha [B,H,T,J,Dk]: one gate per key dimension (the LM setting, App. D.3) */
+  SWILA_GATE_PER_OUT = 2, /* alpha [B,H,T,J,Dv]: one gate per output dimension (Eq. 3.7 as printed) */
+  SWILA_GATE_SCALAR = 3   /* alpha [B,H,T,J]:    one gate per component */
+};
+
+/* algo: which kernel evaluates the recurrence.  Every choice computes the same function. */
+enum {
+  SWILA_ALGO_AUTO = 0,
+  SWILA_ALGO_SCAN = 1,     /* sequential scan, state resident in registers, FP32 FMA pipe */
+  SWILA_ALGO_SCAN_WIDE = 2 /* the same scan with 256-thread blocks (twice the columns per
+                              block); ungated shapes with Dk >= 64 only */
+};
+
+typedef struct {
+  int32_t B, H, T;          /* batch, heads, tokens (T >= 0; ignored by swila_decode_step) */
+  int32_t Dk, Dv;           /* key / value head dimension; Dk in {16, 64, 128}; Dv % 8 == 0 */
+  int32_t J;                /* mixture components, in {1, 2, 4, 8} */
+  int32_t io_dtype;         /* SWILA_IO_*: dtype of q, k, v, o and of every *_logit tensor */
+  int32_t flags;            /* SWILA_TEMPORAL | SWILA_GATED | SWILA_POST_DECAY */
+  int32_t gate_granularity; /* SWILA_GATE_*; must be NONE iff GATED is clear */
+  int32_t algo;             /* SWILA_ALGO_* */
+} swila_shape_t;
+
+/* Per-token gate tensors: the layer's learned projections evaluated at every token,
+ * BEFORE their activation (App. B.2, B.3).  Logit tensors have the io dtype; alpha is
+ * always fp32 and already in [0, 1]. */
+typedef struct {
+  const void *beta_logit;  /* [B,H,T,J,Dv]  beta = sigmoid(.)                        */
+  const void *pik_logit;   /* [B,H,T,J,Dv]  key-side prior  = softmax over J         */
+  const void *piq_logit;   /* [B,H,T,J,Dv]  query-side prior = softmax over J        */
+  const void *gk_logit;    /* [B,H,T,Dv]    TEMPORAL only: g^k = sigmoid(.), else NULL */
+  const void *gq_logit;    /* [B,H,T,Dv]    TEMPORAL only: g^q = sigmoid(.), else NULL */
+  const float *alpha;      /* GATED only: decay, shape by gate_granularity, else NULL */
+} swila_gates_t;
+
+/* Carried state, always fp32. */
+typedef struct {
+  float *W;         /* [B,H,J,Dv,Dk] */
+  float *r_prev;    /* [B,H,J,Dv]  TEMPORAL only: previous posterior r_{t-1}   (App. B.3) */
+  float *rho_prev;  /* [B,H,J,Dv]  TEMPORAL only: previous query prior rhobar_{t-1}       */
+} swila_state_t;
+
+/* Library version (major*10000 + minor*100 + patch). */
+int swila_version(void);
+
+/* Static, never-NULL description of a status code. */
+const char *swila_strerror(int status);
+
+/* Text of the most recent CUDA error seen by the calling thread ("" if none). */
+const char *swila_last_cuda_error(void);
+
+/* Bytes of state->W and of each of state->r_prev / state->rho_prev for `shape`
+ * (0 if the shape is invalid). */
+size_t swila_state_w_bytes(const swila_shape_t *shape);
+size_t swila_state_r_bytes(const swila_shape_t *shape);
+
+/* Initial state: W = 0 and, when TEMPORAL, r_prev = rho_prev = 1/J (the paper does not
+ * state an initial distribution; uniform keeps both carried quantities distributions). */
+int swila_state_init(const swila_shape_t *shape, swila_state_t *state, void *stream);
+
+/*
+ * Prefill: run the recurrence of Eqs. 3.3-3.5 (with the variants selected in
+ * shape->flags) over all T tokens of q,k [B,H,T,Dk], v [B,H,T,Dv] and write o [B,H,T,Dv].
+ *   state_in  : initial state; NULL means the state of swila_state_init.
+ *   state_out : receives the state after token T; NULL discards it; may alias state_in
+ *               (each thread block reads its slice completely before writing it).
+ *   r_debug   : NULL, or fp32 [B,H,T,J,Dv] receiving the responsibilities r of Eq. 3.4.
+ * T == 0 copies state_in to state_out and touches nothing else.
+ */
+int swila_forward(const swila_shape_t *shape, const void *q, const void *k, const void *v,
+                  const swila_gates_t *gates, const swila_state_t *state_in,
+                  swila_state_t *state_out, void *o, float *r_debug, void *stream);
+
+/*
+ * Decode: one token of the same recurrence on a carried state, updated in place
+ * (generation, App. D.4).  q,k [B,H,1,Dk]; v, o [B,H,1,Dv]; gate tensors with T = 1.
+ * shape->T is ignored.  The arithmetic and its order are those of swila_forward, so a
+ * prefill of T tokens equals, bit for bit, T decode steps.
+ */
+int swila_decode_step(const swila_shape_t *shape, const void *q, const void *k, const void *v,
+                      const swila_gates_t *gates, swila_state_t *state, void *o, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SWILA_H_ */

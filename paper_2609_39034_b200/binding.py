@@ -1,0 +1,153 @@
+"""Thin ctypes binding of libswila.so: argument marshalling only.
+
+Every step of the recurrence runs inside the CUDA library; this module turns torch
+tensors into raw device pointers and mirrors the C structs of include/swila.h.  There
+is no CPU fallback: importing this module raises if the library has not been built."""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+from .workloads import Workload
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libswila.so")
+
+SWILA_OK = 0
+ERR_NULL, ERR_SHAPE, ERR_UNSUPPORTED, ERR_ALIGN, ERR_ALIAS, ERR_CUDA, ERR_SIZE = -1, -2, -3, -4, -5, -6, -7
+IO_FP32, IO_BF16 = 0, 1
+ALGO_AUTO, ALGO_SCAN, ALGO_SCAN_WIDE = 0, 1, 2
+
+EXPORTS = ("swila_version", "swila_strerror", "swila_last_cuda_error", "swila_state_w_bytes",
+           "swila_state_r_bytes", "swila_state_init", "swila_forward", "swila_decode_step")
+
+
+class Shape(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("B", "H", "T", "Dk", "Dv", "J", "io_dtype", "flags", "gate_granularity", "algo")]
+
+
+class Gates(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in
+                ("beta_logit", "pik_logit", "piq_logit", "gk_logit", "gq_logit", "alpha")]
+
+
+class State(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("W", "r_prev", "rho_prev")]
+
+
+class SwilaError(RuntimeError):
+    def __init__(self, status: int):
+        self.status = status
+        msg = lib.swila_strerror(status).decode()
+        if status == ERR_CUDA:
+            msg += ": " + lib.swila_last_cuda_error().decode()
+        super().__init__(f"swila status {status}: {msg}")
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2609_39034_b200.build` "
+            "(there is no fallback implementation)")
+    L = ctypes.CDLL(LIB_PATH)
+    L.swila_version.restype = ctypes.c_int
+    L.swila_strerror.restype = ctypes.c_char_p
+    L.swila_strerror.argtypes = [ctypes.c_int]
+    L.swila_last_cuda_error.restype = ctypes.c_char_p
+    for f in (L.swila_state_w_bytes, L.swila_state_r_bytes):
+        f.restype = ctypes.c_size_t
+        f.argtypes = [ctypes.POINTER(Shape)]
+    L.swila_state_init.restype = ctypes.c_int
+    L.swila_state_init.argtypes = [ctypes.POINTER(Shape), ctypes.POINTER(State), ctypes.c_void_p]
+    L.swila_forward.restype = ctypes.c_int
+    L.swila_forward.argtypes = [ctypes.POINTER(Shape), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                ctypes.POINTER(Gates), ctypes.POINTER(State), ctypes.POINTER(State),
+                                ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+    L.swila_decode_step.restype = ctypes.c_int
+    L.swila_decode_step.argtypes = [ctypes.POINTER(Shape), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                    ctypes.POINTER(Gates), ctypes.POINTER(State), ctypes.c_void_p, ctypes.c_void_p]
+    return L
+
+
+lib = _load()
+
+
+def make_shape(w: Workload, T: Optional[int] = None, algo: int = ALGO_AUTO) -> Shape:
+    return Shape(w.B, w.H, w.T if T is None else T, w.Dk, w.Dv, w.J,
+                 IO_BF16 if w.io_dtype == "bf16" else IO_FP32, w.flags, w.gate_granularity, algo)
+
+
+def _p(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "device-resident contiguous tensors only"
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _gates(inp: dict) -> Gates:
+    return Gates(*[(_p(inp.get(n)) or ctypes.c_void_p(None)).value for n in
+                   ("beta_logit", "pik_logit", "piq_logit", "gk_logit", "gq_logit", "alpha")])
+
+
+def _state(W, r, rho) -> State:
+    return State(W.data_ptr(), r.data_ptr() if r is not None else None, rho.data_ptr() if rho is not None else None)
+
+
+def check(status: int) -> None:
+    if status != SWILA_OK:
+        raise SwilaError(status)
+
+
+def state_alloc(w: Workload, device="cuda", init: bool = True, stream=None) -> dict:
+    """Allocate (torch) and optionally initialise (library) a carried state."""
+    st = {"W": torch.empty((w.B, w.H, w.J, w.Dv, w.Dk), device=device, dtype=torch.float32),
+          "r_prev": None, "rho_prev": None}
+    if w.temporal:
+        st["r_prev"] = torch.empty((w.B, w.H, w.J, w.Dv), device=device, dtype=torch.float32)
+        st["rho_prev"] = torch.empty((w.B, w.H, w.J, w.Dv), device=device, dtype=torch.float32)
+    if init:
+        sh = make_shape(w)
+        s = _state(st["W"], st["r_prev"], st["rho_prev"])
+        check(lib.swila_state_init(ctypes.byref(sh), ctypes.byref(s), _stream(stream)))
+    return st
+
+
+def swila_forward(w: Workload, inp: dict, *, state_in: Optional[dict] = None, state_out: Optional[dict] = None,
+                  o: Optional[torch.Tensor] = None, r_debug: Optional[torch.Tensor] = None,
+                  algo: int = ALGO_AUTO, stream=None, T: Optional[int] = None) -> torch.Tensor:
+    """Prefill over inp's q,k,v and gate tensors (device tensors laid out as in
+    include/swila.h).  state_in / state_out: dicts with W (and r_prev, rho_prev when
+    TEMPORAL), or None (initial state / discard).  Returns o."""
+    T = inp["q"].shape[2] if T is None else T
+    sh = make_shape(w, T=T, algo=algo)
+    if o is None:
+        o = torch.empty((w.B, w.H, T, w.Dv), device=inp["q"].device, dtype=w.torch_io_dtype)
+    g = _gates(inp)
+    sin = _state(state_in["W"], state_in.get("r_prev"), state_in.get("rho_prev")) if state_in else None
+    sout = _state(state_out["W"], state_out.get("r_prev"), state_out.get("rho_prev")) if state_out else None
+    check(lib.swila_forward(ctypes.byref(sh), _p(inp["q"]), _p(inp["k"]), _p(inp["v"]), ctypes.byref(g),
+                            ctypes.byref(sin) if sin else None, ctypes.byref(sout) if sout else None,
+                            _p(o), _p(r_debug), _stream(stream)))
+    return o
+
+
+def swila_decode_step(w: Workload, inp: dict, state: dict, *, o: Optional[torch.Tensor] = None,
+                      algo: int = ALGO_AUTO, stream=None) -> torch.Tensor:
+    """One token on a carried state (updated in place).  Returns o [B,H,1,Dv]."""
+    sh = make_shape(w, T=1, algo=algo)
+    if o is None:
+        o = torch.empty((w.B, w.H, 1, w.Dv), device=inp["q"].device, dtype=w.torch_io_dtype)
+    g = _gates(inp)
+    st = _state(state["W"], state.get("r_prev"), state.get("rho_prev"))
+    check(lib.swila_decode_step(ctypes.byref(sh), _p(inp["q"]), _p(inp["k"]), _p(inp["v"]), ctypes.byref(g),
+                                ctypes.byref(st), _p(o), _stream(stream)))
+    return o

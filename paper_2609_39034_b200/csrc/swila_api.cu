@@ -1,0 +1,203 @@
+// C-ABI entry points of the SwiLA library: host-side validation and kernel dispatch.
+// No device memory is allocated here and no state is kept between calls.
+#include <string.h>
+
+#include "swila_common.cuh"
+
+namespace swila {
+#define SWILA_DECL(DK, GATE, POST) template <> int scan_dispatch<DK, GATE, POST>(const LaunchArgs &);
+#define SWILA_DECL_DK(DK) \
+  SWILA_DECL(DK, 0, false) SWILA_DECL(DK, 1, false) SWILA_DECL(DK, 1, true) SWILA_DECL(DK, 2, false) SWILA_DECL(DK, 2, true)
+SWILA_DECL_DK(16)
+SWILA_DECL_DK(64)
+SWILA_DECL_DK(128)
+
+static thread_local char g_cuda_err[256] = "";
+
+static int cuda_fail(cudaError_t e) {
+  strncpy(g_cuda_err, cudaGetErrorString(e), sizeof(g_cuda_err) - 1);
+  g_cuda_err[sizeof(g_cuda_err) - 1] = 0;
+  return SWILA_ERR_CUDA;
+}
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int check_shape(const swila_shape_t *s, bool need_T) {
+  if (!s) return SWILA_ERR_NULL;
+  if (s->B <= 0 || s->H <= 0 || s->Dk <= 0 || s->Dv <= 0 || s->J <= 0) return SWILA_ERR_SHAPE;
+  if (need_T && s->T < 0) return SWILA_ERR_SHAPE;
+  if (s->Dv % 8 != 0) return SWILA_ERR_SHAPE;
+  if (s->Dk != 16 && s->Dk != 64 && s->Dk != 128) return SWILA_ERR_UNSUPPORTED;
+  if (s->J != 1 && s->J != 2 && s->J != 4 && s->J != 8) return SWILA_ERR_UNSUPPORTED;
+  if (s->io_dtype != SWILA_IO_FP32 && s->io_dtype != SWILA_IO_BF16) return SWILA_ERR_UNSUPPORTED;
+  if (s->flags & ~(SWILA_TEMPORAL | SWILA_GATED | SWILA_POST_DECAY)) return SWILA_ERR_UNSUPPORTED;
+  const bool gated = (s->flags & SWILA_GATED) != 0;
+  if (!gated && (s->flags & SWILA_POST_DECAY)) return SWILA_ERR_UNSUPPORTED;
+  if (gated != (s->gate_granularity != SWILA_GATE_NONE)) return SWILA_ERR_UNSUPPORTED;
+  if (s->gate_granularity < SWILA_GATE_NONE || s->gate_granularity > SWILA_GATE_SCALAR) return SWILA_ERR_UNSUPPORTED;
+  if (s->algo != SWILA_ALGO_AUTO && s->algo != SWILA_ALGO_SCAN && s->algo != SWILA_ALGO_SCAN_WIDE)
+    return SWILA_ERR_UNSUPPORTED;
+  return SWILA_OK;
+}
+
+static size_t w_elems(const swila_shape_t *s) { return (size_t)s->B * s->H * s->J * s->Dv * s->Dk; }
+static size_t r_elems(const swila_shape_t *s) { return (size_t)s->B * s->H * s->J * s->Dv; }
+
+static bool overlaps(const void *a, size_t na, const void *b, size_t nb) {
+  if (!a || !b || na == 0 || nb == 0) return false;
+  const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+  return a0 < b0 + nb && b0 < a0 + na;
+}
+
+static int run(const swila_shape_t *s, int T, const void *q, const void *k, const void *v, const swila_gates_t *g,
+               const swila_state_t *sin, swila_state_t *sout, void *o, float *r_debug, void *stream) {
+  const bool temporal = (s->flags & SWILA_TEMPORAL) != 0;
+  const bool gated = (s->flags & SWILA_GATED) != 0;
+  if (!q || !k || !v || !g || !o) return SWILA_ERR_NULL;
+  if (!g->beta_logit || !g->pik_logit || !g->piq_logit) return SWILA_ERR_NULL;
+  if (temporal && (!g->gk_logit || !g->gq_logit)) return SWILA_ERR_NULL;
+  if (gated && !g->alpha) return SWILA_ERR_NULL;
+  if (sin && !sin->W) return SWILA_ERR_NULL;
+  if (sout && !sout->W) return SWILA_ERR_NULL;
+  if (temporal && sin && (!sin->r_prev || !sin->rho_prev)) return SWILA_ERR_NULL;
+  if (temporal && sout && (!sout->r_prev || !sout->rho_prev)) return SWILA_ERR_NULL;
+  const void *ptrs[] = {q, k, v, o, g->beta_logit, g->pik_logit, g->piq_logit, temporal ? g->gk_logit : nullptr,
+                        temporal ? g->gq_logit : nullptr, gated ? (const void *)g->alpha : nullptr,
+                        sin ? sin->W : nullptr, sout ? sout->W : nullptr, r_debug};
+  for (const void *p : ptrs)
+    if (p && !aligned16(p)) return SWILA_ERR_ALIGN;
+  const size_t es = s->io_dtype == SWILA_IO_BF16 ? 2 : 4;
+  const size_t ntok = (size_t)s->B * s->H * (size_t)T;
+  const size_t o_bytes = ntok * s->Dv * es;
+  const size_t gate_bytes = ntok * s->J * s->Dv * es;
+  if (overlaps(o, o_bytes, q, ntok * s->Dk * es) || overlaps(o, o_bytes, k, ntok * s->Dk * es) ||
+      overlaps(o, o_bytes, v, ntok * s->Dv * es) || overlaps(o, o_bytes, g->beta_logit, gate_bytes) ||
+      overlaps(o, o_bytes, g->pik_logit, gate_bytes) || overlaps(o, o_bytes, g->piq_logit, gate_bytes))
+    return SWILA_ERR_ALIAS;
+
+  LaunchArgs a;
+  memset(&a, 0, sizeof(a));
+  a.p.B = s->B; a.p.H = s->H; a.p.T = T; a.p.Dv = s->Dv;
+  a.p.temporal = temporal ? 1 : 0;
+  a.p.gran = s->gate_granularity;
+  a.p.q = q; a.p.k = k; a.p.v = v;
+  a.p.beta_logit = g->beta_logit; a.p.pik_logit = g->pik_logit; a.p.piq_logit = g->piq_logit;
+  a.p.gk_logit = temporal ? g->gk_logit : nullptr;
+  a.p.gq_logit = temporal ? g->gq_logit : nullptr;
+  a.p.alpha = gated ? g->alpha : nullptr;
+  a.p.W_in = sin ? sin->W : nullptr;
+  a.p.r_in = (sin && temporal) ? sin->r_prev : nullptr;
+  a.p.rho_in = (sin && temporal) ? sin->rho_prev : nullptr;
+  a.p.W_out = sout ? sout->W : nullptr;
+  a.p.r_out = (sout && temporal) ? sout->r_prev : nullptr;
+  a.p.rho_out = (sout && temporal) ? sout->rho_prev : nullptr;
+  a.p.o = o;
+  a.p.r_debug = r_debug;
+  a.Dk = s->Dk; a.J = s->J; a.io_dtype = s->io_dtype;
+  a.gate_mode = !gated ? 0 : (s->gate_granularity == SWILA_GATE_PER_KEY ? 1 : 2);
+  a.post = (s->flags & SWILA_POST_DECAY) ? 1 : 0;
+  a.algo = s->algo;
+  a.stream = (cudaStream_t)stream;
+
+  int rc = -1000;
+#define SWILA_CASE(DK)                                                                          \
+  case DK:                                                                                      \
+    if (a.gate_mode == 0) rc = scan_dispatch<DK, 0, false>(a);                                  \
+    else if (a.gate_mode == 1) rc = a.post ? scan_dispatch<DK, 1, true>(a) : scan_dispatch<DK, 1, false>(a); \
+    else rc = a.post ? scan_dispatch<DK, 2, true>(a) : scan_dispatch<DK, 2, false>(a);          \
+    break;
+  switch (s->Dk) {
+    SWILA_CASE(16)
+    SWILA_CASE(64)
+    SWILA_CASE(128)
+    default: break;
+  }
+  if (rc == -1000) return SWILA_ERR_UNSUPPORTED;
+  if (rc != 0) return cuda_fail((cudaError_t)rc);
+  return SWILA_OK;
+}
+
+__global__ void fill_kernel(float *p, size_t n, float val) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) p[i] = val;
+}
+
+}  // namespace swila
+
+using namespace swila;
+
+extern "C" {
+
+int swila_version(void) { return 100; }
+
+const char *swila_strerror(int status) {
+  switch (status) {
+    case SWILA_OK: return "ok";
+    case SWILA_ERR_NULL: return "a required pointer is NULL";
+    case SWILA_ERR_SHAPE: return "invalid shape (non-positive dimension, or Dv not a multiple of 8)";
+    case SWILA_ERR_UNSUPPORTED: return "unsupported Dk / J / dtype / flag combination";
+    case SWILA_ERR_ALIGN: return "a pointer is not 16-byte aligned";
+    case SWILA_ERR_ALIAS: return "the output overlaps an input";
+    case SWILA_ERR_CUDA: return "a CUDA runtime call failed (see swila_last_cuda_error)";
+    case SWILA_ERR_SIZE: return "problem exceeds a size limit of this entry point";
+    default: return "unknown status";
+  }
+}
+
+const char *swila_last_cuda_error(void) { return g_cuda_err; }
+
+size_t swila_state_w_bytes(const swila_shape_t *s) { return check_shape(s, false) == SWILA_OK ? w_elems(s) * 4 : 0; }
+size_t swila_state_r_bytes(const swila_shape_t *s) { return check_shape(s, false) == SWILA_OK ? r_elems(s) * 4 : 0; }
+
+int swila_state_init(const swila_shape_t *s, swila_state_t *st, void *stream) {
+  int rc = check_shape(s, false);
+  if (rc) return rc;
+  if (!st || !st->W) return SWILA_ERR_NULL;
+  const bool temporal = (s->flags & SWILA_TEMPORAL) != 0;
+  if (temporal && (!st->r_prev || !st->rho_prev)) return SWILA_ERR_NULL;
+  cudaStream_t cs = (cudaStream_t)stream;
+  cudaError_t e = cudaMemsetAsync(st->W, 0, w_elems(s) * 4, cs);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (temporal) {
+    const size_t n = r_elems(s);
+    const unsigned grid = (unsigned)((n + 255) / 256 < 1024 ? (n + 255) / 256 : 1024);
+    fill_kernel<<<grid, 256, 0, cs>>>(st->r_prev, n, 1.0f / s->J);
+    fill_kernel<<<grid, 256, 0, cs>>>(st->rho_prev, n, 1.0f / s->J);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  return SWILA_OK;
+}
+
+int swila_forward(const swila_shape_t *s, const void *q, const void *k, const void *v, const swila_gates_t *g,
+                  const swila_state_t *state_in, swila_state_t *state_out, void *o, float *r_debug, void *stream) {
+  int rc = check_shape(s, true);
+  if (rc) return rc;
+  if (s->T == 0) {  // nothing to scan: the state passes through
+    if (!state_out) return SWILA_OK;
+    if (!state_out->W) return SWILA_ERR_NULL;
+    const bool temporal = (s->flags & SWILA_TEMPORAL) != 0;
+    if (temporal && (!state_out->r_prev || !state_out->rho_prev)) return SWILA_ERR_NULL;
+    if (!state_in) return swila_state_init(s, state_out, stream);
+    if (!state_in->W || (temporal && (!state_in->r_prev || !state_in->rho_prev))) return SWILA_ERR_NULL;
+    cudaStream_t cs = (cudaStream_t)stream;
+    cudaError_t e = cudaSuccess;
+    if (state_in->W != state_out->W)
+      e = cudaMemcpyAsync(state_out->W, state_in->W, w_elems(s) * 4, cudaMemcpyDeviceToDevice, cs);
+    if (e == cudaSuccess && temporal && state_in->r_prev != state_out->r_prev)
+      e = cudaMemcpyAsync(state_out->r_prev, state_in->r_prev, r_elems(s) * 4, cudaMemcpyDeviceToDevice, cs);
+    if (e == cudaSuccess && temporal && state_in->rho_prev != state_out->rho_prev)
+      e = cudaMemcpyAsync(state_out->rho_prev, state_in->rho_prev, r_elems(s) * 4, cudaMemcpyDeviceToDevice, cs);
+    return e == cudaSuccess ? SWILA_OK : cuda_fail(e);
+  }
+  return run(s, s->T, q, k, v, g, state_in, state_out, o, r_debug, stream);
+}
+
+int swila_decode_step(const swila_shape_t *s, const void *q, const void *k, const void *v, const swila_gates_t *g,
+                      swila_state_t *state, void *o, void *stream) {
+  int rc = check_shape(s, false);
+  if (rc) return rc;
+  if (!state) return SWILA_ERR_NULL;
+  return run(s, 1, q, k, v, g, state, state, o, nullptr, stream);
+}
+
+}  // extern "C"

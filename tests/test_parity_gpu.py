@@ -1,0 +1,165 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the fp64 CPU oracle on
+the same seeded inputs -- element by element at sizes spanning several token blocks,
+several column slices and ragged tails."""
+import pytest
+import torch
+
+from paper_2609_39034_b200 import workloads as wl
+from tests._gpu_util import assert_close, gpu_forward, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def binding():
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    from paper_2609_39034_b200 import binding as b
+
+    return b
+
+
+def _case(name, config, **kw):
+    return wl.CONFIGS[config].with_(name=name, **kw)
+
+
+# reduced copies of the five benchmark shapes: T not a multiple of the token block, more
+# than one column slice, ragged last slice where Dv allows
+SMALL = [
+    _case("c0", 0),
+    _case("c0_ragged", 0, T=37, Dv=24),
+    _case("c1_small", 1, B=2, H=3, T=203),
+    _case("c1_ragged_cols", 1, B=1, H=2, T=61, Dv=72),
+    _case("c2_small", 2, B=1, H=2, T=150),
+    _case("c2_gauss", 2, B=1, H=2, T=99, recipe="gauss"),
+    _case("c3_small", 3, B=3, H=2, T=200),
+    _case("c4_small", 4, B=2, H=2, T=77),
+    _case("j1_d128", 2, B=1, H=2, T=50, J=1, recipe="gauss"),
+    _case("j2_d128_fp32", 2, B=1, H=2, T=50, J=2, recipe="gauss", io_dtype="fp32"),
+    _case("j8_d128", 2, B=1, H=1, T=50, J=8, recipe="gauss"),
+    _case("j1_d64_fp32", 1, B=1, H=2, T=50, J=1, io_dtype="fp32"),
+    _case("j2_d64", 1, B=1, H=2, T=50, J=2),
+    _case("j4_d16_bf16", 0, T=45, J=4, io_dtype="bf16"),
+    _case("j8_d16", 0, T=45, J=8),
+]
+
+
+@pytest.mark.parametrize("w", SMALL, ids=lambda w: w.name)
+@pytest.mark.parametrize("stress", [False, True], ids=["calm", "stress"])
+def test_vanilla_matches_oracle(binding, oracle, w, stress):
+    inp = wl.make_inputs(w, stress=stress)
+    ref = oracle.forward_inputs(inp, want_r=True)
+    got = gpu_forward(binding, w, to_dev(inp), want_r=True)
+    assert_close(w, got, ref, w.name)
+
+
+VARIANTS = [
+    dict(temporal=True),
+    dict(gated=True),                                   # pre-decay, one gate per key dim (the LM setting)
+    dict(temporal=True, gated=True),
+    dict(gated=True, post_decay=True),
+    dict(gated=True, granularity=wl.GRAN_PER_OUT),
+    dict(gated=True, granularity=wl.GRAN_SCALAR, post_decay=True),
+    dict(temporal=True, gated=True, granularity=wl.GRAN_SCALAR),
+]
+VAR_SHAPES = [SMALL[0], SMALL[2], SMALL[3], SMALL[4], SMALL[6], SMALL[10]]
+
+
+@pytest.mark.parametrize("w0", VAR_SHAPES, ids=lambda w: w.name)
+@pytest.mark.parametrize("var", VARIANTS, ids=lambda v: "+".join(f"{k}={v[k]}" for k in v))
+def test_variants_match_oracle(binding, oracle, w0, var):
+    w = w0.variant(**var)
+    inp = wl.make_inputs(w, stress=True)
+    ref = oracle.forward_inputs(inp, flags=w.flags, gran=w.gate_granularity, want_r=True)
+    got = gpu_forward(binding, w, to_dev(inp), want_r=True)
+    assert_close(w, got, ref, w.name)
+
+
+@pytest.mark.parametrize("w", [SMALL[2], SMALL[4]], ids=lambda w: w.name)
+def test_wide_blocks_match_oracle(binding, oracle, w):
+    inp = wl.make_inputs(w, stress=True)
+    ref = oracle.forward_inputs(inp)
+    got = gpu_forward(binding, w, to_dev(inp), algo=binding.ALGO_SCAN_WIDE)
+    assert_close(w, got, ref, w.name)
+
+
+@pytest.mark.parametrize("w0", [SMALL[2], SMALL[4], SMALL[0]], ids=lambda w: w.name)
+@pytest.mark.parametrize("var", [dict(), dict(temporal=True, gated=True)], ids=["vanilla", "gated_temporal"])
+def test_prefill_then_decode_equals_prefill_bitwise(binding, w0, var):
+    """State carried across calls -- one long prefill, a split prefill, and a prefill followed
+    by single-token decode steps -- gives the same bits (same instruction sequence per token)."""
+    w = w0.variant(**var).with_(T=41)
+    inp = to_dev(wl.make_inputs(w, stress=True))
+    full = gpu_forward(binding, w, inp)
+    # split at a point that is not a token-block boundary
+    st = {"W": inp["W0"].clone(), "r_prev": inp["r0"].clone() if w.temporal else None,
+          "rho_prev": inp["rho0"].clone() if w.temporal else None}
+    outs = []
+    a = wl.slice_time(inp, 0, 13)
+    outs.append(binding.swila_forward(w, a, state_in=st, state_out=st))  # in place
+    b = wl.slice_time(inp, 13, 30)
+    outs.append(binding.swila_forward(w, b, state_in=st, state_out=st))
+    for t in range(30, 41):
+        outs.append(binding.swila_decode_step(w, wl.slice_time(inp, t, t + 1), st))
+    torch.cuda.synchronize()
+    o = torch.cat(outs, dim=2).cpu()
+    assert torch.equal(o, full["o"])
+    assert torch.equal(st["W"].cpu(), full["W"])
+    if w.temporal:
+        assert torch.equal(st["r_prev"].cpu(), full["r_prev"])
+        assert torch.equal(st["rho_prev"].cpu(), full["rho_prev"])
+
+
+def test_default_initial_state_and_discarded_state(binding, oracle):
+    w = SMALL[2].variant(temporal=True)
+    inp = wl.make_inputs(w)  # zero W0, uniform r0 / rho0
+    ref = oracle.forward_inputs(inp, flags=w.flags)
+    dev = to_dev(inp)
+    o = binding.swila_forward(w, dev, state_in=None, state_out=None)
+    torch.cuda.synchronize()
+    assert wl.rel_err(o.cpu(), torch.from_numpy(ref["o"])) < 2e-2
+    st = binding.state_alloc(w, init=True)
+    torch.cuda.synchronize()
+    assert float(st["W"].abs().max()) == 0.0
+    assert torch.equal(st["r_prev"].cpu(), inp["r0"]) and torch.equal(st["rho_prev"].cpu(), inp["rho0"])
+
+
+def test_zero_tokens_passes_the_state_through(binding):
+    w = SMALL[1].variant(temporal=True).with_(T=0)
+    inp = to_dev(wl.make_inputs(w.with_(T=4), stress=True))
+    sin = {"W": inp["W0"], "r_prev": inp["r0"], "rho_prev": inp["rho0"]}
+    sout = binding.state_alloc(w, init=False)
+    empty = wl.slice_time(inp, 0, 0)
+    for n in empty:  # zero-element tensors still need a pointer
+        if empty[n] is not None and empty[n].numel() == 0:
+            empty[n] = inp[n]
+    binding.swila_forward(w, empty, state_in=sin, state_out=sout, T=0, o=torch.empty(8, device="cuda"))
+    torch.cuda.synchronize()
+    for n in ("W", "r_prev", "rho_prev"):
+        assert torch.equal(sout[n], sin[n])
+
+
+def test_outputs_stay_inside_their_buffers(binding):
+    """Canary words around o and the output state must survive a call with ragged tails."""
+    w = SMALL[3]  # T=61, Dv=72: ragged token block and ragged last column slice
+    inp = to_dev(wl.make_inputs(w, stress=True))
+    pad = 64
+    n_o = w.B * w.H * w.T * w.Dv
+    big_o = torch.full((n_o + 2 * pad,), 7.0, device="cuda", dtype=w.torch_io_dtype)
+    o = big_o[pad:pad + n_o].view(w.B, w.H, w.T, w.Dv)
+    n_w = w.B * w.H * w.J * w.Dv * w.Dk
+    big_w = torch.full((n_w + 2 * pad,), 7.0, device="cuda", dtype=torch.float32)
+    st = {"W": big_w[pad:pad + n_w].view(w.B, w.H, w.J, w.Dv, w.Dk), "r_prev": None, "rho_prev": None}
+    binding.swila_forward(w, inp, state_in={"W": inp["W0"]}, state_out=st, o=o)
+    torch.cuda.synchronize()
+    for big, n in ((big_o, n_o), (big_w, n_w)):
+        assert bool((big[:pad] == 7.0).all()) and bool((big[pad + n:] == 7.0).all())
+    assert not bool((o == 7.0).all())
+
+
+def test_inputs_are_not_written(binding):
+    w = SMALL[2].variant(temporal=True, gated=True)
+    inp = to_dev(wl.make_inputs(w, stress=True))
+    before = {n: x.clone() for n, x in inp.items() if x is not None}
+    gpu_forward(binding, w, inp)
+    for n, x in before.items():
+        assert torch.equal(x, inp[n]), n
