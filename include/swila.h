@@ -68,7 +68,7 @@ enum {
   SWILA_ALGO_AUTO = 0,
   SWILA_ALGO_SCAN = 1,     /* sequential scan, state resident in registers, FP32 FMA pipe */
   SWILA_ALGO_SCAN_WIDE = 2 /* the same scan with 256-thread blocks (twice the columns per
-                              block); ungated shapes with Dk >= 64 only */
+                              block); ungated shapes with Dk = 128 only */
 };
 
 typedef struct {

@@ -21,7 +21,7 @@ int pick(const LaunchArgs &a) {
     return launch_scan<IO, J, DK, 32, TB, GATE, POST>(a);
   } else {
     if (a.algo == SWILA_ALGO_SCAN_WIDE) {
-      if constexpr (GATE == 0) return launch_scan<IO, J, DK, 256, TB, GATE, POST>(a);
+      if constexpr (GATE == 0 && DK == 128) return launch_scan<IO, J, DK, 256, TB, GATE, POST>(a);
       return -1000;
     }
     return launch_scan<IO, J, DK, 128, TB, GATE, POST>(a);

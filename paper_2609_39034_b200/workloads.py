@@ -101,7 +101,7 @@ def _l2n(x: torch.Tensor) -> torch.Tensor:
 
 def _head_proj(theta: torch.Tensor, x: torch.Tensor) -> torch.Tensor:
     """theta [H, M, Dk] applied to x [B, H, T, Dk] -> [B, H, T, M]."""
-    return torch.einsum("hmd,bhtd->bhtm", theta, x)
+    return torch.einsum("hmd,bhtd->bhtm", theta, x).contiguous()
 
 
 def make_inputs(w: Workload, *, device="cpu", stress: bool = False, seed_offset: int = 0,
@@ -164,10 +164,11 @@ def make_inputs(w: Workload, *, device="cpu", stress: bool = False, seed_offset:
             gk_l = gq_l = None
         k_for_alpha = k
 
-    out["q"], out["k"], out["v"] = q.to(io), k.to(io), v.to(io)
-    out["beta_logit"], out["pik_logit"], out["piq_logit"] = beta_l.to(io), pik_l.to(io), piq_l.to(io)
-    out["gk_logit"] = gk_l.to(io) if gk_l is not None else None
-    out["gq_logit"] = gq_l.to(io) if gq_l is not None else None
+    out["q"], out["k"], out["v"] = q.to(io).contiguous(), k.to(io).contiguous(), v.to(io).contiguous()
+    out["beta_logit"], out["pik_logit"] = beta_l.to(io).contiguous(), pik_l.to(io).contiguous()
+    out["piq_logit"] = piq_l.to(io).contiguous()
+    out["gk_logit"] = gk_l.to(io).contiguous() if gk_l is not None else None
+    out["gq_logit"] = gq_l.to(io).contiguous() if gq_l is not None else None
 
     if w.gated:
         # Decay values in (0,1), mostly near 1 (sigmoid(3) ~ 0.95), key-dependent.
