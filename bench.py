@@ -1,0 +1,391 @@
+#!/usr/bin/env python
+"""Benchmark of the SwiLA recurrence on B200.
+
+A step is one pass of the whole hot path -- one ``swila_forward`` over the language-model
+shaped prefill workload (B=4, H=16, T=8192, Dk=Dv=128, J=4, bf16 inputs, fp32 state) with
+inputs resident in HBM.  Reported beside it: the same call end to end from pinned host
+buffers (``e2e``), the batched decode leg (B=256 streams, H=32, 1024 single-token steps),
+the roofline of the scan kernel, and the fp64 CPU oracle timed on the host cores.
+
+    python bench.py --gpus 1 --steps 10 --warmup 3
+    python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N ...   (independent replicas)
+    python bench.py --impl reference      (the CPU oracle alone, same metric and workload)
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2609_39034_b200 import workloads as wl  # noqa: E402
+
+METRIC = "swila_fwd_tokens_per_s"
+UNIT = "tokens/s"
+HEADLINE = 2  # config index of the workload the metric is quoted on
+
+# DRAM traffic of one scan launch on the headline workload, from the ncu capture
+# summarised in profiles/scan_lm_prefill.md (dram__bytes_read.sum + dram__bytes_write.sum).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 2.188e9
+
+
+# ----------------------------------------------------------------------------------------------
+def algorithmic_bytes(w: wl.Workload) -> float:
+    """HBM bytes one prefill must move: q, k, v, o, three gate tensors, plus the state once
+    each way."""
+    es = 2 if w.io_dtype == "bf16" else 4
+    per_tok_head = (2 * w.Dk + 2 * w.Dv + 3 * w.J * w.Dv) * es
+    if w.temporal:
+        per_tok_head += 2 * w.Dv * es
+    if w.gated:
+        per = {wl.GRAN_PER_KEY: w.Dk, wl.GRAN_PER_OUT: w.Dv, wl.GRAN_SCALAR: 1}[w.gate_granularity]
+        per_tok_head += w.J * per * 4
+    state = 2 * w.J * w.Dk * w.Dv * 4
+    return float(w.B * w.H * (w.T * per_tok_head + state))
+
+
+def algorithmic_flops(w: wl.Workload, T=None) -> float:
+    """FP32 flops of the recurrence: prediction, update and readout are J*Dk*Dv FMAs each."""
+    T = w.T if T is None else T
+    return 6.0 * w.J * w.Dk * w.Dv * w.B * w.H * T
+
+
+class ClockSampler:
+    """nvidia-smi samples (SM clock, throttle reasons) taken DURING a timed region."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        fd, self.path = tempfile.mkstemp(suffix=".csv")
+        os.close(fd)
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        clocks, reasons, mx, power = [], set(), None, []
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for ln in open(self.path):
+            parts = [x.strip() for x in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                clocks.append(float(parts[0]))
+                mx = float(parts[1])
+                power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        os.unlink(self.path)
+        if clocks:
+            out.update(sm_mhz=statistics.median(clocks), sm_max_mhz=mx, reasons=sorted(reasons),
+                       samples=len(clocks), power_w_max=max(power))
+        return out
+
+
+def time_steps(fn, steps: int, stream) -> float:
+    """Milliseconds for `steps` back-to-back calls of fn, CUDA events on `stream`."""
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(steps):
+        fn()
+    b.record(stream)
+    b.synchronize()
+    return a.elapsed_time(b)
+
+
+# ----------------------------------------------------------------------------------------------
+def cpu_baseline(w: wl.Workload, n_bh: int, repeats: int = 1, warmup: int = 0):
+    """The fp64 oracle, as it stands, on the first n_bh (batch, head) pairs of workload w
+    (all T tokens, all Dv columns).  Returns (tokens/s, seconds per pass, threads)."""
+    from oracle import swila_oracle
+
+    small = w.with_(B=1, H=n_bh)
+    inp = wl.make_inputs(small)  # CPU tensors; same shapes and dtypes as the workload's rows
+    cores = swila_oracle.threads()
+    for _ in range(warmup):
+        swila_oracle.forward_inputs(inp)
+    ts = []
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        swila_oracle.forward_inputs(inp)
+        ts.append(time.perf_counter() - t0)
+    sec = sum(ts) / len(ts)
+    # a token counts once for all H heads of the workload
+    tokens = n_bh * w.T / w.H
+    return tokens / sec, sec, cores
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = wl.CONFIGS[HEADLINE]
+    n_bh = 2
+    val, sec, cores = cpu_baseline(w, n_bh, repeats=max(1, args.steps), warmup=args.warmup)
+    sample = f"{n_bh} of {w.B * w.H} (batch, head) rows of {w.name}, all {w.T} tokens and {w.Dv} columns, per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "B": w.B, "H": w.H, "T": w.T, "Dk": w.Dk, "Dv": w.Dv, "J": w.J,
+                   "note": "fp64 CPU oracle on a bounded sample; tokens/s scaled by sampled rows / H"},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------
+def measure_fma_peak(binding, stream) -> float:
+    """FP32 FMA-chain microbenchmark (scalar FMAs, 16 chains/thread, 8 blocks/SM): TFLOP/s."""
+    scratch = torch.zeros(4, device="cuda")
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    best = 0.0
+    for _ in range(3):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        n = binding.bench_fma_chain(False, 16, sms * 8, 20000, scratch)
+        b.record(stream)
+        b.synchronize()
+        best = max(best, 2.0 * n / (a.elapsed_time(b) * 1e-3) / 1e12)
+    return best
+
+
+def decode_leg(binding, args, stream, dev_index):
+    """Config 4: B=256 streams, H=32; states from a seeded 4096-token prefill fed in chunks of
+    256 tokens, then `decode_steps` single-token calls with fresh inputs, timed back to back."""
+    w = wl.CONFIGS[4]
+    if args.decode_batch:
+        w = w.with_(B=args.decode_batch)
+    st = binding.state_alloc(w)
+    chunk = wl.DECODE_PREFILL_CHUNK
+    for c in range(args.decode_prefill // chunk):
+        inp = wl.make_inputs(w.with_(T=chunk), device="cuda", seed_offset=1 + c)
+        binding.swila_forward(w, inp, state_in=st, state_out=st)
+        torch.cuda.synchronize()
+        del inp
+    steps = args.decode_steps
+    ins = [wl.decode_step_inputs(w, s, device="cuda") for s in range(steps)]
+    o = torch.empty((w.B, w.H, 1, w.Dv), device="cuda", dtype=w.torch_io_dtype)
+    # warm-up on a scratch copy of the state
+    warm = {k: (v.clone() if v is not None else None) for k, v in st.items()}
+    for s in range(min(8, steps)):
+        binding.swila_decode_step(w, ins[s], warm, o=o)
+    torch.cuda.synchronize()
+    del warm
+    sampler = ClockSampler(dev_index)
+    sampler.start()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for s in range(steps):
+        binding.swila_decode_step(w, ins[s], st, o=o)
+    b.record(stream)
+    b.synchronize()
+    clocks = sampler.stop()
+    ms = a.elapsed_time(b)
+    es = 2
+    per_bh_inputs = (2 * w.Dk + 2 * w.Dv + 3 * w.J * w.Dv) * es
+    bytes_step = w.B * w.H * (per_bh_inputs + 2 * w.J * w.Dk * w.Dv * 4)
+    peaks = _peaks()
+    ach = bytes_step * steps / (ms * 1e-3) / 1e9
+    return {
+        "workload": w.name, "B": w.B, "H": w.H, "Dk": w.Dk, "Dv": w.Dv, "J": w.J, "prefill_tokens": args.decode_prefill,
+        "steps": steps, "steps_per_s": steps / (ms * 1e-3), "tokens_per_s": w.B * steps / (ms * 1e-3),
+        "ms_per_step": ms / steps, "gpu_launches": steps,
+        "roofline": {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": ach / peaks["hbm_gbs"], "peak_source": peaks["source"], "traffic": None,
+                     "algorithmic_bytes_per_launch": bytes_step},
+        "clocks": clocks,
+    }
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": float(d["hbm_gbs"]), "source": "measured (MEASURED_PEAKS.json)"}
+    return {"hbm_gbs": 6650.0, "source": "fallback"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--algo", type=int, default=0, help="SWILA_ALGO_* kernel choice (0 = auto)")
+    ap.add_argument("--no-decode", action="store_true", help="skip the batched decode leg")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    ap.add_argument("--decode-steps", type=int, default=wl.DECODE_STEPS)
+    ap.add_argument("--decode-prefill", type=int, default=4096)
+    ap.add_argument("--decode-batch", type=int, default=0, help="override B of the decode leg (0 = 256)")
+    ap.add_argument("--batch", type=int, default=0, help="override B of the prefill workload (profiling only)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device; there is no CPU fallback"
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    from paper_2609_39034_b200 import build as swila_build
+
+    if rank == 0 or world == 1:
+        swila_build.build()
+    if world > 1:
+        dist.barrier()
+    from paper_2609_39034_b200 import binding
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    w = wl.CONFIGS[HEADLINE]
+    if args.batch:
+        w = w.with_(B=args.batch)
+    stream = torch.cuda.current_stream()
+    inp = wl.make_inputs(w, device="cuda")
+    st_out = binding.state_alloc(w, init=False)
+    o = torch.empty((w.B, w.H, w.T, w.Dv), device="cuda", dtype=w.torch_io_dtype)
+
+    def step():
+        binding.swila_forward(w, inp, state_in=None, state_out=st_out, o=o, algo=args.algo)
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms = time_steps(step, args.steps, stream)
+    barrier()
+    clocks = sampler.stop()
+    if world > 1:
+        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / args.steps
+    value = world * w.B * w.T / (ms_per_step * 1e-3)
+
+    # ---- roofline of the scan kernel (one launch per step) ----
+    props = torch.cuda.get_device_properties(local)
+    peaks = _peaks()
+    fma_peak_nominal = props.multi_processor_count * 128 * 2 * 1.965e9 / 1e12  # TFLOP/s at the max SM clock
+    fma_peak_measured = measure_fma_peak(binding, stream)
+    flops = algorithmic_flops(w)
+    ach_tflops = flops / (ms_per_step * 1e-3) / 1e12
+    abytes = algorithmic_bytes(w)
+    roofline = {
+        "bound": "alu", "achieved": ach_tflops, "peak": fma_peak_nominal, "unit": "TFLOP/s",
+        "frac": ach_tflops / fma_peak_nominal,
+        "peak_source": "derived: SMs x 128 FP32 lanes x 2 x 1.965 GHz",
+        "peak_measured_fma_chain": fma_peak_measured, "frac_of_measured_fma_chain": ach_tflops / fma_peak_measured,
+        "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if not args.batch else None,
+        "algorithmic_bytes_per_launch": abytes, "algorithmic_flops_per_launch": flops,
+        "hbm_achieved_gbs": abytes / (ms_per_step * 1e-3) / 1e9, "hbm_peak_gbs": peaks["hbm_gbs"],
+        "hbm_frac": abytes / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"], "hbm_peak_source": peaks["source"],
+        "kernel": "swila_scan_kernel",
+    }
+
+    # ---- end to end from pinned host buffers through the C ABI ----
+    e2e = None
+    if not args.no_e2e:
+        names = ("q", "k", "v", "beta_logit", "pik_logit", "piq_logit")
+        host = {n: inp[n].cpu().pin_memory() for n in names}
+        host.update(gk_logit=None, gq_logit=None, alpha=None)
+        o_host = torch.empty(o.shape, dtype=o.dtype).pin_memory()
+        ws = torch.empty(binding.host_workspace_bytes(w), device="cuda", dtype=torch.uint8)
+
+        def step_host():
+            binding.swila_forward_host(w, host, ws, state_in=None, state_out=None, o=o_host, algo=args.algo)
+
+        n_e2e = max(2, min(args.steps, 5))
+        step_host()
+        barrier()
+        ms_e = time_steps(step_host, n_e2e, stream)
+        barrier()
+        if world > 1:
+            t = torch.tensor([ms_e], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e = float(t.item())
+        h2d = sum(host[n].numel() * host[n].element_size() for n in names)
+        d2h = o_host.numel() * o_host.element_size()
+        e2e = {"value": world * w.B * w.T / (ms_e / n_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": ms_e / n_e2e, "steps": n_e2e,
+               "note": "swila_forward_host: pinned host inputs -> device workspace -> kernel -> o to pinned host"}
+        del host, o_host, ws
+    del inp, o, st_out
+    torch.cuda.empty_cache()
+
+    decode = None
+    if not args.no_decode:
+        decode = decode_leg(binding, args, stream, local)
+        torch.cuda.empty_cache()
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        n_bh = 32
+        val, sec, cores = cpu_baseline(wl.CONFIGS[HEADLINE], n_bh)
+        cpu = {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "seconds": sec,
+               "sample": f"{n_bh} of {wl.CONFIGS[HEADLINE].B * wl.CONFIGS[HEADLINE].H} (batch, head) rows, all tokens "
+                         f"and columns, one pass; tokens/s = rows*T/H / s"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "B": w.B, "H": w.H, "T": w.T, "Dk": w.Dk, "Dv": w.Dv, "J": w.J,
+                       "io_dtype": w.io_dtype, "state_dtype": "fp32", "algo": args.algo,
+                       "l2": "inputs (2.1 GB) larger than L2; no flush needed",
+                       "multi_gpu": "independent replicas, no collective"},
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": args.steps,
+            "clocks": clocks, "decode": decode,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -67,8 +67,10 @@ enum {
 enum {
   SWILA_ALGO_AUTO = 0,
   SWILA_ALGO_SCAN = 1,     /* sequential scan, state resident in registers, FP32 FMA pipe */
-  SWILA_ALGO_SCAN_WIDE = 2 /* the same scan with 256-thread blocks (twice the columns per
+  SWILA_ALGO_SCAN_WIDE = 2, /* the same scan with 256-thread blocks (twice the columns per
                               block); ungated shapes with Dk = 128 only */
+  SWILA_ALGO_SCAN_NARROW = 3 /* the same scan with 16 key dimensions per lane (more, lighter
+                              warps); ungated shapes with Dk = 128, J >= 4 only */
 };
 
 typedef struct {
@@ -139,6 +141,35 @@ int swila_forward(const swila_shape_t *shape, const void *q, const void *k, cons
  */
 int swila_decode_step(const swila_shape_t *shape, const void *q, const void *k, const void *v,
                       const swila_gates_t *gates, swila_state_t *state, void *o, void *stream);
+
+/*
+ * Prefill with HOST buffers: the same computation as swila_forward (Eqs. 3.3-3.5), for callers
+ * whose tensors live in host memory.  q, k, v, every pointer inside `gates`, `state_in`,
+ * `state_out` and o are HOST pointers (pinned memory makes the copies asynchronous);
+ * `workspace` is a DEVICE buffer of at least swila_forward_host_workspace_bytes(shape)
+ * bytes, owned by the caller and reusable across calls.  On `stream` the call enqueues the
+ * host-to-device copies, the kernel, and the device-to-host copies of o and of the final
+ * state; it returns without synchronising.  state_in == NULL starts from the initial
+ * state; state_out == NULL discards the final state.  Errors as swila_forward, plus
+ * SWILA_ERR_SIZE when the workspace is too small.
+ */
+size_t swila_forward_host_workspace_bytes(const swila_shape_t *shape);
+int swila_forward_host(const swila_shape_t *shape, const void *q, const void *k, const void *v,
+                       const swila_gates_t *gates, const swila_state_t *state_in,
+                       swila_state_t *state_out, void *o, void *workspace, size_t workspace_bytes,
+                       void *stream);
+
+/*
+ * Measurement helper (no counterpart in the paper): launches an FP32 FMA-chain
+ * microbenchmark whose rate is the denominator of the scan kernel's roofline (the
+ * recurrence costs 3*J*Dk*Dv FP32 FMAs per token and head, Sec. 3.2).  Every thread of
+ * `blocks` blocks of 256 threads runs `iters` rounds of 2*`chains` independent register
+ * FMAs; packed != 0 uses the packed f32x2 form.  chains in {4, 8, 16}.  scratch_out: device
+ * pointer to >= 4 bytes (practically never written).  *fma_per_launch (HOST pointer) receives
+ * the number of FMAs one launch performs; time the launch with CUDA events on `stream`.
+ */
+int swila_bench_fma_chain(int packed, int chains, int blocks, int iters, float *scratch_out,
+                          double *fma_per_launch, void *stream);
 
 #ifdef __cplusplus
 }

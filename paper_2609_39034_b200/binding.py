@@ -19,10 +19,11 @@ LIB_PATH = os.path.join(_HERE, "libswila.so")
 SWILA_OK = 0
 ERR_NULL, ERR_SHAPE, ERR_UNSUPPORTED, ERR_ALIGN, ERR_ALIAS, ERR_CUDA, ERR_SIZE = -1, -2, -3, -4, -5, -6, -7
 IO_FP32, IO_BF16 = 0, 1
-ALGO_AUTO, ALGO_SCAN, ALGO_SCAN_WIDE = 0, 1, 2
+ALGO_AUTO, ALGO_SCAN, ALGO_SCAN_WIDE, ALGO_SCAN_NARROW = 0, 1, 2, 3
 
 EXPORTS = ("swila_version", "swila_strerror", "swila_last_cuda_error", "swila_state_w_bytes",
-           "swila_state_r_bytes", "swila_state_init", "swila_forward", "swila_decode_step")
+           "swila_state_r_bytes", "swila_state_init", "swila_forward", "swila_decode_step",
+           "swila_bench_fma_chain", "swila_forward_host", "swila_forward_host_workspace_bytes")
 
 
 class Shape(ctypes.Structure):
@@ -70,6 +71,15 @@ def _load() -> ctypes.CDLL:
     L.swila_decode_step.restype = ctypes.c_int
     L.swila_decode_step.argtypes = [ctypes.POINTER(Shape), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                     ctypes.POINTER(Gates), ctypes.POINTER(State), ctypes.c_void_p, ctypes.c_void_p]
+    L.swila_forward_host_workspace_bytes.restype = ctypes.c_size_t
+    L.swila_forward_host_workspace_bytes.argtypes = [ctypes.POINTER(Shape)]
+    L.swila_forward_host.restype = ctypes.c_int
+    L.swila_forward_host.argtypes = [ctypes.POINTER(Shape), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                     ctypes.POINTER(Gates), ctypes.POINTER(State), ctypes.POINTER(State),
+                                     ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+    L.swila_bench_fma_chain.restype = ctypes.c_int
+    L.swila_bench_fma_chain.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
+                                        ctypes.POINTER(ctypes.c_double), ctypes.c_void_p]
     return L
 
 
@@ -81,10 +91,10 @@ def make_shape(w: Workload, T: Optional[int] = None, algo: int = ALGO_AUTO) -> S
                  IO_BF16 if w.io_dtype == "bf16" else IO_FP32, w.flags, w.gate_granularity, algo)
 
 
-def _p(t: Optional[torch.Tensor]):
+def _p(t: Optional[torch.Tensor], host: bool = False):
     if t is None:
         return None
-    assert t.is_cuda and t.is_contiguous(), "device-resident contiguous tensors only"
+    assert t.is_contiguous() and t.is_cuda != host, "contiguous tensors on the side the entry point expects"
     return ctypes.c_void_p(t.data_ptr())
 
 
@@ -93,8 +103,8 @@ def _stream(stream) -> ctypes.c_void_p:
     return ctypes.c_void_p(s.cuda_stream)
 
 
-def _gates(inp: dict) -> Gates:
-    return Gates(*[(_p(inp.get(n)) or ctypes.c_void_p(None)).value for n in
+def _gates(inp: dict, host: bool = False) -> Gates:
+    return Gates(*[(_p(inp.get(n), host) or ctypes.c_void_p(None)).value for n in
                    ("beta_logit", "pik_logit", "piq_logit", "gk_logit", "gq_logit", "alpha")])
 
 
@@ -150,4 +160,36 @@ def swila_decode_step(w: Workload, inp: dict, state: dict, *, o: Optional[torch.
     st = _state(state["W"], state.get("r_prev"), state.get("rho_prev"))
     check(lib.swila_decode_step(ctypes.byref(sh), _p(inp["q"]), _p(inp["k"]), _p(inp["v"]), ctypes.byref(g),
                                 ctypes.byref(st), _p(o), _stream(stream)))
+    return o
+
+
+def bench_fma_chain(packed: bool, chains: int, blocks: int, iters: int, scratch: torch.Tensor, stream=None) -> float:
+    """Launch the FMA-chain microbenchmark once; returns the FMAs it performs."""
+    n = ctypes.c_double(0.0)
+    check(lib.swila_bench_fma_chain(int(packed), chains, blocks, iters, _p(scratch), ctypes.byref(n), _stream(stream)))
+    return n.value
+
+
+def host_workspace_bytes(w: Workload, T: Optional[int] = None) -> int:
+    sh = make_shape(w, T=T)
+    return int(lib.swila_forward_host_workspace_bytes(ctypes.byref(sh)))
+
+
+def swila_forward_host(w: Workload, inp: dict, workspace: torch.Tensor, *, state_in: Optional[dict] = None,
+                       state_out: Optional[dict] = None, o: Optional[torch.Tensor] = None, algo: int = ALGO_AUTO,
+                       stream=None) -> torch.Tensor:
+    """Prefill on HOST tensors (pinned for asynchronous copies) staged through the caller's
+    device ``workspace`` (a uint8 CUDA tensor).  Returns the host tensor o; synchronise the
+    stream before reading it."""
+    T = inp["q"].shape[2]
+    sh = make_shape(w, T=T, algo=algo)
+    if o is None:
+        o = torch.empty((w.B, w.H, T, w.Dv), dtype=w.torch_io_dtype).pin_memory()
+    g = _gates(inp, host=True)
+    sin = _state(state_in["W"], state_in.get("r_prev"), state_in.get("rho_prev")) if state_in else None
+    sout = _state(state_out["W"], state_out.get("r_prev"), state_out.get("rho_prev")) if state_out else None
+    check(lib.swila_forward_host(ctypes.byref(sh), _p(inp["q"], True), _p(inp["k"], True), _p(inp["v"], True),
+                                 ctypes.byref(g), ctypes.byref(sin) if sin else None,
+                                 ctypes.byref(sout) if sout else None, _p(o, True), _p(workspace),
+                                 workspace.numel() * workspace.element_size(), _stream(stream)))
     return o

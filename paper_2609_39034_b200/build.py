@@ -19,6 +19,7 @@ LIB = os.path.join(HERE, "libswila.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
+NVCC_FLAGS += os.environ.get("SWILA_NVCC_EXTRA", "").split()  # developer experiments only
 DKS = (16, 64, 128)
 GATE_MODES = ((0, 0), (1, 0), (1, 1), (2, 0), (2, 1))  # (decay mode, post-decay)
 

@@ -35,7 +35,8 @@ static int check_shape(const swila_shape_t *s, bool need_T) {
   if (!gated && (s->flags & SWILA_POST_DECAY)) return SWILA_ERR_UNSUPPORTED;
   if (gated != (s->gate_granularity != SWILA_GATE_NONE)) return SWILA_ERR_UNSUPPORTED;
   if (s->gate_granularity < SWILA_GATE_NONE || s->gate_granularity > SWILA_GATE_SCALAR) return SWILA_ERR_UNSUPPORTED;
-  if (s->algo != SWILA_ALGO_AUTO && s->algo != SWILA_ALGO_SCAN && s->algo != SWILA_ALGO_SCAN_WIDE)
+  if (s->algo != SWILA_ALGO_AUTO && s->algo != SWILA_ALGO_SCAN && s->algo != SWILA_ALGO_SCAN_WIDE &&
+      s->algo != SWILA_ALGO_SCAN_NARROW)
     return SWILA_ERR_UNSUPPORTED;
   return SWILA_OK;
 }
@@ -198,6 +199,96 @@ int swila_decode_step(const swila_shape_t *s, const void *q, const void *k, cons
   if (rc) return rc;
   if (!state) return SWILA_ERR_NULL;
   return run(s, 1, q, k, v, g, state, state, o, nullptr, stream);
+}
+
+}  // extern "C"
+
+// ---- host-buffer front end --------------------------------------------------------------
+namespace swila {
+static size_t up256(size_t n) { return (n + 255) & ~(size_t)255; }
+struct HostPlan {
+  size_t q, k, v, beta, pik, piq, gk, gq, alpha, W, r, rho, o, total;
+  size_t n_qk, n_v, n_gate, n_tg, n_alpha, n_W, n_r;
+};
+static HostPlan host_plan(const swila_shape_t *s) {
+  HostPlan h;
+  const size_t es = s->io_dtype == SWILA_IO_BF16 ? 2 : 4;
+  const size_t ntok = (size_t)s->B * s->H * (size_t)s->T;
+  const bool temporal = (s->flags & SWILA_TEMPORAL) != 0, gated = (s->flags & SWILA_GATED) != 0;
+  h.n_qk = ntok * s->Dk * es;
+  h.n_v = ntok * s->Dv * es;
+  h.n_gate = ntok * s->J * s->Dv * es;
+  h.n_tg = temporal ? ntok * s->Dv * es : 0;
+  const size_t per = s->gate_granularity == SWILA_GATE_PER_KEY ? (size_t)s->Dk
+                     : s->gate_granularity == SWILA_GATE_PER_OUT ? (size_t)s->Dv : 1;
+  h.n_alpha = gated ? ntok * s->J * per * 4 : 0;
+  h.n_W = w_elems(s) * 4;
+  h.n_r = temporal ? r_elems(s) * 4 : 0;
+  size_t off = 0;
+  auto take = [&](size_t n) { size_t o = off; off += up256(n); return o; };
+  h.q = take(h.n_qk); h.k = take(h.n_qk); h.v = take(h.n_v);
+  h.beta = take(h.n_gate); h.pik = take(h.n_gate); h.piq = take(h.n_gate);
+  h.gk = take(h.n_tg); h.gq = take(h.n_tg); h.alpha = take(h.n_alpha);
+  h.W = take(h.n_W); h.r = take(h.n_r); h.rho = take(h.n_r);
+  h.o = take(h.n_v);
+  h.total = off;
+  return h;
+}
+}  // namespace swila
+
+extern "C" {
+
+size_t swila_forward_host_workspace_bytes(const swila_shape_t *s) {
+  if (check_shape(s, true) != SWILA_OK) return 0;
+  return host_plan(s).total;
+}
+
+int swila_forward_host(const swila_shape_t *s, const void *q, const void *k, const void *v, const swila_gates_t *g,
+                       const swila_state_t *state_in, swila_state_t *state_out, void *o, void *workspace,
+                       size_t workspace_bytes, void *stream) {
+  int rc = check_shape(s, true);
+  if (rc) return rc;
+  if (!q || !k || !v || !g || !o || !workspace) return SWILA_ERR_NULL;
+  const bool temporal = (s->flags & SWILA_TEMPORAL) != 0, gated = (s->flags & SWILA_GATED) != 0;
+  if (!g->beta_logit || !g->pik_logit || !g->piq_logit) return SWILA_ERR_NULL;
+  if (temporal && (!g->gk_logit || !g->gq_logit)) return SWILA_ERR_NULL;
+  if (gated && !g->alpha) return SWILA_ERR_NULL;
+  if (state_in && (!state_in->W || (temporal && (!state_in->r_prev || !state_in->rho_prev)))) return SWILA_ERR_NULL;
+  if (state_out && (!state_out->W || (temporal && (!state_out->r_prev || !state_out->rho_prev)))) return SWILA_ERR_NULL;
+  if (!aligned16(workspace)) return SWILA_ERR_ALIGN;
+  const HostPlan h = host_plan(s);
+  if (workspace_bytes < h.total) return SWILA_ERR_SIZE;
+  char *ws = (char *)workspace;
+  cudaStream_t cs = (cudaStream_t)stream;
+  cudaError_t e = cudaSuccess;
+  auto up = [&](size_t off, const void *src, size_t n) {
+    if (e == cudaSuccess && n) e = cudaMemcpyAsync(ws + off, src, n, cudaMemcpyHostToDevice, cs);
+  };
+  up(h.q, q, h.n_qk); up(h.k, k, h.n_qk); up(h.v, v, h.n_v);
+  up(h.beta, g->beta_logit, h.n_gate); up(h.pik, g->pik_logit, h.n_gate); up(h.piq, g->piq_logit, h.n_gate);
+  if (temporal) { up(h.gk, g->gk_logit, h.n_tg); up(h.gq, g->gq_logit, h.n_tg); }
+  if (gated) up(h.alpha, g->alpha, h.n_alpha);
+  swila_state_t dstate = {(float *)(ws + h.W), temporal ? (float *)(ws + h.r) : nullptr,
+                          temporal ? (float *)(ws + h.rho) : nullptr};
+  if (state_in) {
+    up(h.W, state_in->W, h.n_W);
+    if (temporal) { up(h.r, state_in->r_prev, h.n_r); up(h.rho, state_in->rho_prev, h.n_r); }
+  }
+  if (e != cudaSuccess) return cuda_fail(e);
+  swila_gates_t dg = {ws + h.beta, ws + h.pik, ws + h.piq, temporal ? ws + h.gk : nullptr,
+                      temporal ? ws + h.gq : nullptr, gated ? (const float *)(ws + h.alpha) : nullptr};
+  rc = swila_forward(s, ws + h.q, ws + h.k, ws + h.v, &dg, state_in ? &dstate : nullptr,
+                     state_out ? &dstate : nullptr, ws + h.o, nullptr, stream);
+  if (rc) return rc;
+  auto down = [&](void *dst, size_t off, size_t n) {
+    if (e == cudaSuccess && n) e = cudaMemcpyAsync(dst, ws + off, n, cudaMemcpyDeviceToHost, cs);
+  };
+  down(o, h.o, h.n_v);
+  if (state_out) {
+    down(state_out->W, h.W, h.n_W);
+    if (temporal) { down(state_out->r_prev, h.r, h.n_r); down(state_out->rho_prev, h.rho, h.n_r); }
+  }
+  return e == cudaSuccess ? SWILA_OK : cuda_fail(e);
 }
 
 }  // extern "C"

@@ -75,6 +75,23 @@ __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
+// Two FP32 FMAs / multiplies on a register pair.  SWILA_SCALAR_FMA selects plain scalar
+// instructions instead of the packed f32x2 forms.
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
+#ifdef SWILA_SCALAR_FMA
+  return make_float2(fmaf(a.x, b.x, c.x), fmaf(a.y, b.y, c.y));
+#else
+  return __ffma2_rn(a, b, c);
+#endif
+}
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) {
+#ifdef SWILA_SCALAR_FMA
+  return make_float2(a.x * b.x, a.y * b.y);
+#else
+  return __fmul2_rn(a, b);
+#endif
+}
+
 // J consecutive floats from shared memory with the widest aligned loads.
 template <int J>
 __device__ __forceinline__ void lds_vec(const float *p, float (&out)[J]) {

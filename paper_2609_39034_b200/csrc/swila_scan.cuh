@@ -28,14 +28,18 @@
 
 namespace swila {
 
-template <typename IO, int J, int DK, int NT, int TB, int GATE>
+template <typename IO_, int J_, int DK_, int NT_, int TB_, int GATE_, int LCAP_ = 64>
 struct ScanCfg {
+  using IO = IO_;
+  static constexpr int J = J_, DK = DK_, NT = NT_, TB = TB_, GATE = GATE_;
   static constexpr int L0 = (J * DK >= 128) ? (128 / J) : DK;
-  static constexpr int L = L0 > 64 ? 64 : L0;                 // key dims per lane (J*L <= 128 state registers)
+  static constexpr int L = L0 > LCAP_ ? LCAP_ : L0;           // key dims per lane (J*L <= 128 state registers)
   static constexpr int G = DK / L;                            // lanes per output column
   static constexpr int COLS = NT / G;                         // output columns per block
   static constexpr int ES = (int)sizeof(IO);
   static constexpr int S = 3;                                 // raw ring depth
+  // resident blocks per SM the register budget is sized for
+  static constexpr int MIN_BLOCKS = (NT <= 128) ? ((J * L <= 64 && NT * 4 <= 512) ? 4 : 2) : 1;
   static_assert(L >= 4 && L % 4 == 0 && G >= 1 && G <= 32 && (G & (G - 1)) == 0, "lane split");
   static_assert((COLS * ES) % 16 == 0, "column slice must be a whole number of 16-byte chunks");
 
@@ -75,10 +79,12 @@ struct ScanCfg {
 };
 
 // ---- issue the cp.async copies of one token block into a raw stage ---------------------
-template <typename IO, int J, int DK, int NT, int TB, int GATE>
+template <class C>
 __device__ __forceinline__ void issue_block(const ScanParams &p, unsigned char *raw, size_t tok0, int t0,
                                             int col0, int tid) {
-  using C = ScanCfg<IO, J, DK, NT, TB, GATE>;
+  using IO = typename C::IO;
+  constexpr int J = C::J, DK = C::DK, NT = C::NT, TB = C::TB, GATE = C::GATE;
+  (void)J; (void)DK; (void)NT; (void)TB; (void)GATE;
   constexpr int ES = C::ES, COLS = C::COLS;
   const int nvalid = min(TB, p.T - t0);
   // chunks per token; both candidates are compile-time constants so the divisions below
@@ -140,10 +146,12 @@ __device__ __forceinline__ void issue_block(const ScanParams &p, unsigned char *
 }
 
 // ---- cook one raw block into fp32 operands ---------------------------------------------
-template <typename IO, int J, int DK, int NT, int TB, int GATE>
+template <class C>
 __device__ __forceinline__ void cook_block(const ScanParams &p, const unsigned char *raw, float *ck, size_t tok0,
                                            int t0, int col0, int tid) {
-  using C = ScanCfg<IO, J, DK, NT, TB, GATE>;
+  using IO = typename C::IO;
+  constexpr int J = C::J, DK = C::DK, NT = C::NT, TB = C::TB, GATE = C::GATE;
+  (void)J; (void)DK; (void)NT; (void)TB; (void)GATE;
   constexpr int COLS = C::COLS;
   const int nvalid = min(TB, p.T - t0);
   // k, q: straight conversion
@@ -220,10 +228,12 @@ __device__ __forceinline__ void cook_block(const ScanParams &p, const unsigned c
 }
 
 // ---- write a finished block of outputs ---------------------------------------------------
-template <typename IO, int J, int DK, int NT, int TB, int GATE>
+template <class C>
 __device__ __forceinline__ void flush_o(const ScanParams &p, const unsigned char *ob, size_t tok0, int t0, int col0,
                                         int tid) {
-  using C = ScanCfg<IO, J, DK, NT, TB, GATE>;
+  using IO = typename C::IO;
+  constexpr int J = C::J, DK = C::DK, NT = C::NT, TB = C::TB, GATE = C::GATE;
+  (void)J; (void)DK; (void)NT; (void)TB; (void)GATE;
   const int nvalid = min(TB, p.T - t0);
   for (int c = tid; c < nvalid * C::C_V; c += NT) {
     const int s = c / C::C_V, cc = c - s * C::C_V;
@@ -236,9 +246,11 @@ __device__ __forceinline__ void flush_o(const ScanParams &p, const unsigned char
 }
 
 // ---- the kernel ---------------------------------------------------------------------------
-template <typename IO, int J, int DK, int NT, int TB, int GATE, bool POST>
-__global__ void __launch_bounds__(NT, (NT <= 128 ? 2 : 1)) swila_scan_kernel(const __grid_constant__ ScanParams p) {
-  using C = ScanCfg<IO, J, DK, NT, TB, GATE>;
+template <class C, bool POST>
+__global__ void __launch_bounds__(C::NT, C::MIN_BLOCKS) swila_scan_kernel(const __grid_constant__ ScanParams p) {
+  using IO = typename C::IO;
+  constexpr int J = C::J, DK = C::DK, NT = C::NT, TB = C::TB, GATE = C::GATE;
+  (void)J; (void)DK; (void)NT; (void)TB; (void)GATE;
   constexpr int L = C::L, G = C::G, COLS = C::COLS, S = C::S;
   extern __shared__ __align__(16) unsigned char smem[];
   float *cooked = reinterpret_cast<float *>(smem + C::OFF_COOKED);
@@ -278,23 +290,23 @@ __global__ void __launch_bounds__(NT, (NT <= 128 ? 2 : 1)) swila_scan_kernel(con
   // prologue: fill the ring, cook block 0
 #pragma unroll
   for (int b = 0; b < S - 1; ++b) {
-    if (b < nblocks) issue_block<IO, J, DK, NT, TB, GATE>(p, smem + b * C::RAW_BYTES, tok0, b * TB, col0, tid);
+    if (b < nblocks) issue_block<C>(p, smem + b * C::RAW_BYTES, tok0, b * TB, col0, tid);
     cp_async_commit();
   }
   cp_async_wait<S - 2>();
   __syncthreads();
-  if (nblocks > 0) cook_block<IO, J, DK, NT, TB, GATE>(p, smem, cooked, tok0, 0, col0, tid);
+  if (nblocks > 0) cook_block<C>(p, smem, cooked, tok0, 0, col0, tid);
 
   for (int nb = 0; nb < nblocks; ++nb) {
     const int t0 = nb * TB;
     cp_async_wait<S - 3>();  // block nb+1 has landed (this thread's copies)
     __syncthreads();         // ... everyone's; cooked[nb&1] visible; block nb-1 fully consumed
     if (nb + S - 1 < nblocks)
-      issue_block<IO, J, DK, NT, TB, GATE>(p, smem + ((nb + S - 1) % S) * C::RAW_BYTES, tok0, (nb + S - 1) * TB, col0, tid);
+      issue_block<C>(p, smem + ((nb + S - 1) % S) * C::RAW_BYTES, tok0, (nb + S - 1) * TB, col0, tid);
     cp_async_commit();
-    if (nb > 0) flush_o<IO, J, DK, NT, TB, GATE>(p, obuf + ((nb - 1) & 1) * C::O_BYTES, tok0, t0 - TB, col0, tid);
+    if (nb > 0) flush_o<C>(p, obuf + ((nb - 1) & 1) * C::O_BYTES, tok0, t0 - TB, col0, tid);
     if (nb + 1 < nblocks)
-      cook_block<IO, J, DK, NT, TB, GATE>(p, smem + ((nb + 1) % S) * C::RAW_BYTES, cooked + ((nb + 1) & 1) * C::COOKED_FLOATS,
+      cook_block<C>(p, smem + ((nb + 1) % S) * C::RAW_BYTES, cooked + ((nb + 1) & 1) * C::COOKED_FLOATS,
                                           tok0, t0 + TB, col0, tid);
 
     const float *ck = cooked + (nb & 1) * C::COOKED_FLOATS;
@@ -313,9 +325,9 @@ __global__ void __launch_bounds__(NT, (NT <= 128 ? 2 : 1)) swila_scan_kernel(con
       if constexpr (GATE == 2) lds_vec<J>(ck + C::K_AR + (s * COLS + lcol) * J, arow);
 
       // ---- pass A: predictions w_jd . k_t (on the decayed state when pre-decay, Eq. 3.8) ----
-      float2 acc0[J], acc1[J];
+      float2 acc[J];
 #pragma unroll
-      for (int j = 0; j < J; ++j) acc0[j] = acc1[j] = make_float2(0.f, 0.f);
+      for (int j = 0; j < J; ++j) acc[j] = make_float2(0.f, 0.f);
 #pragma unroll
       for (int i = 0; i < L / 4; ++i) {
         const float4 k4 = *reinterpret_cast<const float4 *>(kt + (i * G + g) * 4);
@@ -324,22 +336,22 @@ __global__ void __launch_bounds__(NT, (NT <= 128 ? 2 : 1)) swila_scan_kernel(con
         for (int j = 0; j < J; ++j) {
           if constexpr (GATE == 1 && !POST) {
             const float4 a4 = *reinterpret_cast<const float4 *>(araw + (s * J + j) * DK + (i * G + g) * 4);
-            w[j][2 * i] = __fmul2_rn(w[j][2 * i], make_float2(a4.x, a4.y));
-            w[j][2 * i + 1] = __fmul2_rn(w[j][2 * i + 1], make_float2(a4.z, a4.w));
+            w[j][2 * i] = mul2(w[j][2 * i], make_float2(a4.x, a4.y));
+            w[j][2 * i + 1] = mul2(w[j][2 * i + 1], make_float2(a4.z, a4.w));
           }
           if constexpr (GATE == 2 && !POST) {
             const float2 a2 = make_float2(arow[j], arow[j]);
-            w[j][2 * i] = __fmul2_rn(w[j][2 * i], a2);
-            w[j][2 * i + 1] = __fmul2_rn(w[j][2 * i + 1], a2);
+            w[j][2 * i] = mul2(w[j][2 * i], a2);
+            w[j][2 * i + 1] = mul2(w[j][2 * i + 1], a2);
           }
-          acc0[j] = __ffma2_rn(w[j][2 * i], klo, acc0[j]);
-          acc1[j] = __ffma2_rn(w[j][2 * i + 1], khi, acc1[j]);
+          acc[j] = fma2(w[j][2 * i], klo, acc[j]);
+          acc[j] = fma2(w[j][2 * i + 1], khi, acc[j]);
         }
       }
       float delta[J];
 #pragma unroll
       for (int j = 0; j < J; ++j) {
-        float pk = (acc0[j].x + acc0[j].y) + (acc1[j].x + acc1[j].y);
+        float pk = acc[j].x + acc[j].y;
 #pragma unroll
         for (int off = 1; off < G; off <<= 1) pk += __shfl_xor_sync(0xffffffffu, pk, off);
         delta[j] = v - pk;
@@ -388,7 +400,7 @@ __global__ void __launch_bounds__(NT, (NT <= 128 ? 2 : 1)) swila_scan_kernel(con
 
       // ---- pass B: M-step (Eq. 3.3 / 3.7) and readout on the updated state (Eq. 3.5) ----
 #pragma unroll
-      for (int j = 0; j < J; ++j) acc0[j] = acc1[j] = make_float2(0.f, 0.f);
+      for (int j = 0; j < J; ++j) acc[j] = make_float2(0.f, 0.f);
 #pragma unroll
       for (int i = 0; i < L / 4; ++i) {
         const float4 k4 = *reinterpret_cast<const float4 *>(kt + (i * G + g) * 4);
@@ -399,30 +411,30 @@ __global__ void __launch_bounds__(NT, (NT <= 128 ? 2 : 1)) swila_scan_kernel(con
         for (int j = 0; j < J; ++j) {
           if constexpr (GATE == 1 && POST) {
             const float4 a4 = *reinterpret_cast<const float4 *>(araw + (s * J + j) * DK + (i * G + g) * 4);
-            w[j][2 * i] = __fmul2_rn(w[j][2 * i], make_float2(a4.x, a4.y));
-            w[j][2 * i + 1] = __fmul2_rn(w[j][2 * i + 1], make_float2(a4.z, a4.w));
+            w[j][2 * i] = mul2(w[j][2 * i], make_float2(a4.x, a4.y));
+            w[j][2 * i + 1] = mul2(w[j][2 * i + 1], make_float2(a4.z, a4.w));
           }
           if constexpr (GATE == 2 && POST) {
             const float2 a2 = make_float2(arow[j], arow[j]);
-            w[j][2 * i] = __fmul2_rn(w[j][2 * i], a2);
-            w[j][2 * i + 1] = __fmul2_rn(w[j][2 * i + 1], a2);
+            w[j][2 * i] = mul2(w[j][2 * i], a2);
+            w[j][2 * i + 1] = mul2(w[j][2 * i + 1], a2);
           }
-          w[j][2 * i] = __ffma2_rn(c2[j], klo, w[j][2 * i]);
-          w[j][2 * i + 1] = __ffma2_rn(c2[j], khi, w[j][2 * i + 1]);
-          acc0[j] = __ffma2_rn(w[j][2 * i], qlo, acc0[j]);
-          acc1[j] = __ffma2_rn(w[j][2 * i + 1], qhi, acc1[j]);
+          w[j][2 * i] = fma2(c2[j], klo, w[j][2 * i]);
+          w[j][2 * i + 1] = fma2(c2[j], khi, w[j][2 * i + 1]);
+          acc[j] = fma2(w[j][2 * i], qlo, acc[j]);
+          acc[j] = fma2(w[j][2 * i + 1], qhi, acc[j]);
         }
       }
       float o = 0.f;
 #pragma unroll
-      for (int j = 0; j < J; ++j) o = fmaf(pq[j], (acc0[j].x + acc0[j].y) + (acc1[j].x + acc1[j].y), o);
+      for (int j = 0; j < J; ++j) o = fmaf(pq[j], acc[j].x + acc[j].y, o);
 #pragma unroll
       for (int off = 1; off < G; off <<= 1) o += __shfl_xor_sync(0xffffffffu, o, off);
       if (g == 0) from_f32(ob[s * COLS + lcol], o);
     }
   }
   __syncthreads();
-  if (nblocks > 0) flush_o<IO, J, DK, NT, TB, GATE>(p, obuf + ((nblocks - 1) & 1) * C::O_BYTES, tok0, (nblocks - 1) * TB, col0, tid);
+  if (nblocks > 0) flush_o<C>(p, obuf + ((nblocks - 1) & 1) * C::O_BYTES, tok0, (nblocks - 1) * TB, col0, tid);
 
   // ---- registers -> state slice ----
   if (p.W_out && col_ok) {
@@ -445,10 +457,12 @@ __global__ void __launch_bounds__(NT, (NT <= 128 ? 2 : 1)) swila_scan_kernel(con
 }
 
 // ---- host-side launch of one instantiation -----------------------------------------------
-template <typename IO, int J, int DK, int NT, int TB, int GATE, bool POST>
+template <class C, bool POST>
 int launch_scan(const LaunchArgs &a) {
-  using C = ScanCfg<IO, J, DK, NT, TB, GATE>;
-  auto kern = swila_scan_kernel<IO, J, DK, NT, TB, GATE, POST>;
+  using IO = typename C::IO;
+  constexpr int J = C::J, DK = C::DK, NT = C::NT, TB = C::TB, GATE = C::GATE;
+  (void)J; (void)DK; (void)NT; (void)TB; (void)GATE;
+  auto kern = swila_scan_kernel<C, POST>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
   if (e != cudaSuccess) return (int)e;
   const long long nslice = (a.p.Dv + C::COLS - 1) / C::COLS;

@@ -18,13 +18,17 @@ int pick(const LaunchArgs &a) {
   // tokens per staged block: fp32 rows are twice as wide, keep two blocks per SM resident
   constexpr int TB = sizeof(IO) == 2 ? 8 : 4;
   if constexpr (DK == 16) {
-    return launch_scan<IO, J, DK, 32, TB, GATE, POST>(a);
+    return launch_scan<ScanCfg<IO, J, DK, 32, TB, GATE>, POST>(a);
   } else {
     if (a.algo == SWILA_ALGO_SCAN_WIDE) {
-      if constexpr (GATE == 0 && DK == 128) return launch_scan<IO, J, DK, 256, TB, GATE, POST>(a);
+      if constexpr (GATE == 0 && DK == 128) return launch_scan<ScanCfg<IO, J, DK, 256, TB, GATE>, POST>(a);
       return -1000;
     }
-    return launch_scan<IO, J, DK, 128, TB, GATE, POST>(a);
+    if (a.algo == SWILA_ALGO_SCAN_NARROW) {
+      if constexpr (GATE == 0 && DK == 128 && J >= 4) return launch_scan<ScanCfg<IO, J, DK, 128, TB, GATE, 16>, POST>(a);
+      return -1000;
+    }
+    return launch_scan<ScanCfg<IO, J, DK, 128, TB, GATE>, POST>(a);
   }
 }
 template <typename IO>
