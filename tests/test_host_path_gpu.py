@@ -1,0 +1,50 @@
+"""GPU: the host-buffer entry point (pinned host tensors staged through a caller-owned device
+workspace) gives exactly the device-pointer entry point's results, and matches the oracle."""
+import pytest
+import torch
+
+from paper_2609_39034_b200 import workloads as wl
+from tests._gpu_util import assert_close, gpu_forward, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def binding():
+    assert torch.cuda.is_available()
+    from paper_2609_39034_b200 import binding as b
+
+    return b
+
+
+def _pin(inp):
+    return {n: (x.pin_memory() if x is not None else None) for n, x in inp.items()}
+
+
+@pytest.mark.parametrize("var", [dict(), dict(temporal=True, gated=True)], ids=["vanilla", "gated_temporal"])
+def test_host_entry_equals_device_entry(binding, oracle, var):
+    w = wl.CONFIGS[1].with_(B=2, H=3, T=75).variant(**var)
+    inp = wl.make_inputs(w, stress=True)
+    ref = oracle.forward_inputs(inp, flags=w.flags, gran=w.gate_granularity)
+    dev = gpu_forward(binding, w, to_dev(inp))
+    host = _pin(inp)
+    ws = torch.empty(binding.host_workspace_bytes(w), device="cuda", dtype=torch.uint8)
+    sin = {"W": host["W0"], "r_prev": host["r0"], "rho_prev": host["rho0"]}
+    sout = {"W": torch.empty_like(inp["W0"]).pin_memory(),
+            "r_prev": torch.empty_like(inp["r0"]).pin_memory() if w.temporal else None,
+            "rho_prev": torch.empty_like(inp["rho0"]).pin_memory() if w.temporal else None}
+    o = binding.swila_forward_host(w, host, ws, state_in=sin, state_out=sout)
+    torch.cuda.synchronize()
+    assert torch.equal(o, dev["o"]) and torch.equal(sout["W"], dev["W"])
+    if w.temporal:
+        assert torch.equal(sout["r_prev"], dev["r_prev"]) and torch.equal(sout["rho_prev"], dev["rho_prev"])
+    assert_close(w, {"o": o, "W": sout["W"], "r_prev": sout["r_prev"], "rho_prev": sout["rho_prev"]}, ref, "host")
+
+
+def test_host_entry_rejects_a_small_workspace(binding):
+    w = wl.CONFIGS[0]
+    host = _pin(wl.make_inputs(w))
+    ws = torch.empty(binding.host_workspace_bytes(w) - 256, device="cuda", dtype=torch.uint8)
+    with pytest.raises(binding.SwilaError) as e:
+        binding.swila_forward_host(w, host, ws)
+    assert e.value.status == binding.ERR_SIZE
