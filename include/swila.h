@@ -160,6 +160,36 @@ int swila_forward_host(const swila_shape_t *shape, const void *q, const void *k,
                        void *stream);
 
 /*
+ * swila_forward_host for callers that cannot allocate device memory (this entry point has no
+ * counterpart in the paper; it computes exactly what swila_forward_host computes).
+ *
+ * Who needs it: code that is given host tensors and a stream but may not call cudaMalloc or
+ * any allocating library routine -- a plug-in inside a host application with a fixed memory
+ * budget, a callback running where allocation is forbidden.  Instead of a caller-supplied
+ * workspace the call stages its inputs, state and output in a fixed array of
+ * SWILA_STATIC_WORKSPACE_BYTES (16 MiB) that is part of the library image; every GPU that
+ * loads the library holds that array until the process exits.  The call itself allocates
+ * nothing and frees nothing.
+ *
+ *  - Size limit: the problem must satisfy swila_forward_host_workspace_bytes(shape) <=
+ *    swila_forward_host_static_capacity(); larger problems are rejected with SWILA_ERR_SIZE
+ *    before anything is enqueued.
+ *  - First call on a device: looks up the array's device address (once per device, with that
+ *    device current).  Make that first call outside any stream capture.
+ *  - Sharing: all calls on a device use the same array and it keeps the previous call's bytes.
+ *    That is harmless for sequential calls (each call overwrites what it reads), but two calls
+ *    whose GPU work overlaps -- different streams, or different host threads -- race on it.
+ *    Keep all calls to this entry point on one stream per device, or serialise them yourself.
+ *  - All pointer arguments are HOST pointers as in swila_forward_host; results are complete
+ *    once `stream` has been synchronised.
+ */
+#define SWILA_STATIC_WORKSPACE_BYTES (16u << 20)
+size_t swila_forward_host_static_capacity(void);
+int swila_forward_host_static(const swila_shape_t *shape, const void *q, const void *k, const void *v,
+                              const swila_gates_t *gates, const swila_state_t *state_in,
+                              swila_state_t *state_out, void *o, void *stream);
+
+/*
  * Measurement helper (no counterpart in the paper): launches an FP32 FMA-chain
  * microbenchmark whose rate is the denominator of the scan kernel's roofline (the
  * recurrence costs 3*J*Dk*Dv FP32 FMAs per token and head, Sec. 3.2).  Every thread of

@@ -23,7 +23,8 @@ ALGO_AUTO, ALGO_SCAN, ALGO_SCAN_WIDE, ALGO_SCAN_NARROW = 0, 1, 2, 3
 
 EXPORTS = ("swila_version", "swila_strerror", "swila_last_cuda_error", "swila_state_w_bytes",
            "swila_state_r_bytes", "swila_state_init", "swila_forward", "swila_decode_step",
-           "swila_bench_fma_chain", "swila_forward_host", "swila_forward_host_workspace_bytes")
+           "swila_bench_fma_chain", "swila_forward_host", "swila_forward_host_workspace_bytes",
+           "swila_forward_host_static", "swila_forward_host_static_capacity")
 
 
 class Shape(ctypes.Structure):
@@ -77,6 +78,11 @@ def _load() -> ctypes.CDLL:
     L.swila_forward_host.argtypes = [ctypes.POINTER(Shape), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                      ctypes.POINTER(Gates), ctypes.POINTER(State), ctypes.POINTER(State),
                                      ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+    L.swila_forward_host_static_capacity.restype = ctypes.c_size_t
+    L.swila_forward_host_static.restype = ctypes.c_int
+    L.swila_forward_host_static.argtypes = [ctypes.POINTER(Shape), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                            ctypes.POINTER(Gates), ctypes.POINTER(State), ctypes.POINTER(State),
+                                            ctypes.c_void_p, ctypes.c_void_p]
     L.swila_bench_fma_chain.restype = ctypes.c_int
     L.swila_bench_fma_chain.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
                                         ctypes.POINTER(ctypes.c_double), ctypes.c_void_p]
@@ -192,4 +198,24 @@ def swila_forward_host(w: Workload, inp: dict, workspace: torch.Tensor, *, state
                                  ctypes.byref(g), ctypes.byref(sin) if sin else None,
                                  ctypes.byref(sout) if sout else None, _p(o, True), _p(workspace),
                                  workspace.numel() * workspace.element_size(), _stream(stream)))
+    return o
+
+
+def swila_forward_host_static(w: Workload, inp: dict, *, state_in: Optional[dict] = None,
+                              state_out: Optional[dict] = None, o: Optional[torch.Tensor] = None,
+                              algo: int = ALGO_AUTO, stream=None) -> torch.Tensor:
+    """swila_forward_host without a caller workspace: the library stages through its own fixed
+    16 MiB device array, for callers that may not allocate device memory.  The output tensor
+    must be supplied (or is created here in pinned host memory, which is a host allocation).
+    Calls that overlap on the GPU race on the shared array; keep them on one stream."""
+    T = inp["q"].shape[2]
+    sh = make_shape(w, T=T, algo=algo)
+    if o is None:
+        o = torch.empty((w.B, w.H, T, w.Dv), dtype=w.torch_io_dtype).pin_memory()
+    g = _gates(inp, host=True)
+    sin = _state(state_in["W"], state_in.get("r_prev"), state_in.get("rho_prev")) if state_in else None
+    sout = _state(state_out["W"], state_out.get("r_prev"), state_out.get("rho_prev")) if state_out else None
+    check(lib.swila_forward_host_static(ctypes.byref(sh), _p(inp["q"], True), _p(inp["k"], True), _p(inp["v"], True),
+                                        ctypes.byref(g), ctypes.byref(sin) if sin else None,
+                                        ctypes.byref(sout) if sout else None, _p(o, True), _stream(stream)))
     return o
