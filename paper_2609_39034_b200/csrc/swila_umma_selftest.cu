@@ -1,0 +1,87 @@
+// Self-test of the tcgen05 plumbing used by the chunked kernel: D[128 x N] = A[128 x K] * B[N x K]^T
+// in TF32 with A placed in tensor memory by the threads, B in shared memory (K-major, no
+// swizzle), the result read back from tensor memory.  One block of 128 threads.
+#include "../../include/swila.h"
+#include "swila_umma.cuh"
+
+namespace {
+using namespace swila::umma;
+
+template <int N, int K>
+__global__ void __launch_bounds__(128) umma_selftest_kernel(const float *A, const float *B, float *D, int *status) {
+  __shared__ __align__(128) float sB[N * K];
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ uint32_t tmem_base_s;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  constexpr uint32_t TM_COLS = 256;  // A: K columns at 0, D: N columns at 128
+
+  if (warp == 0) tmem_alloc(&tmem_base_s, TM_COLS);
+  if (tid == 0) {
+    mbar_init(&bar, 1);
+    mbar_fence_init();
+  }
+  // B -> shared, chunk-major canonical layout: 16-byte unit (row n, k-chunk c) at (c*N + n)*16
+  for (int i = tid; i < N * (K / 4); i += 128) {
+    const int n = i % N, c = i / N;
+    const float4 v = *reinterpret_cast<const float4 *>(B + (size_t)n * K + c * 4);
+    *reinterpret_cast<float4 *>(sB + (size_t)(c * N + n) * 4) = v;
+  }
+  fence_async_smem();
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tbase = tmem_base_s;
+  const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+
+  // A row `tid` -> TMEM lane tid, columns 0..K-1
+#pragma unroll
+  for (int c = 0; c < K / 16; ++c) {
+    float v[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = A[(size_t)tid * K + c * 16 + i];
+    tmem_st16(tbase + lane_base + c * 16, v);
+  }
+  tmem_st_wait();
+  tc_fence_before_sync();
+  __syncthreads();
+
+  if (tid == 0) {
+    tc_fence_after_sync();
+    constexpr uint32_t idesc = idesc_tf32(128, N);
+#pragma unroll
+    for (int ks = 0; ks < K / 8; ++ks) {
+      const uint64_t bdesc = smem_desc_kmajor(smem_u32(sB) + ks * 2 * (N * 16), N * 16, 128);
+      mma_tf32_ts(tbase + 128, tbase + ks * 8, bdesc, idesc, ks > 0);
+    }
+    mma_commit(&bar);
+  }
+  const bool ok = mbar_wait(&bar, 0);
+  tc_fence_after_sync();
+  if (ok) {
+#pragma unroll
+    for (int c = 0; c < N / 16; ++c) {
+      float v[16];
+      tmem_ld16(tbase + lane_base + 128 + c * 16, v);
+      tmem_ld_wait();
+#pragma unroll
+      for (int i = 0; i < 16; ++i) D[(size_t)tid * N + c * 16 + i] = v[i];
+    }
+  } else if (tid == 0) {
+    *status = 1;  // the MMA never signalled completion
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tbase, TM_COLS);
+}
+}  // namespace
+
+extern "C" int swila_selftest_tf32_mma(const float *A, const float *B, float *D, int N, int K, int *status,
+                                       void *stream) {
+  if (!A || !B || !D || !status) return SWILA_ERR_NULL;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (N == 32 && K == 32) umma_selftest_kernel<32, 32><<<1, 128, 0, st>>>(A, B, D, status);
+  else if (N == 128 && K == 32) umma_selftest_kernel<128, 32><<<1, 128, 0, st>>>(A, B, D, status);
+  else if (N == 32 && K == 128) umma_selftest_kernel<32, 128><<<1, 128, 0, st>>>(A, B, D, status);
+  else return SWILA_ERR_UNSUPPORTED;
+  return cudaGetLastError() == cudaSuccess ? SWILA_OK : SWILA_ERR_CUDA;
+}
