@@ -69,8 +69,12 @@ enum {
   SWILA_ALGO_SCAN = 1,     /* sequential scan, state resident in registers, FP32 FMA pipe */
   SWILA_ALGO_SCAN_WIDE = 2, /* the same scan with 256-thread blocks (twice the columns per
                               block); ungated shapes with Dk = 128 only */
-  SWILA_ALGO_SCAN_NARROW = 3 /* the same scan with 16 key dimensions per lane (more, lighter
+  SWILA_ALGO_SCAN_NARROW = 3, /* the same scan with 16 key dimensions per lane (more, lighter
                               warps); ungated shapes with Dk = 128, J >= 4 only */
+  SWILA_ALGO_CHUNK = 4     /* chunked form: the state-times-token contractions of 32-token chunks
+                              on the tcgen05 tensor cores (TF32 hi/lo split, FP32 accumulation in
+                              tensor memory), the E-step and intra-chunk corrections on the FP32
+                              ALUs.  bf16 io, Dk in {64, 128}, no TEMPORAL / GATED */
 };
 
 typedef struct {
@@ -110,6 +114,11 @@ const char *swila_strerror(int status);
 
 /* Text of the most recent CUDA error seen by the calling thread ("" if none). */
 const char *swila_last_cuda_error(void);
+
+/* Device-side health of the current device: SWILA_OK, or SWILA_ERR_CUDA if a kernel of this
+ * library gave up on a bounded wait since the last call (the flag is cleared).  Synchronises
+ * the device; meant for tests and debugging, never needed on the normal path. */
+int swila_device_status(void);
 
 /* Bytes of state->W and of each of state->r_prev / state->rho_prev for `shape`
  * (0 if the shape is invalid). */

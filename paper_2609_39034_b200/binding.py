@@ -19,12 +19,12 @@ LIB_PATH = os.path.join(_HERE, "libswila.so")
 SWILA_OK = 0
 ERR_NULL, ERR_SHAPE, ERR_UNSUPPORTED, ERR_ALIGN, ERR_ALIAS, ERR_CUDA, ERR_SIZE = -1, -2, -3, -4, -5, -6, -7
 IO_FP32, IO_BF16 = 0, 1
-ALGO_AUTO, ALGO_SCAN, ALGO_SCAN_WIDE, ALGO_SCAN_NARROW = 0, 1, 2, 3
+ALGO_AUTO, ALGO_SCAN, ALGO_SCAN_WIDE, ALGO_SCAN_NARROW, ALGO_CHUNK = 0, 1, 2, 3, 4
 
 EXPORTS = ("swila_version", "swila_strerror", "swila_last_cuda_error", "swila_state_w_bytes",
            "swila_state_r_bytes", "swila_state_init", "swila_forward", "swila_decode_step",
            "swila_bench_fma_chain", "swila_forward_host", "swila_forward_host_workspace_bytes",
-           "swila_forward_host_static", "swila_forward_host_static_capacity", "swila_selftest_tf32_mma")
+           "swila_forward_host_static", "swila_forward_host_static_capacity", "swila_selftest_tf32_mma", "swila_device_status")
 
 
 class Shape(ctypes.Structure):
@@ -86,6 +86,7 @@ def _load() -> ctypes.CDLL:
     L.swila_selftest_tf32_mma.restype = ctypes.c_int
     L.swila_selftest_tf32_mma.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
                                           ctypes.c_void_p, ctypes.c_void_p]
+    L.swila_device_status.restype = ctypes.c_int
     L.swila_bench_fma_chain.restype = ctypes.c_int
     L.swila_bench_fma_chain.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
                                         ctypes.POINTER(ctypes.c_double), ctypes.c_void_p]
@@ -234,3 +235,8 @@ def selftest_tf32_mma(A: torch.Tensor, B: torch.Tensor) -> torch.Tensor:
     if int(status.item()) != 0:
         raise RuntimeError("tcgen05 self-test: the MMA did not signal completion")
     return D
+
+
+def device_status() -> None:
+    """Synchronise and raise if a kernel of the library recorded a device-side failure."""
+    check(lib.swila_device_status())

@@ -12,6 +12,9 @@ SWILA_DECL_DK(16)
 SWILA_DECL_DK(64)
 SWILA_DECL_DK(128)
 
+int chunk_dispatch(const LaunchArgs &a);
+int chunk_error_fetch(int *flag);
+
 static thread_local char g_cuda_err[256] = "";
 
 static int cuda_fail(cudaError_t e) {
@@ -36,7 +39,7 @@ static int check_shape(const swila_shape_t *s, bool need_T) {
   if (gated != (s->gate_granularity != SWILA_GATE_NONE)) return SWILA_ERR_UNSUPPORTED;
   if (s->gate_granularity < SWILA_GATE_NONE || s->gate_granularity > SWILA_GATE_SCALAR) return SWILA_ERR_UNSUPPORTED;
   if (s->algo != SWILA_ALGO_AUTO && s->algo != SWILA_ALGO_SCAN && s->algo != SWILA_ALGO_SCAN_WIDE &&
-      s->algo != SWILA_ALGO_SCAN_NARROW)
+      s->algo != SWILA_ALGO_SCAN_NARROW && s->algo != SWILA_ALGO_CHUNK)
     return SWILA_ERR_UNSUPPORTED;
   return SWILA_OK;
 }
@@ -101,6 +104,12 @@ static int run(const swila_shape_t *s, int T, const void *q, const void *k, cons
   a.stream = (cudaStream_t)stream;
 
   int rc = -1000;
+  if (s->algo == SWILA_ALGO_CHUNK) {
+    rc = chunk_dispatch(a);
+    if (rc == -1000) return SWILA_ERR_UNSUPPORTED;
+    if (rc != 0) return cuda_fail((cudaError_t)rc);
+    return SWILA_OK;
+  }
 #define SWILA_CASE(DK)                                                                          \
   case DK:                                                                                      \
     if (a.gate_mode == 0) rc = scan_dispatch<DK, 0, false>(a);                                  \
@@ -145,6 +154,17 @@ const char *swila_strerror(int status) {
 }
 
 const char *swila_last_cuda_error(void) { return g_cuda_err; }
+
+int swila_device_status(void) {
+  int flag = 0;
+  cudaError_t e = (cudaError_t)chunk_error_fetch(&flag);
+  if (e != cudaSuccess) return cuda_fail(e);
+  if (flag) {
+    strncpy(g_cuda_err, "a tensor-core completion wait expired inside the chunked kernel", sizeof(g_cuda_err) - 1);
+    return SWILA_ERR_CUDA;
+  }
+  return SWILA_OK;
+}
 
 size_t swila_state_w_bytes(const swila_shape_t *s) { return check_shape(s, false) == SWILA_OK ? w_elems(s) * 4 : 0; }
 size_t swila_state_r_bytes(const swila_shape_t *s) { return check_shape(s, false) == SWILA_OK ? r_elems(s) * 4 : 0; }

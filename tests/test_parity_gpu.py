@@ -82,6 +82,40 @@ def test_wide_blocks_match_oracle(binding, oracle, w):
     assert_close(w, got, ref, w.name)
 
 
+CHUNK_SHAPES = [w for w in SMALL if w.io_dtype == "bf16" and w.Dk in (64, 128)] + [
+    _case("c2_one_chunk", 2, B=1, H=1, T=32, recipe="gauss"),
+    _case("c2_short", 2, B=1, H=1, T=5, recipe="gauss"),
+    _case("c2_long", 2, B=1, H=2, T=1000, recipe="gauss"),
+]
+
+
+@pytest.mark.parametrize("w", CHUNK_SHAPES, ids=lambda w: w.name)
+@pytest.mark.parametrize("stress", [False, True], ids=["calm", "stress"])
+def test_chunked_tensor_core_kernel_matches_oracle(binding, oracle, w, stress):
+    """The chunked form (contractions on the tcgen05 tensor cores) computes the same recurrence."""
+    inp = wl.make_inputs(w, stress=stress)
+    ref = oracle.forward_inputs(inp, want_r=True)
+    got = gpu_forward(binding, w, to_dev(inp), want_r=True, algo=binding.ALGO_CHUNK)
+    binding.device_status()
+    assert_close(w, got, ref, w.name)
+
+
+def test_chunked_kernel_state_carry(binding, oracle):
+    """Chunked prefill -> scan decode steps -> chunked prefill on one carried state."""
+    w = SMALL[4].with_(T=90)
+    inp = wl.make_inputs(w, stress=True)
+    ref = oracle.forward_inputs(inp)
+    dev = to_dev(inp)
+    st = {"W": dev["W0"].clone(), "r_prev": None, "rho_prev": None}
+    outs = [binding.swila_forward(w, wl.slice_time(dev, 0, 40), state_in=st, state_out=st, algo=binding.ALGO_CHUNK)]
+    outs += [binding.swila_decode_step(w, wl.slice_time(dev, t, t + 1), st) for t in range(40, 45)]
+    outs.append(binding.swila_forward(w, wl.slice_time(dev, 45, 90), state_in=st, state_out=st, algo=binding.ALGO_CHUNK))
+    torch.cuda.synchronize()
+    binding.device_status()
+    got = {"o": torch.cat(outs, dim=2).cpu(), "W": st["W"].cpu()}
+    assert_close(w, got, ref, "carry")
+
+
 @pytest.mark.parametrize("w0", [SMALL[2], SMALL[4], SMALL[0]], ids=lambda w: w.name)
 @pytest.mark.parametrize("var", [dict(), dict(temporal=True, gated=True)], ids=["vanilla", "gated_temporal"])
 def test_prefill_then_decode_equals_prefill_bitwise(binding, w0, var):
