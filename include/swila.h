@@ -215,7 +215,7 @@ int swila_bench_fma_chain(int packed, int chains, int blocks, int iters, float *
  * D[128 x N] = A[128 x K] * B[N x K]^T with TF32 operands and FP32 accumulation on the tcgen05
  * path (A through tensor memory, B through shared memory).  A [128,K], B [N,K], D [128,N] are
  * DEVICE fp32 row-major; *status (DEVICE int, zeroed by the caller) is set non-zero if the MMA
- * never completed.  (N, K) in {(32,32), (128,32), (32,128)}.
+ * never completed.  (N, K) in {(32,32), (128,32), (32,128), (64,128)}.
  */
 int swila_selftest_tf32_mma(const float *A, const float *B, float *D, int N, int K, int *status, void *stream);
 

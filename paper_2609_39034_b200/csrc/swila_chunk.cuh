@@ -19,9 +19,16 @@
 // ~22 significant bits.  bf16 inputs k, q are exact in TF32.  The triangular part (the sums over
 // s inside the chunk) and the E-step stay on the FP32 ALUs, one thread per row.
 //
-// One block = 128 threads = 128 rows = COLS = 128/J output columns of one (batch, head); thread r
-// serves row (d = r / J, j = r % J), which is also its tensor-memory lane, so the J components
-// of a column sit in adjacent lanes of one warp and the E-step normalisation is a few shuffles.
+// One block owns 128 rows = COLS = 128/J output columns of one (batch, head) and is split into
+// three roles that run concurrently and meet on mbarriers:
+//   row warps 0-3    thread r serves row (d = r / J, j = r % J), which is also its tensor-memory
+//                    lane; the J components of a column sit in adjacent lanes, so the E-step
+//                    normalisation is a few shuffles.  They run the sequential part of a chunk.
+//   helper warps 4-7 stage the next chunk (cp.async), convert K and Q into the tensor cores'
+//                    shared-memory operand layout, move the Gram matrices from tensor memory to
+//                    shared memory, refresh the low part of W after each update, and write the
+//                    chunk's outputs -- all while the row warps are busy.
+//   warp 8, lane 0   issues every tcgen05.mma and commits them to the barriers.
 #pragma once
 
 #include "swila_common.cuh"
@@ -29,19 +36,20 @@
 
 namespace swila {
 
-// Set when a bounded wait on a tensor-core completion barrier expires (never expected).
+// Set when a bounded wait on a completion barrier expires (never expected).
 static __device__ int g_chunk_error = 0;
 
 template <int J_, int DK_>
 struct ChunkCfg {
   static constexpr int J = J_, DK = DK_;
-  static constexpr int C = 32;           // tokens per chunk
-  static constexpr int NT = 128;         // threads = rows
-  static constexpr int COLS = NT / J;    // output columns per block
-  static constexpr int ES = 2;           // bf16 io
+  static constexpr int C = 32;            // tokens per chunk
+  static constexpr int NROW = 128;        // row threads = rows of the tile
+  static constexpr int NT = 288;          // 4 row warps + 4 helper warps + 1 MMA warp
+  static constexpr int COLS = NROW / J;   // output columns per block
+  static constexpr int ES = 2;            // bf16 io
   // tensor-memory columns
-  static constexpr int TM_W = 0, TM_WLO = DK, TM_P0 = 2 * DK, TM_Q0 = TM_P0 + C, TM_GKK = TM_Q0 + C,
-                       TM_GKQ = TM_GKK + C, TM_CHI = TM_GKQ + C, TM_CLO = TM_CHI + C, TM_USED = TM_CLO + C;
+  static constexpr int TM_W = 0, TM_WLO = DK, TM_PQ = 2 * DK, TM_G = TM_PQ + 2 * C, TM_CHI = TM_G + 2 * C,
+                       TM_CLO = TM_CHI + C, TM_USED = TM_CLO + C;
   static constexpr int TM_ALLOC = 512;
   static_assert(TM_USED <= TM_ALLOC, "tensor memory budget");
   // raw stage (bytes): k, q [C][DK], v [C][COLS], beta/pik/piq [C][J][COLS], all bf16
@@ -52,144 +60,212 @@ struct ChunkCfg {
   static constexpr int R_PK = R_B + C * J * COLS * ES;
   static constexpr int R_PQ = R_PK + C * J * COLS * ES;
   static constexpr int RAW_BYTES = R_PQ + C * J * COLS * ES;
-  static constexpr int C_K = DK * ES / 16, C_V = COLS * ES / 16;
-  static constexpr int CH = 2 * C_K + C_V + 3 * J * C_V;  // 16-byte copies per token
+  static constexpr int C_K = DK * ES / 16, C_V = COLS * ES / 16;  // 16-byte units per token row / column slice
   // shared memory map (bytes)
   static constexpr int OFF_RAW = 0;
-  static constexpr int OFF_KB = OFF_RAW + 2 * RAW_BYTES;  // [DK/4][C][4] fp32: K, K-major, rows = tokens
-  static constexpr int OFF_QB = OFF_KB + C * DK * 4;      // same for Q
-  static constexpr int OFF_KT = OFF_QB + C * DK * 4;      // [C/4][DK][4] fp32: K transposed, rows = key dims
-  static constexpr int OFF_BS = OFF_KT + C * DK * 4;      // [C][NT] fp32 beta
-  static constexpr int OFF_LK = OFF_BS + C * NT * 4;      // [C][NT] fp32 base-2 key-prior logits
-  static constexpr int OFF_PQ = OFF_LK + C * NT * 4;      // [C][NT] fp32 query prior
-  static constexpr int OFF_PR = OFF_PQ + C * NT * 4;      // [C][NT] fp32 prior-weighted readouts
-  static constexpr int OFF_G = OFF_PR + C * NT * 4;       // Gkk [C][C], Gkq [C][C] fp32
-  static constexpr int OFF_MISC = OFF_G + 2 * C * C * 4;  // barriers, tensor-memory base
-  static constexpr int SMEM_BYTES = OFF_MISC + 64;
+  static constexpr int OFF_KQ = OFF_RAW + 2 * RAW_BYTES;   // [DK/4][2C][4] fp32: rows 0..C-1 = K, C..2C-1 = Q tokens
+  static constexpr int OFF_KT = OFF_KQ + 2 * C * DK * 4;   // [C/4][DK][4] fp32: K transposed (rows = key dims)
+  static constexpr int OFF_PR = OFF_KT + C * DK * 4;       // 2 x [C][NROW] fp32 prior-weighted readouts
+  static constexpr int OFF_G = OFF_PR + 2 * C * NROW * 4;  // 2 x { Gkk [C][C], Gkq [C][C] } fp32
+  static constexpr int OFF_BAR = OFF_G + 2 * 2 * C * C * 4;
+  static constexpr int SMEM_BYTES = OFF_BAR + 128;
   static_assert(RAW_BYTES % 16 == 0 && (COLS * ES) % 16 == 0, "alignment");
   static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 };
 
-template <class Cf>
-__device__ __forceinline__ void chunk_issue_raw(const ScanParams &p, unsigned char *raw, size_t tok0, int t0, int col0,
-                                                int tid) {
-  constexpr int J = Cf::J, DK = Cf::DK, C = Cf::C, COLS = Cf::COLS, ES = Cf::ES, CH = Cf::CH;
-  const int nvalid = min(C, p.T - t0);
-  for (int c = tid; c < C * CH; c += Cf::NT) {
-    const int s = c / CH;
-    int cc = c - s * CH;
-    const size_t tok = tok0 + (size_t)(t0 + s);
-    bool valid = s < nvalid;
-    const char *src;
-    unsigned char *dst;
-    if (cc < 2 * Cf::C_K) {
-      const bool isq = cc >= Cf::C_K;
-      if (isq) cc -= Cf::C_K;
-      src = (const char *)(isq ? p.q : p.k) + (tok * DK) * ES + cc * 16;
-      dst = raw + (isq ? Cf::R_Q : Cf::R_K) + s * DK * ES + cc * 16;
-    } else {
-      cc -= 2 * Cf::C_K;
-      if (cc < Cf::C_V) {
-        const int col = col0 + cc * (16 / ES);
-        valid = valid && col < p.Dv;
-        src = (const char *)p.v + (tok * p.Dv + col) * ES;
-        dst = raw + Cf::R_V + s * COLS * ES + cc * 16;
-      } else {
-        cc -= Cf::C_V;
-        const int which = cc / (J * Cf::C_V);
-        cc -= which * (J * Cf::C_V);
-        const int j = cc / Cf::C_V;
-        cc -= j * Cf::C_V;
-        const int col = col0 + cc * (16 / ES);
-        valid = valid && col < p.Dv;
-        const void *base = which == 0 ? p.beta_logit : (which == 1 ? p.pik_logit : p.piq_logit);
-        src = (const char *)base + ((tok * J + j) * (size_t)p.Dv + col) * ES;
-        dst = raw + (which == 0 ? Cf::R_B : (which == 1 ? Cf::R_PK : Cf::R_PQ)) + ((s * J + j) * COLS) * ES + cc * 16;
-      }
-    }
-    cp_async16(dst, valid ? (const void *)src : (const void *)p.k, valid ? 16 : 0);
-  }
-}
+// barrier slots
+enum { B_E = 0, B_G, B_U, B_KQ, B_KT, B_WLO, B_GS, B_C, B_COUNT };
 
 // hi/lo split of an FP32 value for TF32 operands: hi keeps the bits the tensor core reads
 // (it ignores the 13 low mantissa bits), lo is the exact remainder.
 __device__ __forceinline__ float tf32_hi(float x) { return __uint_as_float(__float_as_uint(x) & 0xffffe000u); }
 
+// cp.async staging of one chunk by the 128 helper threads (h = 0..127)
+template <class Cf>
+__device__ __forceinline__ void chunk_issue_raw(const ScanParams &p, unsigned char *raw, size_t tok0, int t0, int col0,
+                                                int h) {
+  constexpr int J = Cf::J, DK = Cf::DK, C = Cf::C, ES = Cf::ES, C_K = Cf::C_K, C_V = Cf::C_V;
+  const int nvalid = min(C, p.T - t0);
+  const size_t tokb = tok0 + (size_t)t0;
+  const char *kb = (const char *)p.k + tokb * DK * ES;
+  const char *qb = (const char *)p.q + tokb * DK * ES;
+#pragma unroll
+  for (int u = h; u < C * C_K; u += 128) {  // k and q rows of the chunk are contiguous in global memory
+    const bool valid = (u / C_K) < nvalid;
+    cp_async16(raw + Cf::R_K + u * 16, valid ? kb + u * 16 : (const char *)p.k, valid ? 16 : 0);
+    cp_async16(raw + Cf::R_Q + u * 16, valid ? qb + u * 16 : (const char *)p.k, valid ? 16 : 0);
+  }
+#pragma unroll
+  for (int u = h; u < C * C_V; u += 128) {
+    const int tok = u / C_V, cu = u % C_V;
+    const int col = col0 + cu * 8;
+    const bool valid = tok < nvalid && col < p.Dv;
+    cp_async16(raw + Cf::R_V + u * 16, valid ? (const char *)p.v + ((tokb + tok) * p.Dv + col) * ES : (const char *)p.k,
+               valid ? 16 : 0);
+  }
+#pragma unroll
+  for (int u = h; u < C * J * C_V; u += 128) {
+    const int cu = u % C_V, jj = (u / C_V) % J, tok = u / (C_V * J);
+    const int col = col0 + cu * 8;
+    const bool valid = tok < nvalid && col < p.Dv;
+    const size_t off = (((tokb + tok) * J + jj) * (size_t)p.Dv + col) * ES;
+    cp_async16(raw + Cf::R_B + u * 16, valid ? (const char *)p.beta_logit + off : (const char *)p.k, valid ? 16 : 0);
+    cp_async16(raw + Cf::R_PK + u * 16, valid ? (const char *)p.pik_logit + off : (const char *)p.k, valid ? 16 : 0);
+    cp_async16(raw + Cf::R_PQ + u * 16, valid ? (const char *)p.piq_logit + off : (const char *)p.k, valid ? 16 : 0);
+  }
+}
+
 template <class Cf>
 __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_constant__ ScanParams p) {
   using namespace umma;
-  constexpr int J = Cf::J, DK = Cf::DK, C = Cf::C, NT = Cf::NT, COLS = Cf::COLS;
+  constexpr int J = Cf::J, DK = Cf::DK, C = Cf::C, NROW = Cf::NROW, COLS = Cf::COLS;
   extern __shared__ __align__(128) unsigned char smem[];
-  float *Kb = reinterpret_cast<float *>(smem + Cf::OFF_KB);
-  float *Qb = reinterpret_cast<float *>(smem + Cf::OFF_QB);
+  float *KQ = reinterpret_cast<float *>(smem + Cf::OFF_KQ);
   float *Kt = reinterpret_cast<float *>(smem + Cf::OFF_KT);
-  float *bs = reinterpret_cast<float *>(smem + Cf::OFF_BS);
-  float *lks = reinterpret_cast<float *>(smem + Cf::OFF_LK);
-  float *pqs = reinterpret_cast<float *>(smem + Cf::OFF_PQ);
-  float *prs = reinterpret_cast<float *>(smem + Cf::OFF_PR);
-  float *Gkk = reinterpret_cast<float *>(smem + Cf::OFF_G);
-  float *Gkq = Gkk + C * C;
-  uint64_t *bar1 = reinterpret_cast<uint64_t *>(smem + Cf::OFF_MISC);
-  uint64_t *bar2 = bar1 + 1;
-  uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(bar2 + 1);
+  float *prs_all = reinterpret_cast<float *>(smem + Cf::OFF_PR);
+  float *G_all = reinterpret_cast<float *>(smem + Cf::OFF_G);
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + Cf::OFF_BAR);
+  uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(bars + B_COUNT);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int nslice = (p.Dv + COLS - 1) / COLS;
   const int bh = blockIdx.x / nslice;
   const int col0 = (blockIdx.x - bh * nslice) * COLS;
-  const int dl = tid / J, j = tid % J;
-  const int col = col0 + dl;
-  const bool col_ok = col < p.Dv;
   const size_t tok0 = (size_t)bh * p.T;
-  const int jbase = lane - j;  // first lane of this column's J-lane group
+  const int nchunks = (p.T + C - 1) / C;
 
-  if (warp == 0) tmem_alloc(tmem_base_s, Cf::TM_ALLOC);
+  if (warp == 8) tmem_alloc(tmem_base_s, Cf::TM_ALLOC);
   if (tid == 0) {
-    mbar_init(bar1, 1);
-    mbar_init(bar2, 1);
+    mbar_init(&bars[B_E], 1);
+    mbar_init(&bars[B_G], 1);
+    mbar_init(&bars[B_U], 1);
+    mbar_init(&bars[B_KQ], 128);
+    mbar_init(&bars[B_KT], 128);
+    mbar_init(&bars[B_WLO], 128);
+    mbar_init(&bars[B_GS], 32);
+    mbar_init(&bars[B_C], 128);
     mbar_fence_init();
   }
-  const int nchunks = (p.T + C - 1) / C;
-  chunk_issue_raw<Cf>(p, smem + Cf::OFF_RAW, tok0, 0, col0, tid);
-  cp_async_commit();
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
-  const uint32_t tb = *tmem_base_s + ((uint32_t)(warp * 32) << 16);  // this warp's lane quarter
   const uint32_t tb0 = *tmem_base_s;
-
-  // ---- initial state row -> tensor memory (W and its low part) ----
-  {
-    const float *src = (p.W_in && col_ok) ? p.W_in + (((size_t)bh * J + j) * p.Dv + col) * DK : nullptr;
-#pragma unroll
-    for (int cc = 0; cc < DK / 16; ++cc) {
-      float w[16], lo[16];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (src) t = __ldcs(reinterpret_cast<const float4 *>(src + cc * 16 + i * 4));
-        w[4 * i] = t.x; w[4 * i + 1] = t.y; w[4 * i + 2] = t.z; w[4 * i + 3] = t.w;
-      }
-#pragma unroll
-      for (int i = 0; i < 16; ++i) lo[i] = w[i] - tf32_hi(w[i]);
-      tmem_st16(tb + Cf::TM_W + cc * 16, w);
-      tmem_st16(tb + Cf::TM_WLO + cc * 16, lo);
-    }
-    tmem_st_wait();
-  }
-
+  const uint32_t tb = tb0 + ((uint32_t)((warp & 3) * 32) << 16);  // this warp's lane quarter
   bool failed = false;
-  for (int n = 0; n < nchunks && !failed; ++n) {
-    const int t0 = n * C;
-    const int nvalid = min(C, p.T - t0);
-    unsigned char *raw = smem + Cf::OFF_RAW + (n & 1) * Cf::RAW_BYTES;
-    cp_async_wait<0>();
-    __syncthreads();  // raw chunk n landed for everyone; previous chunk fully consumed
-    if (n + 1 < nchunks) chunk_issue_raw<Cf>(p, smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES, tok0, t0 + C, col0, tid);
-    cp_async_commit();
 
-    // ---- cook: K, Q -> fp32 K-major operand tiles (16-byte unit (row, k-chunk c) at (c*rows + row)*16) ----
-    {
+  if (warp < 4) {
+    // =============================== row warps ===============================================
+    const int r = tid;
+    const int dl = r / J, j = r % J;
+    const int col = col0 + dl;
+    const bool col_ok = col < p.Dv;
+    const int jbase = lane - j;
+    if (!mbar_wait(&bars[B_KQ], 0) || !mbar_wait(&bars[B_GS], 0)) failed = true;
+    for (int n = 0; n < nchunks && !failed; ++n) {
+      const int t0 = n * C;
+      const int nvalid = min(C, p.T - t0);
+      const unsigned char *raw = smem + Cf::OFF_RAW + (n & 1) * Cf::RAW_BYTES;
+      const __nv_bfloat16 *rv = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_V);
+      const __nv_bfloat16 *rb = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_B);
+      const __nv_bfloat16 *rpk = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_PK);
+      const __nv_bfloat16 *rpq = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_PQ);
+      const float *Gkk = G_all + (n & 1) * 2 * C * C;
+      const float *Gkq = Gkk + C * C;
+      float *prs = prs_all + (n & 1) * C * NROW;
+
+      if (!mbar_wait(&bars[B_E], n & 1)) { failed = true; break; }
+      tc_fence_after_sync();
+      float pred[C], qd[C], cs[16];
+#pragma unroll
+      for (int cc = 0; cc < C / 16; ++cc) {
+        float a[16], b[16];
+        tmem_ld16(tb + Cf::TM_PQ + cc * 16, a);
+        tmem_ld16(tb + Cf::TM_PQ + C + cc * 16, b);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 16; ++i) { pred[cc * 16 + i] = a[i]; qd[cc * 16 + i] = b[i]; }
+      }
+
+      // ---- sequential part of the chunk: E-step and triangular corrections, one row per thread ----
+#pragma unroll
+      for (int t = 0; t < C; ++t) {
+        const int gi = (t * J + j) * COLS + dl;
+        // gate activations of this row (App. B.2); independent of the state, off the serial chain
+        const float be = sigmoid_approx(__bfloat162float(rb[gi]));
+        const float lk = __bfloat162float(rpk[gi]) * kLog2e;
+        const float xq = __bfloat162float(rpq[gi]) * kLog2e;
+        float mq = xq;
+#pragma unroll
+        for (int off = 1; off < J; off <<= 1) mq = fmaxf(mq, __shfl_xor_sync(0xffffffffu, mq, off));
+        const float eq = ex2_approx(xq - mq);
+        float sq = eq;
+#pragma unroll
+        for (int off = 1; off < J; off <<= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
+        const float piq = eq * rcp_approx(sq);
+        const float v = __bfloat162float(rv[t * COLS + dl]);
+        // serial chain: prediction error -> responsibilities (Eq. 3.4) -> update coefficient (Eq. 3.3)
+        const float delta = v - pred[t];
+        const float a = fmaf(-kHalfLog2e * delta, delta, lk);
+        float all[J];
+#pragma unroll
+        for (int jj = 0; jj < J; ++jj) all[jj] = __shfl_sync(0xffffffffu, a, jbase + jj);
+        float m = all[0];
+#pragma unroll
+        for (int jj = 1; jj < J; ++jj) m = fmaxf(m, all[jj]);
+        float sum = 0.f;
+#pragma unroll
+        for (int jj = 0; jj < J; ++jj) sum += ex2_approx(all[jj] - m);
+        const float rr = ex2_approx(a - m) * rcp_approx(sum);
+        float c = be * rr * delta;
+        if (t >= nvalid) c = 0.f;  // padding tokens of the last chunk leave the state alone
+        cs[t & 15] = c;
+        if (p.r_debug != nullptr && col_ok && t < nvalid)
+          p.r_debug[((tok0 + (size_t)(t0 + t)) * J + j) * p.Dv + col] = rr;
+        // push this token's update into the later predictions / readouts of the chunk
+#pragma unroll
+        for (int u = t + 1; u < C; ++u) pred[u] = fmaf(c, Gkk[t * C + u], pred[u]);
+#pragma unroll
+        for (int u = t; u < C; ++u) qd[u] = fmaf(c, Gkq[t * C + u], qd[u]);
+        prs[t * NROW + r] = piq * qd[t];
+        if ((t & 15) == 15) {  // 16 update coefficients complete: park them in tensor memory (hi / lo)
+          float hi[16], lo[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) { hi[i] = tf32_hi(cs[i]); lo[i] = cs[i] - hi[i]; }
+          tmem_st16(tb + Cf::TM_CHI + (t - 15), hi);
+          tmem_st16(tb + Cf::TM_CLO + (t - 15), lo);
+        }
+      }
+      tmem_st_wait();
+      tc_fence_before_sync();
+      // the next chunk's operands must be in place before this chunk is handed over (keeps every
+      // barrier at most one phase ahead of its waiters)
+      if (n + 1 < nchunks && (!mbar_wait(&bars[B_KQ], (n + 1) & 1) || !mbar_wait(&bars[B_GS], (n + 1) & 1))) failed = true;
+      mbar_arrive(&bars[B_C]);
+    }
+    // ---- final state row -> global ----
+    if (!failed && !mbar_wait(&bars[B_U], (nchunks - 1) & 1)) failed = true;
+    if (!failed && p.W_out && col_ok) {
+      tc_fence_after_sync();
+      float *dst = p.W_out + (((size_t)bh * J + j) * p.Dv + col) * DK;
+#pragma unroll
+      for (int cc = 0; cc < DK / 16; ++cc) {
+        float w[16];
+        tmem_ld16(tb + Cf::TM_W + cc * 16, w);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          __stcs(reinterpret_cast<float4 *>(dst + cc * 16 + i * 4), make_float4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]));
+      }
+    }
+  } else if (warp < 8) {
+    // =============================== helper warps ============================================
+    const int h = tid - 128;
+    const int dl = h / J, j = h % J;
+    const int col = col0 + dl;
+    const bool col_ok = col < p.Dv;
+
+    // K, Q of a raw stage -> stacked fp32 operand tile (16-byte unit (row, k-chunk c) at (c*2C + row)*16)
+    auto cook_kq = [&](const unsigned char *raw) {
       const __nv_bfloat16 *rk = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_K);
       const __nv_bfloat16 *rq = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_Q);
       // diagonal walk over 8-token x 16-chunk blocks: conflict-free 8-byte reads and 16-byte writes
@@ -197,7 +273,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
 #pragma unroll 2
       for (int blk = 0; blk < NBLK; ++blk) {
         const int tb8 = blk % (C / 8), cb16 = blk / (C / 8);
-        const int s = tid >> 4, u = tid & 15;
+        const int s = h >> 4, u = h & 15;
         const int t = tb8 * 8 + ((u + s) & 7), c = cb16 * 16 + u;
         const uint2 kr = *reinterpret_cast<const uint2 *>(rk + t * DK + c * 4);
         const uint2 qr = *reinterpret_cast<const uint2 *>(rq + t * DK + c * 4);
@@ -206,11 +282,15 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         kf.z = __uint_as_float(kr.y << 16); kf.w = __uint_as_float(kr.y & 0xffff0000u);
         qf.x = __uint_as_float(qr.x << 16); qf.y = __uint_as_float(qr.x & 0xffff0000u);
         qf.z = __uint_as_float(qr.y << 16); qf.w = __uint_as_float(qr.y & 0xffff0000u);
-        *reinterpret_cast<float4 *>(Kb + (c * C + t) * 4) = kf;
-        *reinterpret_cast<float4 *>(Qb + (c * C + t) * 4) = qf;
+        *reinterpret_cast<float4 *>(KQ + (c * 2 * C + t) * 4) = kf;
+        *reinterpret_cast<float4 *>(KQ + (c * 2 * C + C + t) * 4) = qf;
       }
-      // K transposed: unit (row d', k-chunk c4) holds K[4 c4 .. 4 c4 + 3][d']
-      for (int e = tid; e < (C / 4) * DK; e += NT) {
+    };
+    // K of a raw stage, transposed: unit (row d', k-chunk c4) holds K[4 c4 .. 4 c4 + 3][d']
+    auto cook_kt = [&](const unsigned char *raw) {
+      const __nv_bfloat16 *rk = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_K);
+#pragma unroll 2
+      for (int e = h; e < (C / 4) * DK; e += 128) {
         const int dd = e % DK, c4 = e / DK;
         float4 f;
         f.x = __bfloat162float(rk[(4 * c4 + 0) * DK + dd]);
@@ -219,72 +299,16 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         f.w = __bfloat162float(rk[(4 * c4 + 3) * DK + dd]);
         *reinterpret_cast<float4 *>(Kt + (c4 * DK + dd) * 4) = f;
       }
-      // this row's gate activations for the chunk (App. B.2): beta = sigmoid, priors = softmax over j
-      const __nv_bfloat16 *rb = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_B);
-      const __nv_bfloat16 *rpk = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_PK);
-      const __nv_bfloat16 *rpq = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_PQ);
-#pragma unroll 4
-      for (int t = 0; t < C; ++t) {
-        const int gi = (t * J + j) * COLS + dl;
-        const float be = sigmoid_approx(__bfloat162float(rb[gi]));
-        const float lk = __bfloat162float(rpk[gi]) * kLog2e;
-        const float x = __bfloat162float(rpq[gi]) * kLog2e;
-        float m = x;
-#pragma unroll
-        for (int off = 1; off < J; off <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-        const float e = ex2_approx(x - m);
-        float sum = e;
-#pragma unroll
-        for (int off = 1; off < J; off <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
-        bs[t * NT + tid] = be;
-        lks[t * NT + tid] = lk;
-        pqs[t * NT + tid] = e * rcp_approx(sum);
-      }
-    }
-    fence_async_smem();
-    tc_fence_before_sync();
-    __syncthreads();
-
-    // ---- tensor cores: P0 = W K^T, Q0 = W Q^T (hi and lo parts of W), Gram matrices ----
-    if (tid == 0) {
-      tc_fence_after_sync();
-      constexpr uint32_t idC = idesc_tf32(128, C);
-      const uint64_t bk0 = smem_desc_kmajor(smem_u32(Kb), C * 16, 128);
-      const uint64_t bq0 = smem_desc_kmajor(smem_u32(Qb), C * 16, 128);
-#pragma unroll 1
-      for (int ks = 0; ks < DK / 8; ++ks) {
-        const uint64_t bk = bk0 + (uint64_t)(ks * 2 * C);  // start address advances in 16-byte units
-        const uint64_t bq = bq0 + (uint64_t)(ks * 2 * C);
-        mma_tf32_ts(tb0 + Cf::TM_P0, tb0 + Cf::TM_W + ks * 8, bk, idC, ks > 0);
-        mma_tf32_ts(tb0 + Cf::TM_Q0, tb0 + Cf::TM_W + ks * 8, bq, idC, ks > 0);
-        mma_tf32_ts(tb0 + Cf::TM_P0, tb0 + Cf::TM_WLO + ks * 8, bk, idC, true);
-        mma_tf32_ts(tb0 + Cf::TM_Q0, tb0 + Cf::TM_WLO + ks * 8, bq, idC, true);
-        mma_tf32_ss(tb0 + Cf::TM_GKK, bk, bk, idC, ks > 0);  // rows >= C of the A tile are don't-care
-        mma_tf32_ss(tb0 + Cf::TM_GKQ, bk, bq, idC, ks > 0);
-      }
-      mma_commit(bar1);
-    }
-    failed = !mbar_wait(bar1, n & 1);
-    failed = __syncthreads_or(failed);
-    if (failed) break;
-    tc_fence_after_sync();
-
-    float pred[C], qd[C], cs[16];
-#pragma unroll
-    for (int cc = 0; cc < C / 16; ++cc) {
-      float a[16], b[16];
-      tmem_ld16(tb + Cf::TM_P0 + cc * 16, a);
-      tmem_ld16(tb + Cf::TM_Q0 + cc * 16, b);
-      tmem_ld_wait();
-#pragma unroll
-      for (int i = 0; i < 16; ++i) { pred[cc * 16 + i] = a[i]; qd[cc * 16 + i] = b[i]; }
-    }
-    if (warp == 0) {  // lanes 0..C-1 hold the Gram rows: spill them to shared memory for everyone
+    };
+    // Gram rows (tensor-memory lanes 0..C-1, helper warp 4 only) -> shared memory
+    auto spill_gram = [&](int n) {
+      float *Gkk = G_all + (n & 1) * 2 * C * C;
+      float *Gkq = Gkk + C * C;
 #pragma unroll
       for (int cc = 0; cc < C / 16; ++cc) {
         float a[16], b[16];
-        tmem_ld16(tb + Cf::TM_GKK + cc * 16, a);
-        tmem_ld16(tb + Cf::TM_GKQ + cc * 16, b);
+        tmem_ld16(tb + Cf::TM_G + cc * 16, a);
+        tmem_ld16(tb + Cf::TM_G + C + cc * 16, b);
         tmem_ld_wait();
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -292,119 +316,172 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
           *reinterpret_cast<float4 *>(Gkq + lane * C + cc * 16 + i * 4) = make_float4(b[4 * i], b[4 * i + 1], b[4 * i + 2], b[4 * i + 3]);
         }
       }
-    }
-    tc_fence_before_sync();
-    __syncthreads();
+      tc_fence_before_sync();
+    };
 
-    // ---- sequential part of the chunk: E-step and the triangular corrections, one row per thread ----
-    const __nv_bfloat16 *rv = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_V);
-#pragma unroll
-    for (int t = 0; t < C; ++t) {
-      const float v = __bfloat162float(rv[t * COLS + dl]);
-      const float delta = v - pred[t];
-      const float a = fmaf(-kHalfLog2e * delta, delta, lks[t * NT + tid]);
-      float all[J];
-#pragma unroll
-      for (int jj = 0; jj < J; ++jj) all[jj] = __shfl_sync(0xffffffffu, a, jbase + jj);
-      float m = all[0];
-#pragma unroll
-      for (int jj = 1; jj < J; ++jj) m = fmaxf(m, all[jj]);
-      float sum = 0.f;
-#pragma unroll
-      for (int jj = 0; jj < J; ++jj) sum += ex2_approx(all[jj] - m);
-      const float r = ex2_approx(a - m) * rcp_approx(sum);
-      float c = bs[t * NT + tid] * r * delta;
-      if (t >= nvalid) c = 0.f;  // padding tokens of the last chunk leave the state alone
-      cs[t & 15] = c;
-      if (p.r_debug != nullptr && col_ok && t < nvalid)
-        p.r_debug[((tok0 + (size_t)(t0 + t)) * J + j) * p.Dv + col] = r;
-      // push this token's update into the later predictions / readouts of the chunk
-#pragma unroll
-      for (int u = t + 1; u < C; ++u) pred[u] = fmaf(c, Gkk[t * C + u], pred[u]);
-#pragma unroll
-      for (int u = t; u < C; ++u) qd[u] = fmaf(c, Gkq[t * C + u], qd[u]);
-      prs[t * NT + tid] = pqs[t * NT + tid] * qd[t];
-      if ((t & 15) == 15) {  // 16 update coefficients complete: park them in tensor memory (hi / lo)
-        float hi[16], lo[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) { hi[i] = tf32_hi(cs[i]); lo[i] = cs[i] - hi[i]; }
-        tmem_st16(tb + Cf::TM_CHI + (t - 15), hi);
-        tmem_st16(tb + Cf::TM_CLO + (t - 15), lo);
-      }
-    }
-
-    // ---- W += Cmat K on the tensor cores ----
-    tmem_st_wait();
-    tc_fence_before_sync();
-    __syncthreads();
-    if (tid == 0) {
-      tc_fence_after_sync();
-      constexpr uint32_t idD = idesc_tf32(128, DK);
-      const uint64_t bt0 = smem_desc_kmajor(smem_u32(Kt), DK * 16, 128);
-#pragma unroll 1
-      for (int ks = 0; ks < C / 8; ++ks) {
-        const uint64_t bt = bt0 + (uint64_t)(ks * 2 * DK);
-        mma_tf32_ts(tb0 + Cf::TM_W, tb0 + Cf::TM_CHI + ks * 8, bt, idD, true);
-        mma_tf32_ts(tb0 + Cf::TM_W, tb0 + Cf::TM_CLO + ks * 8, bt, idD, true);
-      }
-      mma_commit(bar2);
-    }
-
-    // ---- outputs of the chunk (overlaps the update MMAs): o_td = sum_j of the weighted readouts ----
+    // ---- prologue: stage chunks 0 and 1, state row -> tensor memory, operands of chunk 0 ----
+    chunk_issue_raw<Cf>(p, smem + Cf::OFF_RAW, tok0, 0, col0, h);
+    cp_async_commit();
+    if (nchunks > 1) chunk_issue_raw<Cf>(p, smem + Cf::OFF_RAW + Cf::RAW_BYTES, tok0, C, col0, h);
+    cp_async_commit();
     {
-      constexpr int GROUPS = COLS / 8;  // 8 outputs = 16 bytes per store
-      for (int e = tid; e < C * GROUPS; e += NT) {
-        const int t = e / GROUPS, g8 = e - t * GROUPS;
-        if (t < nvalid && col0 + g8 * 8 < p.Dv) {
-          __align__(16) __nv_bfloat16 out[8];
+      const float *src = (p.W_in && col_ok) ? p.W_in + (((size_t)bh * J + j) * p.Dv + col) * DK : nullptr;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            float o = 0.f;
+      for (int cc = 0; cc < DK / 16; ++cc) {
+        float w[16], lo[16];
 #pragma unroll
-            for (int jj = 0; jj < J; ++jj) o += prs[t * NT + (g8 * 8 + i) * J + jj];
-            out[i] = __float2bfloat16_rn(o);
-          }
-          *reinterpret_cast<uint4 *>((__nv_bfloat16 *)p.o + (tok0 + (size_t)(t0 + t)) * p.Dv + col0 + g8 * 8) =
-              *reinterpret_cast<const uint4 *>(out);
+        for (int i = 0; i < 4; ++i) {
+          float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (src) t = __ldcs(reinterpret_cast<const float4 *>(src + cc * 16 + i * 4));
+          w[4 * i] = t.x; w[4 * i + 1] = t.y; w[4 * i + 2] = t.z; w[4 * i + 3] = t.w;
+        }
+#pragma unroll
+        for (int i = 0; i < 16; ++i) lo[i] = w[i] - tf32_hi(w[i]);
+        tmem_st16(tb + Cf::TM_W + cc * 16, w);
+        tmem_st16(tb + Cf::TM_WLO + cc * 16, lo);
+      }
+      tmem_st_wait();
+      tc_fence_before_sync();
+      mbar_arrive(&bars[B_WLO]);
+    }
+    cp_async_wait<1>();
+    named_bar_sync(1, 128);  // every helper's copies of chunk 0 have landed
+    cook_kq(smem + Cf::OFF_RAW);
+    fence_async_smem();
+    mbar_arrive(&bars[B_KQ]);
+    cook_kt(smem + Cf::OFF_RAW);
+    fence_async_smem();
+    mbar_arrive(&bars[B_KT]);
+    if (warp == 4) {
+      if (!mbar_wait(&bars[B_G], 0)) failed = true;
+      tc_fence_after_sync();
+      if (!failed) spill_gram(0);
+      mbar_arrive(&bars[B_GS]);
+    }
+
+    for (int n = 0; n < nchunks && !failed; ++n) {
+      const bool more = n + 1 < nchunks;
+      const unsigned char *raw_next = smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES;
+      // (1) operands of chunk n+1: its raw stage has landed; the K/Q tile is free once E(n) is done
+      if (more) {
+        cp_async_wait<0>();
+        named_bar_sync(1, 128);
+        if (!mbar_wait(&bars[B_E], n & 1)) { failed = true; break; }
+        cook_kq(raw_next);
+        fence_async_smem();
+        mbar_arrive(&bars[B_KQ]);
+        if (warp == 4) {  // (2) Gram matrices of chunk n+1
+          if (!mbar_wait(&bars[B_G], (n + 1) & 1)) { failed = true; }
+          tc_fence_after_sync();
+          if (!failed) spill_gram(n + 1);
+          mbar_arrive(&bars[B_GS]);
         }
       }
+      // (3) chunk n is finished by the row warps: write its outputs, stage chunk n+2
+      if (!mbar_wait(&bars[B_C], n & 1)) { failed = true; break; }
+      {
+        const float *prs = prs_all + (n & 1) * C * NROW;
+        const int t0 = n * C;
+        const int nvalid = min(C, p.T - t0);
+        constexpr int GROUPS = COLS / 8;  // 8 outputs = 16 bytes per store
+        for (int e = h; e < C * GROUPS; e += 128) {
+          const int t = e / GROUPS, g8 = e - t * GROUPS;
+          if (t < nvalid && col0 + g8 * 8 < p.Dv) {
+            __align__(16) __nv_bfloat16 out[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              float o = 0.f;
+#pragma unroll
+              for (int jj = 0; jj < J; ++jj) o += prs[t * NROW + (g8 * 8 + i) * J + jj];
+              out[i] = __float2bfloat16_rn(o);
+            }
+            *reinterpret_cast<uint4 *>((__nv_bfloat16 *)p.o + (tok0 + (size_t)(t0 + t)) * p.Dv + col0 + g8 * 8) =
+                *reinterpret_cast<const uint4 *>(out);
+          }
+        }
+      }
+      if (n + 2 < nchunks) chunk_issue_raw<Cf>(p, smem + Cf::OFF_RAW + (n & 1) * Cf::RAW_BYTES, tok0, (n + 2) * C, col0, h);
+      cp_async_commit();
+      // (4) W has been updated with chunk n: refresh its low part, then the transposed K of chunk n+1
+      if (more) {
+        if (!mbar_wait(&bars[B_U], n & 1)) { failed = true; break; }
+        tc_fence_after_sync();
+#pragma unroll
+        for (int cc = 0; cc < DK / 16; ++cc) {
+          float w[16];
+          tmem_ld16(tb + Cf::TM_W + cc * 16, w);
+          tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) w[i] = w[i] - tf32_hi(w[i]);
+          tmem_st16(tb + Cf::TM_WLO + cc * 16, w);
+        }
+        tmem_st_wait();
+        tc_fence_before_sync();
+        mbar_arrive(&bars[B_WLO]);
+        cook_kt(raw_next);
+        fence_async_smem();
+        mbar_arrive(&bars[B_KT]);
+      }
     }
-
-    failed = !mbar_wait(bar2, n & 1);
-    failed = __syncthreads_or(failed);
-    if (failed) break;
+    cp_async_wait<0>();
+  } else if (lane == 0) {
+    // =============================== MMA issuer ==============================================
+    constexpr uint32_t idE = idesc_tf32(128, 2 * C);  // [P0 | Q0] and [Gkk | Gkq]: N = 2C
+    constexpr uint32_t idU = idesc_tf32(128, DK);
+    const uint64_t kq0 = smem_desc_kmajor(smem_u32(KQ), 2 * C * 16, 128);
+    const uint64_t kt0 = smem_desc_kmajor(smem_u32(Kt), DK * 16, 128);
+    auto gram = [&]() {
+#pragma unroll 1
+      for (int ks = 0; ks < DK / 8; ++ks) {
+        const uint64_t d = kq0 + (uint64_t)(ks * 2 * 2 * C);  // start address advances in 16-byte units
+        mma_tf32_ss(tb0 + Cf::TM_G, d, d, idE, ks > 0);        // rows >= C of the A tile are don't-care
+      }
+      mma_commit(&bars[B_G]);
+    };
+    auto w_times_kq = [&](int w_col, bool first) {
+#pragma unroll 1
+      for (int ks = 0; ks < DK / 8; ++ks)
+        mma_tf32_ts(tb0 + Cf::TM_PQ, tb0 + w_col + ks * 8, kq0 + (uint64_t)(ks * 2 * 2 * C), idE, !(first && ks == 0));
+    };
+    if (!mbar_wait(&bars[B_KQ], 0)) failed = true;
     tc_fence_after_sync();
-    // ---- refresh the low part of W ----
-#pragma unroll
-    for (int cc = 0; cc < DK / 16; ++cc) {
-      float w[16];
-      tmem_ld16(tb + Cf::TM_W + cc * 16, w);
-      tmem_ld_wait();
-#pragma unroll
-      for (int i = 0; i < 16; ++i) w[i] = w[i] - tf32_hi(w[i]);
-      tmem_st16(tb + Cf::TM_WLO + cc * 16, w);
+    if (!failed) gram();
+    if (!failed && !mbar_wait(&bars[B_WLO], 0)) failed = true;
+    tc_fence_after_sync();
+    if (!failed) {
+      w_times_kq(Cf::TM_W, true);
+      w_times_kq(Cf::TM_WLO, false);
+      mma_commit(&bars[B_E]);
     }
-    tmem_st_wait();
-  }
-  cp_async_wait<0>();
-  if (failed && tid == 0) atomicExch(&g_chunk_error, 1);
-
-  // ---- final state row -> global ----
-  if (!failed && p.W_out && col_ok) {
-    float *dst = p.W_out + (((size_t)bh * J + j) * p.Dv + col) * DK;
-#pragma unroll
-    for (int cc = 0; cc < DK / 16; ++cc) {
-      float w[16];
-      tmem_ld16(tb + Cf::TM_W + cc * 16, w);
-      tmem_ld_wait();
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-        __stcs(reinterpret_cast<float4 *>(dst + cc * 16 + i * 4), make_float4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]));
+    for (int n = 0; n < nchunks && !failed; ++n) {
+      const bool more = n + 1 < nchunks;
+      if (more) {
+        if (!mbar_wait(&bars[B_KQ], (n + 1) & 1)) { failed = true; break; }
+        tc_fence_after_sync();
+        gram();
+      }
+      if (!mbar_wait(&bars[B_C], n & 1) || !mbar_wait(&bars[B_KT], n & 1)) { failed = true; break; }
+      tc_fence_after_sync();
+#pragma unroll 1
+      for (int ks = 0; ks < C / 8; ++ks) {  // W += Cmat K (Eq. 3.3 summed over the chunk)
+        const uint64_t bt = kt0 + (uint64_t)(ks * 2 * DK);
+        mma_tf32_ts(tb0 + Cf::TM_W, tb0 + Cf::TM_CHI + ks * 8, bt, idU, true);
+        mma_tf32_ts(tb0 + Cf::TM_W, tb0 + Cf::TM_CLO + ks * 8, bt, idU, true);
+      }
+      mma_commit(&bars[B_U]);
+      if (more) {
+        w_times_kq(Cf::TM_W, true);  // executes after the update: MMAs of one thread run in order
+        if (!mbar_wait(&bars[B_WLO], (n + 1) & 1)) { failed = true; break; }
+        tc_fence_after_sync();
+        w_times_kq(Cf::TM_WLO, false);
+        mma_commit(&bars[B_E]);
+      }
     }
   }
+  if (failed) atomicExch(&g_chunk_error, 1);
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 0) tmem_dealloc(*tmem_base_s, Cf::TM_ALLOC);
+  if (warp == 8) tmem_dealloc(tb0, Cf::TM_ALLOC);
 }
 
 template <int J, int DK>

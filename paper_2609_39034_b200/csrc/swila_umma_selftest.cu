@@ -20,7 +20,7 @@ __global__ void __launch_bounds__(128) umma_selftest_kernel(const float *A, cons
     mbar_init(&bar, 1);
     mbar_fence_init();
   }
-  // B -> shared, chunk-major canonical layout: 16-byte unit (row n, k-chunk c) at (c*N + n)*16
+  // B [N][K] -> shared, K-major tile: 16-byte unit (row n, k-chunk c) at (c*N + n)*16
   for (int i = tid; i < N * (K / 4); i += 128) {
     const int n = i % N, c = i / N;
     const float4 v = *reinterpret_cast<const float4 *>(B + (size_t)n * K + c * 4);
@@ -82,6 +82,7 @@ extern "C" int swila_selftest_tf32_mma(const float *A, const float *B, float *D,
   if (N == 32 && K == 32) umma_selftest_kernel<32, 32><<<1, 128, 0, st>>>(A, B, D, status);
   else if (N == 128 && K == 32) umma_selftest_kernel<128, 32><<<1, 128, 0, st>>>(A, B, D, status);
   else if (N == 32 && K == 128) umma_selftest_kernel<32, 128><<<1, 128, 0, st>>>(A, B, D, status);
+  else if (N == 64 && K == 128) umma_selftest_kernel<64, 128><<<1, 128, 0, st>>>(A, B, D, status);
   else return SWILA_ERR_UNSUPPORTED;
   return cudaGetLastError() == cudaSuccess ? SWILA_OK : SWILA_ERR_CUDA;
 }

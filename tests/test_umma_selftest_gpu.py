@@ -12,7 +12,7 @@ def _tf32(x: torch.Tensor) -> torch.Tensor:
     return (x.view(torch.int32) & ~0x1FFF).view(torch.float32)
 
 
-@pytest.mark.parametrize("N,K", [(32, 32), (128, 32), (32, 128)])
+@pytest.mark.parametrize("N,K", [(32, 32), (128, 32), (32, 128), (64, 128)])
 def test_tf32_mma_matches_matmul(N, K):
     assert torch.cuda.is_available()
     from paper_2609_39034_b200 import binding
