@@ -38,6 +38,12 @@ namespace swila {
 
 // Set when a bounded wait on a completion barrier expires (never expected).
 static __device__ int g_chunk_error = 0;
+#ifdef SWILA_CHUNK_PROFILE
+static __device__ long long g_chunk_prof[8];
+#define PROF_ADD(i, who) do { if (tid == (who) && blockIdx.x == 0) { long long now_ = clock64(); g_chunk_prof[i] += now_ - prof_t; prof_t = now_; } } while (0)
+#else
+#define PROF_ADD(i, who) do {} while (0)
+#endif
 
 template <int J_, int DK_>
 struct ChunkCfg {
@@ -52,24 +58,28 @@ struct ChunkCfg {
                        TM_CLO = TM_CHI + C, TM_USED = TM_CLO + C;
   static constexpr int TM_ALLOC = 512;
   static_assert(TM_USED <= TM_ALLOC, "tensor memory budget");
-  // raw stage (bytes): k, q [C][DK], v [C][COLS], beta/pik/piq [C][J][COLS], all bf16
+  // raw stages (bytes), all bf16.  Main part: k, q [C][DK], v [C][COLS], beta/pik [C][J][COLS] (2-deep
+  // ring); the query-prior logits piq [C][J][COLS] live in their own 3-deep ring because the helper
+  // warps still need them for the outputs of chunk n while chunk n+2 is being fetched.
   static constexpr int R_K = 0;
   static constexpr int R_Q = R_K + C * DK * ES;
   static constexpr int R_V = R_Q + C * DK * ES;
   static constexpr int R_B = R_V + C * COLS * ES;
   static constexpr int R_PK = R_B + C * J * COLS * ES;
-  static constexpr int R_PQ = R_PK + C * J * COLS * ES;
-  static constexpr int RAW_BYTES = R_PQ + C * J * COLS * ES;
+  static constexpr int RAW_BYTES = R_PK + C * J * COLS * ES;
+  static constexpr int RPQ_BYTES = C * J * COLS * ES;
   static constexpr int C_K = DK * ES / 16, C_V = COLS * ES / 16;  // 16-byte units per token row / column slice
   // shared memory map (bytes)
   static constexpr int OFF_RAW = 0;
-  static constexpr int OFF_KQ = OFF_RAW + 2 * RAW_BYTES;   // [DK/4][2C][4] fp32: rows 0..C-1 = K, C..2C-1 = Q tokens
+  static constexpr int OFF_RPQ = OFF_RAW + 2 * RAW_BYTES;
+  static constexpr int OFF_KQ = OFF_RPQ + 3 * RPQ_BYTES;   // [DK/4][2C][4] fp32: rows 0..C-1 = K, C..2C-1 = Q tokens
   static constexpr int OFF_KT = OFF_KQ + 2 * C * DK * 4;   // [C/4][DK][4] fp32: K transposed (rows = key dims)
-  static constexpr int OFF_PR = OFF_KT + C * DK * 4;       // 2 x [C][NROW] fp32 prior-weighted readouts
-  static constexpr int OFF_G = OFF_PR + 2 * C * NROW * 4;  // 2 x { Gkk [C][C], Gkq [C][C] } fp32
-  static constexpr int OFF_BAR = OFF_G + 2 * 2 * C * C * 4;
+  static constexpr int OFF_BE = OFF_KT + C * DK * 4;       // 2 x [C][NROW] fp32 beta = sigmoid(logit)
+  static constexpr int OFF_G = OFF_BE + 2 * C * NROW * 4;  // 2 x { Gkk [C][C], Gkq [C][C] } fp32
+  static constexpr int OFF_OST = OFF_G + 2 * 2 * C * C * 4;  // [C][COLS] bf16 output staging
+  static constexpr int OFF_BAR = OFF_OST + C * COLS * ES;
   static constexpr int SMEM_BYTES = OFF_BAR + 128;
-  static_assert(RAW_BYTES % 16 == 0 && (COLS * ES) % 16 == 0, "alignment");
+  static_assert(RAW_BYTES % 16 == 0 && RPQ_BYTES % 16 == 0 && (COLS * ES) % 16 == 0, "alignment");
   static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 };
 
@@ -82,8 +92,8 @@ __device__ __forceinline__ float tf32_hi(float x) { return __uint_as_float(__flo
 
 // cp.async staging of one chunk by the 128 helper threads (h = 0..127)
 template <class Cf>
-__device__ __forceinline__ void chunk_issue_raw(const ScanParams &p, unsigned char *raw, size_t tok0, int t0, int col0,
-                                                int h) {
+__device__ __forceinline__ void chunk_issue_raw(const ScanParams &p, unsigned char *raw, unsigned char *rawpq,
+                                                size_t tok0, int t0, int col0, int h) {
   constexpr int J = Cf::J, DK = Cf::DK, C = Cf::C, ES = Cf::ES, C_K = Cf::C_K, C_V = Cf::C_V;
   const int nvalid = min(C, p.T - t0);
   const size_t tokb = tok0 + (size_t)t0;
@@ -111,7 +121,7 @@ __device__ __forceinline__ void chunk_issue_raw(const ScanParams &p, unsigned ch
     const size_t off = (((tokb + tok) * J + jj) * (size_t)p.Dv + col) * ES;
     cp_async16(raw + Cf::R_B + u * 16, valid ? (const char *)p.beta_logit + off : (const char *)p.k, valid ? 16 : 0);
     cp_async16(raw + Cf::R_PK + u * 16, valid ? (const char *)p.pik_logit + off : (const char *)p.k, valid ? 16 : 0);
-    cp_async16(raw + Cf::R_PQ + u * 16, valid ? (const char *)p.piq_logit + off : (const char *)p.k, valid ? 16 : 0);
+    cp_async16(rawpq + u * 16, valid ? (const char *)p.piq_logit + off : (const char *)p.k, valid ? 16 : 0);
   }
 }
 
@@ -122,8 +132,9 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   extern __shared__ __align__(128) unsigned char smem[];
   float *KQ = reinterpret_cast<float *>(smem + Cf::OFF_KQ);
   float *Kt = reinterpret_cast<float *>(smem + Cf::OFF_KT);
-  float *prs_all = reinterpret_cast<float *>(smem + Cf::OFF_PR);
+  float *be_all = reinterpret_cast<float *>(smem + Cf::OFF_BE);
   float *G_all = reinterpret_cast<float *>(smem + Cf::OFF_G);
+  __nv_bfloat16 *ostage = reinterpret_cast<__nv_bfloat16 *>(smem + Cf::OFF_OST);
   uint64_t *bars = reinterpret_cast<uint64_t *>(smem + Cf::OFF_BAR);
   uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(bars + B_COUNT);
 
@@ -152,6 +163,9 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   const uint32_t tb0 = *tmem_base_s;
   const uint32_t tb = tb0 + ((uint32_t)((warp & 3) * 32) << 16);  // this warp's lane quarter
   bool failed = false;
+#ifdef SWILA_CHUNK_PROFILE
+  long long prof_t = clock64();
+#endif
 
   if (warp < 4) {
     // =============================== row warps ===============================================
@@ -166,43 +180,32 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       const int nvalid = min(C, p.T - t0);
       const unsigned char *raw = smem + Cf::OFF_RAW + (n & 1) * Cf::RAW_BYTES;
       const __nv_bfloat16 *rv = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_V);
-      const __nv_bfloat16 *rb = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_B);
       const __nv_bfloat16 *rpk = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_PK);
-      const __nv_bfloat16 *rpq = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_PQ);
       const float *Gkk = G_all + (n & 1) * 2 * C * C;
-      const float *Gkq = Gkk + C * C;
-      float *prs = prs_all + (n & 1) * C * NROW;
+      const float *bes = be_all + (n & 1) * C * NROW;
 
+      PROF_ADD(0, 0);
       if (!mbar_wait(&bars[B_E], n & 1)) { failed = true; break; }
       tc_fence_after_sync();
-      float pred[C], qd[C], cs[16];
+      PROF_ADD(1, 0);
+      float pred[C], cs[16];
 #pragma unroll
       for (int cc = 0; cc < C / 16; ++cc) {
-        float a[16], b[16];
+        float a[16];
         tmem_ld16(tb + Cf::TM_PQ + cc * 16, a);
-        tmem_ld16(tb + Cf::TM_PQ + C + cc * 16, b);
         tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 16; ++i) { pred[cc * 16 + i] = a[i]; qd[cc * 16 + i] = b[i]; }
+        for (int i = 0; i < 16; ++i) pred[cc * 16 + i] = a[i];
       }
 
-      // ---- sequential part of the chunk: E-step and triangular corrections, one row per thread ----
+      PROF_ADD(2, 0);
+      // ---- sequential part of the chunk: E-step and the triangular key-side corrections ----
 #pragma unroll
       for (int t = 0; t < C; ++t) {
         const int gi = (t * J + j) * COLS + dl;
-        // gate activations of this row (App. B.2); independent of the state, off the serial chain
-        const float be = sigmoid_approx(__bfloat162float(rb[gi]));
         const float lk = __bfloat162float(rpk[gi]) * kLog2e;
-        const float xq = __bfloat162float(rpq[gi]) * kLog2e;
-        float mq = xq;
-#pragma unroll
-        for (int off = 1; off < J; off <<= 1) mq = fmaxf(mq, __shfl_xor_sync(0xffffffffu, mq, off));
-        const float eq = ex2_approx(xq - mq);
-        float sq = eq;
-#pragma unroll
-        for (int off = 1; off < J; off <<= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
-        const float piq = eq * rcp_approx(sq);
         const float v = __bfloat162float(rv[t * COLS + dl]);
+        const float be = bes[t * NROW + r];
         // serial chain: prediction error -> responsibilities (Eq. 3.4) -> update coefficient (Eq. 3.3)
         const float delta = v - pred[t];
         const float a = fmaf(-kHalfLog2e * delta, delta, lk);
@@ -221,12 +224,9 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         cs[t & 15] = c;
         if (p.r_debug != nullptr && col_ok && t < nvalid)
           p.r_debug[((tok0 + (size_t)(t0 + t)) * J + j) * p.Dv + col] = rr;
-        // push this token's update into the later predictions / readouts of the chunk
+        // push this token's update into the later predictions of the chunk
 #pragma unroll
         for (int u = t + 1; u < C; ++u) pred[u] = fmaf(c, Gkk[t * C + u], pred[u]);
-#pragma unroll
-        for (int u = t; u < C; ++u) qd[u] = fmaf(c, Gkq[t * C + u], qd[u]);
-        prs[t * NROW + r] = piq * qd[t];
         if ((t & 15) == 15) {  // 16 update coefficients complete: park them in tensor memory (hi / lo)
           float hi[16], lo[16];
 #pragma unroll
@@ -237,6 +237,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       }
       tmem_st_wait();
       tc_fence_before_sync();
+      PROF_ADD(3, 0);
       // the next chunk's operands must be in place before this chunk is handed over (keeps every
       // barrier at most one phase ahead of its waiters)
       if (n + 1 < nchunks && (!mbar_wait(&bars[B_KQ], (n + 1) & 1) || !mbar_wait(&bars[B_GS], (n + 1) & 1))) failed = true;
@@ -300,6 +301,30 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         *reinterpret_cast<float4 *>(Kt + (c4 * DK + dd) * 4) = f;
       }
     };
+    // beta = sigmoid(logit) of this helper's row for every token of a raw stage (App. B.2)
+    auto cook_be = [&](const unsigned char *raw, float *bes) {
+      const __nv_bfloat16 *rb = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_B);
+#pragma unroll 8
+      for (int t = 0; t < C; ++t) bes[t * NROW + h] = sigmoid_approx(__bfloat162float(rb[(t * J + j) * COLS + dl]));
+    };
+    // low part of W after an update: W_lo = W - hi(W), this helper's tensor-memory lane
+    auto refresh_wlo = [&]() {
+#pragma unroll
+      for (int half = 0; half < DK / 64; ++half) {
+        float w[4][16];
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) tmem_ld16(tb + Cf::TM_W + half * 64 + cc * 16, w[cc]);
+        tmem_ld_wait();
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) w[cc][i] = w[cc][i] - tf32_hi(w[cc][i]);
+          tmem_st16(tb + Cf::TM_WLO + half * 64 + cc * 16, w[cc]);
+        }
+      }
+      tmem_st_wait();
+      tc_fence_before_sync();
+    };
     // Gram rows (tensor-memory lanes 0..C-1, helper warp 4 only) -> shared memory
     auto spill_gram = [&](int n) {
       float *Gkk = G_all + (n & 1) * 2 * C * C;
@@ -320,9 +345,10 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     };
 
     // ---- prologue: stage chunks 0 and 1, state row -> tensor memory, operands of chunk 0 ----
-    chunk_issue_raw<Cf>(p, smem + Cf::OFF_RAW, tok0, 0, col0, h);
+    chunk_issue_raw<Cf>(p, smem + Cf::OFF_RAW, smem + Cf::OFF_RPQ, tok0, 0, col0, h);
     cp_async_commit();
-    if (nchunks > 1) chunk_issue_raw<Cf>(p, smem + Cf::OFF_RAW + Cf::RAW_BYTES, tok0, C, col0, h);
+    if (nchunks > 1)
+      chunk_issue_raw<Cf>(p, smem + Cf::OFF_RAW + Cf::RAW_BYTES, smem + Cf::OFF_RPQ + Cf::RPQ_BYTES, tok0, C, col0, h);
     cp_async_commit();
     {
       const float *src = (p.W_in && col_ok) ? p.W_in + (((size_t)bh * J + j) * p.Dv + col) * DK : nullptr;
@@ -347,6 +373,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     cp_async_wait<1>();
     named_bar_sync(1, 128);  // every helper's copies of chunk 0 have landed
     cook_kq(smem + Cf::OFF_RAW);
+    cook_be(smem + Cf::OFF_RAW, be_all);
     fence_async_smem();
     mbar_arrive(&bars[B_KQ]);
     cook_kt(smem + Cf::OFF_RAW);
@@ -362,66 +389,102 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     for (int n = 0; n < nchunks && !failed; ++n) {
       const bool more = n + 1 < nchunks;
       const unsigned char *raw_next = smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES;
-      // (1) operands of chunk n+1: its raw stage has landed; the K/Q tile is free once E(n) is done
+      // (1) E(n) is done: take this row's Q0 out of tensor memory; the K/Q tile is free again
+      if (!mbar_wait(&bars[B_E], n & 1)) { failed = true; break; }
+      tc_fence_after_sync();
+      float qd[C];
+#pragma unroll
+      for (int cc = 0; cc < C / 16; ++cc) {
+        float a[16];
+        tmem_ld16(tb + Cf::TM_PQ + C + cc * 16, a);
+        tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 16; ++i) qd[cc * 16 + i] = a[i];
+      }
+      tc_fence_before_sync();
+      // (2) operands of chunk n+1 (its raw stage has landed)
+      cp_async_wait<0>();
+      named_bar_sync(1, 128);
       if (more) {
-        cp_async_wait<0>();
-        named_bar_sync(1, 128);
-        if (!mbar_wait(&bars[B_E], n & 1)) { failed = true; break; }
         cook_kq(raw_next);
+        cook_be(raw_next, be_all + ((n + 1) & 1) * C * NROW);
         fence_async_smem();
         mbar_arrive(&bars[B_KQ]);
-        if (warp == 4) {  // (2) Gram matrices of chunk n+1
+        if (warp == 4) {  // Gram matrices of chunk n+1
           if (!mbar_wait(&bars[B_G], (n + 1) & 1)) { failed = true; }
           tc_fence_after_sync();
           if (!failed) spill_gram(n + 1);
           mbar_arrive(&bars[B_GS]);
         }
       }
-      // (3) chunk n is finished by the row warps: write its outputs, stage chunk n+2
+      PROF_ADD(4, 128);
+      // (3) chunk n is finished by the row warps: stage chunk n+2 into the buffers chunk n used
       if (!mbar_wait(&bars[B_C], n & 1)) { failed = true; break; }
-      {
-        const float *prs = prs_all + (n & 1) * C * NROW;
-        const int t0 = n * C;
-        const int nvalid = min(C, p.T - t0);
-        constexpr int GROUPS = COLS / 8;  // 8 outputs = 16 bytes per store
-        for (int e = h; e < C * GROUPS; e += 128) {
-          const int t = e / GROUPS, g8 = e - t * GROUPS;
-          if (t < nvalid && col0 + g8 * 8 < p.Dv) {
-            __align__(16) __nv_bfloat16 out[8];
+      PROF_ADD(5, 128);
+      tc_fence_after_sync();
+      float cq[C];  // this row's update coefficients c = hi + lo, before the row warps reuse the slots
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              float o = 0.f;
+      for (int cc = 0; cc < C / 16; ++cc) {
+        float a[16], b[16];
+        tmem_ld16(tb + Cf::TM_CHI + cc * 16, a);
+        tmem_ld16(tb + Cf::TM_CLO + cc * 16, b);
+        tmem_ld_wait();
 #pragma unroll
-              for (int jj = 0; jj < J; ++jj) o += prs[t * NROW + (g8 * 8 + i) * J + jj];
-              out[i] = __float2bfloat16_rn(o);
-            }
-            *reinterpret_cast<uint4 *>((__nv_bfloat16 *)p.o + (tok0 + (size_t)(t0 + t)) * p.Dv + col0 + g8 * 8) =
-                *reinterpret_cast<const uint4 *>(out);
-          }
-        }
+        for (int i = 0; i < 16; ++i) cq[cc * 16 + i] = a[i] + b[i];
       }
-      if (n + 2 < nchunks) chunk_issue_raw<Cf>(p, smem + Cf::OFF_RAW + (n & 1) * Cf::RAW_BYTES, tok0, (n + 2) * C, col0, h);
+      tc_fence_before_sync();
+      if (n + 2 < nchunks)
+        chunk_issue_raw<Cf>(p, smem + Cf::OFF_RAW + (n & 1) * Cf::RAW_BYTES, smem + Cf::OFF_RPQ + ((n + 2) % 3) * Cf::RPQ_BYTES,
+                            tok0, (n + 2) * C, col0, h);
       cp_async_commit();
       // (4) W has been updated with chunk n: refresh its low part, then the transposed K of chunk n+1
       if (more) {
         if (!mbar_wait(&bars[B_U], n & 1)) { failed = true; break; }
         tc_fence_after_sync();
-#pragma unroll
-        for (int cc = 0; cc < DK / 16; ++cc) {
-          float w[16];
-          tmem_ld16(tb + Cf::TM_W + cc * 16, w);
-          tmem_ld_wait();
-#pragma unroll
-          for (int i = 0; i < 16; ++i) w[i] = w[i] - tf32_hi(w[i]);
-          tmem_st16(tb + Cf::TM_WLO + cc * 16, w);
-        }
-        tmem_st_wait();
-        tc_fence_before_sync();
+        refresh_wlo();
         mbar_arrive(&bars[B_WLO]);
         cook_kt(raw_next);
         fence_async_smem();
         mbar_arrive(&bars[B_KT]);
       }
+      PROF_ADD(6, 128);
+      // (5) readouts of chunk n (Eq. 3.5): w_t.q_t = Q0 + sum_{s<=t} c_s (k_s.q_t), weighted by the query prior
+      {
+        const float *Gkq = G_all + (n & 1) * 2 * C * C + C * C;
+        const __nv_bfloat16 *rpq = reinterpret_cast<const __nv_bfloat16 *>(smem + Cf::OFF_RPQ + (n % 3) * Cf::RPQ_BYTES);
+        const int t0 = n * C;
+        const int nvalid = min(C, p.T - t0);
+#pragma unroll
+        for (int sidx = 0; sidx < C; ++sidx) {
+          const float c = cq[sidx];
+#pragma unroll
+          for (int u = sidx; u < C; ++u) qd[u] = fmaf(c, Gkq[sidx * C + u], qd[u]);
+        }
+#pragma unroll
+        for (int t = 0; t < C; ++t) {
+          const float x = __bfloat162float(rpq[(t * J + j) * COLS + dl]) * kLog2e;
+          float m = x;
+#pragma unroll
+          for (int off = 1; off < J; off <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+          const float e = ex2_approx(x - m);
+          float sum = e, o = e * qd[t];
+#pragma unroll
+          for (int off = 1; off < J; off <<= 1) {
+            sum += __shfl_xor_sync(0xffffffffu, sum, off);
+            o += __shfl_xor_sync(0xffffffffu, o, off);
+          }
+          if (j == 0) ostage[t * COLS + dl] = __float2bfloat16_rn(o * rcp_approx(sum));
+        }
+        named_bar_sync(2, 128);
+        constexpr int GROUPS = COLS / 8;  // 8 outputs = 16 bytes per store
+        for (int e = h; e < C * GROUPS; e += 128) {
+          const int t = e / GROUPS, g8 = e - t * GROUPS;
+          if (t < nvalid && col0 + g8 * 8 < p.Dv)
+            *reinterpret_cast<uint4 *>((__nv_bfloat16 *)p.o + (tok0 + (size_t)(t0 + t)) * p.Dv + col0 + g8 * 8) =
+                *reinterpret_cast<const uint4 *>(ostage + t * COLS + g8 * 8);
+        }
+      }
+      PROF_ADD(7, 128);
     }
     cp_async_wait<0>();
   } else if (lane == 0) {

@@ -29,3 +29,12 @@ int chunk_error_fetch(int *flag) {
 }
 
 }  // namespace swila
+
+#ifdef SWILA_CHUNK_PROFILE
+// Developer build only: per-phase cycle counters of block 0 (reset on read).
+extern "C" int swila_chunk_profile(long long *out8) {
+  long long z[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  if (cudaMemcpyFromSymbol(out8, swila::g_chunk_prof, sizeof(z)) != cudaSuccess) return -1;
+  return cudaMemcpyToSymbol(swila::g_chunk_prof, z, sizeof(z)) == cudaSuccess ? 0 : -1;
+}
+#endif
