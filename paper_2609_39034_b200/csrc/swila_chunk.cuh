@@ -54,7 +54,9 @@ struct ChunkCfg {
   static constexpr int COLS = NROW / J;   // output columns per block
   static constexpr int ES = 2;            // bf16 io
   // tensor-memory columns
-  static constexpr int TM_W = 0, TM_WLO = DK, TM_PQ = 2 * DK, TM_G = TM_PQ + 2 * C, TM_CHI = TM_G + 2 * C,
+  // ([P0 | Q0] is double-buffered: the row warps still read Q0 of chunk n while the tensor cores
+  // already write the products of chunk n+1)
+  static constexpr int TM_W = 0, TM_WLO = DK, TM_PQ = 2 * DK, TM_G = TM_PQ + 4 * C, TM_CHI = TM_G + 2 * C,
                        TM_CLO = TM_CHI + C, TM_USED = TM_CLO + C;
   static constexpr int TM_ALLOC = 512;
   static_assert(TM_USED <= TM_ALLOC, "tensor memory budget");
@@ -76,8 +78,8 @@ struct ChunkCfg {
   static constexpr int OFF_KT = OFF_KQ + 2 * C * DK * 4;   // [C/4][DK][4] fp32: K transposed (rows = key dims)
   static constexpr int OFF_BE = OFF_KT + C * DK * 4;       // 2 x [C][NROW] fp32 beta = sigmoid(logit)
   static constexpr int OFF_G = OFF_BE + 2 * C * NROW * 4;  // 2 x { Gkk [C][C], Gkq [C][C] } fp32
-  static constexpr int OFF_OST = OFF_G + 2 * 2 * C * C * 4;  // [C][COLS] bf16 output staging
-  static constexpr int OFF_BAR = OFF_OST + C * COLS * ES;
+  static constexpr int OFF_OST = OFF_G + 2 * 2 * C * C * 4;  // 2 x [C][COLS] bf16 output staging
+  static constexpr int OFF_BAR = OFF_OST + 2 * C * COLS * ES;
   static constexpr int SMEM_BYTES = OFF_BAR + 128;
   static_assert(RAW_BYTES % 16 == 0 && RPQ_BYTES % 16 == 0 && (COLS * ES) % 16 == 0, "alignment");
   static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
@@ -182,23 +184,22 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       const __nv_bfloat16 *rv = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_V);
       const __nv_bfloat16 *rpk = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_PK);
       const float *Gkk = G_all + (n & 1) * 2 * C * C;
+      const float *Gkq = Gkk + C * C;
       const float *bes = be_all + (n & 1) * C * NROW;
 
-      PROF_ADD(0, 0);
       if (!mbar_wait(&bars[B_E], n & 1)) { failed = true; break; }
       tc_fence_after_sync();
-      PROF_ADD(1, 0);
-      float pred[C], cs[16];
+      float pred[C], qd[C], cs[16];
 #pragma unroll
       for (int cc = 0; cc < C / 16; ++cc) {
-        float a[16];
-        tmem_ld16(tb + Cf::TM_PQ + cc * 16, a);
+        float a[16], b[16];
+        tmem_ld16(tb + Cf::TM_PQ + (n & 1) * 2 * C + cc * 16, a);
+        tmem_ld16(tb + Cf::TM_PQ + (n & 1) * 2 * C + C + cc * 16, b);
         tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 16; ++i) pred[cc * 16 + i] = a[i];
+        for (int i = 0; i < 16; ++i) { pred[cc * 16 + i] = a[i]; qd[cc * 16 + i] = b[i]; }
       }
 
-      PROF_ADD(2, 0);
       // ---- sequential part of the chunk: E-step and the triangular key-side corrections ----
 #pragma unroll
       for (int t = 0; t < C; ++t) {
@@ -224,9 +225,12 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         cs[t & 15] = c;
         if (p.r_debug != nullptr && col_ok && t < nvalid)
           p.r_debug[((tok0 + (size_t)(t0 + t)) * J + j) * p.Dv + col] = rr;
-        // push this token's update into the later predictions of the chunk
+        // push this token's update into the later predictions of the chunk (serial chain) and into
+        // the readouts w.q of this and the later tokens (Eq. 3.5; nothing waits on these)
 #pragma unroll
         for (int u = t + 1; u < C; ++u) pred[u] = fmaf(c, Gkk[t * C + u], pred[u]);
+#pragma unroll
+        for (int u = t; u < C; ++u) qd[u] = fmaf(c, Gkq[t * C + u], qd[u]);
         if ((t & 15) == 15) {  // 16 update coefficients complete: park them in tensor memory (hi / lo)
           float hi[16], lo[16];
 #pragma unroll
@@ -237,11 +241,51 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       }
       tmem_st_wait();
       tc_fence_before_sync();
-      PROF_ADD(3, 0);
       // the next chunk's operands must be in place before this chunk is handed over (keeps every
       // barrier at most one phase ahead of its waiters)
       if (n + 1 < nchunks && (!mbar_wait(&bars[B_KQ], (n + 1) & 1) || !mbar_wait(&bars[B_GS], (n + 1) & 1))) failed = true;
       mbar_arrive(&bars[B_C]);
+
+      // ---- outputs of the chunk (Eq. 3.5), in the shadow of the tensor-core work for chunk n+1:
+      //      o_td = sum_j pi^q_j (w_t.q_t)_j with pi^q = softmax over the J lanes of a column.
+      //      Tokens are handled eight at a time so that the shuffles of different tokens overlap. ----
+      {
+        const __nv_bfloat16 *rpq = reinterpret_cast<const __nv_bfloat16 *>(smem + Cf::OFF_RPQ + (n % 3) * Cf::RPQ_BYTES);
+        __nv_bfloat16 *ost = ostage + (n & 1) * C * COLS;
+#pragma unroll
+        for (int tg = 0; tg < C; tg += 8) {
+          float x[8], m[8], e[8], o[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) { x[i] = __bfloat162float(rpq[((tg + i) * J + j) * COLS + dl]) * kLog2e; m[i] = x[i]; }
+#pragma unroll
+          for (int off = 1; off < J; off <<= 1) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) m[i] = fmaxf(m[i], __shfl_xor_sync(0xffffffffu, m[i], off));
+          }
+#pragma unroll
+          for (int i = 0; i < 8; ++i) { e[i] = ex2_approx(x[i] - m[i]); o[i] = e[i] * qd[tg + i]; }
+#pragma unroll
+          for (int off = 1; off < J; off <<= 1) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              e[i] += __shfl_xor_sync(0xffffffffu, e[i], off);
+              o[i] += __shfl_xor_sync(0xffffffffu, o[i], off);
+            }
+          }
+          if (j == 0) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) ost[(tg + i) * COLS + dl] = __float2bfloat16_rn(o[i] * rcp_approx(e[i]));
+          }
+        }
+        named_bar_sync(2, 128);
+        constexpr int GROUPS = COLS / 8;  // 8 outputs = 16 bytes per store
+        for (int e = r; e < C * GROUPS; e += 128) {
+          const int t = e / GROUPS, g8 = e - t * GROUPS;
+          if (t < nvalid && col0 + g8 * 8 < p.Dv)
+            *reinterpret_cast<uint4 *>((__nv_bfloat16 *)p.o + (tok0 + (size_t)(t0 + t)) * p.Dv + col0 + g8 * 8) =
+                *reinterpret_cast<const uint4 *>(ost + t * COLS + g8 * 8);
+        }
+      }
     }
     // ---- final state row -> global ----
     if (!failed && !mbar_wait(&bars[B_U], (nchunks - 1) & 1)) failed = true;
@@ -389,19 +433,9 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     for (int n = 0; n < nchunks && !failed; ++n) {
       const bool more = n + 1 < nchunks;
       const unsigned char *raw_next = smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES;
-      // (1) E(n) is done: take this row's Q0 out of tensor memory; the K/Q tile is free again
+      // (1) E(n) is done: the K/Q tile is free again
       if (!mbar_wait(&bars[B_E], n & 1)) { failed = true; break; }
       tc_fence_after_sync();
-      float qd[C];
-#pragma unroll
-      for (int cc = 0; cc < C / 16; ++cc) {
-        float a[16];
-        tmem_ld16(tb + Cf::TM_PQ + C + cc * 16, a);
-        tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 16; ++i) qd[cc * 16 + i] = a[i];
-      }
-      tc_fence_before_sync();
       // (2) operands of chunk n+1 (its raw stage has landed)
       cp_async_wait<0>();
       named_bar_sync(1, 128);
@@ -417,22 +451,10 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
           mbar_arrive(&bars[B_GS]);
         }
       }
-      PROF_ADD(4, 128);
+      
       // (3) chunk n is finished by the row warps: stage chunk n+2 into the buffers chunk n used
       if (!mbar_wait(&bars[B_C], n & 1)) { failed = true; break; }
-      PROF_ADD(5, 128);
-      tc_fence_after_sync();
-      float cq[C];  // this row's update coefficients c = hi + lo, before the row warps reuse the slots
-#pragma unroll
-      for (int cc = 0; cc < C / 16; ++cc) {
-        float a[16], b[16];
-        tmem_ld16(tb + Cf::TM_CHI + cc * 16, a);
-        tmem_ld16(tb + Cf::TM_CLO + cc * 16, b);
-        tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 16; ++i) cq[cc * 16 + i] = a[i] + b[i];
-      }
-      tc_fence_before_sync();
+      
       if (n + 2 < nchunks)
         chunk_issue_raw<Cf>(p, smem + Cf::OFF_RAW + (n & 1) * Cf::RAW_BYTES, smem + Cf::OFF_RPQ + ((n + 2) % 3) * Cf::RPQ_BYTES,
                             tok0, (n + 2) * C, col0, h);
@@ -447,44 +469,8 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         fence_async_smem();
         mbar_arrive(&bars[B_KT]);
       }
-      PROF_ADD(6, 128);
-      // (5) readouts of chunk n (Eq. 3.5): w_t.q_t = Q0 + sum_{s<=t} c_s (k_s.q_t), weighted by the query prior
-      {
-        const float *Gkq = G_all + (n & 1) * 2 * C * C + C * C;
-        const __nv_bfloat16 *rpq = reinterpret_cast<const __nv_bfloat16 *>(smem + Cf::OFF_RPQ + (n % 3) * Cf::RPQ_BYTES);
-        const int t0 = n * C;
-        const int nvalid = min(C, p.T - t0);
-#pragma unroll
-        for (int sidx = 0; sidx < C; ++sidx) {
-          const float c = cq[sidx];
-#pragma unroll
-          for (int u = sidx; u < C; ++u) qd[u] = fmaf(c, Gkq[sidx * C + u], qd[u]);
-        }
-#pragma unroll
-        for (int t = 0; t < C; ++t) {
-          const float x = __bfloat162float(rpq[(t * J + j) * COLS + dl]) * kLog2e;
-          float m = x;
-#pragma unroll
-          for (int off = 1; off < J; off <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-          const float e = ex2_approx(x - m);
-          float sum = e, o = e * qd[t];
-#pragma unroll
-          for (int off = 1; off < J; off <<= 1) {
-            sum += __shfl_xor_sync(0xffffffffu, sum, off);
-            o += __shfl_xor_sync(0xffffffffu, o, off);
-          }
-          if (j == 0) ostage[t * COLS + dl] = __float2bfloat16_rn(o * rcp_approx(sum));
-        }
-        named_bar_sync(2, 128);
-        constexpr int GROUPS = COLS / 8;  // 8 outputs = 16 bytes per store
-        for (int e = h; e < C * GROUPS; e += 128) {
-          const int t = e / GROUPS, g8 = e - t * GROUPS;
-          if (t < nvalid && col0 + g8 * 8 < p.Dv)
-            *reinterpret_cast<uint4 *>((__nv_bfloat16 *)p.o + (tok0 + (size_t)(t0 + t)) * p.Dv + col0 + g8 * 8) =
-                *reinterpret_cast<const uint4 *>(ostage + t * COLS + g8 * 8);
-        }
-      }
-      PROF_ADD(7, 128);
+      
+      
     }
     cp_async_wait<0>();
   } else if (lane == 0) {
@@ -501,10 +487,11 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       }
       mma_commit(&bars[B_G]);
     };
-    auto w_times_kq = [&](int w_col, bool first) {
+    auto w_times_kq = [&](int chunk, int w_col, bool first) {
 #pragma unroll 1
       for (int ks = 0; ks < DK / 8; ++ks)
-        mma_tf32_ts(tb0 + Cf::TM_PQ, tb0 + w_col + ks * 8, kq0 + (uint64_t)(ks * 2 * 2 * C), idE, !(first && ks == 0));
+        mma_tf32_ts(tb0 + Cf::TM_PQ + (chunk & 1) * 2 * C, tb0 + w_col + ks * 8, kq0 + (uint64_t)(ks * 2 * 2 * C), idE,
+                    !(first && ks == 0));
     };
     if (!mbar_wait(&bars[B_KQ], 0)) failed = true;
     tc_fence_after_sync();
@@ -512,8 +499,8 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     if (!failed && !mbar_wait(&bars[B_WLO], 0)) failed = true;
     tc_fence_after_sync();
     if (!failed) {
-      w_times_kq(Cf::TM_W, true);
-      w_times_kq(Cf::TM_WLO, false);
+      w_times_kq(0, Cf::TM_W, true);
+      w_times_kq(0, Cf::TM_WLO, false);
       mma_commit(&bars[B_E]);
     }
     for (int n = 0; n < nchunks && !failed; ++n) {
@@ -533,10 +520,10 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       }
       mma_commit(&bars[B_U]);
       if (more) {
-        w_times_kq(Cf::TM_W, true);  // executes after the update: MMAs of one thread run in order
+        w_times_kq(n + 1, Cf::TM_W, true);  // executes after the update: MMAs of one thread run in order
         if (!mbar_wait(&bars[B_WLO], (n + 1) & 1)) { failed = true; break; }
         tc_fence_after_sync();
-        w_times_kq(Cf::TM_WLO, false);
+        w_times_kq(n + 1, Cf::TM_WLO, false);
         mma_commit(&bars[B_E]);
       }
     }
