@@ -3,7 +3,7 @@
 
 A step is one pass of the whole hot path -- one ``swila_forward`` over the language-model
 shaped prefill workload (B=4, H=16, T=8192, Dk=Dv=128, J=4, bf16 inputs, fp32 state) with
-inputs resident in HBM.  Reported beside it: the same call end to end from pinned host
+inputs resident in HBM (the library picks the chunked tensor-core kernel).  Reported beside it: the same call end to end from pinned host
 buffers (``e2e``), the batched decode leg (B=256 streams, H=32, 1024 single-token steps),
 the roofline of the scan kernel, and the fp64 CPU oracle timed on the host cores.
 
@@ -34,9 +34,10 @@ METRIC = "swila_fwd_tokens_per_s"
 UNIT = "tokens/s"
 HEADLINE = 2  # config index of the workload the metric is quoted on
 
-# DRAM traffic of one scan launch on the headline workload, from the ncu capture
-# summarised in profiles/scan_lm_prefill.md (dram__bytes_read.sum + dram__bytes_write.sum).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 2.188e9
+# DRAM traffic of one launch on the headline workload, from the ncu captures summarised in
+# profiles/chunk_lm_prefill.md and profiles/scan_lm_prefill.md (dram__bytes_read.sum +
+# dram__bytes_write.sum; 2.186 GB chunked, 2.188 GB scan).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 2.186e9
 
 
 # ----------------------------------------------------------------------------------------------
@@ -233,8 +234,9 @@ def _peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         d = json.load(open(p))
-        return {"hbm_gbs": float(d["hbm_gbs"]), "source": "measured (MEASURED_PEAKS.json)"}
-    return {"hbm_gbs": 6650.0, "source": "fallback"}
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "source": "measured (MEASURED_PEAKS.json)"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"}
 
 
 def main():
@@ -247,6 +249,7 @@ def main():
     ap.add_argument("--no-decode", action="store_true", help="skip the batched decode leg")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    ap.add_argument("--no-scan", action="store_true", help="skip the scan-kernel comparison leg")
     ap.add_argument("--decode-steps", type=int, default=wl.DECODE_STEPS)
     ap.add_argument("--decode-prefill", type=int, default=4096)
     ap.add_argument("--decode-batch", type=int, default=0, help="override B of the decode leg (0 = 256)")
@@ -307,25 +310,61 @@ def main():
     ms_per_step = ms / args.steps
     value = world * w.B * w.T / (ms_per_step * 1e-3)
 
-    # ---- roofline of the scan kernel (one launch per step) ----
+    # ---- roofline of the kernel the step launches (one launch per step) ----
     props = torch.cuda.get_device_properties(local)
     peaks = _peaks()
     fma_peak_nominal = props.multi_processor_count * 128 * 2 * 1.965e9 / 1e12  # TFLOP/s at the max SM clock
     fma_peak_measured = measure_fma_peak(binding, stream)
     flops = algorithmic_flops(w)
-    ach_tflops = flops / (ms_per_step * 1e-3) / 1e12
     abytes = algorithmic_bytes(w)
-    roofline = {
-        "bound": "alu", "achieved": ach_tflops, "peak": fma_peak_nominal, "unit": "TFLOP/s",
-        "frac": ach_tflops / fma_peak_nominal,
-        "peak_source": "derived: SMs x 128 FP32 lanes x 2 x 1.965 GHz",
-        "peak_measured_fma_chain": fma_peak_measured, "frac_of_measured_fma_chain": ach_tflops / fma_peak_measured,
-        "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if not args.batch else None,
-        "algorithmic_bytes_per_launch": abytes, "algorithmic_flops_per_launch": flops,
-        "hbm_achieved_gbs": abytes / (ms_per_step * 1e-3) / 1e9, "hbm_peak_gbs": peaks["hbm_gbs"],
-        "hbm_frac": abytes / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"], "hbm_peak_source": peaks["source"],
-        "kernel": "swila_scan_kernel",
-    }
+    sec = ms_per_step * 1e-3
+    chunked = args.algo in (0, binding.ALGO_CHUNK)
+    if chunked:
+        # The chunked kernel runs the three state contractions on the tensor cores (TF32), so of the two
+        # bounds -- HBM bytes at the measured copy bandwidth, flops at the TF32 tensor peak -- HBM is the
+        # slower one (0.33 ms vs 0.26 ms on this workload) and is the roofline reported.
+        tf32_peak = peaks["bf16_tflops"] * 0.5
+        roofline = {
+            "bound": "hbm", "achieved": abytes / sec / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": abytes / sec / 1e9 / peaks["hbm_gbs"], "peak_source": peaks["source"],
+            "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if not args.batch else None,
+            "algorithmic_bytes_per_launch": abytes, "algorithmic_flops_per_launch": flops,
+            "kernel": "swila_chunk_kernel",
+            "tensor_bound": {"achieved_tflops": flops / sec / 1e12, "peak_tflops": tf32_peak,
+                             "frac": flops / sec / 1e12 / tf32_peak,
+                             "peak_source": "measured bf16 peak x nominal TF32/bf16 ratio 0.5"},
+            "note": "latency-bound: T tokens are a serial dependency chain per row; see DESIGN.md",
+        }
+    else:
+        ach_tflops = flops / sec / 1e12
+        roofline = {
+            "bound": "alu", "achieved": ach_tflops, "peak": fma_peak_nominal, "unit": "TFLOP/s",
+            "frac": ach_tflops / fma_peak_nominal, "peak_source": "derived: SMs x 128 FP32 lanes x 2 x 1.965 GHz",
+            "peak_measured_fma_chain": fma_peak_measured, "frac_of_measured_fma_chain": ach_tflops / fma_peak_measured,
+            "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if not args.batch else None,
+            "algorithmic_bytes_per_launch": abytes, "algorithmic_flops_per_launch": flops,
+            "hbm_achieved_gbs": abytes / sec / 1e9, "hbm_peak_gbs": peaks["hbm_gbs"], "kernel": "swila_scan_kernel",
+        }
+
+    # ---- the register-resident scan kernel on the same workload (the path of fp32 io, the TEMPORAL /
+    #      GATED variants and decode), with its FP32-ALU roofline ----
+    scan = None
+    if chunked and not args.no_scan:
+        def step_scan():
+            binding.swila_forward(w, inp, state_in=None, state_out=st_out, o=o, algo=binding.ALGO_SCAN)
+        for _ in range(3):
+            step_scan()
+        barrier()
+        n_scan = max(3, min(args.steps, 10))
+        ms_s = time_steps(step_scan, n_scan, stream) / n_scan
+        barrier()
+        ach = flops / (ms_s * 1e-3) / 1e12
+        scan = {"ms_per_step": ms_s, "tokens_per_s": world * w.B * w.T / (ms_s * 1e-3), "steps": n_scan,
+                "roofline": {"bound": "alu", "achieved": ach, "peak": fma_peak_nominal, "unit": "TFLOP/s",
+                             "frac": ach / fma_peak_nominal,
+                             "peak_source": "derived: SMs x 128 FP32 lanes x 2 x 1.965 GHz",
+                             "peak_measured_fma_chain": fma_peak_measured,
+                             "frac_of_measured_fma_chain": ach / fma_peak_measured, "kernel": "swila_scan_kernel"}}
 
     # ---- end to end from pinned host buffers through the C ABI ----
     e2e = None
@@ -380,7 +419,7 @@ def main():
                        "l2": "inputs (2.1 GB) larger than L2; no flush needed",
                        "multi_gpu": "independent replicas, no collective"},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": args.steps,
-            "clocks": clocks, "decode": decode,
+            "clocks": clocks, "decode": decode, "scan": scan,
         }
         print(json.dumps(line))
     if world > 1:

@@ -65,7 +65,7 @@ enum {
 
 /* algo: which kernel evaluates the recurrence.  Every choice computes the same function. */
 enum {
-  SWILA_ALGO_AUTO = 0,
+  SWILA_ALGO_AUTO = 0,     /* CHUNK where it applies and T >= 64, else SCAN */
   SWILA_ALGO_SCAN = 1,     /* sequential scan, state resident in registers, FP32 FMA pipe */
   SWILA_ALGO_SCAN_WIDE = 2, /* the same scan with 256-thread blocks (twice the columns per
                               block); ungated shapes with Dk = 128 only */
@@ -145,8 +145,9 @@ int swila_forward(const swila_shape_t *shape, const void *q, const void *k, cons
 /*
  * Decode: one token of the same recurrence on a carried state, updated in place
  * (generation, App. D.4).  q,k [B,H,1,Dk]; v, o [B,H,1,Dv]; gate tensors with T = 1.
- * shape->T is ignored.  The arithmetic and its order are those of swila_forward, so a
- * prefill of T tokens equals, bit for bit, T decode steps.
+ * shape->T is ignored.  Decode always runs the scan kernel with T = 1: its arithmetic and order
+ * are those of a scan prefill (SWILA_ALGO_SCAN), so a scan prefill of T tokens equals, bit for
+ * bit, T decode steps; against a chunked prefill the two agree to rounding (1e-4 on the state).
  */
 int swila_decode_step(const swila_shape_t *shape, const void *q, const void *k, const void *v,
                       const swila_gates_t *gates, swila_state_t *state, void *o, void *stream);

@@ -187,8 +187,10 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       const float *Gkq = Gkk + C * C;
       const float *bes = be_all + (n & 1) * C * NROW;
 
+      PROF_ADD(0, 0);
       if (!mbar_wait(&bars[B_E], n & 1)) { failed = true; break; }
       tc_fence_after_sync();
+      PROF_ADD(1, 0);
       float pred[C], qd[C], cs[16];
 #pragma unroll
       for (int cc = 0; cc < C / 16; ++cc) {
@@ -241,10 +243,12 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       }
       tmem_st_wait();
       tc_fence_before_sync();
+      PROF_ADD(2, 0);
       // the next chunk's operands must be in place before this chunk is handed over (keeps every
       // barrier at most one phase ahead of its waiters)
       if (n + 1 < nchunks && (!mbar_wait(&bars[B_KQ], (n + 1) & 1) || !mbar_wait(&bars[B_GS], (n + 1) & 1))) failed = true;
       mbar_arrive(&bars[B_C]);
+      PROF_ADD(3, 0);
 
       // ---- outputs of the chunk (Eq. 3.5), in the shadow of the tensor-core work for chunk n+1:
       //      o_td = sum_j pi^q_j (w_t.q_t)_j with pi^q = softmax over the J lanes of a column.
@@ -452,8 +456,10 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         }
       }
       
+      PROF_ADD(4, 128);
       // (3) chunk n is finished by the row warps: stage chunk n+2 into the buffers chunk n used
       if (!mbar_wait(&bars[B_C], n & 1)) { failed = true; break; }
+      PROF_ADD(5, 128);
       
       if (n + 2 < nchunks)
         chunk_issue_raw<Cf>(p, smem + Cf::OFF_RAW + (n & 1) * Cf::RAW_BYTES, smem + Cf::OFF_RPQ + ((n + 2) % 3) * Cf::RPQ_BYTES,
