@@ -54,10 +54,11 @@ struct ChunkCfg {
   static constexpr int COLS = NROW / J;   // output columns per block
   static constexpr int ES = 2;            // bf16 io
   // tensor-memory columns
-  // ([P0 | Q0] is double-buffered: the row warps still read Q0 of chunk n while the tensor cores
-  // already write the products of chunk n+1)
-  static constexpr int TM_W = 0, TM_WLO = DK, TM_PQ = 2 * DK, TM_G = TM_PQ + 4 * C, TM_CHI = TM_G + 2 * C,
-                       TM_CLO = TM_CHI + C, TM_USED = TM_CLO + C;
+  // W, W_lo: the state and its low part; PQ: [P0 | Q0] of the current chunk; QD: the query-side
+  // readouts w_t.q_t of a chunk (double-buffered: the outputs of chunk n are formed while chunk
+  // n+1 runs); G: [K K^T | K Q^T]; CHI / CLO: the update coefficients of the chunk
+  static constexpr int TM_W = 0, TM_WLO = DK, TM_PQ = 2 * DK, TM_QD = TM_PQ + 2 * C, TM_G = TM_QD + 2 * C,
+                       TM_CHI = TM_G + 2 * C, TM_CLO = TM_CHI + C, TM_USED = TM_CLO + C;
   static constexpr int TM_ALLOC = 512;
   static_assert(TM_USED <= TM_ALLOC, "tensor memory budget");
   // raw stages (bytes), all bf16.  Main part: k, q [C][DK], v [C][COLS], beta/pik [C][J][COLS] (2-deep
@@ -73,12 +74,13 @@ struct ChunkCfg {
   static constexpr int C_K = DK * ES / 16, C_V = COLS * ES / 16;  // 16-byte units per token row / column slice
   // shared memory map (bytes)
   static constexpr int OFF_RAW = 0;
-  static constexpr int OFF_RPQ = OFF_RAW + 2 * RAW_BYTES;
-  static constexpr int OFF_KQ = OFF_RPQ + 3 * RPQ_BYTES;   // [DK/4][2C][4] fp32: rows 0..C-1 = K, C..2C-1 = Q tokens
+  static constexpr int OFF_RPQ = OFF_RAW + 2 * RAW_BYTES;  // 4-deep ring of query-prior logits
+  static constexpr int OFF_KQ = OFF_RPQ + 4 * RPQ_BYTES;   // [DK/4][2C][4] fp32: rows 0..C-1 = K, C..2C-1 = Q tokens
   static constexpr int OFF_KT = OFF_KQ + 2 * C * DK * 4;   // [C/4][DK][4] fp32: K transposed (rows = key dims)
   static constexpr int OFF_BE = OFF_KT + C * DK * 4;       // 2 x [C][NROW] fp32 beta = sigmoid(logit)
-  static constexpr int OFF_G = OFF_BE + 2 * C * NROW * 4;  // 2 x { Gkk [C][C], Gkq [C][C] } fp32
-  static constexpr int OFF_OST = OFF_G + 2 * 2 * C * C * 4;  // 2 x [C][COLS] bf16 output staging
+  static constexpr int OFF_G = OFF_BE + 2 * C * NROW * 4;  // 2 x Gkk [C][C] fp32 (K K^T, for the row warps)
+  static constexpr int OFF_BQ = OFF_G + 2 * C * C * 4;     // 2 x { hi, lo } [C/4][C][4] fp32: masked (K Q^T)^T operand tiles
+  static constexpr int OFF_OST = OFF_BQ + 2 * 2 * C * C * 4;  // 2 x [C][COLS] bf16 output staging
   static constexpr int OFF_BAR = OFF_OST + 2 * C * COLS * ES;
   static constexpr int SMEM_BYTES = OFF_BAR + 128;
   static_assert(RAW_BYTES % 16 == 0 && RPQ_BYTES % 16 == 0 && (COLS * ES) % 16 == 0, "alignment");
@@ -86,7 +88,7 @@ struct ChunkCfg {
 };
 
 // barrier slots
-enum { B_E = 0, B_G, B_U, B_KQ, B_KT, B_WLO, B_GS, B_C, B_COUNT };
+enum { B_E = 0, B_G, B_U, B_QD, B_KQ, B_KT, B_WLO, B_GS, B_C, B_COUNT };
 
 // hi/lo split of an FP32 value for TF32 operands: hi keeps the bits the tensor core reads
 // (it ignores the 13 low mantissa bits), lo is the exact remainder.
@@ -136,6 +138,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   float *Kt = reinterpret_cast<float *>(smem + Cf::OFF_KT);
   float *be_all = reinterpret_cast<float *>(smem + Cf::OFF_BE);
   float *G_all = reinterpret_cast<float *>(smem + Cf::OFF_G);
+  float *BQ_all = reinterpret_cast<float *>(smem + Cf::OFF_BQ);
   __nv_bfloat16 *ostage = reinterpret_cast<__nv_bfloat16 *>(smem + Cf::OFF_OST);
   uint64_t *bars = reinterpret_cast<uint64_t *>(smem + Cf::OFF_BAR);
   uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(bars + B_COUNT);
@@ -152,6 +155,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     mbar_init(&bars[B_E], 1);
     mbar_init(&bars[B_G], 1);
     mbar_init(&bars[B_U], 1);
+    mbar_init(&bars[B_QD], 1);
     mbar_init(&bars[B_KQ], 128);
     mbar_init(&bars[B_KT], 128);
     mbar_init(&bars[B_WLO], 128);
@@ -177,62 +181,130 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     const bool col_ok = col < p.Dv;
     const int jbase = lane - j;
     if (!mbar_wait(&bars[B_KQ], 0) || !mbar_wait(&bars[B_GS], 0)) failed = true;
+    // outputs of one chunk (Eq. 3.5): o_td = sum_j pi^q_j (w_t.q_t)_j, pi^q = softmax over the J lanes
+    // of a column; eight tokens at a time so that the shuffles of different tokens overlap
+    auto write_outputs = [&](int n) {
+      const int t0 = n * C;
+      const int nvalid = min(C, p.T - t0);
+      const __nv_bfloat16 *rpq = reinterpret_cast<const __nv_bfloat16 *>(smem + Cf::OFF_RPQ + (n & 3) * Cf::RPQ_BYTES);
+      __nv_bfloat16 *ost = ostage + (n & 1) * C * COLS;
+      tc_fence_after_sync();
+#pragma unroll
+      for (int tg = 0; tg < C; tg += 16) {
+        float qd[16];
+        tmem_ld16(tb + Cf::TM_QD + (n & 1) * C + tg, qd);
+        tmem_ld_wait();
+#pragma unroll
+        for (int th = 0; th < 16; th += 8) {
+          float x[8], m[8], e[8], o[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) { x[i] = __bfloat162float(rpq[((tg + th + i) * J + j) * COLS + dl]) * kLog2e; m[i] = x[i]; }
+#pragma unroll
+          for (int off = 1; off < J; off <<= 1) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) m[i] = fmaxf(m[i], __shfl_xor_sync(0xffffffffu, m[i], off));
+          }
+#pragma unroll
+          for (int i = 0; i < 8; ++i) { e[i] = ex2_approx(x[i] - m[i]); o[i] = e[i] * qd[th + i]; }
+#pragma unroll
+          for (int off = 1; off < J; off <<= 1) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              e[i] += __shfl_xor_sync(0xffffffffu, e[i], off);
+              o[i] += __shfl_xor_sync(0xffffffffu, o[i], off);
+            }
+          }
+          if (j == 0) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) ost[(tg + th + i) * COLS + dl] = __float2bfloat16_rn(o[i] * rcp_approx(e[i]));
+          }
+        }
+      }
+      tc_fence_before_sync();
+      named_bar_sync(2, 128);
+      constexpr int GROUPS = COLS / 8;  // 8 outputs = 16 bytes per store
+      for (int e = r; e < C * GROUPS; e += 128) {
+        const int t = e / GROUPS, g8 = e - t * GROUPS;
+        if (t < nvalid && col0 + g8 * 8 < p.Dv)
+          *reinterpret_cast<uint4 *>((__nv_bfloat16 *)p.o + (tok0 + (size_t)(t0 + t)) * p.Dv + col0 + g8 * 8) =
+              *reinterpret_cast<const uint4 *>(ost + t * COLS + g8 * 8);
+      }
+    };
+
     for (int n = 0; n < nchunks && !failed; ++n) {
       const int t0 = n * C;
       const int nvalid = min(C, p.T - t0);
       const unsigned char *raw = smem + Cf::OFF_RAW + (n & 1) * Cf::RAW_BYTES;
       const __nv_bfloat16 *rv = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_V);
       const __nv_bfloat16 *rpk = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_PK);
-      const float *Gkk = G_all + (n & 1) * 2 * C * C;
-      const float *Gkq = Gkk + C * C;
+      const float *Gkk = G_all + (n & 1) * C * C;
       const float *bes = be_all + (n & 1) * C * NROW;
+
+      // key-prior logits of this row, base 2, shifted by their maximum over the J components: with
+      // a_j = lk_j - delta_j^2 log2(e)/2 <= 0 the E-step needs no further max-subtraction (raw stage n
+      // is in place: the hand-over of chunk n-1 waited for it).  Grouped so the shuffles overlap.
+      float lk[C];
+#pragma unroll
+      for (int tg = 0; tg < C; tg += 8) {
+        float m[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { lk[tg + i] = __bfloat162float(rpk[((tg + i) * J + j) * COLS + dl]) * kLog2e; m[i] = lk[tg + i]; }
+#pragma unroll
+        for (int off = 1; off < J; off <<= 1) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) m[i] = fmaxf(m[i], __shfl_xor_sync(0xffffffffu, m[i], off));
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) lk[tg + i] -= m[i];
+      }
 
       PROF_ADD(0, 0);
       if (!mbar_wait(&bars[B_E], n & 1)) { failed = true; break; }
       tc_fence_after_sync();
       PROF_ADD(1, 0);
-      float pred[C], qd[C], cs[16];
+      float pred[C], cs[16];
 #pragma unroll
       for (int cc = 0; cc < C / 16; ++cc) {
         float a[16], b[16];
-        tmem_ld16(tb + Cf::TM_PQ + (n & 1) * 2 * C + cc * 16, a);
-        tmem_ld16(tb + Cf::TM_PQ + (n & 1) * 2 * C + C + cc * 16, b);
+        tmem_ld16(tb + Cf::TM_PQ + cc * 16, a);
+        tmem_ld16(tb + Cf::TM_PQ + C + cc * 16, b);
         tmem_ld_wait();
+        tmem_st16(tb + Cf::TM_QD + (n & 1) * C + cc * 16, b);  // Q0 seeds the readout accumulator of this chunk
 #pragma unroll
-        for (int i = 0; i < 16; ++i) { pred[cc * 16 + i] = a[i]; qd[cc * 16 + i] = b[i]; }
+        for (int i = 0; i < 16; ++i) pred[cc * 16 + i] = a[i];
       }
 
       // ---- sequential part of the chunk: E-step and the triangular key-side corrections ----
 #pragma unroll
       for (int t = 0; t < C; ++t) {
-        const int gi = (t * J + j) * COLS + dl;
-        const float lk = __bfloat162float(rpk[gi]) * kLog2e;
         const float v = __bfloat162float(rv[t * COLS + dl]);
         const float be = bes[t * NROW + r];
         // serial chain: prediction error -> responsibilities (Eq. 3.4) -> update coefficient (Eq. 3.3)
         const float delta = v - pred[t];
-        const float a = fmaf(-kHalfLog2e * delta, delta, lk);
-        float all[J];
+        const float a = fmaf(-kHalfLog2e * delta, delta, lk[t]);
+        float e = ex2_approx(a);
+        float sum = e;
 #pragma unroll
-        for (int jj = 0; jj < J; ++jj) all[jj] = __shfl_sync(0xffffffffu, a, jbase + jj);
-        float m = all[0];
+        for (int jj = 1; jj < J; ++jj) sum += __shfl_sync(0xffffffffu, e, jbase + ((j + jj) & (J - 1)));
+        if (__any_sync(0xffffffffu, !(sum > 1e-30f))) {
+          // every component is > ~13 standard deviations off: redo the E-step with the maximum subtracted
+          float m = a;
 #pragma unroll
-        for (int jj = 1; jj < J; ++jj) m = fmaxf(m, all[jj]);
-        float sum = 0.f;
+          for (int off = 1; off < J; off <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+          e = ex2_approx(a - m);
+          sum = e;
 #pragma unroll
-        for (int jj = 0; jj < J; ++jj) sum += ex2_approx(all[jj] - m);
-        const float rr = ex2_approx(a - m) * rcp_approx(sum);
-        float c = be * rr * delta;
+          for (int off = 1; off < J; off <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+        }
+        const float rr = e * rcp_approx(sum);
+        float c = (be * delta) * rr;
         if (t >= nvalid) c = 0.f;  // padding tokens of the last chunk leave the state alone
         cs[t & 15] = c;
         if (p.r_debug != nullptr && col_ok && t < nvalid)
           p.r_debug[((tok0 + (size_t)(t0 + t)) * J + j) * p.Dv + col] = rr;
-        // push this token's update into the later predictions of the chunk (serial chain) and into
-        // the readouts w.q of this and the later tokens (Eq. 3.5; nothing waits on these)
+        // push this token's update into the later predictions of the chunk
 #pragma unroll
         for (int u = t + 1; u < C; ++u) pred[u] = fmaf(c, Gkk[t * C + u], pred[u]);
-#pragma unroll
-        for (int u = t; u < C; ++u) qd[u] = fmaf(c, Gkq[t * C + u], qd[u]);
         if ((t & 15) == 15) {  // 16 update coefficients complete: park them in tensor memory (hi / lo)
           float hi[16], lo[16];
 #pragma unroll
@@ -244,53 +316,17 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       tmem_st_wait();
       tc_fence_before_sync();
       PROF_ADD(2, 0);
-      // the next chunk's operands must be in place before this chunk is handed over (keeps every
-      // barrier at most one phase ahead of its waiters)
+      // the next chunk's operands, and the previous chunk's readouts, must be in place before this
+      // chunk is handed over (keeps every barrier at most one phase ahead of its waiters)
       if (n + 1 < nchunks && (!mbar_wait(&bars[B_KQ], (n + 1) & 1) || !mbar_wait(&bars[B_GS], (n + 1) & 1))) failed = true;
+      if (n > 0 && !mbar_wait(&bars[B_QD], (n - 1) & 1)) failed = true;
       mbar_arrive(&bars[B_C]);
       PROF_ADD(3, 0);
-
-      // ---- outputs of the chunk (Eq. 3.5), in the shadow of the tensor-core work for chunk n+1:
-      //      o_td = sum_j pi^q_j (w_t.q_t)_j with pi^q = softmax over the J lanes of a column.
-      //      Tokens are handled eight at a time so that the shuffles of different tokens overlap. ----
-      {
-        const __nv_bfloat16 *rpq = reinterpret_cast<const __nv_bfloat16 *>(smem + Cf::OFF_RPQ + (n % 3) * Cf::RPQ_BYTES);
-        __nv_bfloat16 *ost = ostage + (n & 1) * C * COLS;
-#pragma unroll
-        for (int tg = 0; tg < C; tg += 8) {
-          float x[8], m[8], e[8], o[8];
-#pragma unroll
-          for (int i = 0; i < 8; ++i) { x[i] = __bfloat162float(rpq[((tg + i) * J + j) * COLS + dl]) * kLog2e; m[i] = x[i]; }
-#pragma unroll
-          for (int off = 1; off < J; off <<= 1) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) m[i] = fmaxf(m[i], __shfl_xor_sync(0xffffffffu, m[i], off));
-          }
-#pragma unroll
-          for (int i = 0; i < 8; ++i) { e[i] = ex2_approx(x[i] - m[i]); o[i] = e[i] * qd[tg + i]; }
-#pragma unroll
-          for (int off = 1; off < J; off <<= 1) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              e[i] += __shfl_xor_sync(0xffffffffu, e[i], off);
-              o[i] += __shfl_xor_sync(0xffffffffu, o[i], off);
-            }
-          }
-          if (j == 0) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) ost[(tg + i) * COLS + dl] = __float2bfloat16_rn(o[i] * rcp_approx(e[i]));
-          }
-        }
-        named_bar_sync(2, 128);
-        constexpr int GROUPS = COLS / 8;  // 8 outputs = 16 bytes per store
-        for (int e = r; e < C * GROUPS; e += 128) {
-          const int t = e / GROUPS, g8 = e - t * GROUPS;
-          if (t < nvalid && col0 + g8 * 8 < p.Dv)
-            *reinterpret_cast<uint4 *>((__nv_bfloat16 *)p.o + (tok0 + (size_t)(t0 + t)) * p.Dv + col0 + g8 * 8) =
-                *reinterpret_cast<const uint4 *>(ost + t * COLS + g8 * 8);
-        }
-      }
+      // outputs of the previous chunk, in the shadow of the tensor-core work for chunk n+1
+      if (n > 0 && !failed) write_outputs(n - 1);
     }
+    if (!failed && !mbar_wait(&bars[B_QD], (nchunks - 1) & 1)) failed = true;
+    if (!failed) write_outputs(nchunks - 1);
     // ---- final state row -> global ----
     if (!failed && !mbar_wait(&bars[B_U], (nchunks - 1) & 1)) failed = true;
     if (!failed && p.W_out && col_ok) {
@@ -373,10 +409,13 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       tmem_st_wait();
       tc_fence_before_sync();
     };
-    // Gram rows (tensor-memory lanes 0..C-1, helper warp 4 only) -> shared memory
+    // Gram rows (tensor-memory lanes 0..C-1, helper warp 4 only) -> shared memory: K K^T row-major for the
+    // row warps; K Q^T as the B operand of the readout MMA -- transposed (rows = later token t, K index
+    // = earlier token s = this lane), causally masked (s <= t), split into hi / lo TF32 parts
     auto spill_gram = [&](int n) {
-      float *Gkk = G_all + (n & 1) * 2 * C * C;
-      float *Gkq = Gkk + C * C;
+      float *Gkk = G_all + (n & 1) * C * C;
+      float *Bhi = BQ_all + (n & 1) * 2 * C * C;
+      float *Blo = Bhi + C * C;
 #pragma unroll
       for (int cc = 0; cc < C / 16; ++cc) {
         float a[16], b[16];
@@ -384,12 +423,20 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         tmem_ld16(tb + Cf::TM_G + C + cc * 16, b);
         tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < 4; ++i)
           *reinterpret_cast<float4 *>(Gkk + lane * C + cc * 16 + i * 4) = make_float4(a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
-          *reinterpret_cast<float4 *>(Gkq + lane * C + cc * 16 + i * 4) = make_float4(b[4 * i], b[4 * i + 1], b[4 * i + 2], b[4 * i + 3]);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const int t = cc * 16 + i;
+          const float val = (lane <= t) ? b[i] : 0.f;
+          const float hi = tf32_hi(val);
+          const int idx = ((lane >> 2) * C + t) * 4 + (lane & 3);
+          Bhi[idx] = hi;
+          Blo[idx] = val - hi;
         }
       }
       tc_fence_before_sync();
+      fence_async_smem();
     };
 
     // ---- prologue: stage chunks 0 and 1, state row -> tensor memory, operands of chunk 0 ----
@@ -462,7 +509,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       PROF_ADD(5, 128);
       
       if (n + 2 < nchunks)
-        chunk_issue_raw<Cf>(p, smem + Cf::OFF_RAW + (n & 1) * Cf::RAW_BYTES, smem + Cf::OFF_RPQ + ((n + 2) % 3) * Cf::RPQ_BYTES,
+        chunk_issue_raw<Cf>(p, smem + Cf::OFF_RAW + (n & 1) * Cf::RAW_BYTES, smem + Cf::OFF_RPQ + ((n + 2) & 3) * Cf::RPQ_BYTES,
                             tok0, (n + 2) * C, col0, h);
       cp_async_commit();
       // (4) W has been updated with chunk n: refresh its low part, then the transposed K of chunk n+1
@@ -493,11 +540,25 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       }
       mma_commit(&bars[B_G]);
     };
-    auto w_times_kq = [&](int chunk, int w_col, bool first) {
+    auto w_times_kq = [&](int w_col, bool first) {
 #pragma unroll 1
       for (int ks = 0; ks < DK / 8; ++ks)
-        mma_tf32_ts(tb0 + Cf::TM_PQ + (chunk & 1) * 2 * C, tb0 + w_col + ks * 8, kq0 + (uint64_t)(ks * 2 * 2 * C), idE,
-                    !(first && ks == 0));
+        mma_tf32_ts(tb0 + Cf::TM_PQ, tb0 + w_col + ks * 8, kq0 + (uint64_t)(ks * 2 * 2 * C), idE, !(first && ks == 0));
+    };
+    constexpr uint32_t idQ = idesc_tf32(128, C);
+    // readouts of chunk n: QD += Cmat (K Q^T masked)  -- c_hi B_hi + c_lo B_hi + c_hi B_lo
+    auto readout = [&](int n) {
+      const uint64_t bh0 = smem_desc_kmajor(smem_u32(BQ_all + (n & 1) * 2 * C * C), C * 16, 128);
+      const uint64_t bl0 = smem_desc_kmajor(smem_u32(BQ_all + (n & 1) * 2 * C * C + C * C), C * 16, 128);
+      const uint32_t d = tb0 + Cf::TM_QD + (n & 1) * C;
+#pragma unroll 1
+      for (int ks = 0; ks < C / 8; ++ks) {
+        const uint64_t adv = (uint64_t)(ks * 2 * C);
+        mma_tf32_ts(d, tb0 + Cf::TM_CHI + ks * 8, bh0 + adv, idQ, true);
+        mma_tf32_ts(d, tb0 + Cf::TM_CLO + ks * 8, bh0 + adv, idQ, true);
+        mma_tf32_ts(d, tb0 + Cf::TM_CHI + ks * 8, bl0 + adv, idQ, true);
+      }
+      mma_commit(&bars[B_QD]);
     };
     if (!mbar_wait(&bars[B_KQ], 0)) failed = true;
     tc_fence_after_sync();
@@ -505,8 +566,8 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     if (!failed && !mbar_wait(&bars[B_WLO], 0)) failed = true;
     tc_fence_after_sync();
     if (!failed) {
-      w_times_kq(0, Cf::TM_W, true);
-      w_times_kq(0, Cf::TM_WLO, false);
+      w_times_kq(Cf::TM_W, true);
+      w_times_kq(Cf::TM_WLO, false);
       mma_commit(&bars[B_E]);
     }
     for (int n = 0; n < nchunks && !failed; ++n) {
@@ -525,11 +586,12 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         mma_tf32_ts(tb0 + Cf::TM_W, tb0 + Cf::TM_CLO + ks * 8, bt, idU, true);
       }
       mma_commit(&bars[B_U]);
+      if (more) w_times_kq(Cf::TM_W, true);  // executes after the update: MMAs of one thread run in order
+      readout(n);
       if (more) {
-        w_times_kq(n + 1, Cf::TM_W, true);  // executes after the update: MMAs of one thread run in order
         if (!mbar_wait(&bars[B_WLO], (n + 1) & 1)) { failed = true; break; }
         tc_fence_after_sync();
-        w_times_kq(n + 1, Cf::TM_WLO, false);
+        w_times_kq(Cf::TM_WLO, false);
         mma_commit(&bars[B_E]);
       }
     }
