@@ -129,7 +129,7 @@ __device__ __forceinline__ void chunk_issue_raw(const ScanParams &p, unsigned ch
   }
 }
 
-template <class Cf>
+template <class Cf, bool RDEBUG>
 __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_constant__ ScanParams p) {
   using namespace umma;
   constexpr int J = Cf::J, DK = Cf::DK, C = Cf::C, NROW = Cf::NROW, COLS = Cf::COLS;
@@ -240,23 +240,11 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       const float *Gkk = G_all + (n & 1) * C * C;
       const float *bes = be_all + (n & 1) * C * NROW;
 
-      // key-prior logits of this row, base 2, shifted by their maximum over the J components: with
-      // a_j = lk_j - delta_j^2 log2(e)/2 <= 0 the E-step needs no further max-subtraction (raw stage n
-      // is in place: the hand-over of chunk n-1 waited for it).  Grouped so the shuffles overlap.
+      // key-prior logits of this row in base 2 (raw stage n is in place: the hand-over of chunk n-1
+      // waited for it)
       float lk[C];
 #pragma unroll
-      for (int tg = 0; tg < C; tg += 8) {
-        float m[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) { lk[tg + i] = __bfloat162float(rpk[((tg + i) * J + j) * COLS + dl]) * kLog2e; m[i] = lk[tg + i]; }
-#pragma unroll
-        for (int off = 1; off < J; off <<= 1) {
-#pragma unroll
-          for (int i = 0; i < 8; ++i) m[i] = fmaxf(m[i], __shfl_xor_sync(0xffffffffu, m[i], off));
-        }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) lk[tg + i] -= m[i];
-      }
+      for (int t = 0; t < C; ++t) lk[t] = __bfloat162float(rpk[(t * J + j) * COLS + dl]) * kLog2e;
 
       PROF_ADD(0, 0);
       if (!mbar_wait(&bars[B_E], n & 1)) { failed = true; break; }
@@ -282,26 +270,25 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         // serial chain: prediction error -> responsibilities (Eq. 3.4) -> update coefficient (Eq. 3.3)
         const float delta = v - pred[t];
         const float a = fmaf(-kHalfLog2e * delta, delta, lk[t]);
-        float e = ex2_approx(a);
-        float sum = e;
+        // softmax over the J components with the maximum subtracted (exact, never 0/0); every lane of the
+        // column gathers all J exponents and normalises redundantly: one shuffle round on the chain
+        float all[J];
 #pragma unroll
-        for (int jj = 1; jj < J; ++jj) sum += __shfl_sync(0xffffffffu, e, jbase + ((j + jj) & (J - 1)));
-        if (__any_sync(0xffffffffu, !(sum > 1e-30f))) {
-          // every component is > ~13 standard deviations off: redo the E-step with the maximum subtracted
-          float m = a;
+        for (int jj = 0; jj < J; ++jj) all[jj] = __shfl_sync(0xffffffffu, a, jbase + jj);
+        float m = all[0];
 #pragma unroll
-          for (int off = 1; off < J; off <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
-          e = ex2_approx(a - m);
-          sum = e;
+        for (int jj = 1; jj < J; ++jj) m = fmaxf(m, all[jj]);
+        float sum = 0.f;
 #pragma unroll
-          for (int off = 1; off < J; off <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
-        }
+        for (int jj = 0; jj < J; ++jj) sum += ex2_approx(all[jj] - m);
+        const float e = ex2_approx(a - m);
         const float rr = e * rcp_approx(sum);
         float c = (be * delta) * rr;
         if (t >= nvalid) c = 0.f;  // padding tokens of the last chunk leave the state alone
         cs[t & 15] = c;
-        if (p.r_debug != nullptr && col_ok && t < nvalid)
-          p.r_debug[((tok0 + (size_t)(t0 + t)) * J + j) * p.Dv + col] = rr;
+        if constexpr (RDEBUG) {
+          if (col_ok && t < nvalid) p.r_debug[((tok0 + (size_t)(t0 + t)) * J + j) * p.Dv + col] = rr;
+        }
         // push this token's update into the later predictions of the chunk
 #pragma unroll
         for (int u = t + 1; u < C; ++u) pred[u] = fmaf(c, Gkk[t * C + u], pred[u]);
@@ -586,14 +573,14 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         mma_tf32_ts(tb0 + Cf::TM_W, tb0 + Cf::TM_CLO + ks * 8, bt, idU, true);
       }
       mma_commit(&bars[B_U]);
-      if (more) w_times_kq(Cf::TM_W, true);  // executes after the update: MMAs of one thread run in order
-      readout(n);
       if (more) {
+        w_times_kq(Cf::TM_W, true);  // executes after the update: MMAs of one thread run in order
         if (!mbar_wait(&bars[B_WLO], (n + 1) & 1)) { failed = true; break; }
         tc_fence_after_sync();
         w_times_kq(Cf::TM_WLO, false);
         mma_commit(&bars[B_E]);
       }
+      readout(n);  // not needed before the outputs are formed one chunk later: off the critical path
     }
   }
   if (failed) atomicExch(&g_chunk_error, 1);
@@ -605,7 +592,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
 template <int J, int DK>
 int launch_chunk(const LaunchArgs &a) {
   using Cf = ChunkCfg<J, DK>;
-  auto kern = swila_chunk_kernel<Cf>;
+  auto kern = a.p.r_debug ? swila_chunk_kernel<Cf, true> : swila_chunk_kernel<Cf, false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cf::SMEM_BYTES);
   if (e != cudaSuccess) return (int)e;
   const long long nslice = (a.p.Dv + Cf::COLS - 1) / Cf::COLS;
