@@ -31,6 +31,8 @@
 //   warp 8, lane 0   issues every tcgen05.mma and commits them to the barriers.
 #pragma once
 
+#include <type_traits>
+
 #include "swila_common.cuh"
 #include "swila_umma.cuh"
 
@@ -240,65 +242,110 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       const float *Gkk = G_all + (n & 1) * C * C;
       const float *bes = be_all + (n & 1) * C * NROW;
 
-      // key-prior logits of this row in base 2 (raw stage n is in place: the hand-over of chunk n-1
-      // waited for it)
+      // key-prior logits of this row, base 2, shifted by their maximum over the J components (the softmax
+      // of the E-step is shift-invariant; with the shift every exponent a_j = lk_j - delta_j^2 log2(e)/2 is
+      // <= 0).  Raw stage n is in place: the hand-over of chunk n-1 waited for it.  Grouped so the
+      // shuffles of different tokens overlap.
       float lk[C];
 #pragma unroll
-      for (int t = 0; t < C; ++t) lk[t] = __bfloat162float(rpk[(t * J + j) * COLS + dl]) * kLog2e;
+      for (int tg = 0; tg < C; tg += 8) {
+        float m[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { lk[tg + i] = __bfloat162float(rpk[((tg + i) * J + j) * COLS + dl]) * kLog2e; m[i] = lk[tg + i]; }
+#pragma unroll
+        for (int off = 1; off < J; off <<= 1) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) m[i] = fmaxf(m[i], __shfl_xor_sync(0xffffffffu, m[i], off));
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) lk[tg + i] -= m[i];
+      }
 
       PROF_ADD(0, 0);
       if (!mbar_wait(&bars[B_E], n & 1)) { failed = true; break; }
       tc_fence_after_sync();
       PROF_ADD(1, 0);
-      float pred[C], cs[16];
+      // ---- sequential part of the chunk: E-step and the triangular key-side corrections.  Only one FMA
+      //      of a token's push (into the next token's prediction) sits on the serial chain; the rest is
+      //      deferred into the shuffle latency of the next token's E-step.
+      //      FAST: exponents are taken without a per-token maximum (they are <= 0 after the prior shift);
+      //      the pass reports whether any normaliser underflowed -- every component > ~13 standard
+      //      deviations off -- in which case the chunk is redone with the per-token maximum subtracted. ----
+      auto sequential = [&](auto exact_tag) -> bool {
+        constexpr bool EXACT = decltype(exact_tag)::value;
+        bool bad = false;
+        float pred[C], cs[16];
 #pragma unroll
-      for (int cc = 0; cc < C / 16; ++cc) {
-        float a[16], b[16];
-        tmem_ld16(tb + Cf::TM_PQ + cc * 16, a);
-        tmem_ld16(tb + Cf::TM_PQ + C + cc * 16, b);
-        tmem_ld_wait();
-        tmem_st16(tb + Cf::TM_QD + (n & 1) * C + cc * 16, b);  // Q0 seeds the readout accumulator of this chunk
+        for (int cc = 0; cc < C / 16; ++cc) {
+          float a[16];
+          tmem_ld16(tb + Cf::TM_PQ + cc * 16, a);
+          tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 16; ++i) pred[cc * 16 + i] = a[i];
+          for (int i = 0; i < 16; ++i) pred[cc * 16 + i] = a[i];
+        }
+        float c_prev = 0.f;
+#pragma unroll
+        for (int t = 0; t < C; ++t) {
+          const float v = __bfloat162float(rv[t * COLS + dl]);
+          const float be = bes[t * NROW + r];
+          // serial chain: prediction error -> responsibilities (Eq. 3.4) -> update coefficient (Eq. 3.3)
+          const float delta = v - pred[t];
+          const float a = fmaf(-kHalfLog2e * delta, delta, lk[t]);
+          float e, sum;
+          if constexpr (EXACT) {
+            float all[J];
+#pragma unroll
+            for (int jj = 0; jj < J; ++jj) all[jj] = __shfl_sync(0xffffffffu, a, jbase + jj);
+            float m = all[0];
+#pragma unroll
+            for (int jj = 1; jj < J; ++jj) m = fmaxf(m, all[jj]);
+            sum = 0.f;
+#pragma unroll
+            for (int jj = 0; jj < J; ++jj) sum += ex2_approx(all[jj] - m);
+            e = ex2_approx(a - m);
+          } else {
+            e = ex2_approx(a);
+            sum = e;
+#pragma unroll
+            for (int jj = 1; jj < J; ++jj) sum += __shfl_sync(0xffffffffu, e, jbase + ((j + jj) & (J - 1)));
+            bad = bad || !(sum > 1e-30f);
+          }
+          if (t >= 1) {  // deferred push of token t-1 into the predictions of tokens t+1 ..
+#pragma unroll
+            for (int u = t + 1; u < C; ++u) pred[u] = fmaf(c_prev, Gkk[(t - 1) * C + u], pred[u]);
+          }
+          const float rr = e * rcp_approx(sum);
+          float c = (be * delta) * rr;
+          if (t >= nvalid) c = 0.f;  // padding tokens of the last chunk leave the state alone
+          cs[t & 15] = c;
+          if constexpr (RDEBUG) {
+            if (col_ok && t < nvalid) p.r_debug[((tok0 + (size_t)(t0 + t)) * J + j) * p.Dv + col] = rr;
+          }
+          if (t + 1 < C) pred[t + 1] = fmaf(c, Gkk[t * C + t + 1], pred[t + 1]);  // the push the next token waits for
+          c_prev = c;
+          if ((t & 15) == 15) {  // 16 update coefficients complete: park them in tensor memory (hi / lo)
+            float hi[16], lo[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) { hi[i] = tf32_hi(cs[i]); lo[i] = cs[i] - hi[i]; }
+            tmem_st16(tb + Cf::TM_CHI + (t - 15), hi);
+            tmem_st16(tb + Cf::TM_CLO + (t - 15), lo);
+          }
+        }
+        return bad;
+      };
+      {  // Q0 seeds the readout accumulator of this chunk
+#pragma unroll
+        for (int cc = 0; cc < C / 16; ++cc) {
+          float b[16];
+          tmem_ld16(tb + Cf::TM_PQ + C + cc * 16, b);
+          tmem_ld_wait();
+          tmem_st16(tb + Cf::TM_QD + (n & 1) * C + cc * 16, b);
+        }
       }
-
-      // ---- sequential part of the chunk: E-step and the triangular key-side corrections ----
-#pragma unroll
-      for (int t = 0; t < C; ++t) {
-        const float v = __bfloat162float(rv[t * COLS + dl]);
-        const float be = bes[t * NROW + r];
-        // serial chain: prediction error -> responsibilities (Eq. 3.4) -> update coefficient (Eq. 3.3)
-        const float delta = v - pred[t];
-        const float a = fmaf(-kHalfLog2e * delta, delta, lk[t]);
-        // softmax over the J components with the maximum subtracted (exact, never 0/0); every lane of the
-        // column gathers all J exponents and normalises redundantly: one shuffle round on the chain
-        float all[J];
-#pragma unroll
-        for (int jj = 0; jj < J; ++jj) all[jj] = __shfl_sync(0xffffffffu, a, jbase + jj);
-        float m = all[0];
-#pragma unroll
-        for (int jj = 1; jj < J; ++jj) m = fmaxf(m, all[jj]);
-        float sum = 0.f;
-#pragma unroll
-        for (int jj = 0; jj < J; ++jj) sum += ex2_approx(all[jj] - m);
-        const float e = ex2_approx(a - m);
-        const float rr = e * rcp_approx(sum);
-        float c = (be * delta) * rr;
-        if (t >= nvalid) c = 0.f;  // padding tokens of the last chunk leave the state alone
-        cs[t & 15] = c;
-        if constexpr (RDEBUG) {
-          if (col_ok && t < nvalid) p.r_debug[((tok0 + (size_t)(t0 + t)) * J + j) * p.Dv + col] = rr;
-        }
-        // push this token's update into the later predictions of the chunk
-#pragma unroll
-        for (int u = t + 1; u < C; ++u) pred[u] = fmaf(c, Gkk[t * C + u], pred[u]);
-        if ((t & 15) == 15) {  // 16 update coefficients complete: park them in tensor memory (hi / lo)
-          float hi[16], lo[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) { hi[i] = tf32_hi(cs[i]); lo[i] = cs[i] - hi[i]; }
-          tmem_st16(tb + Cf::TM_CHI + (t - 15), hi);
-          tmem_st16(tb + Cf::TM_CLO + (t - 15), lo);
-        }
+      const bool underflow = sequential(std::false_type{});
+      if (__any_sync(0xffffffffu, underflow)) {
+        tmem_st_wait();
+        sequential(std::true_type{});
       }
       tmem_st_wait();
       tc_fence_before_sync();
