@@ -74,7 +74,7 @@ enum {
   SWILA_ALGO_CHUNK = 4     /* chunked form: the state-times-token contractions of 32-token chunks
                               on the tcgen05 tensor cores (TF32 hi/lo split, FP32 accumulation in
                               tensor memory), the E-step and intra-chunk corrections on the FP32
-                              ALUs.  bf16 io, Dk in {64, 128}, J >= 2, no TEMPORAL / GATED */
+                              ALUs.  bf16 io, Dk in {64, 128}, J >= 4, no TEMPORAL / GATED */
 };
 
 typedef struct {

@@ -69,20 +69,22 @@ struct ChunkCfg {
   static constexpr int R_K = 0;
   static constexpr int R_Q = R_K + C * DK * ES;
   static constexpr int R_V = R_Q + C * DK * ES;
-  static constexpr int R_B = R_V + C * COLS * ES;
-  static constexpr int R_PK = R_B + C * J * COLS * ES;
+  static constexpr int R_B = R_V + C * COLS * ES;   // beta logits; the helpers overwrite them in place with
+                                                    // beta = sigmoid(.) as fp32 [C][NROW], hence the fp32-sized slot
+  static constexpr int R_PK = R_B + C * NROW * 4;
   static constexpr int RAW_BYTES = R_PK + C * J * COLS * ES;
   static constexpr int RPQ_BYTES = C * J * COLS * ES;
+  static constexpr int BQ_LBO = C * 16 + 16;        // padded K-chunk stride of the readout operand tiles (bank spread)
+  static constexpr int BQ_TILE = (C / 4) * BQ_LBO;
   static constexpr int C_K = DK * ES / 16, C_V = COLS * ES / 16;  // 16-byte units per token row / column slice
   // shared memory map (bytes)
   static constexpr int OFF_RAW = 0;
   static constexpr int OFF_RPQ = OFF_RAW + 2 * RAW_BYTES;  // 4-deep ring of query-prior logits
-  static constexpr int OFF_KQ = OFF_RPQ + 4 * RPQ_BYTES;   // [DK/4][2C][4] fp32: rows 0..C-1 = K, C..2C-1 = Q tokens
-  static constexpr int OFF_KT = OFF_KQ + 2 * C * DK * 4;   // [C/4][DK][4] fp32: K transposed (rows = key dims)
-  static constexpr int OFF_BE = OFF_KT + C * DK * 4;       // 2 x [C][NROW] fp32 beta = sigmoid(logit)
-  static constexpr int OFF_G = OFF_BE + 2 * C * NROW * 4;  // 2 x Gkk [C][C] fp32 (K K^T, for the row warps)
-  static constexpr int OFF_BQ = OFF_G + 2 * C * C * 4;     // 2 x { hi, lo } [C/4][C][4] fp32: masked (K Q^T)^T operand tiles
-  static constexpr int OFF_OST = OFF_BQ + 2 * 2 * C * C * 4;  // 2 x [C][COLS] bf16 output staging
+  static constexpr int OFF_KQ = OFF_RPQ + 4 * RPQ_BYTES;   // 2 x [DK/4][2C][4] fp32: rows 0..C-1 = K, C..2C-1 = Q tokens
+  static constexpr int OFF_KT = OFF_KQ + 2 * 2 * C * DK * 4;  // [C/4][DK][4] fp32: K transposed (rows = key dims)
+  static constexpr int OFF_G = OFF_KT + C * DK * 4;        // 2 x Gkk [C][C] fp32 (K K^T, for the row warps)
+  static constexpr int OFF_BQ = OFF_G + 2 * C * C * 4;     // 2 x { hi, lo } masked (K Q^T)^T operand tiles
+  static constexpr int OFF_OST = OFF_BQ + 2 * 2 * BQ_TILE; // 2 x [C][COLS] bf16 output staging
   static constexpr int OFF_BAR = OFF_OST + 2 * C * COLS * ES;
   static constexpr int SMEM_BYTES = OFF_BAR + 128;
   static_assert(RAW_BYTES % 16 == 0 && RPQ_BYTES % 16 == 0 && (COLS * ES) % 16 == 0, "alignment");
@@ -136,11 +138,10 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   using namespace umma;
   constexpr int J = Cf::J, DK = Cf::DK, C = Cf::C, NROW = Cf::NROW, COLS = Cf::COLS;
   extern __shared__ __align__(128) unsigned char smem[];
-  float *KQ = reinterpret_cast<float *>(smem + Cf::OFF_KQ);
+  float *KQ_all = reinterpret_cast<float *>(smem + Cf::OFF_KQ);
   float *Kt = reinterpret_cast<float *>(smem + Cf::OFF_KT);
-  float *be_all = reinterpret_cast<float *>(smem + Cf::OFF_BE);
   float *G_all = reinterpret_cast<float *>(smem + Cf::OFF_G);
-  float *BQ_all = reinterpret_cast<float *>(smem + Cf::OFF_BQ);
+  unsigned char *BQ_all = smem + Cf::OFF_BQ;
   __nv_bfloat16 *ostage = reinterpret_cast<__nv_bfloat16 *>(smem + Cf::OFF_OST);
   uint64_t *bars = reinterpret_cast<uint64_t *>(smem + Cf::OFF_BAR);
   uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(bars + B_COUNT);
@@ -223,7 +224,9 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         }
       }
       tc_fence_before_sync();
+      PROF_ADD(4, 0);
       named_bar_sync(2, 128);
+      PROF_ADD(5, 0);
       constexpr int GROUPS = COLS / 8;  // 8 outputs = 16 bytes per store
       for (int e = r; e < C * GROUPS; e += 128) {
         const int t = e / GROUPS, g8 = e - t * GROUPS;
@@ -231,6 +234,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
           *reinterpret_cast<uint4 *>((__nv_bfloat16 *)p.o + (tok0 + (size_t)(t0 + t)) * p.Dv + col0 + g8 * 8) =
               *reinterpret_cast<const uint4 *>(ost + t * COLS + g8 * 8);
       }
+      PROF_ADD(6, 0);
     };
 
     for (int n = 0; n < nchunks && !failed; ++n) {
@@ -240,26 +244,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       const __nv_bfloat16 *rv = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_V);
       const __nv_bfloat16 *rpk = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_PK);
       const float *Gkk = G_all + (n & 1) * C * C;
-      const float *bes = be_all + (n & 1) * C * NROW;
-
-      // key-prior logits of this row, base 2, shifted by their maximum over the J components (the softmax
-      // of the E-step is shift-invariant; with the shift every exponent a_j = lk_j - delta_j^2 log2(e)/2 is
-      // <= 0).  Raw stage n is in place: the hand-over of chunk n-1 waited for it.  Grouped so the
-      // shuffles of different tokens overlap.
-      float lk[C];
-#pragma unroll
-      for (int tg = 0; tg < C; tg += 8) {
-        float m[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) { lk[tg + i] = __bfloat162float(rpk[((tg + i) * J + j) * COLS + dl]) * kLog2e; m[i] = lk[tg + i]; }
-#pragma unroll
-        for (int off = 1; off < J; off <<= 1) {
-#pragma unroll
-          for (int i = 0; i < 8; ++i) m[i] = fmaxf(m[i], __shfl_xor_sync(0xffffffffu, m[i], off));
-        }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) lk[tg + i] -= m[i];
-      }
+      const float *bes = reinterpret_cast<const float *>(raw + Cf::R_B);
 
       PROF_ADD(0, 0);
       if (!mbar_wait(&bars[B_E], n & 1)) { failed = true; break; }
@@ -268,9 +253,9 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       // ---- sequential part of the chunk: E-step and the triangular key-side corrections.  Only one FMA
       //      of a token's push (into the next token's prediction) sits on the serial chain; the rest is
       //      deferred into the shuffle latency of the next token's E-step.
-      //      FAST: exponents are taken without a per-token maximum (they are <= 0 after the prior shift);
-      //      the pass reports whether any normaliser underflowed -- every component > ~13 standard
-      //      deviations off -- in which case the chunk is redone with the per-token maximum subtracted. ----
+      //      FAST: exponentials are taken without subtracting the per-token maximum; the pass reports whether
+      //      any normaliser left the safe range (all components > ~13 standard deviations off, or extreme
+      //      prior logits), in which case the chunk is redone with the maximum subtracted. ----
       auto sequential = [&](auto exact_tag) -> bool {
         constexpr bool EXACT = decltype(exact_tag)::value;
         bool bad = false;
@@ -290,7 +275,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
           const float be = bes[t * NROW + r];
           // serial chain: prediction error -> responsibilities (Eq. 3.4) -> update coefficient (Eq. 3.3)
           const float delta = v - pred[t];
-          const float a = fmaf(-kHalfLog2e * delta, delta, lk[t]);
+          const float a = fmaf(-kHalfLog2e * delta, delta, __bfloat162float(rpk[(t * J + j) * COLS + dl]) * kLog2e);
           float e, sum;
           if constexpr (EXACT) {
             float all[J];
@@ -308,7 +293,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
             sum = e;
 #pragma unroll
             for (int jj = 1; jj < J; ++jj) sum += __shfl_sync(0xffffffffu, e, jbase + ((j + jj) & (J - 1)));
-            bad = bad || !(sum > 1e-30f);
+            bad = bad || !(sum > 1e-30f && sum < 1e30f);
           }
           if (t >= 1) {  // deferred push of token t-1 into the predictions of tokens t+1 ..
 #pragma unroll
@@ -384,7 +369,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     const bool col_ok = col < p.Dv;
 
     // K, Q of a raw stage -> stacked fp32 operand tile (16-byte unit (row, k-chunk c) at (c*2C + row)*16)
-    auto cook_kq = [&](const unsigned char *raw) {
+    auto cook_kq = [&](const unsigned char *raw, float *KQ) {
       const __nv_bfloat16 *rk = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_K);
       const __nv_bfloat16 *rq = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_Q);
       // diagonal walk over 8-token x 16-chunk blocks: conflict-free 8-byte reads and 16-byte writes
@@ -419,11 +404,17 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         *reinterpret_cast<float4 *>(Kt + (c4 * DK + dd) * 4) = f;
       }
     };
-    // beta = sigmoid(logit) of this helper's row for every token of a raw stage (App. B.2)
-    auto cook_be = [&](const unsigned char *raw, float *bes) {
+    // beta = sigmoid(logit) of this helper's row for every token of a raw stage (App. B.2), written over the
+    // logits: all helpers read their logits first, then all write
+    auto cook_be = [&](unsigned char *raw) {
       const __nv_bfloat16 *rb = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_B);
-#pragma unroll 8
-      for (int t = 0; t < C; ++t) bes[t * NROW + h] = sigmoid_approx(__bfloat162float(rb[(t * J + j) * COLS + dl]));
+      float *bes = reinterpret_cast<float *>(raw + Cf::R_B);
+      float be[C];
+#pragma unroll
+      for (int t = 0; t < C; ++t) be[t] = sigmoid_approx(__bfloat162float(rb[(t * J + j) * COLS + dl]));
+      named_bar_sync(3, 128);
+#pragma unroll
+      for (int t = 0; t < C; ++t) bes[t * NROW + h] = be[t];
     };
     // low part of W after an update: W_lo = W - hi(W), this helper's tensor-memory lane
     auto refresh_wlo = [&]() {
@@ -448,8 +439,8 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     // = earlier token s = this lane), causally masked (s <= t), split into hi / lo TF32 parts
     auto spill_gram = [&](int n) {
       float *Gkk = G_all + (n & 1) * C * C;
-      float *Bhi = BQ_all + (n & 1) * 2 * C * C;
-      float *Blo = Bhi + C * C;
+      float *Bhi = reinterpret_cast<float *>(BQ_all + (n & 1) * 2 * Cf::BQ_TILE);
+      float *Blo = reinterpret_cast<float *>(BQ_all + (n & 1) * 2 * Cf::BQ_TILE + Cf::BQ_TILE);
 #pragma unroll
       for (int cc = 0; cc < C / 16; ++cc) {
         float a[16], b[16];
@@ -464,7 +455,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
           const int t = cc * 16 + i;
           const float val = (lane <= t) ? b[i] : 0.f;
           const float hi = tf32_hi(val);
-          const int idx = ((lane >> 2) * C + t) * 4 + (lane & 3);
+          const int idx = (lane >> 2) * (Cf::BQ_LBO / 4) + t * 4 + (lane & 3);
           Bhi[idx] = hi;
           Blo[idx] = val - hi;
         }
@@ -501,8 +492,8 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     }
     cp_async_wait<1>();
     named_bar_sync(1, 128);  // every helper's copies of chunk 0 have landed
-    cook_kq(smem + Cf::OFF_RAW);
-    cook_be(smem + Cf::OFF_RAW, be_all);
+    cook_kq(smem + Cf::OFF_RAW, KQ_all);
+    cook_be(smem + Cf::OFF_RAW);
     fence_async_smem();
     mbar_arrive(&bars[B_KQ]);
     cook_kt(smem + Cf::OFF_RAW);
@@ -517,16 +508,14 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
 
     for (int n = 0; n < nchunks && !failed; ++n) {
       const bool more = n + 1 < nchunks;
-      const unsigned char *raw_next = smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES;
-      // (1) E(n) is done: the K/Q tile is free again
-      if (!mbar_wait(&bars[B_E], n & 1)) { failed = true; break; }
-      tc_fence_after_sync();
-      // (2) operands of chunk n+1 (its raw stage has landed)
+      unsigned char *raw_next = smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES;
+      // (1) operands of chunk n+1: its raw stage has landed, and the K/Q tile it goes to was last read by
+      //     the MMAs of chunk n-1, which completed before the update of chunk n-1 this warp waited for
       cp_async_wait<0>();
       named_bar_sync(1, 128);
       if (more) {
-        cook_kq(raw_next);
-        cook_be(raw_next, be_all + ((n + 1) & 1) * C * NROW);
+        cook_kq(raw_next, KQ_all + ((n + 1) & 1) * 2 * C * DK);
+        cook_be(raw_next);
         fence_async_smem();
         mbar_arrive(&bars[B_KQ]);
         if (warp == 4) {  // Gram matrices of chunk n+1
@@ -537,10 +526,10 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         }
       }
       
-      PROF_ADD(4, 128);
+      
       // (3) chunk n is finished by the row warps: stage chunk n+2 into the buffers chunk n used
       if (!mbar_wait(&bars[B_C], n & 1)) { failed = true; break; }
-      PROF_ADD(5, 128);
+      
       
       if (n + 2 < nchunks)
         chunk_issue_raw<Cf>(p, smem + Cf::OFF_RAW + (n & 1) * Cf::RAW_BYTES, smem + Cf::OFF_RPQ + ((n + 2) & 3) * Cf::RPQ_BYTES,
@@ -564,9 +553,11 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     // =============================== MMA issuer ==============================================
     constexpr uint32_t idE = idesc_tf32(128, 2 * C);  // [P0 | Q0] and [Gkk | Gkq]: N = 2C
     constexpr uint32_t idU = idesc_tf32(128, DK);
-    const uint64_t kq0 = smem_desc_kmajor(smem_u32(KQ), 2 * C * 16, 128);
+    const uint64_t kq_desc[2] = {smem_desc_kmajor(smem_u32(KQ_all), 2 * C * 16, 128),
+                                 smem_desc_kmajor(smem_u32(KQ_all + 2 * C * DK), 2 * C * 16, 128)};
     const uint64_t kt0 = smem_desc_kmajor(smem_u32(Kt), DK * 16, 128);
-    auto gram = [&]() {
+    auto gram = [&](int chunk) {
+      const uint64_t kq0 = kq_desc[chunk & 1];
 #pragma unroll 1
       for (int ks = 0; ks < DK / 8; ++ks) {
         const uint64_t d = kq0 + (uint64_t)(ks * 2 * 2 * C);  // start address advances in 16-byte units
@@ -574,7 +565,8 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       }
       mma_commit(&bars[B_G]);
     };
-    auto w_times_kq = [&](int w_col, bool first) {
+    auto w_times_kq = [&](int chunk, int w_col, bool first) {
+      const uint64_t kq0 = kq_desc[chunk & 1];
 #pragma unroll 1
       for (int ks = 0; ks < DK / 8; ++ks)
         mma_tf32_ts(tb0 + Cf::TM_PQ, tb0 + w_col + ks * 8, kq0 + (uint64_t)(ks * 2 * 2 * C), idE, !(first && ks == 0));
@@ -582,12 +574,12 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     constexpr uint32_t idQ = idesc_tf32(128, C);
     // readouts of chunk n: QD += Cmat (K Q^T masked)  -- c_hi B_hi + c_lo B_hi + c_hi B_lo
     auto readout = [&](int n) {
-      const uint64_t bh0 = smem_desc_kmajor(smem_u32(BQ_all + (n & 1) * 2 * C * C), C * 16, 128);
-      const uint64_t bl0 = smem_desc_kmajor(smem_u32(BQ_all + (n & 1) * 2 * C * C + C * C), C * 16, 128);
+      const uint64_t bh0 = smem_desc_kmajor(smem_u32(BQ_all + (n & 1) * 2 * Cf::BQ_TILE), Cf::BQ_LBO, 128);
+      const uint64_t bl0 = smem_desc_kmajor(smem_u32(BQ_all + (n & 1) * 2 * Cf::BQ_TILE + Cf::BQ_TILE), Cf::BQ_LBO, 128);
       const uint32_t d = tb0 + Cf::TM_QD + (n & 1) * C;
 #pragma unroll 1
       for (int ks = 0; ks < C / 8; ++ks) {
-        const uint64_t adv = (uint64_t)(ks * 2 * C);
+        const uint64_t adv = (uint64_t)(ks * 2 * (Cf::BQ_LBO / 16));
         mma_tf32_ts(d, tb0 + Cf::TM_CHI + ks * 8, bh0 + adv, idQ, true);
         mma_tf32_ts(d, tb0 + Cf::TM_CLO + ks * 8, bh0 + adv, idQ, true);
         mma_tf32_ts(d, tb0 + Cf::TM_CHI + ks * 8, bl0 + adv, idQ, true);
@@ -596,12 +588,12 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     };
     if (!mbar_wait(&bars[B_KQ], 0)) failed = true;
     tc_fence_after_sync();
-    if (!failed) gram();
+    if (!failed) gram(0);
     if (!failed && !mbar_wait(&bars[B_WLO], 0)) failed = true;
     tc_fence_after_sync();
     if (!failed) {
-      w_times_kq(Cf::TM_W, true);
-      w_times_kq(Cf::TM_WLO, false);
+      w_times_kq(0, Cf::TM_W, true);
+      w_times_kq(0, Cf::TM_WLO, false);
       mma_commit(&bars[B_E]);
     }
     for (int n = 0; n < nchunks && !failed; ++n) {
@@ -609,7 +601,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       if (more) {
         if (!mbar_wait(&bars[B_KQ], (n + 1) & 1)) { failed = true; break; }
         tc_fence_after_sync();
-        gram();
+        gram(n + 1);
       }
       if (!mbar_wait(&bars[B_C], n & 1) || !mbar_wait(&bars[B_KT], n & 1)) { failed = true; break; }
       tc_fence_after_sync();
@@ -621,10 +613,10 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       }
       mma_commit(&bars[B_U]);
       if (more) {
-        w_times_kq(Cf::TM_W, true);  // executes after the update: MMAs of one thread run in order
+        w_times_kq(n + 1, Cf::TM_W, true);  // executes after the update: MMAs of one thread run in order
         if (!mbar_wait(&bars[B_WLO], (n + 1) & 1)) { failed = true; break; }
         tc_fence_after_sync();
-        w_times_kq(Cf::TM_WLO, false);
+        w_times_kq(n + 1, Cf::TM_WLO, false);
         mma_commit(&bars[B_E]);
       }
       readout(n);  // not needed before the outputs are formed one chunk later: off the critical path

@@ -1,5 +1,5 @@
 // Instantiations and dispatch of the chunked tensor-core kernel (bf16 io, ungated, non-temporal,
-// J in {2, 4, 8}: with one component the shared-memory tiles of a 128-column block do not fit).
+// J in {4, 8}: with fewer components a block covers more columns and its shared-memory tiles do not fit).
 #include "swila_chunk.cuh"
 
 namespace swila {
@@ -13,7 +13,6 @@ int chunk_dispatch(const LaunchArgs &a) {
     if (a.Dk == 64) return launch_chunk<JJ, 64>(a);   \
     return -1000;
   switch (a.J) {
-    SWILA_CHUNK_CASE(2)
     SWILA_CHUNK_CASE(4)
     SWILA_CHUNK_CASE(8)
     default: return -1000;
