@@ -246,7 +246,7 @@ __device__ __forceinline__ void flush_o(const ScanParams &p, const unsigned char
 }
 
 // ---- the kernel ---------------------------------------------------------------------------
-template <class C, bool POST>
+template <class C, bool POST, bool RDEBUG>
 __global__ void __launch_bounds__(C::NT, C::MIN_BLOCKS) swila_scan_kernel(const __grid_constant__ ScanParams p) {
   using IO = typename C::IO;
   constexpr int J = C::J, DK = C::DK, NT = C::NT, TB = C::TB, GATE = C::GATE;
@@ -393,9 +393,11 @@ __global__ void __launch_bounds__(C::NT, C::MIN_BLOCKS) swila_scan_kernel(const 
           pq[j] = rho[j];
         }
       }
-      if (p.r_debug != nullptr && g == 0 && col_ok) {
+      if constexpr (RDEBUG) {  // compile-time: a run-time test here would sit on every token's serial chain
+        if (g == 0 && col_ok) {
 #pragma unroll
-        for (int j = 0; j < J; ++j) p.r_debug[((tok0 + (size_t)(t0 + s)) * J + j) * p.Dv + col] = rr[j];
+          for (int j = 0; j < J; ++j) p.r_debug[((tok0 + (size_t)(t0 + s)) * J + j) * p.Dv + col] = rr[j];
+        }
       }
 
       // ---- pass B: M-step (Eq. 3.3 / 3.7) and readout on the updated state (Eq. 3.5) ----
@@ -462,7 +464,7 @@ int launch_scan(const LaunchArgs &a) {
   using IO = typename C::IO;
   constexpr int J = C::J, DK = C::DK, NT = C::NT, TB = C::TB, GATE = C::GATE;
   (void)J; (void)DK; (void)NT; (void)TB; (void)GATE;
-  auto kern = swila_scan_kernel<C, POST>;
+  auto kern = a.p.r_debug ? swila_scan_kernel<C, POST, true> : swila_scan_kernel<C, POST, false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
   if (e != cudaSuccess) return (int)e;
   const long long nslice = (a.p.Dv + C::COLS - 1) / C::COLS;
