@@ -230,6 +230,46 @@ def decode_leg(binding, args, stream, dev_index):
     }
 
 
+def paper_shapes_leg(binding, stream):
+    """Shapes the paper quotes (not the headline): the 374M LM layer (H=8, J=4, D=64) at B=16, T=4096
+    (App. C), and the generation protocol of App. D.4 (2048-token prompt + 128 decoded tokens) at several
+    batch sizes; generation time includes prefill and decode, as in the paper."""
+    out = {}
+    lm = wl.CONFIGS[1].with_(name="lm374m_layer", B=16, H=8, T=4096)
+    inp = wl.make_inputs(lm, device="cuda")
+    st = binding.state_alloc(lm, init=False)
+    o = torch.empty((lm.B, lm.H, lm.T, lm.Dv), device="cuda", dtype=lm.torch_io_dtype)
+    f = lambda: binding.swila_forward(lm, inp, state_in=None, state_out=st, o=o)
+    for _ in range(3):
+        f()
+    torch.cuda.synchronize()
+    ms = time_steps(f, 10, stream) / 10
+    out["lm374m_layer_prefill"] = {"B": lm.B, "H": lm.H, "T": lm.T, "D": lm.Dk, "J": lm.J, "ms": ms,
+                                   "tokens_per_s": lm.B * lm.T / (ms * 1e-3)}
+    del inp, o, st
+    gen_out = []
+    for B in (1, 8, 128):
+        g = wl.CONFIGS[1].with_(name="generation", B=B, H=8, T=2048)
+        prompt = wl.make_inputs(g, device="cuda")
+        steps = [wl.decode_step_inputs(g, s, device="cuda") for s in range(128)]
+        st = binding.state_alloc(g)
+        o = torch.empty((g.B, g.H, g.T, g.Dv), device="cuda", dtype=g.torch_io_dtype)
+        o1 = torch.empty((g.B, g.H, 1, g.Dv), device="cuda", dtype=g.torch_io_dtype)
+
+        def generate():
+            binding.swila_forward(g, prompt, state_in=None, state_out=st, o=o)
+            for s in range(128):
+                binding.swila_decode_step(g, steps[s], st, o=o1)
+
+        generate()
+        torch.cuda.synchronize()
+        ms = time_steps(generate, 3, stream) / 3
+        gen_out.append({"batch": B, "ms_per_call": ms, "tokens_per_s": B * (2048 + 128) / (ms * 1e-3)})
+    out["generation_2048_plus_128"] = {"H": 8, "D": 64, "J": 4, "runs": gen_out,
+                                       "note": "one layer's recurrence only; 1 warm-up + 3 timed calls"}
+    return out
+
+
 def _peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -250,6 +290,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     ap.add_argument("--no-scan", action="store_true", help="skip the scan-kernel comparison leg")
+    ap.add_argument("--paper-shapes", action="store_true", help="also time the shapes the paper itself quotes")
     ap.add_argument("--decode-steps", type=int, default=wl.DECODE_STEPS)
     ap.add_argument("--decode-prefill", type=int, default=4096)
     ap.add_argument("--decode-batch", type=int, default=0, help="override B of the decode leg (0 = 256)")
@@ -401,6 +442,8 @@ def main():
         decode = decode_leg(binding, args, stream, local)
         torch.cuda.empty_cache()
 
+    paper = paper_shapes_leg(binding, stream) if args.paper_shapes else None
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
         n_bh = 32
@@ -419,7 +462,7 @@ def main():
                        "l2": "inputs (2.1 GB) larger than L2; no flush needed",
                        "multi_gpu": "independent replicas, no collective"},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": args.steps,
-            "clocks": clocks, "decode": decode, "scan": scan,
+            "clocks": clocks, "decode": decode, "scan": scan, "paper_shapes": paper,
         }
         print(json.dumps(line))
     if world > 1:

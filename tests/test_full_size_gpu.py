@@ -95,3 +95,35 @@ def test_batched_decode_config_sampled(binding, oracle):
     # decode outputs alone (the last n_decode tokens)
     e_dec = wl.rel_err(o[:, :, -n_decode:], torch.from_numpy(ref["o"][:, :, -n_decode:]))
     assert e_o < TOL_BF16_O and e_dec < TOL_BF16_O and e_w < TOL_STATE, (e_o, e_dec, e_w)
+
+
+def test_paper_native_shapes(binding, oracle):
+    """Shapes the paper itself quotes: the 374M language-model layer (H=8, J=4, D=64) at B=16, T=4096
+    (App. C), and the generation protocol of App. D.4 -- a 2048-token prompt followed by 128 decoded
+    tokens -- at batch 8.  Sampled rows are replayed by the oracle."""
+    lm = wl.CONFIGS[1].with_(name="lm374m_layer", B=16, H=8, T=4096)
+    inp = wl.make_inputs(lm, device="cuda", stress=True)
+    st = binding.state_alloc(lm, init=False)
+    o = binding.swila_forward(lm, inp, state_in={"W": inp["W0"]}, state_out=st)
+    torch.cuda.synchronize()
+    bh, cols = _sample(lm, 8, 16, seed=11)
+    _check_sample(lm, oracle, inp, o, st["W"], bh, cols, lm.name)
+
+    gen = wl.CONFIGS[1].with_(name="generation", B=8, H=8, T=2048)
+    bh, cols = _sample(gen, 8, 8, seed=12)
+    prompt = wl.make_inputs(gen, device="cuda")
+    st = binding.state_alloc(gen)
+    outs = [binding.swila_forward(gen, prompt, state_in=st, state_out=st)]
+    hist = [wl.slice_rows(prompt, bh.cuda(), cols.cuda())]
+    for s in range(128):
+        step = wl.decode_step_inputs(gen, s, device="cuda")
+        outs.append(binding.swila_decode_step(gen, step, st))
+        hist.append(wl.slice_rows(step, bh.cuda(), cols.cuda()))
+    torch.cuda.synchronize()
+    names = ("q", "k", "v", "beta_logit", "pik_logit", "piq_logit")
+    full = {n: torch.cat([h[n].cpu() for h in hist], dim=2) for n in names}
+    ref = oracle.forward(full["q"], full["k"], full["v"], full["beta_logit"], full["pik_logit"], full["piq_logit"])
+    o = torch.cat(outs, dim=2).reshape(gen.B * gen.H, -1, gen.Dv)[bh.cuda()][..., cols.cuda()].unsqueeze(1).cpu()
+    W = st["W"].reshape(gen.B * gen.H, gen.J, gen.Dv, gen.Dk)[bh.cuda()][:, :, cols.cuda()].unsqueeze(1).cpu()
+    assert wl.rel_err(o, torch.from_numpy(ref["o"])) < TOL_BF16_O
+    assert wl.rel_err(W, torch.from_numpy(ref["W"])) < TOL_STATE
