@@ -112,6 +112,23 @@ class ClockSampler:
         return out
 
 
+def max_over_ranks(ms: float, world: int, device="cpu") -> float:
+    """The slowest rank's time: every multi-GPU number is the maximum over ranks (all-reduce MAX on
+    whatever process group is initialised; identity for a single process)."""
+    if world <= 1:
+        return float(ms)
+    import torch.distributed as dist
+
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_s(world: int, B: int, T: int, ms_per_step: float) -> float:
+    """Independent replicas (weak scaling): every rank processes its own B x T tokens per step."""
+    return world * B * T / (ms_per_step * 1e-3)
+
+
 def time_steps(fn, steps: int, stream) -> float:
     """Milliseconds for `steps` back-to-back calls of fn, CUDA events on `stream`."""
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -344,12 +361,9 @@ def main():
     ms = time_steps(step, args.steps, stream)
     barrier()
     clocks = sampler.stop()
-    if world > 1:
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, world, "cuda")
     ms_per_step = ms / args.steps
-    value = world * w.B * w.T / (ms_per_step * 1e-3)
+    value = whole_job_tokens_per_s(world, w.B, w.T, ms_per_step)
 
     # ---- roofline of the kernel the step launches (one launch per step) ----
     props = torch.cuda.get_device_properties(local)
@@ -424,13 +438,10 @@ def main():
         barrier()
         ms_e = time_steps(step_host, n_e2e, stream)
         barrier()
-        if world > 1:
-            t = torch.tensor([ms_e], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e = float(t.item())
+        ms_e = max_over_ranks(ms_e, world, "cuda")
         h2d = sum(host[n].numel() * host[n].element_size() for n in names)
         d2h = o_host.numel() * o_host.element_size()
-        e2e = {"value": world * w.B * w.T / (ms_e / n_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        e2e = {"value": whole_job_tokens_per_s(world, w.B, w.T, ms_e / n_e2e), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h, "ms_per_step": ms_e / n_e2e, "steps": n_e2e,
                "note": "swila_forward_host: pinned host inputs -> device workspace -> kernel -> o to pinned host"}
         del host, o_host, ws
