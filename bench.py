@@ -34,10 +34,9 @@ METRIC = "swila_fwd_tokens_per_s"
 UNIT = "tokens/s"
 HEADLINE = 2  # config index of the workload the metric is quoted on
 
-# DRAM traffic of one launch on the headline workload, from the ncu captures summarised in
-# profiles/chunk_lm_prefill.md and profiles/scan_lm_prefill.md (dram__bytes_read.sum +
-# dram__bytes_write.sum; 2.186 GB chunked, 2.188 GB scan).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 2.186e9
+# DRAM traffic of one launch on the headline workload, from the ncu captures summarised under
+# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum: 2.174 GB chunked kernel, 2.188 GB scan kernel).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 2.174e9
 
 
 # ----------------------------------------------------------------------------------------------
@@ -388,7 +387,7 @@ def main():
             "tensor_bound": {"achieved_tflops": flops / sec / 1e12, "peak_tflops": tf32_peak,
                              "frac": flops / sec / 1e12 / tf32_peak,
                              "peak_source": "measured bf16 peak x nominal TF32/bf16 ratio 0.5"},
-            "note": "latency-bound: T tokens are a serial dependency chain per row; see DESIGN.md",
+            "note": "latency-bound: the T tokens of a row are a serial dependency chain (~180 cycles per token)",
         }
     else:
         ach_tflops = flops / sec / 1e12
