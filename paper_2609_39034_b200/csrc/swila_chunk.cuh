@@ -42,6 +42,7 @@ namespace swila {
 static __device__ int g_chunk_error = 0;
 #ifdef SWILA_CHUNK_PROFILE
 static __device__ long long g_chunk_prof[8];
+static __device__ long long g_chunk_blk[3 * 1024];  // per block: cycles, SM id, start time (ns)
 #define PROF_ADD(i, who) do { if (tid == (who) && blockIdx.x == 0) { long long now_ = clock64(); g_chunk_prof[i] += now_ - prof_t; prof_t = now_; } } while (0)
 #else
 #define PROF_ADD(i, who) do {} while (0)
@@ -51,6 +52,7 @@ template <int J_, int DK_>
 struct ChunkCfg {
   static constexpr int J = J_, DK = DK_;
   static constexpr int C = 32;            // tokens per chunk
+  static constexpr int GT = 8;            // tokens per trip of the row warps' rolled serial loop
   static constexpr int NROW = 128;        // row threads = rows of the tile
   static constexpr int NT = 288;          // 4 row warps + 4 helper warps + 1 MMA warp
   static constexpr int COLS = NROW / J;   // output columns per block
@@ -174,6 +176,15 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   bool failed = false;
 #ifdef SWILA_CHUNK_PROFILE
   long long prof_t = clock64();
+  const long long prof_t0 = prof_t;
+  if (tid == 0 && blockIdx.x < 1024) {
+    unsigned smid;
+    unsigned long long ns;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns));
+    g_chunk_blk[1024 + blockIdx.x] = smid;
+    g_chunk_blk[2048 + blockIdx.x] = (long long)ns;
+  }
 #endif
 
   if (warp < 4) {
@@ -192,35 +203,31 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       const __nv_bfloat16 *rpq = reinterpret_cast<const __nv_bfloat16 *>(smem + Cf::OFF_RPQ + (n & 3) * Cf::RPQ_BYTES);
       __nv_bfloat16 *ost = ostage + (n & 1) * C * COLS;
       tc_fence_after_sync();
+#pragma unroll 1
+      for (int tg = 0; tg < C; tg += 8) {  // rolled: the loop body stays resident in the instruction cache
+        float qd[8], x[8], m[8], e[8], o[8];
+        tmem_ld8(tb + Cf::TM_QD + (n & 1) * C + tg, qd);
 #pragma unroll
-      for (int tg = 0; tg < C; tg += 16) {
-        float qd[16];
-        tmem_ld16(tb + Cf::TM_QD + (n & 1) * C + tg, qd);
+        for (int i = 0; i < 8; ++i) { x[i] = __bfloat162float(rpq[((tg + i) * J + j) * COLS + dl]) * kLog2e; m[i] = x[i]; }
+#pragma unroll
+        for (int off = 1; off < J; off <<= 1) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) m[i] = fmaxf(m[i], __shfl_xor_sync(0xffffffffu, m[i], off));
+        }
         tmem_ld_wait();
 #pragma unroll
-        for (int th = 0; th < 16; th += 8) {
-          float x[8], m[8], e[8], o[8];
+        for (int i = 0; i < 8; ++i) { e[i] = ex2_approx(x[i] - m[i]); o[i] = e[i] * qd[i]; }
 #pragma unroll
-          for (int i = 0; i < 8; ++i) { x[i] = __bfloat162float(rpq[((tg + th + i) * J + j) * COLS + dl]) * kLog2e; m[i] = x[i]; }
+        for (int off = 1; off < J; off <<= 1) {
 #pragma unroll
-          for (int off = 1; off < J; off <<= 1) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) m[i] = fmaxf(m[i], __shfl_xor_sync(0xffffffffu, m[i], off));
+          for (int i = 0; i < 8; ++i) {
+            e[i] += __shfl_xor_sync(0xffffffffu, e[i], off);
+            o[i] += __shfl_xor_sync(0xffffffffu, o[i], off);
           }
+        }
+        if (j == 0) {
 #pragma unroll
-          for (int i = 0; i < 8; ++i) { e[i] = ex2_approx(x[i] - m[i]); o[i] = e[i] * qd[th + i]; }
-#pragma unroll
-          for (int off = 1; off < J; off <<= 1) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-              e[i] += __shfl_xor_sync(0xffffffffu, e[i], off);
-              o[i] += __shfl_xor_sync(0xffffffffu, o[i], off);
-            }
-          }
-          if (j == 0) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) ost[(tg + th + i) * COLS + dl] = __float2bfloat16_rn(o[i] * rcp_approx(e[i]));
-          }
+          for (int i = 0; i < 8; ++i) ost[(tg + i) * COLS + dl] = __float2bfloat16_rn(o[i] * rcp_approx(e[i]));
         }
       }
       tc_fence_before_sync();
@@ -237,6 +244,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       PROF_ADD(6, 0);
     };
 
+#pragma unroll 1
     for (int n = 0; n < nchunks && !failed; ++n) {
       const int t0 = n * C;
       const int nvalid = min(C, p.T - t0);
@@ -258,8 +266,11 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       //      prior logits), in which case the chunk is redone with the maximum subtracted. ----
       auto sequential = [&](auto exact_tag) -> bool {
         constexpr bool EXACT = decltype(exact_tag)::value;
+        constexpr int GT = Cf::GT;
         bool bad = false;
-        float pred[C], cs[16];
+        // pred[i]: prediction of token tg + i of the current trip (slots past the chunk end are dead weight that
+        // keeps the trip's code independent of tg); slot C takes the last token's push
+        float pred[C + 1];
 #pragma unroll
         for (int cc = 0; cc < C / 16; ++cc) {
           float a[16];
@@ -268,53 +279,75 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
 #pragma unroll
           for (int i = 0; i < 16; ++i) pred[cc * 16 + i] = a[i];
         }
+        pred[C] = 0.f;
         float c_prev = 0.f;
+#pragma unroll 1
+        for (int tg = 0; tg < C; tg += GT) {  // rolled: GT tokens of straight-line code stay in the instruction cache
+          float cs[GT];
 #pragma unroll
-        for (int t = 0; t < C; ++t) {
-          const float v = __bfloat162float(rv[t * COLS + dl]);
-          const float be = bes[t * NROW + r];
-          // serial chain: prediction error -> responsibilities (Eq. 3.4) -> update coefficient (Eq. 3.3)
-          const float delta = v - pred[t];
-          const float a = fmaf(-kHalfLog2e * delta, delta, __bfloat162float(rpk[(t * J + j) * COLS + dl]) * kLog2e);
-          float e, sum;
-          if constexpr (EXACT) {
-            float all[J];
+          for (int i = 0; i < GT; ++i) {
+            const int t = tg + i;
+            const float v = __bfloat162float(rv[t * COLS + dl]);
+            const float be = bes[t * NROW + r];
+            // serial chain: prediction error -> responsibilities (Eq. 3.4) -> update coefficient (Eq. 3.3)
+            const float delta = v - pred[i];
+            const float a = fmaf(-kHalfLog2e * delta, delta, __bfloat162float(rpk[(t * J + j) * COLS + dl]) * kLog2e);
+            float e, sum;
+            if constexpr (EXACT) {
+              float all[J];
 #pragma unroll
-            for (int jj = 0; jj < J; ++jj) all[jj] = __shfl_sync(0xffffffffu, a, jbase + jj);
-            float m = all[0];
+              for (int jj = 0; jj < J; ++jj) all[jj] = __shfl_sync(0xffffffffu, a, jbase + jj);
+              float m = all[0];
 #pragma unroll
-            for (int jj = 1; jj < J; ++jj) m = fmaxf(m, all[jj]);
-            sum = 0.f;
+              for (int jj = 1; jj < J; ++jj) m = fmaxf(m, all[jj]);
+              sum = 0.f;
 #pragma unroll
-            for (int jj = 0; jj < J; ++jj) sum += ex2_approx(all[jj] - m);
-            e = ex2_approx(a - m);
-          } else {
-            e = ex2_approx(a);
-            sum = e;
+              for (int jj = 0; jj < J; ++jj) sum += ex2_approx(all[jj] - m);
+              e = ex2_approx(a - m);
+            } else {
+              e = ex2_approx(a);
+              sum = e;
 #pragma unroll
-            for (int jj = 1; jj < J; ++jj) sum += __shfl_sync(0xffffffffu, e, jbase + ((j + jj) & (J - 1)));
-            bad = bad || !(sum > 1e-30f && sum < 1e30f);
+              for (int jj = 1; jj < J; ++jj) sum += __shfl_sync(0xffffffffu, e, jbase + ((j + jj) & (J - 1)));
+              bad = bad || !(sum > 1e-30f && sum < 1e30f);
+            }
+            {  // deferred push of token t-1 into the predictions of tokens t+1 .. (slots i+1 ..)
+              const float4 *gp = reinterpret_cast<const float4 *>(Gkk + max(t - 1, 0) * C + tg);
+#pragma unroll
+              for (int u4 = (i + 1) / 4; u4 < C / 4; ++u4) {
+                const float4 g = gp[u4];
+                if (4 * u4 + 0 > i) pred[4 * u4 + 0] = fmaf(c_prev, g.x, pred[4 * u4 + 0]);
+                if (4 * u4 + 1 > i) pred[4 * u4 + 1] = fmaf(c_prev, g.y, pred[4 * u4 + 1]);
+                if (4 * u4 + 2 > i) pred[4 * u4 + 2] = fmaf(c_prev, g.z, pred[4 * u4 + 2]);
+                if (4 * u4 + 3 > i) pred[4 * u4 + 3] = fmaf(c_prev, g.w, pred[4 * u4 + 3]);
+              }
+            }
+            const float rr = e * rcp_approx(sum);
+            float c = (be * delta) * rr;
+            if (t >= nvalid) c = 0.f;  // padding tokens of the last chunk leave the state alone
+            cs[i] = c;
+            if constexpr (RDEBUG) {
+              if (col_ok && t < nvalid) p.r_debug[((tok0 + (size_t)(t0 + t)) * J + j) * p.Dv + col] = rr;
+            }
+            pred[i + 1] = fmaf(c, Gkk[t * C + t + 1], pred[i + 1]);  // the push the next token waits for
+            c_prev = c;
           }
-          if (t >= 1) {  // deferred push of token t-1 into the predictions of tokens t+1 ..
+          {  // GT update coefficients complete: park them in tensor memory (hi / lo)
+            float hi[GT], lo[GT];
 #pragma unroll
-            for (int u = t + 1; u < C; ++u) pred[u] = fmaf(c_prev, Gkk[(t - 1) * C + u], pred[u]);
+            for (int i = 0; i < GT; ++i) { hi[i] = tf32_hi(cs[i]); lo[i] = cs[i] - hi[i]; }
+            if constexpr (GT == 8) {
+              tmem_st8(tb + Cf::TM_CHI + tg, hi);
+              tmem_st8(tb + Cf::TM_CLO + tg, lo);
+            } else {
+              tmem_st16(tb + Cf::TM_CHI + tg, hi);
+              tmem_st16(tb + Cf::TM_CLO + tg, lo);
+            }
           }
-          const float rr = e * rcp_approx(sum);
-          float c = (be * delta) * rr;
-          if (t >= nvalid) c = 0.f;  // padding tokens of the last chunk leave the state alone
-          cs[t & 15] = c;
-          if constexpr (RDEBUG) {
-            if (col_ok && t < nvalid) p.r_debug[((tok0 + (size_t)(t0 + t)) * J + j) * p.Dv + col] = rr;
-          }
-          if (t + 1 < C) pred[t + 1] = fmaf(c, Gkk[t * C + t + 1], pred[t + 1]);  // the push the next token waits for
-          c_prev = c;
-          if ((t & 15) == 15) {  // 16 update coefficients complete: park them in tensor memory (hi / lo)
-            float hi[16], lo[16];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) { hi[i] = tf32_hi(cs[i]); lo[i] = cs[i] - hi[i]; }
-            tmem_st16(tb + Cf::TM_CHI + (t - 15), hi);
-            tmem_st16(tb + Cf::TM_CLO + (t - 15), lo);
-          }
+          for (int i = 0; i + GT <= C; ++i) pred[i] = pred[i + GT];
+#pragma unroll
+          for (int i = C - GT + 1; i <= C; ++i) pred[i] = 0.f;
         }
         return bad;
       };
@@ -506,6 +539,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       mbar_arrive(&bars[B_GS]);
     }
 
+#pragma unroll 1
     for (int n = 0; n < nchunks && !failed; ++n) {
       const bool more = n + 1 < nchunks;
       unsigned char *raw_next = smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES;
@@ -596,6 +630,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       w_times_kq(0, Cf::TM_WLO, false);
       mma_commit(&bars[B_E]);
     }
+#pragma unroll 1
     for (int n = 0; n < nchunks && !failed; ++n) {
       const bool more = n + 1 < nchunks;
       if (more) {
@@ -626,6 +661,9 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 8) tmem_dealloc(tb0, Cf::TM_ALLOC);
+#ifdef SWILA_CHUNK_PROFILE
+  if (tid == 0 && blockIdx.x < 1024) g_chunk_blk[blockIdx.x] = clock64() - prof_t0;
+#endif
 }
 
 template <int J, int DK>

@@ -36,4 +36,8 @@ extern "C" int swila_chunk_profile(long long *out8) {
   if (cudaMemcpyFromSymbol(out8, swila::g_chunk_prof, sizeof(z)) != cudaSuccess) return -1;
   return cudaMemcpyToSymbol(swila::g_chunk_prof, z, sizeof(z)) == cudaSuccess ? 0 : -1;
 }
+// Developer build only: per block (first 1024) total cycles, SM id and start time in ns.
+extern "C" int swila_chunk_blocks(long long *out3072) {
+  return cudaMemcpyFromSymbol(out3072, swila::g_chunk_blk, 3 * 1024 * sizeof(long long)) == cudaSuccess ? 0 : -1;
+}
 #endif
