@@ -41,9 +41,11 @@ namespace swila {
 // Set when a bounded wait on a completion barrier expires (never expected).
 static __device__ int g_chunk_error = 0;
 #ifdef SWILA_CHUNK_PROFILE
-static __device__ long long g_chunk_prof[8];
+// Developer build only: cycle counters per phase, kept in registers by the first thread of each warp
+// role of block 0 and written out at the end; per-block totals for every block.
+static __device__ long long g_chunk_prof[4 * 8];
 static __device__ long long g_chunk_blk[3 * 1024];  // per block: cycles, SM id, start time (ns)
-#define PROF_ADD(i, who) do { if (tid == (who) && blockIdx.x == 0) { long long now_ = clock64(); g_chunk_prof[i] += now_ - prof_t; prof_t = now_; } } while (0)
+#define PROF_ADD(i, who) do { long long now_ = clock64(); prof_acc[i] += now_ - prof_t; prof_t = now_; } while (0)
 #else
 #define PROF_ADD(i, who) do {} while (0)
 #endif
@@ -65,6 +67,7 @@ struct ChunkCfg {
                        TM_CHI = TM_G + 2 * C, TM_CLO = TM_CHI + C, TM_USED = TM_CLO + C;
   static constexpr int TM_ALLOC = 512;
   static_assert(TM_USED <= TM_ALLOC, "tensor memory budget");
+  static_assert(J == 4 || J == 8, "the output transposition assumes that J divides 8");
   // raw stages (bytes), all bf16.  Main part: k, q [C][DK], v [C][COLS], beta/pik [C][J][COLS] (2-deep
   // ring); the query-prior logits piq [C][J][COLS] live in their own 3-deep ring because the helper
   // warps still need them for the outputs of chunk n while chunk n+2 is being fetched.
@@ -177,6 +180,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
 #ifdef SWILA_CHUNK_PROFILE
   long long prof_t = clock64();
   const long long prof_t0 = prof_t;
+  long long prof_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
   if (tid == 0 && blockIdx.x < 1024) {
     unsigned smid;
     unsigned long long ns;
@@ -205,29 +209,56 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       tc_fence_after_sync();
 #pragma unroll 1
       for (int tg = 0; tg < C; tg += 8) {  // rolled: the loop body stays resident in the instruction cache
-        float qd[8], x[8], m[8], e[8], o[8];
-        tmem_ld8(tb + Cf::TM_QD + (n & 1) * C + tg, qd);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) { x[i] = __bfloat162float(rpq[((tg + i) * J + j) * COLS + dl]) * kLog2e; m[i] = x[i]; }
-#pragma unroll
-        for (int off = 1; off < J; off <<= 1) {
-#pragma unroll
-          for (int i = 0; i < 8; ++i) m[i] = fmaxf(m[i], __shfl_xor_sync(0xffffffffu, m[i], off));
-        }
+        // This lane's readouts of 8 tokens (own component j) are transposed inside the J-lane group of the
+        // column, one exchange round per bit of j, so that the lane ends up with all J components of 8/J
+        // tokens and forms their outputs without any further exchange.
+        constexpr int LJ = (J == 4) ? 2 : 3;
+        float hq[8];
+        tmem_ld8(tb + Cf::TM_QD + (n & 1) * C + tg, hq);
         tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 8; ++i) { e[i] = ex2_approx(x[i] - m[i]); o[i] = e[i] * qd[i]; }
+        for (int rd = 0; rd < LJ; ++rd) {
+          const int nrem = 3 - rd;              // token bits still in the index
+          const int m = J >> (rd + 1);          // partner lane distance
+          const bool mybit = (j & m) != 0;
+          float g[8];
 #pragma unroll
-        for (int off = 1; off < J; off <<= 1) {
+          for (int c = 0; c < (1 << rd); ++c) {
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            e[i] += __shfl_xor_sync(0xffffffffu, e[i], off);
-            o[i] += __shfl_xor_sync(0xffffffffu, o[i], off);
+            for (int rest = 0; rest < (1 << (nrem - 1)); ++rest) {
+              const float lo = hq[(c << nrem) | rest], hi = hq[(c << nrem) | (1 << (nrem - 1)) | rest];
+              const float keep = mybit ? hi : lo, send = mybit ? lo : hi;
+              const float recv = __shfl_xor_sync(0xffffffffu, send, m);
+              g[(((c << 1) | 0) << (nrem - 1)) | rest] = keep;
+              g[(((c << 1) | 1) << (nrem - 1)) | rest] = recv;
+            }
           }
-        }
-        if (j == 0) {
 #pragma unroll
-          for (int i = 0; i < 8; ++i) ost[(tg + i) * COLS + dl] = __float2bfloat16_rn(o[i] * rcp_approx(e[i]));
+          for (int i = 0; i < 8; ++i) hq[i] = g[i];
+        }
+        // hq[(c << (3 - LJ)) | rest]: token tg + (j << (3 - LJ)) + rest, component j ^ pattern(c), where bit
+        // (LJ - 1 - rd) of c says whether the value came from the partner of round rd
+#pragma unroll
+        for (int rest = 0; rest < (8 >> LJ); ++rest) {
+          const int tl = tg + (j << (3 - LJ)) + rest;
+          float x[J];
+          float mx = -3.0e38f;
+#pragma unroll
+          for (int c = 0; c < J; ++c) {
+            int pat = 0;
+#pragma unroll
+            for (int rd = 0; rd < LJ; ++rd) pat |= ((c >> (LJ - 1 - rd)) & 1) ? (J >> (rd + 1)) : 0;
+            x[c] = __bfloat162float(rpq[(tl * J + (j ^ pat)) * COLS + dl]) * kLog2e;
+            mx = fmaxf(mx, x[c]);
+          }
+          float se = 0.f, so = 0.f;
+#pragma unroll
+          for (int c = 0; c < J; ++c) {
+            const float e = ex2_approx(x[c] - mx);
+            se += e;
+            so = fmaf(e, hq[(c << (3 - LJ)) | rest], so);
+          }
+          ost[tl * COLS + dl] = __float2bfloat16_rn(so * rcp_approx(se));
         }
       }
       tc_fence_before_sync();
@@ -311,6 +342,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
               for (int jj = 1; jj < J; ++jj) sum += __shfl_sync(0xffffffffu, e, jbase + ((j + jj) & (J - 1)));
               bad = bad || !(sum > 1e-30f && sum < 1e30f);
             }
+#ifndef SWILA_EXP_NOPUSH
             {  // deferred push of token t-1 into the predictions of tokens t+1 .. (slots i+1 ..)
               const float4 *gp = reinterpret_cast<const float4 *>(Gkk + max(t - 1, 0) * C + tg);
 #pragma unroll
@@ -322,6 +354,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
                 if (4 * u4 + 3 > i) pred[4 * u4 + 3] = fmaf(c_prev, g.w, pred[4 * u4 + 3]);
               }
             }
+#endif
             const float rr = e * rcp_approx(sum);
             float c = (be * delta) * rr;
             if (t >= nvalid) c = 0.f;  // padding tokens of the last chunk leave the state alone
@@ -663,6 +696,9 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   if (warp == 8) tmem_dealloc(tb0, Cf::TM_ALLOC);
 #ifdef SWILA_CHUNK_PROFILE
   if (tid == 0 && blockIdx.x < 1024) g_chunk_blk[blockIdx.x] = clock64() - prof_t0;
+  if (blockIdx.x == 0 && (tid & 127) == 0 && tid < 512) {
+    for (int i = 0; i < 8; ++i) g_chunk_prof[(tid >> 7) * 8 + i] = prof_acc[i];
+  }
 #endif
 }
 

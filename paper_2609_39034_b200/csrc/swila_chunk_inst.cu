@@ -30,11 +30,9 @@ int chunk_error_fetch(int *flag) {
 }  // namespace swila
 
 #ifdef SWILA_CHUNK_PROFILE
-// Developer build only: per-phase cycle counters of block 0 (reset on read).
-extern "C" int swila_chunk_profile(long long *out8) {
-  long long z[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-  if (cudaMemcpyFromSymbol(out8, swila::g_chunk_prof, sizeof(z)) != cudaSuccess) return -1;
-  return cudaMemcpyToSymbol(swila::g_chunk_prof, z, sizeof(z)) == cudaSuccess ? 0 : -1;
+// Developer build only: per-phase cycle counters of block 0, 8 per warp role (rows, helpers, ...).
+extern "C" int swila_chunk_profile(long long *out32) {
+  return cudaMemcpyFromSymbol(out32, swila::g_chunk_prof, 32 * sizeof(long long)) == cudaSuccess ? 0 : -1;
 }
 // Developer build only: per block (first 1024) total cycles, SM id and start time in ns.
 extern "C" int swila_chunk_blocks(long long *out3072) {
