@@ -24,7 +24,7 @@ ALGO_AUTO, ALGO_SCAN, ALGO_SCAN_WIDE, ALGO_SCAN_NARROW, ALGO_CHUNK = 0, 1, 2, 3,
 EXPORTS = ("swila_version", "swila_strerror", "swila_last_cuda_error", "swila_state_w_bytes",
            "swila_state_r_bytes", "swila_state_init", "swila_forward", "swila_decode_step",
            "swila_bench_fma_chain", "swila_forward_host", "swila_forward_host_workspace_bytes",
-           "swila_forward_host_static", "swila_forward_host_static_capacity", "swila_selftest_tf32_mma", "swila_device_status")
+           "swila_forward_host_static", "swila_forward_host_static_capacity", "swila_selftest_tf32_mma", "swila_selftest_bf16_mma", "swila_device_status")
 
 
 class Shape(ctypes.Structure):
@@ -83,6 +83,9 @@ def _load() -> ctypes.CDLL:
     L.swila_forward_host_static.argtypes = [ctypes.POINTER(Shape), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                             ctypes.POINTER(Gates), ctypes.POINTER(State), ctypes.POINTER(State),
                                             ctypes.c_void_p, ctypes.c_void_p]
+    L.swila_selftest_bf16_mma.restype = ctypes.c_int
+    L.swila_selftest_bf16_mma.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
+                                          ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p]
     L.swila_selftest_tf32_mma.restype = ctypes.c_int
     L.swila_selftest_tf32_mma.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
                                           ctypes.c_void_p, ctypes.c_void_p]
@@ -231,6 +234,18 @@ def selftest_tf32_mma(A: torch.Tensor, B: torch.Tensor) -> torch.Tensor:
     D = torch.zeros((128, N), device=A.device, dtype=torch.float32)
     status = torch.zeros(1, device=A.device, dtype=torch.int32)
     check(lib.swila_selftest_tf32_mma(_p(A), _p(B), _p(D), N, K, _p(status), _stream(None)))
+    torch.cuda.synchronize()
+    if int(status.item()) != 0:
+        raise RuntimeError("tcgen05 self-test: the MMA did not signal completion")
+    return D
+
+
+def selftest_bf16_mma(A: torch.Tensor, B: torch.Tensor, a_in_smem: bool = False) -> torch.Tensor:
+    """D = bf16(A) @ bf16(B).T on the tcgen05 path (A [128,K], B [N,K], fp32 on the device)."""
+    N, K = B.shape
+    D = torch.zeros((128, N), device=A.device, dtype=torch.float32)
+    status = torch.zeros(1, device=A.device, dtype=torch.int32)
+    check(lib.swila_selftest_bf16_mma(_p(A), _p(B), _p(D), N, K, int(a_in_smem), _p(status), _stream(None)))
     torch.cuda.synchronize()
     if int(status.item()) != 0:
         raise RuntimeError("tcgen05 self-test: the MMA did not signal completion")

@@ -24,3 +24,17 @@ def test_tf32_mma_matches_matmul(N, K):
     ref = A.double() @ B.double().T
     err = float((D.double() - ref).abs().max() / ref.abs().max())
     assert err < 1e-5, err
+
+
+@pytest.mark.parametrize("N,K,a_in_smem", [(64, 128, False), (128, 32, False), (32, 32, False), (64, 64, True)])
+def test_bf16_mma_matches_matmul(N, K, a_in_smem):
+    assert torch.cuda.is_available()
+    from paper_2609_39034_b200 import binding
+
+    g = torch.Generator(device="cuda").manual_seed(N * 1000 + K + 7)
+    A = torch.randn((128, K), device="cuda", generator=g)
+    B = torch.randn((N, K), device="cuda", generator=g)
+    D = binding.selftest_bf16_mma(A, B, a_in_smem)
+    ref = A.bfloat16().double() @ B.bfloat16().double().T  # the kernel rounds to bf16 the same way
+    err = float((D.double() - ref).abs().max() / ref.abs().max())
+    assert err < 1e-5, err
