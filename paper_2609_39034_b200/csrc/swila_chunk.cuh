@@ -11,31 +11,46 @@
 //   w_C    = w_0 + sum_s c_s k_s                                                        (Eq. 3.3)
 //
 // This is the same recurrence, token by token and exact (no Newton iteration): only the order
-// of the floating-point additions differs from the scan.  The three dense contractions
-//   P0 = W0 K^T, Q0 = W0 Q^T  (M x Dk x C)      and      W += Cmat K  (M x C x Dk)
-// plus the two Gram matrices K K^T, K Q^T run on the tcgen05 tensor cores in TF32 with FP32
-// accumulation in tensor memory; FP32 operands are split as x = hi + lo (hi = the 19 leading
-// bits the hardware keeps, lo = the remainder) and both parts are multiplied, so products carry
-// ~22 significant bits.  bf16 inputs k, q are exact in TF32.  The triangular part (the sums over
-// s inside the chunk) and the E-step stay on the FP32 ALUs, one thread per row.
+// of the floating-point additions differs from the scan.  The dense contractions
+//   P0 = W0 K^T, Q0 = W0 Q^T  (M x Dk x C),   W += Cmat K  (M x C x Dk),   the Gram matrices
+// run on the tcgen05 tensor cores with BF16 operands (K = 16 per instruction) and FP32
+// accumulation in tensor memory.  k and q are bf16 inputs, hence exact operands; every FP32
+// operand (the state, the update coefficients, Gram matrices used as operands) is split as
+// x = hi + lo with hi = bf16(x), lo = bf16(x - hi) and both parts are multiplied (lo x lo is
+// dropped), which keeps 16 significant bits of the operand: a relative error of 4e-6 per product,
+// unbiased, against a parity tolerance of 1e-4.  The triangular part (the sums over s inside the
+// chunk) and the E-step stay on the FP32 ALUs, one thread per row.
+//
+// Across chunks the products of the state with the next chunk's keys and queries are taken off
+// the serial path: with W_{n+1} = W_n + Cmat_n K_n,
+//   W_{n+1} [K;Q]_{n+1}^T = W_n [K;Q]_{n+1}^T  +  Cmat_n (K_n [K;Q]_{n+1}^T),
+// the first term only needs the state BEFORE chunk n's update, so it runs while chunk n is still
+// being processed; after chunk n only the small second term (K = 32) remains.
 //
 // One block owns 128 rows = COLS = 128/J output columns of one (batch, head) and is split into
 // three roles that run concurrently and meet on mbarriers:
 //   row warps 0-3    thread r serves row (d = r / J, j = r % J), which is also its tensor-memory
 //                    lane; the J components of a column sit in adjacent lanes, so the E-step
-//                    normalisation is a few shuffles.  They run the sequential part of a chunk.
-//   helper warps 4-7 stage the next chunk (cp.async), convert K and Q into the tensor cores'
-//                    shared-memory operand layout, move the Gram matrices from tensor memory to
-//                    shared memory, refresh the low part of W after each update, and write the
-//                    chunk's outputs -- all while the row warps are busy.
+//                    normalisation is a few shuffles.  They run the sequential part of a chunk
+//                    and, while the tensor cores finish the hand-over to the next chunk, form the
+//                    outputs of the previous one.
+//   helper warps 4-7 stage chunks (cp.async straight into the tensor cores' operand layout for k
+//                    and q), turn gate logits into gates, move Gram matrices from tensor memory to
+//                    shared memory (plain rows for the row warps, hi / lo operand tiles for the
+//                    MMAs), split the state into its operand parts after each update.
 //   warp 8, lane 0   issues every tcgen05.mma and commits them to the barriers.
 #pragma once
+
+#include <cuda_bf16.h>
 
 #include <type_traits>
 
 #include "swila_common.cuh"
 #include "swila_umma.cuh"
 
+#ifndef SWILA_EXP
+#define SWILA_EXP 0
+#endif
 namespace swila {
 
 // Set when a bounded wait on a completion barrier expires (never expected).
@@ -45,84 +60,107 @@ static __device__ int g_chunk_error = 0;
 // role of block 0 and written out at the end; per-block totals for every block.
 static __device__ long long g_chunk_prof[4 * 8];
 static __device__ long long g_chunk_blk[3 * 1024];  // per block: cycles, SM id, start time (ns)
-#define PROF_ADD(i, who) do { long long now_ = clock64(); prof_acc[i] += now_ - prof_t; prof_t = now_; } while (0)
+#define PROF_ADD(i) do { long long now_ = clock64(); prof_acc[i] += now_ - prof_t; prof_t = now_; } while (0)
 #else
-#define PROF_ADD(i, who) do {} while (0)
+#define PROF_ADD(i) do {} while (0)
 #endif
 
 template <int J_, int DK_>
 struct ChunkCfg {
   static constexpr int J = J_, DK = DK_;
   static constexpr int C = 32;            // tokens per chunk
-  static constexpr int GT = 8;            // tokens per trip of the row warps' rolled serial loop
+  static constexpr int GT = 8;            // tokens per trip of the rolled loops (keeps the hot code inside the instruction cache)
   static constexpr int NROW = 128;        // row threads = rows of the tile
   static constexpr int NT = 288;          // 4 row warps + 4 helper warps + 1 MMA warp
   static constexpr int COLS = NROW / J;   // output columns per block
   static constexpr int ES = 2;            // bf16 io
-  // tensor-memory columns
-  // W, W_lo: the state and its low part; PQ: [P0 | Q0] of the current chunk; QD: the query-side
-  // readouts w_t.q_t of a chunk (double-buffered: the outputs of chunk n are formed while chunk
-  // n+1 runs); G: [K K^T | K Q^T]; CHI / CLO: the update coefficients of the chunk
-  static constexpr int TM_W = 0, TM_WLO = DK, TM_PQ = 2 * DK, TM_QD = TM_PQ + 2 * C, TM_G = TM_QD + 2 * C,
-                       TM_CHI = TM_G + 2 * C, TM_CLO = TM_CHI + C, TM_USED = TM_CLO + C;
+  // tensor-memory columns.  W: the state (FP32 accumulator); WHI / WLO: its bf16 operand parts, two key
+  // dims per column; PQ: [P0 | Q0] = state x [K;Q] of the next chunk to run; QD: the query-side readouts
+  // of a chunk (double-buffered); G: Gram matrices as they leave the tensor cores; CHI / CLO: the bf16
+  // parts of the chunk's update coefficients, two tokens per column
+  static constexpr int TM_W = 0, TM_WHI = DK, TM_WLO = DK + DK / 2, TM_PQ = 2 * DK, TM_QD = TM_PQ + 2 * C,
+                       TM_G = TM_QD + 2 * C, TM_CHI = TM_G + 3 * C, TM_CLO = TM_CHI + C / 2, TM_USED = TM_CLO + C / 2;
   static constexpr int TM_ALLOC = 512;
   static_assert(TM_USED <= TM_ALLOC, "tensor memory budget");
   static_assert(J == 4 || J == 8, "the output transposition assumes that J divides 8");
-  // raw stages (bytes), all bf16.  Main part: k, q [C][DK], v [C][COLS], beta/pik [C][J][COLS] (2-deep
-  // ring); the query-prior logits piq [C][J][COLS] live in their own 3-deep ring because the helper
-  // warps still need them for the outputs of chunk n while chunk n+2 is being fetched.
-  static constexpr int R_K = 0;
-  static constexpr int R_Q = R_K + C * DK * ES;
-  static constexpr int R_V = R_Q + C * DK * ES;
-  static constexpr int R_B = R_V + C * COLS * ES;   // beta logits; the helpers overwrite them in place with
-                                                    // beta = sigmoid(.) as fp32 [C][NROW], hence the fp32-sized slot
+  // K/Q operand tile (bf16, K-major, no swizzle): 16-byte unit (row, c) = 8 key dims 8c..8c+7 of one
+  // token at c*TILE_LBO + row*16, rows [K_even ; Q_even ; K_odd ; Q_odd]: the chunks of both parities
+  // side by side, so that one 128-row A operand covers the keys of two consecutive chunks.  cp.async
+  // writes it directly from global memory.
+  static constexpr int TILE_LBO = 4 * C * 16;
+  static constexpr int TILE_BYTES = (DK / 8) * TILE_LBO;
+  // raw stages (2-deep ring): v [C][COLS] bf16; beta logits [C][J][COLS] bf16, overwritten in place by the
+  // helpers with beta = sigmoid(.) as fp32 [C][NROW] (hence the fp32-sized slot); pik logits [C][J][COLS]
+  // bf16.  The query-prior logits piq [C][J][COLS] live in their own 4-deep ring because the outputs of
+  // chunk n are formed while chunk n+2 is being fetched.
+  static constexpr int R_V = 0;
+  static constexpr int R_B = R_V + C * COLS * ES;
   static constexpr int R_PK = R_B + C * NROW * 4;
   static constexpr int RAW_BYTES = R_PK + C * J * COLS * ES;
   static constexpr int RPQ_BYTES = C * J * COLS * ES;
-  static constexpr int BQ_LBO = C * 16 + 16;        // padded K-chunk stride of the readout operand tiles (bank spread)
-  static constexpr int BQ_TILE = (C / 4) * BQ_LBO;
   static constexpr int C_K = DK * ES / 16, C_V = COLS * ES / 16;  // 16-byte units per token row / column slice
+  // operand tiles written by the helpers (bf16, same unit layout, 8 tokens per unit)
+  static constexpr int KT_LBO = DK * 16;           // K transposed: rows = key dims, K index = tokens
+  static constexpr int KT_BYTES = (C / 8) * KT_LBO;
+  static constexpr int BQ_LBO = C * 16;            // masked (K Q^T)^T: rows = later token, K index = earlier token
+  static constexpr int BQ_TILE = (C / 8) * BQ_LBO;
+  static constexpr int GX_LBO = 2 * C * 16;        // ([K;Q]_{n+1} K_n^T): rows = token of the next chunk
+  static constexpr int GX_TILE = (C / 8) * GX_LBO;
   // shared memory map (bytes)
-  static constexpr int OFF_RAW = 0;
-  static constexpr int OFF_RPQ = OFF_RAW + 2 * RAW_BYTES;  // 4-deep ring of query-prior logits
-  static constexpr int OFF_KQ = OFF_RPQ + 4 * RPQ_BYTES;   // 2 x [DK/4][2C][4] fp32: rows 0..C-1 = K, C..2C-1 = Q tokens
-  static constexpr int OFF_KT = OFF_KQ + 2 * 2 * C * DK * 4;  // [C/4][DK][4] fp32: K transposed (rows = key dims)
-  static constexpr int OFF_G = OFF_KT + C * DK * 4;        // 2 x Gkk [C][C] fp32 (K K^T, for the row warps)
-  static constexpr int OFF_BQ = OFF_G + 2 * C * C * 4;     // 2 x { hi, lo } masked (K Q^T)^T operand tiles
-  static constexpr int OFF_OST = OFF_BQ + 2 * 2 * BQ_TILE; // 2 x [C][COLS] bf16 output staging
+  static constexpr int OFF_TILE = 0;
+  static constexpr int OFF_RAW = OFF_TILE + TILE_BYTES;
+  static constexpr int OFF_RPQ = OFF_RAW + 2 * RAW_BYTES;
+  static constexpr int OFF_KT = OFF_RPQ + 4 * RPQ_BYTES;
+  static constexpr int OFF_G = OFF_KT + KT_BYTES;             // 2 x Gkk [C][C] fp32 (K K^T, for the row warps)
+  static constexpr int OFF_BQ = OFF_G + 2 * C * C * 4;        // 2 x { hi, lo } readout operand tiles
+  static constexpr int OFF_GX = OFF_BQ + 2 * 2 * BQ_TILE;     // { hi, lo } cross-chunk operand tiles
+  static constexpr int OFF_OST = OFF_GX + 2 * GX_TILE;        // 2 x [C][COLS] bf16 output staging
   static constexpr int OFF_BAR = OFF_OST + 2 * C * COLS * ES;
   static constexpr int SMEM_BYTES = OFF_BAR + 128;
   static_assert(RAW_BYTES % 16 == 0 && RPQ_BYTES % 16 == 0 && (COLS * ES) % 16 == 0, "alignment");
   static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 };
 
-// barrier slots
-enum { B_E = 0, B_G, B_U, B_QD, B_KQ, B_KT, B_WLO, B_GS, B_C, B_COUNT };
+// barrier slots.  Committed by the MMA thread: E (state x [K;Q] of a chunk complete), G (Gram batch),
+// U (update of W), QD (readouts).  Arrived by threads: KQ (operand tile and gates of a chunk ready, 128
+// helpers), KT (transposed keys ready, 128 helpers), WP (operand parts of W refreshed, 128 helpers), GS
+// (Gram batch spilled, 2 helper warps), C (chunk finished, 128 rows), PQF ([P0|Q0] taken out of tensor
+// memory, 128 rows), BE (gates of a chunk ready, 128 helpers), OD (outputs of a chunk formed, 128 helpers).
+enum { B_E = 0, B_G, B_U, B_QD, B_KQ, B_KT, B_WP, B_GS, B_C, B_PQF, B_BE, B_OD, B_COUNT };
 
-// hi/lo split of an FP32 value for TF32 operands: hi keeps the bits the tensor core reads
-// (it ignores the 13 low mantissa bits), lo is the exact remainder.
-__device__ __forceinline__ float tf32_hi(float x) { return __uint_as_float(__float_as_uint(x) & 0xffffe000u); }
+// bf16 split of FP32 values: hi = bf16(x) (nearest), lo = bf16(x - hi); pairs packed with the first
+// value in the low half, which is where the tensor cores expect the even K index.
+__device__ __forceinline__ void bf16_split2(float x0, float x1, uint32_t &hi, uint32_t &lo) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+  hi = *reinterpret_cast<const uint32_t *>(&h);
+  const float r0 = x0 - __uint_as_float(hi << 16), r1 = x1 - __uint_as_float(hi & 0xffff0000u);
+  const __nv_bfloat162 l = __floats2bfloat162_rn(r0, r1);
+  lo = *reinterpret_cast<const uint32_t *>(&l);
+}
 
 // cp.async staging of one chunk by the 128 helper threads (h = 0..127)
-template <class Cf>
-__device__ __forceinline__ void chunk_issue_raw(const ScanParams &p, unsigned char *raw, unsigned char *rawpq,
-                                                size_t tok0, int t0, int col0, int h) {
+// FULL: every token of the chunk and every column of the slice exists (no predicates)
+template <class Cf, bool FULL>
+__device__ __forceinline__ void chunk_issue_raw_impl(const ScanParams &p, unsigned char *tile, unsigned char *raw,
+                                                unsigned char *rawpq, size_t tok0, int t0, int col0, int h) {
   constexpr int J = Cf::J, DK = Cf::DK, C = Cf::C, ES = Cf::ES, C_K = Cf::C_K, C_V = Cf::C_V;
   const int nvalid = min(C, p.T - t0);
   const size_t tokb = tok0 + (size_t)t0;
   const char *kb = (const char *)p.k + tokb * DK * ES;
   const char *qb = (const char *)p.q + tokb * DK * ES;
+  unsigned char *trow = tile + ((t0 / C) & 1) * 2 * C * 16;  // this chunk's 2C rows of the operand tile
 #pragma unroll
   for (int u = h; u < C * C_K; u += 128) {  // k and q rows of the chunk are contiguous in global memory
-    const bool valid = (u / C_K) < nvalid;
-    cp_async16(raw + Cf::R_K + u * 16, valid ? kb + u * 16 : (const char *)p.k, valid ? 16 : 0);
-    cp_async16(raw + Cf::R_Q + u * 16, valid ? qb + u * 16 : (const char *)p.k, valid ? 16 : 0);
+    const int tok = u / C_K, c = u % C_K;
+    const bool valid = FULL || tok < nvalid;
+    cp_async16(trow + c * Cf::TILE_LBO + tok * 16, valid ? kb + u * 16 : (const char *)p.k, valid ? 16 : 0);
+    cp_async16(trow + c * Cf::TILE_LBO + (C + tok) * 16, valid ? qb + u * 16 : (const char *)p.k, valid ? 16 : 0);
   }
 #pragma unroll
   for (int u = h; u < C * C_V; u += 128) {
     const int tok = u / C_V, cu = u % C_V;
     const int col = col0 + cu * 8;
-    const bool valid = tok < nvalid && col < p.Dv;
+    const bool valid = FULL || (tok < nvalid && col < p.Dv);
     cp_async16(raw + Cf::R_V + u * 16, valid ? (const char *)p.v + ((tokb + tok) * p.Dv + col) * ES : (const char *)p.k,
                valid ? 16 : 0);
   }
@@ -130,7 +168,7 @@ __device__ __forceinline__ void chunk_issue_raw(const ScanParams &p, unsigned ch
   for (int u = h; u < C * J * C_V; u += 128) {
     const int cu = u % C_V, jj = (u / C_V) % J, tok = u / (C_V * J);
     const int col = col0 + cu * 8;
-    const bool valid = tok < nvalid && col < p.Dv;
+    const bool valid = FULL || (tok < nvalid && col < p.Dv);
     const size_t off = (((tokb + tok) * J + jj) * (size_t)p.Dv + col) * ES;
     cp_async16(raw + Cf::R_B + u * 16, valid ? (const char *)p.beta_logit + off : (const char *)p.k, valid ? 16 : 0);
     cp_async16(raw + Cf::R_PK + u * 16, valid ? (const char *)p.pik_logit + off : (const char *)p.k, valid ? 16 : 0);
@@ -138,15 +176,23 @@ __device__ __forceinline__ void chunk_issue_raw(const ScanParams &p, unsigned ch
   }
 }
 
+template <class Cf>
+__device__ __forceinline__ void chunk_issue_raw(const ScanParams &p, unsigned char *tile, unsigned char *raw,
+                                                unsigned char *rawpq, size_t tok0, int t0, int col0, int h) {
+  if (t0 + Cf::C <= p.T && col0 + Cf::COLS <= p.Dv) chunk_issue_raw_impl<Cf, true>(p, tile, raw, rawpq, tok0, t0, col0, h);
+  else chunk_issue_raw_impl<Cf, false>(p, tile, raw, rawpq, tok0, t0, col0, h);
+}
+
 template <class Cf, bool RDEBUG>
 __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_constant__ ScanParams p) {
   using namespace umma;
   constexpr int J = Cf::J, DK = Cf::DK, C = Cf::C, NROW = Cf::NROW, COLS = Cf::COLS;
   extern __shared__ __align__(128) unsigned char smem[];
-  float *KQ_all = reinterpret_cast<float *>(smem + Cf::OFF_KQ);
-  float *Kt = reinterpret_cast<float *>(smem + Cf::OFF_KT);
+  unsigned char *tile = smem + Cf::OFF_TILE;
+  unsigned char *Kt = smem + Cf::OFF_KT;
   float *G_all = reinterpret_cast<float *>(smem + Cf::OFF_G);
   unsigned char *BQ_all = smem + Cf::OFF_BQ;
+  unsigned char *GX_all = smem + Cf::OFF_GX;
   __nv_bfloat16 *ostage = reinterpret_cast<__nv_bfloat16 *>(smem + Cf::OFF_OST);
   uint64_t *bars = reinterpret_cast<uint64_t *>(smem + Cf::OFF_BAR);
   uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(bars + B_COUNT);
@@ -166,9 +212,12 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     mbar_init(&bars[B_QD], 1);
     mbar_init(&bars[B_KQ], 128);
     mbar_init(&bars[B_KT], 128);
-    mbar_init(&bars[B_WLO], 128);
-    mbar_init(&bars[B_GS], 32);
+    mbar_init(&bars[B_WP], 128);
+    mbar_init(&bars[B_GS], 64);
     mbar_init(&bars[B_C], 128);
+    mbar_init(&bars[B_PQF], 128);
+    mbar_init(&bars[B_BE], 128);
+    mbar_init(&bars[B_OD], 128);
     mbar_fence_init();
   }
   tc_fence_before_sync();
@@ -176,6 +225,11 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   tc_fence_after_sync();
   const uint32_t tb0 = *tmem_base_s;
   const uint32_t tb = tb0 + ((uint32_t)((warp & 3) * 32) << 16);  // this warp's lane quarter
+  // row served by this thread in either 128-thread role
+  const int r = tid & 127;
+  const int dl = r / J, j = r % J;
+  const int col = col0 + dl;
+  const bool col_ok = col < p.Dv;
   bool failed = false;
 #ifdef SWILA_CHUNK_PROFILE
   long long prof_t = clock64();
@@ -191,104 +245,115 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   }
 #endif
 
+  // outputs of one chunk (Eq. 3.5): o_td = sum_j pi^q_j (w_t.q_t)_j, pi^q = softmax over the J
+  // components of a column
+  auto write_outputs = [&](int n) {
+    const int t0 = n * C;
+    const int nvalid = min(C, p.T - t0);
+    const __nv_bfloat16 *rpq = reinterpret_cast<const __nv_bfloat16 *>(smem + Cf::OFF_RPQ + (n & 3) * Cf::RPQ_BYTES);
+    __nv_bfloat16 *ost = ostage + (n & 1) * C * COLS;
+    tc_fence_after_sync();
+#pragma unroll 1
+    for (int tg = 0; tg < C; tg += 8) {  // rolled: the loop body stays resident in the instruction cache
+      // This lane's readouts of 8 tokens (own component j) are transposed inside the J-lane group of the
+      // column, one exchange round per bit of j, so that the lane ends up with all J components of 8/J
+      // tokens and forms their outputs without any further exchange.
+      constexpr int LJ = (J == 4) ? 2 : 3;
+      float hq[8];
+      tmem_ld8(tb + Cf::TM_QD + (n & 1) * C + tg, hq);
+      tmem_ld_wait();
+#pragma unroll
+      for (int rd = 0; rd < LJ; ++rd) {
+        const int nrem = 3 - rd;              // token bits still in the index
+        const int m = J >> (rd + 1);          // partner lane distance
+        const bool mybit = (j & m) != 0;
+        float g[8];
+#pragma unroll
+        for (int c = 0; c < (1 << rd); ++c) {
+#pragma unroll
+          for (int rest = 0; rest < (1 << (nrem - 1)); ++rest) {
+            const float lo = hq[(c << nrem) | rest], hi = hq[(c << nrem) | (1 << (nrem - 1)) | rest];
+            const float keep = mybit ? hi : lo, send = mybit ? lo : hi;
+            const float recv = __shfl_xor_sync(0xffffffffu, send, m);
+            g[(((c << 1) | 0) << (nrem - 1)) | rest] = keep;
+            g[(((c << 1) | 1) << (nrem - 1)) | rest] = recv;
+          }
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) hq[i] = g[i];
+      }
+      // hq[(c << (3 - LJ)) | rest]: token tg + (j << (3 - LJ)) + rest, component j ^ pattern(c), where bit
+      // (LJ - 1 - rd) of c says whether the value came from the partner of round rd
+#pragma unroll
+      for (int rest = 0; rest < (8 >> LJ); ++rest) {
+        const int tl = tg + (j << (3 - LJ)) + rest;
+        float x[J];
+        float mx = -3.0e38f;
+#pragma unroll
+        for (int c = 0; c < J; ++c) {
+          int pat = 0;
+#pragma unroll
+          for (int rd = 0; rd < LJ; ++rd) pat |= ((c >> (LJ - 1 - rd)) & 1) ? (J >> (rd + 1)) : 0;
+          x[c] = __bfloat162float(rpq[(tl * J + (j ^ pat)) * COLS + dl]) * kLog2e;
+          mx = fmaxf(mx, x[c]);
+        }
+        float se = 0.f, so = 0.f;
+#pragma unroll
+        for (int c = 0; c < J; ++c) {
+          const float e = ex2_approx(x[c] - mx);
+          se += e;
+          so = fmaf(e, hq[(c << (3 - LJ)) | rest], so);
+        }
+        ost[tl * COLS + dl] = __float2bfloat16_rn(so * rcp_approx(se));
+      }
+    }
+    tc_fence_before_sync();
+    named_bar_sync(2, 128);
+    constexpr int GROUPS = COLS / 8;  // 8 outputs = 16 bytes per store
+    for (int e = r; e < C * GROUPS; e += 128) {
+      const int t = e / GROUPS, g8 = e - t * GROUPS;
+      if (t < nvalid && col0 + g8 * 8 < p.Dv)
+        *reinterpret_cast<uint4 *>((__nv_bfloat16 *)p.o + (tok0 + (size_t)(t0 + t)) * p.Dv + col0 + g8 * 8) =
+            *reinterpret_cast<const uint4 *>(ost + t * COLS + g8 * 8);
+    }
+  };
+
   if (warp < 4) {
     // =============================== row warps ===============================================
-    const int r = tid;
-    const int dl = r / J, j = r % J;
-    const int col = col0 + dl;
-    const bool col_ok = col < p.Dv;
     const int jbase = lane - j;
-    if (!mbar_wait(&bars[B_KQ], 0) || !mbar_wait(&bars[B_GS], 0)) failed = true;
-    // outputs of one chunk (Eq. 3.5): o_td = sum_j pi^q_j (w_t.q_t)_j, pi^q = softmax over the J lanes
-    // of a column; eight tokens at a time so that the shuffles of different tokens overlap
-    auto write_outputs = [&](int n) {
-      const int t0 = n * C;
-      const int nvalid = min(C, p.T - t0);
-      const __nv_bfloat16 *rpq = reinterpret_cast<const __nv_bfloat16 *>(smem + Cf::OFF_RPQ + (n & 3) * Cf::RPQ_BYTES);
-      __nv_bfloat16 *ost = ostage + (n & 1) * C * COLS;
-      tc_fence_after_sync();
-#pragma unroll 1
-      for (int tg = 0; tg < C; tg += 8) {  // rolled: the loop body stays resident in the instruction cache
-        // This lane's readouts of 8 tokens (own component j) are transposed inside the J-lane group of the
-        // column, one exchange round per bit of j, so that the lane ends up with all J components of 8/J
-        // tokens and forms their outputs without any further exchange.
-        constexpr int LJ = (J == 4) ? 2 : 3;
-        float hq[8];
-        tmem_ld8(tb + Cf::TM_QD + (n & 1) * C + tg, hq);
-        tmem_ld_wait();
-#pragma unroll
-        for (int rd = 0; rd < LJ; ++rd) {
-          const int nrem = 3 - rd;              // token bits still in the index
-          const int m = J >> (rd + 1);          // partner lane distance
-          const bool mybit = (j & m) != 0;
-          float g[8];
-#pragma unroll
-          for (int c = 0; c < (1 << rd); ++c) {
-#pragma unroll
-            for (int rest = 0; rest < (1 << (nrem - 1)); ++rest) {
-              const float lo = hq[(c << nrem) | rest], hi = hq[(c << nrem) | (1 << (nrem - 1)) | rest];
-              const float keep = mybit ? hi : lo, send = mybit ? lo : hi;
-              const float recv = __shfl_xor_sync(0xffffffffu, send, m);
-              g[(((c << 1) | 0) << (nrem - 1)) | rest] = keep;
-              g[(((c << 1) | 1) << (nrem - 1)) | rest] = recv;
-            }
-          }
-#pragma unroll
-          for (int i = 0; i < 8; ++i) hq[i] = g[i];
-        }
-        // hq[(c << (3 - LJ)) | rest]: token tg + (j << (3 - LJ)) + rest, component j ^ pattern(c), where bit
-        // (LJ - 1 - rd) of c says whether the value came from the partner of round rd
-#pragma unroll
-        for (int rest = 0; rest < (8 >> LJ); ++rest) {
-          const int tl = tg + (j << (3 - LJ)) + rest;
-          float x[J];
-          float mx = -3.0e38f;
-#pragma unroll
-          for (int c = 0; c < J; ++c) {
-            int pat = 0;
-#pragma unroll
-            for (int rd = 0; rd < LJ; ++rd) pat |= ((c >> (LJ - 1 - rd)) & 1) ? (J >> (rd + 1)) : 0;
-            x[c] = __bfloat162float(rpq[(tl * J + (j ^ pat)) * COLS + dl]) * kLog2e;
-            mx = fmaxf(mx, x[c]);
-          }
-          float se = 0.f, so = 0.f;
-#pragma unroll
-          for (int c = 0; c < J; ++c) {
-            const float e = ex2_approx(x[c] - mx);
-            se += e;
-            so = fmaf(e, hq[(c << (3 - LJ)) | rest], so);
-          }
-          ost[tl * COLS + dl] = __float2bfloat16_rn(so * rcp_approx(se));
-        }
-      }
-      tc_fence_before_sync();
-      PROF_ADD(4, 0);
-      named_bar_sync(2, 128);
-      PROF_ADD(5, 0);
-      constexpr int GROUPS = COLS / 8;  // 8 outputs = 16 bytes per store
-      for (int e = r; e < C * GROUPS; e += 128) {
-        const int t = e / GROUPS, g8 = e - t * GROUPS;
-        if (t < nvalid && col0 + g8 * 8 < p.Dv)
-          *reinterpret_cast<uint4 *>((__nv_bfloat16 *)p.o + (tok0 + (size_t)(t0 + t)) * p.Dv + col0 + g8 * 8) =
-              *reinterpret_cast<const uint4 *>(ost + t * COLS + g8 * 8);
-      }
-      PROF_ADD(6, 0);
-    };
-
+    if (!mbar_wait(&bars[B_BE], 0) || !mbar_wait(&bars[B_GS], 0)) failed = true;
 #pragma unroll 1
     for (int n = 0; n < nchunks && !failed; ++n) {
       const int t0 = n * C;
       const int nvalid = min(C, p.T - t0);
       const unsigned char *raw = smem + Cf::OFF_RAW + (n & 1) * Cf::RAW_BYTES;
       const __nv_bfloat16 *rv = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_V);
+      const float *bes = reinterpret_cast<const float *>(raw + Cf::R_B);
       const __nv_bfloat16 *rpk = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_PK);
       const float *Gkk = G_all + (n & 1) * C * C;
-      const float *bes = reinterpret_cast<const float *>(raw + Cf::R_B);
 
-      PROF_ADD(0, 0);
+      PROF_ADD(0);
       if (!mbar_wait(&bars[B_E], n & 1)) { failed = true; break; }
       tc_fence_after_sync();
-      PROF_ADD(1, 0);
+      PROF_ADD(1);
+      // [P0 | Q0] out of tensor memory: P0 to registers, Q0 seeds the readout accumulator of this chunk;
+      // then the tensor cores may overwrite the region with the next chunk's products
+      float pred0[C];
+#pragma unroll
+      for (int cc = 0; cc < C / 16; ++cc) {
+        float a[16], b[16];
+        tmem_ld16(tb + Cf::TM_PQ + cc * 16, a);
+        tmem_ld16(tb + Cf::TM_PQ + C + cc * 16, b);
+        tmem_ld_wait();
+        tmem_st16(tb + Cf::TM_QD + (n & 1) * C + cc * 16, b);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) pred0[cc * 16 + i] = a[i];
+      }
+      tmem_st_wait();
+      tc_fence_before_sync();
+      mbar_arrive(&bars[B_PQF]);
+      PROF_ADD(4);
+
       // ---- sequential part of the chunk: E-step and the triangular key-side corrections.  Only one FMA
       //      of a token's push (into the next token's prediction) sits on the serial chain; the rest is
       //      deferred into the shuffle latency of the next token's E-step.
@@ -303,17 +368,11 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         // keeps the trip's code independent of tg); slot C takes the last token's push
         float pred[C + 1];
 #pragma unroll
-        for (int cc = 0; cc < C / 16; ++cc) {
-          float a[16];
-          tmem_ld16(tb + Cf::TM_PQ + cc * 16, a);
-          tmem_ld_wait();
-#pragma unroll
-          for (int i = 0; i < 16; ++i) pred[cc * 16 + i] = a[i];
-        }
+        for (int t = 0; t < C; ++t) pred[t] = pred0[t];
         pred[C] = 0.f;
         float c_prev = 0.f;
 #pragma unroll 1
-        for (int tg = 0; tg < C; tg += GT) {  // rolled: GT tokens of straight-line code stay in the instruction cache
+        for (int tg = 0; tg < C; tg += GT) {
           float cs[GT];
 #pragma unroll
           for (int i = 0; i < GT; ++i) {
@@ -342,7 +401,6 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
               for (int jj = 1; jj < J; ++jj) sum += __shfl_sync(0xffffffffu, e, jbase + ((j + jj) & (J - 1)));
               bad = bad || !(sum > 1e-30f && sum < 1e30f);
             }
-#ifndef SWILA_EXP_NOPUSH
             {  // deferred push of token t-1 into the predictions of tokens t+1 .. (slots i+1 ..)
               const float4 *gp = reinterpret_cast<const float4 *>(Gkk + max(t - 1, 0) * C + tg);
 #pragma unroll
@@ -354,7 +412,6 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
                 if (4 * u4 + 3 > i) pred[4 * u4 + 3] = fmaf(c_prev, g.w, pred[4 * u4 + 3]);
               }
             }
-#endif
             const float rr = e * rcp_approx(sum);
             float c = (be * delta) * rr;
             if (t >= nvalid) c = 0.f;  // padding tokens of the last chunk leave the state alone
@@ -365,17 +422,19 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
             pred[i + 1] = fmaf(c, Gkk[t * C + t + 1], pred[i + 1]);  // the push the next token waits for
             c_prev = c;
           }
-          {  // GT update coefficients complete: park them in tensor memory (hi / lo)
-            float hi[GT], lo[GT];
+          // the coefficient columns are still operands of the previous chunk's update and readout MMAs until
+          // those complete (normally long before the first trip ends)
+          if (tg == 0 && n > 0) {
+            PROF_ADD(6);
+            if (!mbar_wait(&bars[B_QD], (n - 1) & 1)) failed = true;
+            PROF_ADD(7);
+          }
+          {  // GT update coefficients complete: park their bf16 parts in tensor memory, two tokens per column
+            uint32_t hi[GT / 2], lo[GT / 2];
 #pragma unroll
-            for (int i = 0; i < GT; ++i) { hi[i] = tf32_hi(cs[i]); lo[i] = cs[i] - hi[i]; }
-            if constexpr (GT == 8) {
-              tmem_st8(tb + Cf::TM_CHI + tg, hi);
-              tmem_st8(tb + Cf::TM_CLO + tg, lo);
-            } else {
-              tmem_st16(tb + Cf::TM_CHI + tg, hi);
-              tmem_st16(tb + Cf::TM_CLO + tg, lo);
-            }
+            for (int i = 0; i < GT / 2; ++i) bf16_split2(cs[2 * i], cs[2 * i + 1], hi[i], lo[i]);
+            tmem_st4(tb + Cf::TM_CHI + tg / 2, hi);
+            tmem_st4(tb + Cf::TM_CLO + tg / 2, lo);
           }
 #pragma unroll
           for (int i = 0; i + GT <= C; ++i) pred[i] = pred[i + GT];
@@ -384,34 +443,23 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         }
         return bad;
       };
-      {  // Q0 seeds the readout accumulator of this chunk
-#pragma unroll
-        for (int cc = 0; cc < C / 16; ++cc) {
-          float b[16];
-          tmem_ld16(tb + Cf::TM_PQ + C + cc * 16, b);
-          tmem_ld_wait();
-          tmem_st16(tb + Cf::TM_QD + (n & 1) * C + cc * 16, b);
-        }
-      }
-      const bool underflow = sequential(std::false_type{});
-      if (__any_sync(0xffffffffu, underflow)) {
+      const bool unsafe = sequential(std::false_type{});
+      PROF_ADD(5);
+      if (__any_sync(0xffffffffu, unsafe)) {
         tmem_st_wait();
         sequential(std::true_type{});
       }
       tmem_st_wait();
       tc_fence_before_sync();
-      PROF_ADD(2, 0);
-      // the next chunk's operands, and the previous chunk's readouts, must be in place before this
-      // chunk is handed over (keeps every barrier at most one phase ahead of its waiters)
-      if (n + 1 < nchunks && (!mbar_wait(&bars[B_KQ], (n + 1) & 1) || !mbar_wait(&bars[B_GS], (n + 1) & 1))) failed = true;
-      if (n > 0 && !mbar_wait(&bars[B_QD], (n - 1) & 1)) failed = true;
+      PROF_ADD(2);
+      // what the next steps rely on must be in place before this chunk is handed over (this also keeps every
+      // barrier at most one phase ahead of its waiters): operands, gates and Gram rows of chunk n+1
+      // gates and Gram rows of chunk n+1, and the helpers done with the readout buffer that chunk n+1 will seed
+      if (n + 1 < nchunks && (!mbar_wait(&bars[B_BE], (n + 1) & 1) || !mbar_wait(&bars[B_GS], (n + 1) & 1))) failed = true;
+      if (n > 0 && !mbar_wait(&bars[B_OD], (n - 1) & 1)) failed = true;
       mbar_arrive(&bars[B_C]);
-      PROF_ADD(3, 0);
-      // outputs of the previous chunk, in the shadow of the tensor-core work for chunk n+1
-      if (n > 0 && !failed) write_outputs(n - 1);
+      PROF_ADD(3);
     }
-    if (!failed && !mbar_wait(&bars[B_QD], (nchunks - 1) & 1)) failed = true;
-    if (!failed) write_outputs(nchunks - 1);
     // ---- final state row -> global ----
     if (!failed && !mbar_wait(&bars[B_U], (nchunks - 1) & 1)) failed = true;
     if (!failed && p.W_out && col_ok) {
@@ -429,45 +477,20 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     }
   } else if (warp < 8) {
     // =============================== helper warps ============================================
-    const int h = tid - 128;
-    const int dl = h / J, j = h % J;
-    const int col = col0 + dl;
-    const bool col_ok = col < p.Dv;
-
-    // K, Q of a raw stage -> stacked fp32 operand tile (16-byte unit (row, k-chunk c) at (c*2C + row)*16)
-    auto cook_kq = [&](const unsigned char *raw, float *KQ) {
-      const __nv_bfloat16 *rk = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_K);
-      const __nv_bfloat16 *rq = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_Q);
-      // diagonal walk over 8-token x 16-chunk blocks: conflict-free 8-byte reads and 16-byte writes
-      constexpr int NBLK = (C / 8) * (DK / 4 / 16);
-#pragma unroll 2
-      for (int blk = 0; blk < NBLK; ++blk) {
-        const int tb8 = blk % (C / 8), cb16 = blk / (C / 8);
-        const int s = h >> 4, u = h & 15;
-        const int t = tb8 * 8 + ((u + s) & 7), c = cb16 * 16 + u;
-        const uint2 kr = *reinterpret_cast<const uint2 *>(rk + t * DK + c * 4);
-        const uint2 qr = *reinterpret_cast<const uint2 *>(rq + t * DK + c * 4);
-        float4 kf, qf;
-        kf.x = __uint_as_float(kr.x << 16); kf.y = __uint_as_float(kr.x & 0xffff0000u);
-        kf.z = __uint_as_float(kr.y << 16); kf.w = __uint_as_float(kr.y & 0xffff0000u);
-        qf.x = __uint_as_float(qr.x << 16); qf.y = __uint_as_float(qr.x & 0xffff0000u);
-        qf.z = __uint_as_float(qr.y << 16); qf.w = __uint_as_float(qr.y & 0xffff0000u);
-        *reinterpret_cast<float4 *>(KQ + (c * 2 * C + t) * 4) = kf;
-        *reinterpret_cast<float4 *>(KQ + (c * 2 * C + C + t) * 4) = qf;
-      }
-    };
-    // K of a raw stage, transposed: unit (row d', k-chunk c4) holds K[4 c4 .. 4 c4 + 3][d']
-    auto cook_kt = [&](const unsigned char *raw) {
-      const __nv_bfloat16 *rk = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_K);
-#pragma unroll 2
-      for (int e = h; e < (C / 4) * DK; e += 128) {
-        const int dd = e % DK, c4 = e / DK;
-        float4 f;
-        f.x = __bfloat162float(rk[(4 * c4 + 0) * DK + dd]);
-        f.y = __bfloat162float(rk[(4 * c4 + 1) * DK + dd]);
-        f.z = __bfloat162float(rk[(4 * c4 + 2) * DK + dd]);
-        f.w = __bfloat162float(rk[(4 * c4 + 3) * DK + dd]);
-        *reinterpret_cast<float4 *>(Kt + (c4 * DK + dd) * 4) = f;
+    const int h = r;
+    // K of a chunk, transposed: unit (row d', c) holds K[8c .. 8c+7][d'], read from the operand tile
+    auto cook_kt = [&](int m) {
+      const unsigned char *trow = tile + (m & 1) * 2 * C * 16;
+#pragma unroll 1
+      for (int e = h; e < (C / 8) * DK; e += 128) {
+        const int dd = e % DK, c = e / DK;
+        const unsigned char *src = trow + (dd >> 3) * Cf::TILE_LBO + (8 * c) * 16 + (dd & 7) * 2;
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          w[i] = (uint32_t)*reinterpret_cast<const unsigned short *>(src + (2 * i) * 16) |
+                 ((uint32_t)*reinterpret_cast<const unsigned short *>(src + (2 * i + 1) * 16) << 16);
+        *reinterpret_cast<uint4 *>(Kt + c * Cf::KT_LBO + dd * 16) = make_uint4(w[0], w[1], w[2], w[3]);
       }
     };
     // beta = sigmoid(logit) of this helper's row for every token of a raw stage (App. B.2), written over the
@@ -482,65 +505,79 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
 #pragma unroll
       for (int t = 0; t < C; ++t) bes[t * NROW + h] = be[t];
     };
-    // low part of W after an update: W_lo = W - hi(W), this helper's tensor-memory lane
-    auto refresh_wlo = [&]() {
+    // operand parts of W after an update, this helper's tensor-memory lane
+    auto refresh_parts = [&]() {
 #pragma unroll
-      for (int half = 0; half < DK / 64; ++half) {
-        float w[4][16];
-#pragma unroll
-        for (int cc = 0; cc < 4; ++cc) tmem_ld16(tb + Cf::TM_W + half * 64 + cc * 16, w[cc]);
+      for (int cc = 0; cc < DK / 16; ++cc) {
+        float w[16];
+        uint32_t hi[8], lo[8];
+        tmem_ld16(tb + Cf::TM_W + cc * 16, w);
         tmem_ld_wait();
 #pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-#pragma unroll
-          for (int i = 0; i < 16; ++i) w[cc][i] = w[cc][i] - tf32_hi(w[cc][i]);
-          tmem_st16(tb + Cf::TM_WLO + half * 64 + cc * 16, w[cc]);
-        }
+        for (int i = 0; i < 8; ++i) bf16_split2(w[2 * i], w[2 * i + 1], hi[i], lo[i]);
+        tmem_st8(tb + Cf::TM_WHI + cc * 8, reinterpret_cast<const float(&)[8]>(hi));
+        tmem_st8(tb + Cf::TM_WLO + cc * 8, reinterpret_cast<const float(&)[8]>(lo));
       }
       tmem_st_wait();
       tc_fence_before_sync();
     };
-    // Gram rows (tensor-memory lanes 0..C-1, helper warp 4 only) -> shared memory: K K^T row-major for the
-    // row warps; K Q^T as the B operand of the readout MMA -- transposed (rows = later token t, K index
-    // = earlier token s = this lane), causally masked (s <= t), split into hi / lo TF32 parts
-    auto spill_gram = [&](int n) {
-      float *Gkk = G_all + (n & 1) * C * C;
-      float *Bhi = reinterpret_cast<float *>(BQ_all + (n & 1) * 2 * Cf::BQ_TILE);
-      float *Blo = reinterpret_cast<float *>(BQ_all + (n & 1) * 2 * Cf::BQ_TILE + Cf::BQ_TILE);
+    // 32 FP32 values of this lane's Gram row -> bf16 hi / lo operand units (row `row` of a tile with `lbo`)
+    auto store_parts = [&](const float (&x)[C], unsigned char *thi, unsigned char *tlo, int lbo, int row) {
 #pragma unroll
-      for (int cc = 0; cc < C / 16; ++cc) {
-        float a[16], b[16];
-        tmem_ld16(tb + Cf::TM_G + cc * 16, a);
-        tmem_ld16(tb + Cf::TM_G + C + cc * 16, b);
+      for (int c = 0; c < C / 8; ++c) {
+        uint32_t hi[4], lo[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) bf16_split2(x[8 * c + 2 * i], x[8 * c + 2 * i + 1], hi[i], lo[i]);
+        *reinterpret_cast<uint4 *>(thi + c * lbo + row * 16) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        *reinterpret_cast<uint4 *>(tlo + c * lbo + row * 16) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+      }
+    };
+    // The Gram batch of chunk m is [K_e;Q_e;K_o;Q_o] x [K_m;Q_m | K_{m-1}]^T; the two helper warps whose
+    // tensor-memory lanes hold the rows of chunk m's keys and queries spill it:
+    //   key rows   (lane s):  K_m K_m^T as plain FP32 rows for the row warps;
+    //   query rows (lane t):  Q_m K_m^T, causally masked (s <= t), as the hi / lo operand of the readout MMA;
+    //   both:                 [K_m;Q_m] K_{m-1}^T as the hi / lo operand of the cross-chunk MMA.
+    auto spill_gram = [&](int m) {
+      const bool qrows = (warp & 1) != 0;
+      float a[C];
+#pragma unroll
+      for (int cc = 0; cc < C / 16; ++cc) tmem_ld16(tb + Cf::TM_G + cc * 16, reinterpret_cast<float(&)[16]>(a[cc * 16]));
+      tmem_ld_wait();
+      if (!qrows) {
+        float *Gkk = G_all + (m & 1) * C * C;
+#pragma unroll
+        for (int i = 0; i < C / 4; ++i)
+          *reinterpret_cast<float4 *>(Gkk + lane * C + i * 4) = make_float4(a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
+      } else {
+#pragma unroll
+        for (int s = 0; s < C; ++s) a[s] = (s <= lane) ? a[s] : 0.f;
+        unsigned char *bq = BQ_all + (m & 1) * 2 * Cf::BQ_TILE;
+        store_parts(a, bq, bq + Cf::BQ_TILE, Cf::BQ_LBO, lane);
+      }
+      if (m > 0) {
+#pragma unroll
+        for (int cc = 0; cc < C / 16; ++cc)
+          tmem_ld16(tb + Cf::TM_G + 2 * C + cc * 16, reinterpret_cast<float(&)[16]>(a[cc * 16]));
         tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-          *reinterpret_cast<float4 *>(Gkk + lane * C + cc * 16 + i * 4) = make_float4(a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const int t = cc * 16 + i;
-          const float val = (lane <= t) ? b[i] : 0.f;
-          const float hi = tf32_hi(val);
-          const int idx = (lane >> 2) * (Cf::BQ_LBO / 4) + t * 4 + (lane & 3);
-          Bhi[idx] = hi;
-          Blo[idx] = val - hi;
-        }
+        store_parts(a, GX_all, GX_all + Cf::GX_TILE, Cf::GX_LBO, (qrows ? C : 0) + lane);
       }
       tc_fence_before_sync();
       fence_async_smem();
     };
+    const bool spill_mine[2] = {warp < 6, warp >= 6};  // which parity of chunks this warp's lanes hold
 
     // ---- prologue: stage chunks 0 and 1, state row -> tensor memory, operands of chunk 0 ----
-    chunk_issue_raw<Cf>(p, smem + Cf::OFF_RAW, smem + Cf::OFF_RPQ, tok0, 0, col0, h);
+    chunk_issue_raw<Cf>(p, tile, smem + Cf::OFF_RAW, smem + Cf::OFF_RPQ, tok0, 0, col0, h);
     cp_async_commit();
     if (nchunks > 1)
-      chunk_issue_raw<Cf>(p, smem + Cf::OFF_RAW + Cf::RAW_BYTES, smem + Cf::OFF_RPQ + Cf::RPQ_BYTES, tok0, C, col0, h);
+      chunk_issue_raw<Cf>(p, tile, smem + Cf::OFF_RAW + Cf::RAW_BYTES, smem + Cf::OFF_RPQ + Cf::RPQ_BYTES, tok0, C, col0, h);
     cp_async_commit();
     {
       const float *src = (p.W_in && col_ok) ? p.W_in + (((size_t)bh * J + j) * p.Dv + col) * DK : nullptr;
 #pragma unroll
       for (int cc = 0; cc < DK / 16; ++cc) {
-        float w[16], lo[16];
+        float w[16];
+        uint32_t hi[8], lo[8];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -548,146 +585,205 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
           w[4 * i] = t.x; w[4 * i + 1] = t.y; w[4 * i + 2] = t.z; w[4 * i + 3] = t.w;
         }
 #pragma unroll
-        for (int i = 0; i < 16; ++i) lo[i] = w[i] - tf32_hi(w[i]);
+        for (int i = 0; i < 8; ++i) bf16_split2(w[2 * i], w[2 * i + 1], hi[i], lo[i]);
         tmem_st16(tb + Cf::TM_W + cc * 16, w);
-        tmem_st16(tb + Cf::TM_WLO + cc * 16, lo);
+        tmem_st8(tb + Cf::TM_WHI + cc * 8, reinterpret_cast<const float(&)[8]>(hi));
+        tmem_st8(tb + Cf::TM_WLO + cc * 8, reinterpret_cast<const float(&)[8]>(lo));
       }
       tmem_st_wait();
       tc_fence_before_sync();
-      mbar_arrive(&bars[B_WLO]);
+      mbar_arrive(&bars[B_WP]);
+    }
+    if (nchunks == 1) {  // the odd half of the operand tile is read (as don't-care rows) by the Gram batch: make it finite
+      for (int e = h; e < (DK / 8) * 2 * C; e += 128)
+        *reinterpret_cast<uint4 *>(tile + (e / (2 * C)) * Cf::TILE_LBO + (2 * C + e % (2 * C)) * 16) = make_uint4(0, 0, 0, 0);
     }
     cp_async_wait<1>();
     named_bar_sync(1, 128);  // every helper's copies of chunk 0 have landed
-    cook_kq(smem + Cf::OFF_RAW, KQ_all);
-    cook_be(smem + Cf::OFF_RAW);
     fence_async_smem();
     mbar_arrive(&bars[B_KQ]);
-    cook_kt(smem + Cf::OFF_RAW);
+    cook_be(smem + Cf::OFF_RAW);
+    mbar_arrive(&bars[B_BE]);
+    cook_kt(0);
     fence_async_smem();
     mbar_arrive(&bars[B_KT]);
-    if (warp == 4) {
+    if (nchunks > 1) {
+      cp_async_wait<0>();
+      named_bar_sync(1, 128);
+      fence_async_smem();
+      mbar_arrive(&bars[B_KQ]);
+    }
+    if (spill_mine[0]) {
       if (!mbar_wait(&bars[B_G], 0)) failed = true;
       tc_fence_after_sync();
       if (!failed) spill_gram(0);
       mbar_arrive(&bars[B_GS]);
     }
 
+    // Per chunk n, in the order of what the other roles wait for first.
 #pragma unroll 1
     for (int n = 0; n < nchunks && !failed; ++n) {
       const bool more = n + 1 < nchunks;
-      unsigned char *raw_next = smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES;
-      // (1) operands of chunk n+1: its raw stage has landed, and the K/Q tile it goes to was last read by
-      //     the MMAs of chunk n-1, which completed before the update of chunk n-1 this warp waited for
-      cp_async_wait<0>();
-      named_bar_sync(1, 128);
+      PROF_ADD(0);
       if (more) {
-        cook_kq(raw_next, KQ_all + ((n + 1) & 1) * 2 * C * DK);
-        cook_be(raw_next);
-        fence_async_smem();
-        mbar_arrive(&bars[B_KQ]);
-        if (warp == 4) {  // Gram matrices of chunk n+1
-          if (!mbar_wait(&bars[B_G], (n + 1) & 1)) { failed = true; }
+        // (1) gates of chunk n+1 for the row warps, then its Gram batch
+#if SWILA_EXP != 2
+        cook_be(smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES);
+#endif
+        mbar_arrive(&bars[B_BE]);
+        PROF_ADD(1);
+        if (spill_mine[(n + 1) & 1]) {
+          if (!mbar_wait(&bars[B_G], (n + 1) & 1)) failed = true;
           tc_fence_after_sync();
           if (!failed) spill_gram(n + 1);
           mbar_arrive(&bars[B_GS]);
         }
       }
-      
-      
+      PROF_ADD(2);
+      // (2) outputs of chunk n-1, whose readouts completed shortly after chunk n started
+      if (n > 0) {
+        if (!mbar_wait(&bars[B_QD], (n - 1) & 1)) { failed = true; break; }
+#if SWILA_EXP != 1
+        write_outputs(n - 1);
+#endif
+        mbar_arrive(&bars[B_OD]);
+      }
+      PROF_ADD(3);
       // (3) chunk n is finished by the row warps: stage chunk n+2 into the buffers chunk n used
       if (!mbar_wait(&bars[B_C], n & 1)) { failed = true; break; }
-      
-      
+      PROF_ADD(4);
       if (n + 2 < nchunks)
-        chunk_issue_raw<Cf>(p, smem + Cf::OFF_RAW + (n & 1) * Cf::RAW_BYTES, smem + Cf::OFF_RPQ + ((n + 2) & 3) * Cf::RPQ_BYTES,
+        chunk_issue_raw<Cf>(p, tile, smem + Cf::OFF_RAW + (n & 1) * Cf::RAW_BYTES, smem + Cf::OFF_RPQ + ((n + 2) & 3) * Cf::RPQ_BYTES,
                             tok0, (n + 2) * C, col0, h);
       cp_async_commit();
-      // (4) W has been updated with chunk n: refresh its low part, then the transposed K of chunk n+1
+      // (4) W has been updated with chunk n: split it into operand parts again
+      if (!mbar_wait(&bars[B_U], n & 1)) { failed = true; break; }
+      PROF_ADD(5);
       if (more) {
-        if (!mbar_wait(&bars[B_U], n & 1)) { failed = true; break; }
         tc_fence_after_sync();
-        refresh_wlo();
-        mbar_arrive(&bars[B_WLO]);
-        cook_kt(raw_next);
+#if SWILA_EXP != 3
+        refresh_parts();
+#endif
+        mbar_arrive(&bars[B_WP]);
+      }
+      PROF_ADD(6);
+      // (5) chunk n+2 has landed: its keys and queries already sit in the operand tile
+      if (n + 2 < nchunks) {
+        cp_async_wait<0>();
+        named_bar_sync(1, 128);
+        fence_async_smem();
+        mbar_arrive(&bars[B_KQ]);
+      }
+      // (6) transposed K of chunk n+1 (the update of chunk n has released the tile)
+      if (more) {
+        cook_kt(n + 1);
         fence_async_smem();
         mbar_arrive(&bars[B_KT]);
       }
-      
-      
+      PROF_ADD(7);
     }
     cp_async_wait<0>();
+    if (!failed && !mbar_wait(&bars[B_QD], (nchunks - 1) & 1)) failed = true;
+    if (!failed) write_outputs(nchunks - 1);
   } else if (lane == 0) {
     // =============================== MMA issuer ==============================================
-    constexpr uint32_t idE = idesc_tf32(128, 2 * C);  // [P0 | Q0] and [Gkk | Gkq]: N = 2C
-    constexpr uint32_t idU = idesc_tf32(128, DK);
-    const uint64_t kq_desc[2] = {smem_desc_kmajor(smem_u32(KQ_all), 2 * C * 16, 128),
-                                 smem_desc_kmajor(smem_u32(KQ_all + 2 * C * DK), 2 * C * 16, 128)};
-    const uint64_t kt0 = smem_desc_kmajor(smem_u32(Kt), DK * 16, 128);
-    auto gram = [&](int chunk) {
-      const uint64_t kq0 = kq_desc[chunk & 1];
+    constexpr uint32_t idE = idesc_bf16(128, 2 * C);  // N = 2C: [P0 | Q0], Gram batch, cross-chunk term
+    constexpr uint32_t idU = idesc_bf16(128, DK);
+    constexpr uint32_t idQ = idesc_bf16(128, C);
+    const uint64_t tile_a = smem_desc_kmajor(smem_u32(tile), Cf::TILE_LBO, 128);  // all 128 rows, as an A operand
+    const uint64_t kq_b[2] = {smem_desc_kmajor(smem_u32(tile), Cf::TILE_LBO, 128),
+                              smem_desc_kmajor(smem_u32(tile) + 2 * C * 16, Cf::TILE_LBO, 128)};  // [K;Q] (or K) of a parity
+    const uint64_t kt0 = smem_desc_kmajor(smem_u32(Kt), Cf::KT_LBO, 128);
+    const uint64_t gx_hi = smem_desc_kmajor(smem_u32(GX_all), Cf::GX_LBO, 128);
+    const uint64_t gx_lo = smem_desc_kmajor(smem_u32(GX_all + Cf::GX_TILE), Cf::GX_LBO, 128);
+    constexpr uint64_t TILE_ADV = 2 * (Cf::TILE_LBO / 16);  // start-address advance per 16 key dims, 16-byte units
+    // Gram batch of chunk m: every row of the tile against [K;Q] of chunk m and against K of chunk m-1
+    auto gram = [&](int m) {
 #pragma unroll 1
-      for (int ks = 0; ks < DK / 8; ++ks) {
-        const uint64_t d = kq0 + (uint64_t)(ks * 2 * 2 * C);  // start address advances in 16-byte units
-        mma_tf32_ss(tb0 + Cf::TM_G, d, d, idE, ks > 0);        // rows >= C of the A tile are don't-care
+      for (int ks = 0; ks < DK / 16; ++ks)
+        mma_bf16_ss(tb0 + Cf::TM_G, tile_a + ks * TILE_ADV, kq_b[m & 1] + ks * TILE_ADV, idE, ks > 0);
+      if (m > 0) {
+#pragma unroll 1
+        for (int ks = 0; ks < DK / 16; ++ks)
+          mma_bf16_ss(tb0 + Cf::TM_G + 2 * C, tile_a + ks * TILE_ADV, kq_b[(m - 1) & 1] + ks * TILE_ADV, idQ, ks > 0);
       }
       mma_commit(&bars[B_G]);
     };
-    auto w_times_kq = [&](int chunk, int w_col, bool first) {
-      const uint64_t kq0 = kq_desc[chunk & 1];
+    // [P0 | Q0] of chunk m from the state as it is now (hi and lo parts)
+    auto w_times_kq = [&](int m) {
 #pragma unroll 1
-      for (int ks = 0; ks < DK / 8; ++ks)
-        mma_tf32_ts(tb0 + Cf::TM_PQ, tb0 + w_col + ks * 8, kq0 + (uint64_t)(ks * 2 * 2 * C), idE, !(first && ks == 0));
+      for (int ks = 0; ks < DK / 16; ++ks)
+        mma_bf16_ts(tb0 + Cf::TM_PQ, tb0 + Cf::TM_WHI + ks * 8, kq_b[m & 1] + ks * TILE_ADV, idE, ks > 0);
+#pragma unroll 1
+      for (int ks = 0; ks < DK / 16; ++ks)
+        mma_bf16_ts(tb0 + Cf::TM_PQ, tb0 + Cf::TM_WLO + ks * 8, kq_b[m & 1] + ks * TILE_ADV, idE, true);
     };
-    constexpr uint32_t idQ = idesc_tf32(128, C);
+    // + Cmat (K_prev [K;Q]^T): the update of the chunk that just finished, seen by the next chunk's products
+    auto cross = [&]() {
+#pragma unroll 1
+      for (int ks = 0; ks < C / 16; ++ks) {
+        const uint64_t adv = (uint64_t)(ks * 2 * (Cf::GX_LBO / 16));
+        mma_bf16_ts(tb0 + Cf::TM_PQ, tb0 + Cf::TM_CHI + ks * 8, gx_hi + adv, idE, true);
+        mma_bf16_ts(tb0 + Cf::TM_PQ, tb0 + Cf::TM_CLO + ks * 8, gx_hi + adv, idE, true);
+        mma_bf16_ts(tb0 + Cf::TM_PQ, tb0 + Cf::TM_CHI + ks * 8, gx_lo + adv, idE, true);
+      }
+      mma_commit(&bars[B_E]);
+    };
     // readouts of chunk n: QD += Cmat (K Q^T masked)  -- c_hi B_hi + c_lo B_hi + c_hi B_lo
     auto readout = [&](int n) {
       const uint64_t bh0 = smem_desc_kmajor(smem_u32(BQ_all + (n & 1) * 2 * Cf::BQ_TILE), Cf::BQ_LBO, 128);
       const uint64_t bl0 = smem_desc_kmajor(smem_u32(BQ_all + (n & 1) * 2 * Cf::BQ_TILE + Cf::BQ_TILE), Cf::BQ_LBO, 128);
       const uint32_t d = tb0 + Cf::TM_QD + (n & 1) * C;
 #pragma unroll 1
-      for (int ks = 0; ks < C / 8; ++ks) {
+      for (int ks = 0; ks < C / 16; ++ks) {
         const uint64_t adv = (uint64_t)(ks * 2 * (Cf::BQ_LBO / 16));
-        mma_tf32_ts(d, tb0 + Cf::TM_CHI + ks * 8, bh0 + adv, idQ, true);
-        mma_tf32_ts(d, tb0 + Cf::TM_CLO + ks * 8, bh0 + adv, idQ, true);
-        mma_tf32_ts(d, tb0 + Cf::TM_CHI + ks * 8, bl0 + adv, idQ, true);
+        mma_bf16_ts(d, tb0 + Cf::TM_CHI + ks * 8, bh0 + adv, idQ, true);
+        mma_bf16_ts(d, tb0 + Cf::TM_CLO + ks * 8, bh0 + adv, idQ, true);
+        mma_bf16_ts(d, tb0 + Cf::TM_CHI + ks * 8, bl0 + adv, idQ, true);
       }
       mma_commit(&bars[B_QD]);
     };
-    if (!mbar_wait(&bars[B_KQ], 0)) failed = true;
-    tc_fence_after_sync();
-    if (!failed) gram(0);
-    if (!failed && !mbar_wait(&bars[B_WLO], 0)) failed = true;
+    if (!mbar_wait(&bars[B_KQ], 0) || !mbar_wait(&bars[B_WP], 0)) failed = true;
     tc_fence_after_sync();
     if (!failed) {
-      w_times_kq(0, Cf::TM_W, true);
-      w_times_kq(0, Cf::TM_WLO, false);
+      gram(0);
+      w_times_kq(0);
       mma_commit(&bars[B_E]);
     }
 #pragma unroll 1
     for (int n = 0; n < nchunks && !failed; ++n) {
       const bool more = n + 1 < nchunks;
       if (more) {
-        if (!mbar_wait(&bars[B_KQ], (n + 1) & 1)) { failed = true; break; }
+        // ahead of the serial path: Gram batch and state x [K;Q] of chunk n+1 with the state before chunk n's
+        // update (W is final up to chunk n-1 and split into parts; [P0|Q0] of chunk n has been taken out)
+        if (!mbar_wait(&bars[B_KQ], (n + 1) & 1) || !mbar_wait(&bars[B_PQF], n & 1)) { failed = true; break; }
+        if (n > 0 && !mbar_wait(&bars[B_WP], n & 1)) { failed = true; break; }
         tc_fence_after_sync();
+        PROF_ADD(0);
         gram(n + 1);
+        w_times_kq(n + 1);
+        PROF_ADD(1);
       }
-      if (!mbar_wait(&bars[B_C], n & 1) || !mbar_wait(&bars[B_KT], n & 1)) { failed = true; break; }
+      if (!mbar_wait(&bars[B_C], n & 1)) { failed = true; break; }
+      PROF_ADD(2);
+      if (more) {
+        if (!mbar_wait(&bars[B_GS], (n + 1) & 1)) { failed = true; break; }
+        tc_fence_after_sync();
+        cross();  // -> E(n+1): the only tensor work between two chunks of the row warps
+      }
+      PROF_ADD(3);
+      if (!mbar_wait(&bars[B_KT], n & 1)) { failed = true; break; }
       tc_fence_after_sync();
+      PROF_ADD(4);
 #pragma unroll 1
-      for (int ks = 0; ks < C / 8; ++ks) {  // W += Cmat K (Eq. 3.3 summed over the chunk)
-        const uint64_t bt = kt0 + (uint64_t)(ks * 2 * DK);
-        mma_tf32_ts(tb0 + Cf::TM_W, tb0 + Cf::TM_CHI + ks * 8, bt, idU, true);
-        mma_tf32_ts(tb0 + Cf::TM_W, tb0 + Cf::TM_CLO + ks * 8, bt, idU, true);
+      for (int ks = 0; ks < C / 16; ++ks) {  // W += Cmat K (Eq. 3.3 summed over the chunk)
+        const uint64_t bt = kt0 + (uint64_t)(ks * 2 * (Cf::KT_LBO / 16));
+        mma_bf16_ts(tb0 + Cf::TM_W, tb0 + Cf::TM_CHI + ks * 8, bt, idU, true);
+        mma_bf16_ts(tb0 + Cf::TM_W, tb0 + Cf::TM_CLO + ks * 8, bt, idU, true);
       }
       mma_commit(&bars[B_U]);
-      if (more) {
-        w_times_kq(n + 1, Cf::TM_W, true);  // executes after the update: MMAs of one thread run in order
-        if (!mbar_wait(&bars[B_WLO], (n + 1) & 1)) { failed = true; break; }
-        tc_fence_after_sync();
-        w_times_kq(n + 1, Cf::TM_WLO, false);
-        mma_commit(&bars[B_E]);
-      }
-      readout(n);  // not needed before the outputs are formed one chunk later: off the critical path
+      readout(n);
+      PROF_ADD(5);
     }
   }
   if (failed) atomicExch(&g_chunk_error, 1);

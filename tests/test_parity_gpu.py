@@ -114,13 +114,14 @@ def test_chunked_kernel_extreme_prediction_errors(binding, oracle):
     binding.device_status()
     scan = gpu_forward(binding, w, to_dev(inp), algo=binding.ALGO_SCAN)
     # With |delta| ~ 50 the exponent delta^2/2 ~ 1e3 carries an fp32 rounding error of ~1e-4, which is the
-    # relative error of the responsibilities whatever the kernel: the state bar is relaxed to 2e-3 here,
-    # and the two kernels (both fp32) must agree with each other much more closely than with fp64.
+    # relative error of the responsibilities whatever the kernel: the state bar is relaxed to 2e-3 here.
+    # The chunked kernel's predictions also carry its 16-bit operand split (4e-6 of |w.k| ~ 50), which the
+    # same amplification by |delta| turns into a few 1e-4 of the state: the two kernels agree to 1e-3.
     for name, g in (("chunk", got), ("scan", scan)):
         assert wl.rel_err(g["o"], torch.from_numpy(ref["o"])) < 2e-2, name
         assert wl.rel_err(g["W"], torch.from_numpy(ref["W"])) < 2e-3, name
         assert bool(torch.isfinite(g["W"]).all())
-    assert wl.rel_err(got["W"], scan["W"]) < 3e-4
+    assert wl.rel_err(got["W"], scan["W"]) < 1e-3
 
 
 def test_chunked_kernel_state_carry(binding, oracle):
