@@ -43,6 +43,7 @@
 
 #include <cuda_bf16.h>
 
+#include <atomic>
 #include <type_traits>
 
 #include "swila_common.cuh"
@@ -60,10 +61,28 @@ static __device__ int g_chunk_error = 0;
 // role of block 0 and written out at the end; per-block totals for every block.
 static __device__ long long g_chunk_prof[4 * 8];
 static __device__ long long g_chunk_blk[3 * 1024];  // per block: cycles, SM id, start time (ns)
+#ifdef SWILA_CHUNK_PHASES
 #define PROF_ADD(i) do { long long now_ = clock64(); prof_acc[i] += now_ - prof_t; prof_t = now_; } while (0)
 #else
 #define PROF_ADD(i) do {} while (0)
 #endif
+#else
+#define PROF_ADD(i) do {} while (0)
+#endif
+
+// How the (tile, chunk) work items are spread over the blocks of a launch.  The ntiles * nch chunks, tile
+// after tile, are cut into equal runs of `per` chunks, one run per block; within a run the piece that
+// ends in the middle of a tile comes first and the piece that starts in the middle of a tile comes last.  The block that owns
+// the head of a split tile leaves the state in the state output and releases flags[tile] = epoch; the
+// block that owns the tail acquires it before loading that state.  With per == nch every block owns
+// exactly one tile and no block ever waits.
+struct ChunkSched {
+  int ntiles, nch, per;
+  unsigned epoch;
+  unsigned *flags;
+};
+constexpr int kChunkFlagSlots = 8, kChunkFlagTiles = 4096;
+static __device__ unsigned g_chunk_flags[kChunkFlagSlots][kChunkFlagTiles];
 
 template <int J_, int DK_>
 struct ChunkCfg {
@@ -115,7 +134,8 @@ struct ChunkCfg {
   static constexpr int OFF_BQ = OFF_G + 2 * C * C * 4;        // 2 x { hi, lo } readout operand tiles
   static constexpr int OFF_GX = OFF_BQ + 2 * 2 * BQ_TILE;     // { hi, lo } cross-chunk operand tiles
   static constexpr int OFF_OST = OFF_GX + 2 * GX_TILE;        // 2 x [C][COLS] bf16 output staging
-  static constexpr int OFF_BAR = OFF_OST + 2 * C * COLS * ES;
+  static constexpr int OFF_P0 = OFF_OST + 2 * C * COLS * ES;  // [C/4][NROW] float4: a chunk's P0 rows, kept for the rare redo
+  static constexpr int OFF_BAR = OFF_P0 + C * NROW * 4;
   static constexpr int SMEM_BYTES = OFF_BAR + 128;
   static_assert(RAW_BYTES % 16 == 0 && RPQ_BYTES % 16 == 0 && (COLS * ES) % 16 == 0, "alignment");
   static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
@@ -142,9 +162,9 @@ __device__ __forceinline__ void bf16_split2(float x0, float x1, uint32_t &hi, ui
 // FULL: every token of the chunk and every column of the slice exists (no predicates)
 template <class Cf, bool FULL>
 __device__ __forceinline__ void chunk_issue_raw_impl(const ScanParams &p, unsigned char *tile, unsigned char *raw,
-                                                unsigned char *rawpq, size_t tok0, int t0, int col0, int h) {
+                                                unsigned char *rawpq, size_t tok0, int Tseg, int t0, int col0, int h) {
   constexpr int J = Cf::J, DK = Cf::DK, C = Cf::C, ES = Cf::ES, C_K = Cf::C_K, C_V = Cf::C_V;
-  const int nvalid = min(C, p.T - t0);
+  const int nvalid = min(C, Tseg - t0);
   const size_t tokb = tok0 + (size_t)t0;
   const char *kb = (const char *)p.k + tokb * DK * ES;
   const char *qb = (const char *)p.q + tokb * DK * ES;
@@ -178,13 +198,14 @@ __device__ __forceinline__ void chunk_issue_raw_impl(const ScanParams &p, unsign
 
 template <class Cf>
 __device__ __forceinline__ void chunk_issue_raw(const ScanParams &p, unsigned char *tile, unsigned char *raw,
-                                                unsigned char *rawpq, size_t tok0, int t0, int col0, int h) {
-  if (t0 + Cf::C <= p.T && col0 + Cf::COLS <= p.Dv) chunk_issue_raw_impl<Cf, true>(p, tile, raw, rawpq, tok0, t0, col0, h);
-  else chunk_issue_raw_impl<Cf, false>(p, tile, raw, rawpq, tok0, t0, col0, h);
+                                                unsigned char *rawpq, size_t tok0, int Tseg, int t0, int col0, int h) {
+  if (t0 + Cf::C <= Tseg && col0 + Cf::COLS <= p.Dv) chunk_issue_raw_impl<Cf, true>(p, tile, raw, rawpq, tok0, Tseg, t0, col0, h);
+  else chunk_issue_raw_impl<Cf, false>(p, tile, raw, rawpq, tok0, Tseg, t0, col0, h);
 }
 
 template <class Cf, bool RDEBUG>
-__global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_constant__ ScanParams p) {
+__global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_constant__ ScanParams p,
+                                                                     const __grid_constant__ ChunkSched sched) {
   using namespace umma;
   constexpr int J = Cf::J, DK = Cf::DK, C = Cf::C, NROW = Cf::NROW, COLS = Cf::COLS;
   extern __shared__ __align__(128) unsigned char smem[];
@@ -194,17 +215,73 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   unsigned char *BQ_all = smem + Cf::OFF_BQ;
   unsigned char *GX_all = smem + Cf::OFF_GX;
   __nv_bfloat16 *ostage = reinterpret_cast<__nv_bfloat16 *>(smem + Cf::OFF_OST);
+  float4 *p0s = reinterpret_cast<float4 *>(smem + Cf::OFF_P0);
   uint64_t *bars = reinterpret_cast<uint64_t *>(smem + Cf::OFF_BAR);
   uint32_t *tmem_base_s = reinterpret_cast<uint32_t *>(bars + B_COUNT);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int nslice = (p.Dv + COLS - 1) / COLS;
-  const int bh = blockIdx.x / nslice;
-  const int col0 = (blockIdx.x - bh * nslice) * COLS;
-  const size_t tok0 = (size_t)bh * p.T;
-  const int nchunks = (p.T + C - 1) / C;
-
+  uint32_t *fail_s = tmem_base_s + 1;  // set by any thread whose bounded wait expired: no further piece is started
+  // this block's run of chunks and the pieces (tile, first chunk, end chunk) it falls into
+  const long long run0 = (long long)blockIdx.x * sched.per;
+  const long long run1 = min((long long)sched.ntiles * sched.nch, run0 + sched.per);
+  const int tile_first = (int)(run0 / sched.nch), chunk_first = (int)(run0 % sched.nch);
+  const int npieces = run1 > run0 ? (int)((run1 - 1) / sched.nch) - tile_first + 1 : 0;
   if (warp == 8) tmem_alloc(tmem_base_s, Cf::TM_ALLOC);
+  if (tid == 0) *fail_s = 0;
+  const uint32_t tb_lane = ((uint32_t)((warp & 3) * 32) << 16);  // this warp's lane quarter
+  // row served by this thread in either 128-thread role
+  const int r = tid & 127;
+  const int dl = r / J, j = r % J;
+#ifdef SWILA_CHUNK_PROFILE
+  long long prof_t = clock64();
+  const long long prof_t0 = prof_t;
+  long long prof_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  if (tid == 0 && blockIdx.x < 1024) {
+    unsigned smid;
+    unsigned long long ns;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns));
+    g_chunk_blk[1024 + blockIdx.x] = smid;
+    g_chunk_blk[2048 + blockIdx.x] = (long long)ns;
+  }
+#endif
+
+#pragma unroll 1
+  for (int pi = 0; pi < npieces; ++pi) {
+    // the piece being processed (uniform over the block).  Order: a trailing piece that ends inside a tile
+    // (a head, whose state another block waits for) first, whole tiles next, a leading piece that starts
+    // inside a tile (a tail, which waits for another block's head) last.  A head is shorter than a run, so
+    // it is finished before the block that owns the tail gets there.
+    const bool has_tail = chunk_first > 0;
+    const bool has_head = run1 % sched.nch != 0 && !(npieces == 1 && has_tail);
+    int ps;
+    if (has_head && pi == 0) {
+      ps = npieces - 1;
+    } else {
+      const int k = pi - (has_head ? 1 : 0);
+      const int mid = npieces - (has_head ? 1 : 0) - (has_tail ? 1 : 0);
+      ps = k < mid ? k + (has_tail ? 1 : 0) : 0;
+    }
+    const int tl = tile_first + ps;
+    const int cb = ps == 0 ? chunk_first : 0;
+    const int ce = (int)min((long long)sched.nch, run1 - (long long)tl * sched.nch);
+    const int bh = tl / nslice;
+    const int col0 = (tl - bh * nslice) * COLS;
+    const int nchunks = ce - cb;
+    const int Tseg = min(p.T, ce * C) - cb * C;
+    const size_t tok0 = (size_t)bh * p.T + (size_t)cb * C;
+    const bool from_flag = cb > 0, to_flag = ce < sched.nch;  // state handed over from / to another block
+    unsigned *const flag = sched.flags + tl;
+    const int col = col0 + dl;
+    const bool col_ok = col < p.Dv;
+    bool failed = false;
+  if (pi > 0) {  // every barrier of the previous piece is quiescent: all its phases were waited for
+    __syncthreads();
+    if (tid == 0) {
+      for (int b = 0; b < B_COUNT; ++b) mbar_inval(&bars[b]);
+    }
+  }
   if (tid == 0) {
     mbar_init(&bars[B_E], 1);
     mbar_init(&bars[B_G], 1);
@@ -223,33 +300,15 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
+  if (*fail_s) break;
   const uint32_t tb0 = *tmem_base_s;
-  const uint32_t tb = tb0 + ((uint32_t)((warp & 3) * 32) << 16);  // this warp's lane quarter
-  // row served by this thread in either 128-thread role
-  const int r = tid & 127;
-  const int dl = r / J, j = r % J;
-  const int col = col0 + dl;
-  const bool col_ok = col < p.Dv;
-  bool failed = false;
-#ifdef SWILA_CHUNK_PROFILE
-  long long prof_t = clock64();
-  const long long prof_t0 = prof_t;
-  long long prof_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-  if (tid == 0 && blockIdx.x < 1024) {
-    unsigned smid;
-    unsigned long long ns;
-    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns));
-    g_chunk_blk[1024 + blockIdx.x] = smid;
-    g_chunk_blk[2048 + blockIdx.x] = (long long)ns;
-  }
-#endif
+  const uint32_t tb = tb0 + tb_lane;
 
   // outputs of one chunk (Eq. 3.5): o_td = sum_j pi^q_j (w_t.q_t)_j, pi^q = softmax over the J
   // components of a column
   auto write_outputs = [&](int n) {
     const int t0 = n * C;
-    const int nvalid = min(C, p.T - t0);
+    const int nvalid = min(C, Tseg - t0);
     const __nv_bfloat16 *rpq = reinterpret_cast<const __nv_bfloat16 *>(smem + Cf::OFF_RPQ + (n & 3) * Cf::RPQ_BYTES);
     __nv_bfloat16 *ost = ostage + (n & 1) * C * COLS;
     tc_fence_after_sync();
@@ -325,7 +384,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
 #pragma unroll 1
     for (int n = 0; n < nchunks && !failed; ++n) {
       const int t0 = n * C;
-      const int nvalid = min(C, p.T - t0);
+      const int nvalid = min(C, Tseg - t0);
       const unsigned char *raw = smem + Cf::OFF_RAW + (n & 1) * Cf::RAW_BYTES;
       const __nv_bfloat16 *rv = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_V);
       const float *bes = reinterpret_cast<const float *>(raw + Cf::R_B);
@@ -348,6 +407,9 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         tmem_st16(tb + Cf::TM_QD + (n & 1) * C + cc * 16, b);
 #pragma unroll
         for (int i = 0; i < 16; ++i) pred0[cc * 16 + i] = a[i];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)  // copy for the redo path, so that the values need not stay in registers
+          p0s[((cc * 4 + i) * NROW + r)] = make_float4(a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
       }
       tmem_st_wait();
       tc_fence_before_sync();
@@ -447,6 +509,11 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       PROF_ADD(5);
       if (__any_sync(0xffffffffu, unsafe)) {
         tmem_st_wait();
+#pragma unroll
+        for (int i = 0; i < C / 4; ++i) {  // P0 again, from the copy in shared memory
+          const float4 v4 = p0s[i * NROW + r];
+          pred0[4 * i] = v4.x; pred0[4 * i + 1] = v4.y; pred0[4 * i + 2] = v4.z; pred0[4 * i + 3] = v4.w;
+        }
         sequential(std::true_type{});
       }
       tmem_st_wait();
@@ -474,6 +541,11 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         for (int i = 0; i < 4; ++i)
           __stcs(reinterpret_cast<float4 *>(dst + cc * 16 + i * 4), make_float4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]));
       }
+    }
+    if (to_flag) {  // the rest of this tile belongs to another block: publish the state
+      __threadfence();
+      named_bar_sync(4, 128);
+      if (r == 0 && !failed) st_release_gpu(flag, sched.epoch);
     }
   } else if (warp < 8) {
     // =============================== helper warps ============================================
@@ -567,13 +639,26 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     const bool spill_mine[2] = {warp < 6, warp >= 6};  // which parity of chunks this warp's lanes hold
 
     // ---- prologue: stage chunks 0 and 1, state row -> tensor memory, operands of chunk 0 ----
-    chunk_issue_raw<Cf>(p, tile, smem + Cf::OFF_RAW, smem + Cf::OFF_RPQ, tok0, 0, col0, h);
+    chunk_issue_raw<Cf>(p, tile, smem + Cf::OFF_RAW, smem + Cf::OFF_RPQ, tok0, Tseg, 0, col0, h);
     cp_async_commit();
     if (nchunks > 1)
-      chunk_issue_raw<Cf>(p, tile, smem + Cf::OFF_RAW + Cf::RAW_BYTES, smem + Cf::OFF_RPQ + Cf::RPQ_BYTES, tok0, C, col0, h);
+      chunk_issue_raw<Cf>(p, tile, smem + Cf::OFF_RAW + Cf::RAW_BYTES, smem + Cf::OFF_RPQ + Cf::RPQ_BYTES, tok0, Tseg, C, col0, h);
     cp_async_commit();
+    if (from_flag) {  // the head of this tile was processed by another block: wait for its state
+      if (h == 0) {
+        bool seen = false;
+        for (int spin = 0; spin < (1 << 21) && !seen; ++spin) {
+          seen = ld_acquire_gpu(flag) == sched.epoch;
+          if (!seen) __nanosleep(100);
+        }
+        if (!seen) *fail_s = 1;
+      }
+      named_bar_sync(1, 128);
+      if (*fail_s) failed = true;
+    }
     {
-      const float *src = (p.W_in && col_ok) ? p.W_in + (((size_t)bh * J + j) * p.Dv + col) * DK : nullptr;
+      const float *w_src = from_flag ? p.W_out : p.W_in;
+      const float *src = (w_src && col_ok && !failed) ? w_src + (((size_t)bh * J + j) * p.Dv + col) * DK : nullptr;
 #pragma unroll
       for (int cc = 0; cc < DK / 16; ++cc) {
         float w[16];
@@ -581,7 +666,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
           float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (src) t = __ldcs(reinterpret_cast<const float4 *>(src + cc * 16 + i * 4));
+          if (src) t = __ldcg(reinterpret_cast<const float4 *>(src + cc * 16 + i * 4));
           w[4 * i] = t.x; w[4 * i + 1] = t.y; w[4 * i + 2] = t.z; w[4 * i + 3] = t.w;
         }
 #pragma unroll
@@ -654,7 +739,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       PROF_ADD(4);
       if (n + 2 < nchunks)
         chunk_issue_raw<Cf>(p, tile, smem + Cf::OFF_RAW + (n & 1) * Cf::RAW_BYTES, smem + Cf::OFF_RPQ + ((n + 2) & 3) * Cf::RPQ_BYTES,
-                            tok0, (n + 2) * C, col0, h);
+                            tok0, Tseg, (n + 2) * C, col0, h);
       cp_async_commit();
       // (4) W has been updated with chunk n: split it into operand parts again
       if (!mbar_wait(&bars[B_U], n & 1)) { failed = true; break; }
@@ -786,16 +871,37 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       PROF_ADD(5);
     }
   }
-  if (failed) atomicExch(&g_chunk_error, 1);
+  if (failed) {
+    atomicExch(&g_chunk_error, 1);
+    *fail_s = 1;
+  }
+  }  // pieces
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 8) tmem_dealloc(tb0, Cf::TM_ALLOC);
+  if (warp == 8) tmem_dealloc(*tmem_base_s, Cf::TM_ALLOC);
 #ifdef SWILA_CHUNK_PROFILE
   if (tid == 0 && blockIdx.x < 1024) g_chunk_blk[blockIdx.x] = clock64() - prof_t0;
   if (blockIdx.x == 0 && (tid & 127) == 0 && tid < 512) {
     for (int i = 0; i < 8; ++i) g_chunk_prof[(tid >> 7) * 8 + i] = prof_acc[i];
   }
 #endif
+}
+
+// Number of SMs of the current device (one block is resident per SM).
+inline int chunk_sm_count() {
+  int dev = 0, n = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+  return n;
+}
+
+// Launch counter shared by every instantiation: the value a launch publishes in the hand-over flags
+// (never 0, the flags' initial value).
+inline unsigned chunk_next_epoch() {
+  static std::atomic<unsigned> counter{0};
+  unsigned e = ++counter;
+  if (e == 0) e = ++counter;
+  return e;
 }
 
 template <int J, int DK>
@@ -805,9 +911,35 @@ int launch_chunk(const LaunchArgs &a) {
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cf::SMEM_BYTES);
   if (e != cudaSuccess) return (int)e;
   const long long nslice = (a.p.Dv + Cf::COLS - 1) / Cf::COLS;
-  const long long grid = nslice * a.p.B * a.p.H;
-  if (grid <= 0 || grid > 0x7fffffffLL) return (int)cudaErrorInvalidConfiguration;
-  kern<<<(unsigned)grid, Cf::NT, Cf::SMEM_BYTES, a.stream>>>(a.p);
+  const long long ntiles = nslice * a.p.B * a.p.H;
+  const long long nch = (a.p.T + Cf::C - 1) / Cf::C;
+  if (ntiles <= 0 || ntiles > 0x7fffffffLL || nch <= 0 || nch > 0x7fffffffLL) return (int)cudaErrorInvalidConfiguration;
+  ChunkSched sc{(int)ntiles, (int)nch, (int)nch, 0u, nullptr};
+  ScanParams prm = a.p;
+
+  // More tiles than SMs, not a whole number of waves: cut the chunk sequence into one equal run per SM
+  // instead of whole tiles, so that the last wave is not half empty.  The state of a split tile travels
+  // through the state output, hence only when that is given; blocks of such a launch wait for each other,
+  // hence the cooperative launch (all blocks resident or no launch at all).
+  const int nsm = chunk_sm_count();
+  if (nsm > 0 && a.p.W_out && ntiles > nsm && ntiles <= kChunkFlagTiles && nch >= 16) {
+    const long long total = ntiles * nch;
+    const long long per = (total + nsm - 1) / nsm;
+    const long long plain = ((ntiles + nsm - 1) / nsm) * nch;
+    if (per >= nch && per * 100 <= plain * 97) {
+      unsigned *flags = nullptr;
+      if (cudaGetSymbolAddress((void **)&flags, g_chunk_flags) == cudaSuccess) {
+        const unsigned epoch = chunk_next_epoch();
+        ChunkSched ss{(int)ntiles, (int)nch, (int)per, epoch, flags + (size_t)(epoch % kChunkFlagSlots) * kChunkFlagTiles};
+        const long long grid = (total + per - 1) / per;
+        void *args[] = {(void *)&prm, (void *)&ss};
+        e = cudaLaunchCooperativeKernel((const void *)kern, dim3((unsigned)grid), dim3(Cf::NT), args, Cf::SMEM_BYTES, a.stream);
+        if (e == cudaSuccess) return (int)cudaGetLastError();
+        (void)cudaGetLastError();  // not launched (e.g. the blocks cannot all be resident): fall back to whole tiles
+      }
+    }
+  }
+  kern<<<(unsigned)ntiles, Cf::NT, Cf::SMEM_BYTES, a.stream>>>(prm, sc);
   return (int)cudaGetLastError();
 }
 
