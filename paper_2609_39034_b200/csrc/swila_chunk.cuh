@@ -647,9 +647,13 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     if (from_flag) {  // the head of this tile was processed by another block: wait for its state
       if (h == 0) {
         bool seen = false;
-        for (int spin = 0; spin < (1 << 21) && !seen; ++spin) {
+        const unsigned long long t_begin = global_timer_ns();
+        while (!seen) {  // bounded by wall time (about two seconds)
           seen = ld_acquire_gpu(flag) == sched.epoch;
-          if (!seen) __nanosleep(100);
+          if (!seen) {
+            if (global_timer_ns() - t_begin > 2000000000ull) break;
+            __nanosleep(100);
+          }
         }
         if (!seen) *fail_s = 1;
       }
@@ -692,17 +696,19 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     cook_kt(0);
     fence_async_smem();
     mbar_arrive(&bars[B_KT]);
+    // every helper waits for the first Gram batch: its completion also tells that the MMA thread has consumed
+    // the first phase of KQ, so the second one may be completed
+    if (!mbar_wait(&bars[B_G], 0)) failed = true;
+    if (spill_mine[0]) {
+      tc_fence_after_sync();
+      if (!failed) spill_gram(0);
+      mbar_arrive(&bars[B_GS]);
+    }
     if (nchunks > 1) {
       cp_async_wait<0>();
       named_bar_sync(1, 128);
       fence_async_smem();
       mbar_arrive(&bars[B_KQ]);
-    }
-    if (spill_mine[0]) {
-      if (!mbar_wait(&bars[B_G], 0)) failed = true;
-      tc_fence_after_sync();
-      if (!failed) spill_gram(0);
-      mbar_arrive(&bars[B_GS]);
     }
 
     // Per chunk n, in the order of what the other roles wait for first.

@@ -31,12 +31,35 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait for the phase with the given parity; false on expiry.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, uint32_t max_spins = (1u << 22)) {
+// Bounded wait for the phase with the given parity; false on expiry.  The bound is wall time (about two
+// seconds, checked every 256 polls): one poll may itself suspend the thread for a while, so a poll count
+// alone would not bound the wait.
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __noinline__ bool mbar_wait_poll(uint32_t bar_addr, uint32_t parity) {
+  const unsigned long long t0 = global_timer_ns();
 #pragma unroll 1
-  for (uint32_t i = 0; i < max_spins; ++i)
+  for (uint32_t i = 1;; ++i) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar_addr), "r"(parity)
+        : "memory");
+    if (ok) return true;
+    if ((i & 255u) == 0 && global_timer_ns() - t0 > 2000000000ull) return false;
+  }
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+#pragma unroll 1
+  for (int i = 0; i < 1024; ++i)  // the common case: complete already, or within a few thousand cycles
     if (mbar_try_wait(bar, parity)) return true;
-  return false;
+  return mbar_wait_poll(smem_u32(bar), parity);
 }
 
 // Arrive (release) on a barrier of this block from an ordinary thread.

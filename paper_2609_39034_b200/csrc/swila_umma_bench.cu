@@ -35,7 +35,7 @@ __global__ void __launch_bounds__(128) umma_rate_kernel(int reps, long long *cyc
       }
     }
     mma_commit(&bar);
-    const bool ok = mbar_wait(&bar, 0, 1u << 26);
+    const bool ok = mbar_wait(&bar, 0);
     const long long t1 = clock64();
     cycles[0] = ok ? (t1 - t0) : -1;
   }
