@@ -39,7 +39,7 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-__device__ __noinline__ bool mbar_wait_poll(uint32_t bar_addr, uint32_t parity) {
+static __device__ __noinline__ bool mbar_wait_poll(uint32_t bar_addr, uint32_t parity) {
   const unsigned long long t0 = global_timer_ns();
 #pragma unroll 1
   for (uint32_t i = 1;; ++i) {
