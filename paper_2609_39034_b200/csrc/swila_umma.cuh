@@ -39,27 +39,14 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-static __device__ __noinline__ bool mbar_wait_poll(uint32_t bar_addr, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_timer_ns();
 #pragma unroll 1
   for (uint32_t i = 1;; ++i) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar_addr), "r"(parity)
-        : "memory");
-    if (ok) return true;
+    if (mbar_try_wait(bar, parity)) return true;
     if ((i & 255u) == 0 && global_timer_ns() - t0 > 2000000000ull) return false;
   }
-}
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
-#pragma unroll 1
-  for (int i = 0; i < 1024; ++i)  // the common case: complete already, or within a few thousand cycles
-    if (mbar_try_wait(bar, parity)) return true;
-  return mbar_wait_poll(smem_u32(bar), parity);
 }
 
 // Arrive (release) on a barrier of this block from an ordinary thread.
