@@ -72,9 +72,13 @@ enum {
   SWILA_ALGO_SCAN_NARROW = 3, /* the same scan with 16 key dimensions per lane (more, lighter
                               warps); ungated shapes with Dk = 128, J >= 4 only */
   SWILA_ALGO_CHUNK = 4     /* chunked form: the state-times-token contractions of 32-token chunks
-                              on the tcgen05 tensor cores (TF32 hi/lo split, FP32 accumulation in
-                              tensor memory), the E-step and intra-chunk corrections on the FP32
-                              ALUs.  bf16 io, Dk in {64, 128}, J >= 4, no TEMPORAL / GATED */
+                              on the tcgen05 tensor cores (bf16 hi/lo operand split, FP32
+                              accumulation in tensor memory), the E-step and intra-chunk
+                              corrections on the FP32 ALUs.  bf16 io, Dk in {64, 128}, J in {4, 8},
+                              no TEMPORAL / GATED.  When a state output is given and the tiles do
+                              not fill a whole number of waves, the launch is cooperative and
+                              balances chunks over the SMs; up to 8 such launches may overlap on
+                              one device */
 };
 
 typedef struct {

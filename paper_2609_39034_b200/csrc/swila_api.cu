@@ -106,12 +106,15 @@ static int run(const swila_shape_t *s, int T, const void *q, const void *k, cons
   int rc = -1000;
   // AUTO: the chunked tensor-core kernel whenever it applies and the sequence is long enough to
   // amortise its per-chunk set-up; the scan otherwise (fp32 io, TEMPORAL / GATED, decode).
-  const bool chunk_ok = s->io_dtype == SWILA_IO_BF16 && s->flags == 0 && (s->Dk == 64 || s->Dk == 128) && s->J >= 4;
+  const bool chunk_ok = s->io_dtype == SWILA_IO_BF16 && s->flags == 0 && (s->Dk == 64 || s->Dk == 128) &&
+                        (s->J == 4 || s->J == 8);
   if (s->algo == SWILA_ALGO_CHUNK || (s->algo == SWILA_ALGO_AUTO && chunk_ok && T >= 64)) {
     rc = chunk_dispatch(a);
-    if (rc == -1000) return SWILA_ERR_UNSUPPORTED;
-    if (rc != 0) return cuda_fail((cudaError_t)rc);
-    return SWILA_OK;
+    if (rc == -1000 && s->algo == SWILA_ALGO_CHUNK) return SWILA_ERR_UNSUPPORTED;
+    if (rc != -1000) {
+      if (rc != 0) return cuda_fail((cudaError_t)rc);
+      return SWILA_OK;
+    }
   }
 #define SWILA_CASE(DK)                                                                          \
   case DK:                                                                                      \
