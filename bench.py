@@ -36,8 +36,6 @@ HEADLINE = 2  # config index of the workload the metric is quoted on
 
 # DRAM traffic of one launch on the headline workload, from the ncu captures summarised under
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum: 2.174 GB chunked kernel, 2.188 GB scan kernel).
-# The chunked kernel's capture predates its bf16-operand generation; its path to HBM (every input byte
-# staged once with cp.async, every output byte stored once) is the same in both.
 NCU_TRAFFIC_BYTES_PER_LAUNCH = 2.174e9
 
 

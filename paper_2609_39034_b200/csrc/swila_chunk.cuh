@@ -76,8 +76,12 @@ static __device__ long long g_chunk_blk[3 * 1024];  // per block: cycles, SM id,
 // the head of a split tile leaves the state in the state output and releases flags[tile] = epoch; the
 // block that owns the tail acquires it before loading that state.  With per == nch every block owns
 // exactly one tile and no block ever waits.
+// `gang` > 1: the blocks come in gangs of `gang` = column slices per (batch, head); the schedule above is then
+// laid over (batch, head) units and the blocks of a gang walk it in step, one column slice each, so that the
+// slices of one (batch, head) -- which share every 128-byte line of the gate tensors and all of k and q --
+// are fetched at the same time and meet in L2 (without this the DRAM read traffic doubles).
 struct ChunkSched {
-  int ntiles, nch, per;
+  int ntiles, nch, per, gang;
   unsigned epoch;
   unsigned *flags;
 };
@@ -223,7 +227,8 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   const int nslice = (p.Dv + COLS - 1) / COLS;
   uint32_t *fail_s = tmem_base_s + 1;  // set by any thread whose bounded wait expired: no further piece is started
   // this block's run of chunks and the pieces (tile, first chunk, end chunk) it falls into
-  const long long run0 = (long long)blockIdx.x * sched.per;
+  const int gang_slice = (int)(blockIdx.x % sched.gang);
+  const long long run0 = (long long)(blockIdx.x / sched.gang) * sched.per;
   const long long run1 = min((long long)sched.ntiles * sched.nch, run0 + sched.per);
   const int tile_first = (int)(run0 / sched.nch), chunk_first = (int)(run0 % sched.nch);
   const int npieces = run1 > run0 ? (int)((run1 - 1) / sched.nch) - tile_first + 1 : 0;
@@ -266,13 +271,13 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     const int tl = tile_first + ps;
     const int cb = ps == 0 ? chunk_first : 0;
     const int ce = (int)min((long long)sched.nch, run1 - (long long)tl * sched.nch);
-    const int bh = tl / nslice;
-    const int col0 = (tl - bh * nslice) * COLS;
+    const int bh = sched.gang > 1 ? tl : tl / nslice;
+    const int col0 = (sched.gang > 1 ? gang_slice : tl - bh * nslice) * COLS;
     const int nchunks = ce - cb;
     const int Tseg = min(p.T, ce * C) - cb * C;
     const size_t tok0 = (size_t)bh * p.T + (size_t)cb * C;
     const bool from_flag = cb > 0, to_flag = ce < sched.nch;  // state handed over from / to another block
-    unsigned *const flag = sched.flags + tl;
+    unsigned *const flag = sched.flags + (sched.gang > 1 ? tl * sched.gang + gang_slice : tl);
     const int col = col0 + dl;
     const bool col_ok = col < p.Dv;
     bool failed = false;
@@ -920,24 +925,28 @@ int launch_chunk(const LaunchArgs &a) {
   const long long ntiles = nslice * a.p.B * a.p.H;
   const long long nch = (a.p.T + Cf::C - 1) / Cf::C;
   if (ntiles <= 0 || ntiles > 0x7fffffffLL || nch <= 0 || nch > 0x7fffffffLL) return (int)cudaErrorInvalidConfiguration;
-  ChunkSched sc{(int)ntiles, (int)nch, (int)nch, 0u, nullptr};
+  ChunkSched sc{(int)ntiles, (int)nch, (int)nch, 1, 0u, nullptr};
   ScanParams prm = a.p;
 
-  // More tiles than SMs, not a whole number of waves: cut the chunk sequence into one equal run per SM
-  // instead of whole tiles, so that the last wave is not half empty.  The state of a split tile travels
-  // through the state output, hence only when that is given; blocks of such a launch wait for each other,
-  // hence the cooperative launch (all blocks resident or no launch at all).
+  // More tiles than SMs, not a whole number of waves: cut the chunk sequence into equal runs instead of whole
+  // tiles, so that the last wave is not half empty.  The runs are laid over (batch, head) units and walked by
+  // gangs of nslice blocks (one column slice each, see ChunkSched).  The state of a split tile travels through
+  // the state output, hence only when that is given; blocks of such a launch wait for each other, hence the
+  // cooperative launch (all blocks resident or no launch at all).
   const int nsm = chunk_sm_count();
-  if (nsm > 0 && a.p.W_out && ntiles > nsm && ntiles <= kChunkFlagTiles && nch >= 16) {
-    const long long total = ntiles * nch;
-    const long long per = (total + nsm - 1) / nsm;
+  const long long nbh = (long long)a.p.B * a.p.H;
+  const long long gangs = nslice > 0 ? nsm / nslice : 0;
+  if (gangs > 0 && a.p.W_out && nbh > gangs && ntiles <= kChunkFlagTiles && nch >= 16) {
+    const long long total = nbh * nch;
+    const long long per = (total + gangs - 1) / gangs;
     const long long plain = ((ntiles + nsm - 1) / nsm) * nch;
     if (per >= nch && per * 100 <= plain * 97) {
       unsigned *flags = nullptr;
       if (cudaGetSymbolAddress((void **)&flags, g_chunk_flags) == cudaSuccess) {
         const unsigned epoch = chunk_next_epoch();
-        ChunkSched ss{(int)ntiles, (int)nch, (int)per, epoch, flags + (size_t)(epoch % kChunkFlagSlots) * kChunkFlagTiles};
-        const long long grid = (total + per - 1) / per;
+        ChunkSched ss{(int)nbh, (int)nch, (int)per, (int)nslice, epoch,
+                      flags + (size_t)(epoch % kChunkFlagSlots) * kChunkFlagTiles};
+        const long long grid = ((total + per - 1) / per) * nslice;
         void *args[] = {(void *)&prm, (void *)&ss};
         e = cudaLaunchCooperativeKernel((const void *)kern, dim3((unsigned)grid), dim3(Cf::NT), args, Cf::SMEM_BYTES, a.stream);
         if (e == cudaSuccess) return (int)cudaGetLastError();
