@@ -49,9 +49,6 @@
 #include "swila_common.cuh"
 #include "swila_umma.cuh"
 
-#ifndef SWILA_EXP
-#define SWILA_EXP 0
-#endif
 namespace swila {
 
 // Set when a bounded wait on a completion barrier expires (never expected).
@@ -723,9 +720,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       PROF_ADD(0);
       if (more) {
         // (1) gates of chunk n+1 for the row warps, then its Gram batch
-#if SWILA_EXP != 2
         cook_be(smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES);
-#endif
         mbar_arrive(&bars[B_BE]);
         PROF_ADD(1);
         if (spill_mine[(n + 1) & 1]) {
@@ -739,9 +734,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       // (2) outputs of chunk n-1, whose readouts completed shortly after chunk n started
       if (n > 0) {
         if (!mbar_wait(&bars[B_QD], (n - 1) & 1)) { failed = true; break; }
-#if SWILA_EXP != 1
         write_outputs(n - 1);
-#endif
         mbar_arrive(&bars[B_OD]);
       }
       PROF_ADD(3);
@@ -757,9 +750,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       PROF_ADD(5);
       if (more) {
         tc_fence_after_sync();
-#if SWILA_EXP != 3
         refresh_parts();
-#endif
         mbar_arrive(&bars[B_WP]);
       }
       PROF_ADD(6);
