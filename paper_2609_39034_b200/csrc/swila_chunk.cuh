@@ -41,6 +41,7 @@
 //   warp 8, lane 0   issues every tcgen05.mma and commits them to the barriers.
 #pragma once
 
+#include <cuda.h>  // CUtensorMap and its enums (types only; the encoder is fetched through the runtime)
 #include <cuda_bf16.h>
 
 #include <atomic>
@@ -107,17 +108,24 @@ struct ChunkCfg {
   // token at c*TILE_LBO + row*16, rows [K_even ; Q_even ; K_odd ; Q_odd]: the chunks of both parities
   // side by side, so that one 128-row A operand covers the keys of two consecutive chunks.  cp.async
   // writes it directly from global memory.
-  static constexpr int TILE_LBO = 4 * C * 16;
+  static constexpr int TILE_LBO = 4 * C * 16 + 16;  // + 16: consecutive columns start 4 banks apart (conflict-free
+                                                    // cp.async stores and transposing reads)
   static constexpr int TILE_BYTES = (DK / 8) * TILE_LBO;
   // raw stages (2-deep ring): v [C][COLS] bf16; beta logits [C][J][COLS] bf16, overwritten in place by the
   // helpers with beta = sigmoid(.) as fp32 [C][NROW] (hence the fp32-sized slot); pik logits [C][J][COLS]
   // bf16.  The query-prior logits piq [C][J][COLS] live in their own 4-deep ring because the outputs of
   // chunk n are formed while chunk n+2 is being fetched.
+  // Gate rows are fetched 8 columns wider than the slice (GROW = COLS + 8, the extra columns are never read):
+  // the 16-byte skew between rows spreads the J lanes of a column over different banks.
+  static constexpr int GROW = COLS + 8;
   static constexpr int R_V = 0;
   static constexpr int R_B = R_V + C * COLS * ES;
   static constexpr int R_PK = R_B + C * NROW * 4;
-  static constexpr int RAW_BYTES = R_PK + C * J * COLS * ES;
-  static constexpr int RPQ_BYTES = C * J * COLS * ES;
+  static constexpr int RAW_BYTES = R_PK + C * J * GROW * ES;
+  static constexpr int RPQ_BYTES = C * J * GROW * ES;
+  // bytes one chunk's tensor copies deliver: v and three gate tensors (k and q come by cp.async)
+  static constexpr int STAGE_TX_BYTES = C * COLS * ES + 3 * C * J * GROW * ES;
+  static_assert(C * J * GROW * ES <= C * NROW * 4, "the beta logits must fit the slot their gates overwrite");
   static constexpr int C_K = DK * ES / 16, C_V = COLS * ES / 16;  // 16-byte units per token row / column slice
   // operand tiles written by the helpers (bf16, same unit layout, 8 tokens per unit)
   static constexpr int KT_LBO = DK * 16;           // K transposed: rows = key dims, K index = tokens
@@ -138,16 +146,18 @@ struct ChunkCfg {
   static constexpr int OFF_P0 = OFF_OST + 2 * C * COLS * ES;  // [C/4][NROW] float4: a chunk's P0 rows, kept for the rare redo
   static constexpr int OFF_BAR = OFF_P0 + C * NROW * 4;
   static constexpr int SMEM_BYTES = OFF_BAR + 128;
-  static_assert(RAW_BYTES % 16 == 0 && RPQ_BYTES % 16 == 0 && (COLS * ES) % 16 == 0, "alignment");
+  static_assert(RAW_BYTES % 128 == 0 && RPQ_BYTES % 128 == 0 && R_B % 128 == 0 && R_PK % 128 == 0 && OFF_RAW % 128 == 0 &&
+                    OFF_RPQ % 128 == 0 && TILE_LBO % 16 == 0 && (COLS * ES) % 16 == 0 && (GROW * ES) % 16 == 0,
+                "destinations of the tensor copies are 128-byte aligned, their rows multiples of 16 bytes");
   static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 };
 
 // barrier slots.  Committed by the MMA thread: E (state x [K;Q] of a chunk complete), G (Gram batch),
-// U (update of W), QD (readouts).  Arrived by threads: KQ (operand tile and gates of a chunk ready, 128
-// helpers), KT (transposed keys ready, 128 helpers), WP (operand parts of W refreshed, 128 helpers), GS
+// U (update of W), QD (readouts).  Completed by the tensor copies: KQ0 / KQ1 (everything staged for an even /
+// odd chunk has landed).  Arrived by threads: KT (transposed keys ready, 128 helpers), WP (operand parts of W refreshed, 128 helpers), GS
 // (Gram batch spilled, 2 helper warps), C (chunk finished, 128 rows), PQF ([P0|Q0] taken out of tensor
 // memory, 128 rows), BE (gates of a chunk ready, 128 helpers), OD (outputs of a chunk formed, 128 helpers).
-enum { B_E = 0, B_G, B_U, B_QD, B_KQ, B_KT, B_WP, B_GS, B_C, B_PQF, B_BE, B_OD, B_COUNT };
+enum { B_E = 0, B_G, B_U, B_QD, B_KQ0, B_KQ1, B_KT, B_WP, B_GS, B_C, B_PQF, B_BE, B_OD, B_COUNT };
 
 // bf16 split of FP32 values: hi = bf16(x) (nearest), lo = bf16(x - hi); pairs packed with the first
 // value in the low half, which is where the tensor cores expect the even K index.
@@ -159,54 +169,53 @@ __device__ __forceinline__ void bf16_split2(float x0, float x1, uint32_t &hi, ui
   lo = *reinterpret_cast<const uint32_t *>(&l);
 }
 
-// cp.async staging of one chunk by the 128 helper threads (h = 0..127)
-// FULL: every token of the chunk and every column of the slice exists (no predicates)
-template <class Cf, bool FULL>
-__device__ __forceinline__ void chunk_issue_raw_impl(const ScanParams &p, unsigned char *tile, unsigned char *raw,
-                                                unsigned char *rawpq, size_t tok0, int Tseg, int t0, int col0, int h) {
-  constexpr int J = Cf::J, DK = Cf::DK, C = Cf::C, ES = Cf::ES, C_K = Cf::C_K, C_V = Cf::C_V;
-  const int nvalid = min(C, Tseg - t0);
-  const size_t tokb = tok0 + (size_t)t0;
+// Tensor maps of the six streamed inputs (built by the host for every launch), see chunk_make_maps.
+struct ChunkMaps {
+  CUtensorMap k, q, v, be, pk, pq;
+};
+
+// Staging of chunk m of a piece.  v and the gate logits: tiled bulk tensor copies (TMA) issued by ONE thread straight
+// into the raw stage; tokens past the end of the sequence and columns past Dv are filled with zeros by the copy
+// engine, and the bytes land on `bar`.  k and q: 16-byte cp.async by all 128 helper threads (h = 0..127) into the
+// operand tile, whose 16-byte columns are too narrow for efficient tensor copies; the threads arrive on `bar`
+// themselves once their copies have landed.
+template <class Cf>
+__device__ __forceinline__ void chunk_stage(const ScanParams &p, const ChunkMaps &maps, unsigned char *tile,
+                                            unsigned char *raw, unsigned char *rawpq, int bh, int tok, int T_end, int col0,
+                                            int m, int h, uint64_t *bar) {
+  using namespace umma;
+  constexpr int DK = Cf::DK, C = Cf::C, ES = Cf::ES, C_K = Cf::C_K;
+  if (h == 0) {
+    fence_async_smem();  // the buffers were last read through ordinary loads
+    mbar_arrive_expect_tx(bar, Cf::STAGE_TX_BYTES);
+    tma_load_3d(raw + Cf::R_V, &maps.v, col0, tok, bh, bar);
+    tma_load_4d(raw + Cf::R_B, &maps.be, col0, 0, tok, bh, bar);
+    tma_load_4d(raw + Cf::R_PK, &maps.pk, col0, 0, tok, bh, bar);
+    tma_load_4d(rawpq, &maps.pq, col0, 0, tok, bh, bar);
+  }
+  const int nvalid = min(C, T_end - tok);
+  const size_t tokb = (size_t)bh * p.T + (size_t)tok;
   const char *kb = (const char *)p.k + tokb * DK * ES;
   const char *qb = (const char *)p.q + tokb * DK * ES;
-  unsigned char *trow = tile + ((t0 / C) & 1) * 2 * C * 16;  // this chunk's 2C rows of the operand tile
+  unsigned char *trow = tile + (m & 1) * 2 * C * 16;  // this chunk's 2C rows of the operand tile
+  // One warp instruction copies 8 columns x 4 tokens: each quarter-warp reads 128 contiguous bytes of one token
+  // and writes 8 columns of the tile, which the padded column stride puts into 8 different bank groups.
+  static_assert(C_K % 8 == 0, "key dims come in groups of 64");
+  constexpr int NINSTR = (C_K / 8) * (C / 4);  // per tensor and chunk
 #pragma unroll
-  for (int u = h; u < C * C_K; u += 128) {  // k and q rows of the chunk are contiguous in global memory
-    const int tok = u / C_K, c = u % C_K;
-    const bool valid = FULL || tok < nvalid;
-    cp_async16(trow + c * Cf::TILE_LBO + tok * 16, valid ? kb + u * 16 : (const char *)p.k, valid ? 16 : 0);
-    cp_async16(trow + c * Cf::TILE_LBO + (C + tok) * 16, valid ? qb + u * 16 : (const char *)p.k, valid ? 16 : 0);
+  for (int id = h >> 5; id < NINSTR; id += 4) {
+    const int c = (id % (C_K / 8)) * 8 + (h & 7), t = (id / (C_K / 8)) * 4 + ((h >> 3) & 3);
+    const bool valid = t < nvalid;
+    cp_async16(trow + c * Cf::TILE_LBO + t * 16, valid ? kb + (t * C_K + c) * 16 : (const char *)p.k, valid ? 16 : 0);
+    cp_async16(trow + c * Cf::TILE_LBO + (C + t) * 16, valid ? qb + (t * C_K + c) * 16 : (const char *)p.k, valid ? 16 : 0);
   }
-#pragma unroll
-  for (int u = h; u < C * C_V; u += 128) {
-    const int tok = u / C_V, cu = u % C_V;
-    const int col = col0 + cu * 8;
-    const bool valid = FULL || (tok < nvalid && col < p.Dv);
-    cp_async16(raw + Cf::R_V + u * 16, valid ? (const char *)p.v + ((tokb + tok) * p.Dv + col) * ES : (const char *)p.k,
-               valid ? 16 : 0);
-  }
-#pragma unroll
-  for (int u = h; u < C * J * C_V; u += 128) {
-    const int cu = u % C_V, jj = (u / C_V) % J, tok = u / (C_V * J);
-    const int col = col0 + cu * 8;
-    const bool valid = FULL || (tok < nvalid && col < p.Dv);
-    const size_t off = (((tokb + tok) * J + jj) * (size_t)p.Dv + col) * ES;
-    cp_async16(raw + Cf::R_B + u * 16, valid ? (const char *)p.beta_logit + off : (const char *)p.k, valid ? 16 : 0);
-    cp_async16(raw + Cf::R_PK + u * 16, valid ? (const char *)p.pik_logit + off : (const char *)p.k, valid ? 16 : 0);
-    cp_async16(rawpq + u * 16, valid ? (const char *)p.piq_logit + off : (const char *)p.k, valid ? 16 : 0);
-  }
-}
-
-template <class Cf>
-__device__ __forceinline__ void chunk_issue_raw(const ScanParams &p, unsigned char *tile, unsigned char *raw,
-                                                unsigned char *rawpq, size_t tok0, int Tseg, int t0, int col0, int h) {
-  if (t0 + Cf::C <= Tseg && col0 + Cf::COLS <= p.Dv) chunk_issue_raw_impl<Cf, true>(p, tile, raw, rawpq, tok0, Tseg, t0, col0, h);
-  else chunk_issue_raw_impl<Cf, false>(p, tile, raw, rawpq, tok0, Tseg, t0, col0, h);
+  cp_async_commit();
 }
 
 template <class Cf, bool RDEBUG>
 __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_constant__ ScanParams p,
-                                                                     const __grid_constant__ ChunkSched sched) {
+                                                                     const __grid_constant__ ChunkSched sched,
+                                                                     const __grid_constant__ ChunkMaps maps) {
   using namespace umma;
   constexpr int J = Cf::J, DK = Cf::DK, C = Cf::C, NROW = Cf::NROW, COLS = Cf::COLS;
   extern __shared__ __align__(128) unsigned char smem[];
@@ -273,6 +282,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     const int nchunks = ce - cb;
     const int Tseg = min(p.T, ce * C) - cb * C;
     const size_t tok0 = (size_t)bh * p.T + (size_t)cb * C;
+    const int tseg0 = cb * C;  // first token of the piece inside its sequence
     const bool from_flag = cb > 0, to_flag = ce < sched.nch;  // state handed over from / to another block
     unsigned *const flag = sched.flags + (sched.gang > 1 ? tl * sched.gang + gang_slice : tl);
     const int col = col0 + dl;
@@ -289,7 +299,8 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     mbar_init(&bars[B_G], 1);
     mbar_init(&bars[B_U], 1);
     mbar_init(&bars[B_QD], 1);
-    mbar_init(&bars[B_KQ], 128);
+    mbar_init(&bars[B_KQ0], 129);  // the tensor copies' issuer + 128 helpers (their cp.async of k and q)
+    mbar_init(&bars[B_KQ1], 129);
     mbar_init(&bars[B_KT], 128);
     mbar_init(&bars[B_WP], 128);
     mbar_init(&bars[B_GS], 64);
@@ -355,7 +366,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
           int pat = 0;
 #pragma unroll
           for (int rd = 0; rd < LJ; ++rd) pat |= ((c >> (LJ - 1 - rd)) & 1) ? (J >> (rd + 1)) : 0;
-          x[c] = __bfloat162float(rpq[(tl * J + (j ^ pat)) * COLS + dl]) * kLog2e;
+          x[c] = __bfloat162float(rpq[(tl * J + (j ^ pat)) * Cf::GROW + dl]) * kLog2e;
           mx = fmaxf(mx, x[c]);
         }
         float se = 0.f, so = 0.f;
@@ -445,7 +456,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
             const float be = bes[t * NROW + r];
             // serial chain: prediction error -> responsibilities (Eq. 3.4) -> update coefficient (Eq. 3.3)
             const float delta = v - pred[i];
-            const float a = fmaf(-kHalfLog2e * delta, delta, __bfloat162float(rpk[(t * J + j) * COLS + dl]) * kLog2e);
+            const float a = fmaf(-kHalfLog2e * delta, delta, __bfloat162float(rpk[(t * J + j) * Cf::GROW + dl]) * kLog2e);
             float e, sum;
             if constexpr (EXACT) {
               float all[J];
@@ -574,7 +585,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       float *bes = reinterpret_cast<float *>(raw + Cf::R_B);
       float be[C];
 #pragma unroll
-      for (int t = 0; t < C; ++t) be[t] = sigmoid_approx(__bfloat162float(rb[(t * J + j) * COLS + dl]));
+      for (int t = 0; t < C; ++t) be[t] = sigmoid_approx(__bfloat162float(rb[(t * J + j) * Cf::GROW + dl]));
       named_bar_sync(3, 128);
 #pragma unroll
       for (int t = 0; t < C; ++t) bes[t * NROW + h] = be[t];
@@ -641,11 +652,24 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     const bool spill_mine[2] = {warp < 6, warp >= 6};  // which parity of chunks this warp's lanes hold
 
     // ---- prologue: stage chunks 0 and 1, state row -> tensor memory, operands of chunk 0 ----
-    chunk_issue_raw<Cf>(p, tile, smem + Cf::OFF_RAW, smem + Cf::OFF_RPQ, tok0, Tseg, 0, col0, h);
-    cp_async_commit();
-    if (nchunks > 1)
-      chunk_issue_raw<Cf>(p, tile, smem + Cf::OFF_RAW + Cf::RAW_BYTES, smem + Cf::OFF_RPQ + Cf::RPQ_BYTES, tok0, Tseg, C, col0, h);
-    cp_async_commit();
+    // stage chunk m of this piece (one thread; the buffers it overwrites were last read through ordinary loads,
+    // hence the proxy fence)
+    auto stage = [&](int m) {
+      chunk_stage<Cf>(p, maps, tile, smem + Cf::OFF_RAW + (m & 1) * Cf::RAW_BYTES, smem + Cf::OFF_RPQ + (m & 3) * Cf::RPQ_BYTES,
+                      bh, tseg0 + m * C, tseg0 + Tseg, col0, m, h, &bars[B_KQ0 + (m & 1)]);
+    };
+    // this thread's cp.async of chunk m (all but the `pending` most recent groups) have landed: tell the barrier
+    // of m's parity, then wait until everything staged for the chunk is there (the barrier completes once per
+    // chunk of that parity)
+    auto staged = [&](int m, auto pending) {
+      cp_async_wait<decltype(pending)::value>();
+      fence_async_smem();
+      mbar_arrive(&bars[B_KQ0 + (m & 1)]);
+      return mbar_wait(&bars[B_KQ0 + (m & 1)], (m >> 1) & 1);
+    };
+    stage(0);
+    if (nchunks > 1) stage(1);
+    else cp_async_commit();
     if (from_flag) {  // the head of this tile was processed by another block: wait for its state
       if (h == 0) {
         bool seen = false;
@@ -689,28 +713,17 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       for (int e = h; e < (DK / 8) * 2 * C; e += 128)
         *reinterpret_cast<uint4 *>(tile + (e / (2 * C)) * Cf::TILE_LBO + (2 * C + e % (2 * C)) * 16) = make_uint4(0, 0, 0, 0);
     }
-    cp_async_wait<1>();
-    named_bar_sync(1, 128);  // every helper's copies of chunk 0 have landed
-    fence_async_smem();
-    mbar_arrive(&bars[B_KQ]);
+    if (!staged(0, std::integral_constant<int, 1>{})) failed = true;
     cook_be(smem + Cf::OFF_RAW);
     mbar_arrive(&bars[B_BE]);
     cook_kt(0);
     fence_async_smem();
     mbar_arrive(&bars[B_KT]);
-    // every helper waits for the first Gram batch: its completion also tells that the MMA thread has consumed
-    // the first phase of KQ, so the second one may be completed
-    if (!mbar_wait(&bars[B_G], 0)) failed = true;
     if (spill_mine[0]) {
+      if (!mbar_wait(&bars[B_G], 0)) failed = true;
       tc_fence_after_sync();
       if (!failed) spill_gram(0);
       mbar_arrive(&bars[B_GS]);
-    }
-    if (nchunks > 1) {
-      cp_async_wait<0>();
-      named_bar_sync(1, 128);
-      fence_async_smem();
-      mbar_arrive(&bars[B_KQ]);
     }
 
     // Per chunk n, in the order of what the other roles wait for first.
@@ -720,6 +733,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       PROF_ADD(0);
       if (more) {
         // (1) gates of chunk n+1 for the row warps, then its Gram batch
+        if (!staged(n + 1, std::integral_constant<int, 0>{})) { failed = true; break; }
         cook_be(smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES);
         mbar_arrive(&bars[B_BE]);
         PROF_ADD(1);
@@ -741,10 +755,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       // (3) chunk n is finished by the row warps: stage chunk n+2 into the buffers chunk n used
       if (!mbar_wait(&bars[B_C], n & 1)) { failed = true; break; }
       PROF_ADD(4);
-      if (n + 2 < nchunks)
-        chunk_issue_raw<Cf>(p, tile, smem + Cf::OFF_RAW + (n & 1) * Cf::RAW_BYTES, smem + Cf::OFF_RPQ + ((n + 2) & 3) * Cf::RPQ_BYTES,
-                            tok0, Tseg, (n + 2) * C, col0, h);
-      cp_async_commit();
+      if (n + 2 < nchunks) stage(n + 2);
       // (4) W has been updated with chunk n: split it into operand parts again
       if (!mbar_wait(&bars[B_U], n & 1)) { failed = true; break; }
       PROF_ADD(5);
@@ -754,14 +765,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         mbar_arrive(&bars[B_WP]);
       }
       PROF_ADD(6);
-      // (5) chunk n+2 has landed: its keys and queries already sit in the operand tile
-      if (n + 2 < nchunks) {
-        cp_async_wait<0>();
-        named_bar_sync(1, 128);
-        fence_async_smem();
-        mbar_arrive(&bars[B_KQ]);
-      }
-      // (6) transposed K of chunk n+1 (the update of chunk n has released the tile)
+      // (5) transposed K of chunk n+1 (the update of chunk n has released the tile)
       if (more) {
         cook_kt(n + 1);
         fence_async_smem();
@@ -769,7 +773,6 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       }
       PROF_ADD(7);
     }
-    cp_async_wait<0>();
     if (!failed && !mbar_wait(&bars[B_QD], (nchunks - 1) & 1)) failed = true;
     if (!failed) write_outputs(nchunks - 1);
   } else if (lane == 0) {
@@ -830,7 +833,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       }
       mma_commit(&bars[B_QD]);
     };
-    if (!mbar_wait(&bars[B_KQ], 0) || !mbar_wait(&bars[B_WP], 0)) failed = true;
+    if (!mbar_wait(&bars[B_KQ0], 0) || !mbar_wait(&bars[B_WP], 0)) failed = true;
     tc_fence_after_sync();
     if (!failed) {
       gram(0);
@@ -843,7 +846,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       if (more) {
         // ahead of the serial path: Gram batch and state x [K;Q] of chunk n+1 with the state before chunk n's
         // update (W is final up to chunk n-1 and split into parts; [P0|Q0] of chunk n has been taken out)
-        if (!mbar_wait(&bars[B_KQ], (n + 1) & 1) || !mbar_wait(&bars[B_PQF], n & 1)) { failed = true; break; }
+        if (!mbar_wait(&bars[B_KQ0 + ((n + 1) & 1)], ((n + 1) >> 1) & 1) || !mbar_wait(&bars[B_PQF], n & 1)) { failed = true; break; }
         if (n > 0 && !mbar_wait(&bars[B_WP], n & 1)) { failed = true; break; }
         tc_fence_after_sync();
         PROF_ADD(0);
@@ -889,6 +892,63 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
 #endif
 }
 
+// cuTensorMapEncodeTiled, fetched through the runtime so that the library does not link against the driver.
+typedef CUresult (*ChunkEncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                       const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                       CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+inline ChunkEncodeTiledFn chunk_encode_fn() {
+  static ChunkEncodeTiledFn fn = [] {
+    void *sym = nullptr;
+    cudaDriverEntryPointQueryResult res;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &res) != cudaSuccess ||
+        res != cudaDriverEntryPointSuccess)
+      sym = nullptr;
+    return (ChunkEncodeTiledFn)sym;
+  }();
+  return fn;
+}
+
+// One bf16 tensor map: `rank` dimensions (innermost first) of sizes `dims` with byte strides `strides` (for dimensions
+// 1 .. rank-1) and a copy box of `box` elements; no swizzle, out-of-range elements read as zero.
+inline bool chunk_encode(CUtensorMap *map, const void *base, int rank, const cuuint64_t *dims, const cuuint64_t *strides,
+                         const cuuint32_t *box) {
+  ChunkEncodeTiledFn fn = chunk_encode_fn();
+  if (!fn) return false;
+  const cuuint32_t ones[4] = {1, 1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base), dims, strides, box, ones,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Tensor maps of one launch.  k, q [BH][T][DK] are seen as (8 key dims, DK/8, T, BH) so that one box is the
+// 16-byte column c of 32 tokens, which is how the operand tile stores them; v [BH][T][Dv] as (Dv, T, BH); the gate
+// logits [BH][T][J][Dv] as (Dv, J, T, BH) with a box of GROW columns, all J components, 32 tokens.
+template <class Cf>
+bool chunk_make_maps(const ScanParams &p, ChunkMaps *m) {
+  const cuuint64_t BH = (cuuint64_t)p.B * p.H, T = (cuuint64_t)p.T, Dv = (cuuint64_t)p.Dv, J = Cf::J, DK = Cf::DK;
+  {
+    const cuuint64_t dims[4] = {8, DK / 8, T, BH};
+    const cuuint64_t strides[3] = {16, DK * 2, T * DK * 2};
+    const cuuint32_t box[4] = {8, 1, (cuuint32_t)Cf::C, 1};
+    if (!chunk_encode(&m->k, p.k, 4, dims, strides, box) || !chunk_encode(&m->q, p.q, 4, dims, strides, box)) return false;
+  }
+  {
+    const cuuint64_t dims[3] = {Dv, T, BH};
+    const cuuint64_t strides[2] = {Dv * 2, T * Dv * 2};
+    const cuuint32_t box[3] = {(cuuint32_t)Cf::COLS, (cuuint32_t)Cf::C, 1};
+    if (!chunk_encode(&m->v, p.v, 3, dims, strides, box)) return false;
+  }
+  {
+    const cuuint64_t dims[4] = {Dv, J, T, BH};
+    const cuuint64_t strides[3] = {Dv * 2, J * Dv * 2, T * J * Dv * 2};
+    const cuuint32_t box[4] = {(cuuint32_t)Cf::GROW, (cuuint32_t)Cf::J, (cuuint32_t)Cf::C, 1};
+    if (!chunk_encode(&m->be, p.beta_logit, 4, dims, strides, box) || !chunk_encode(&m->pk, p.pik_logit, 4, dims, strides, box) ||
+        !chunk_encode(&m->pq, p.piq_logit, 4, dims, strides, box))
+      return false;
+  }
+  return true;
+}
+
 // Number of SMs of the current device (one block is resident per SM).
 inline int chunk_sm_count() {
   int dev = 0, n = 0;
@@ -918,6 +978,8 @@ int launch_chunk(const LaunchArgs &a) {
   if (ntiles <= 0 || ntiles > 0x7fffffffLL || nch <= 0 || nch > 0x7fffffffLL) return (int)cudaErrorInvalidConfiguration;
   ChunkSched sc{(int)ntiles, (int)nch, (int)nch, 1, 0u, nullptr};
   ScanParams prm = a.p;
+  ChunkMaps maps;
+  if (!chunk_make_maps<Cf>(a.p, &maps)) return (int)cudaErrorInvalidValue;
 
   // More tiles than SMs, not a whole number of waves: cut the chunk sequence into equal runs instead of whole
   // tiles, so that the last wave is not half empty.  The runs are laid over (batch, head) units and walked by
@@ -938,14 +1000,14 @@ int launch_chunk(const LaunchArgs &a) {
         ChunkSched ss{(int)nbh, (int)nch, (int)per, (int)nslice, epoch,
                       flags + (size_t)(epoch % kChunkFlagSlots) * kChunkFlagTiles};
         const long long grid = ((total + per - 1) / per) * nslice;
-        void *args[] = {(void *)&prm, (void *)&ss};
+        void *args[] = {(void *)&prm, (void *)&ss, (void *)&maps};
         e = cudaLaunchCooperativeKernel((const void *)kern, dim3((unsigned)grid), dim3(Cf::NT), args, Cf::SMEM_BYTES, a.stream);
         if (e == cudaSuccess) return (int)cudaGetLastError();
         (void)cudaGetLastError();  // not launched (e.g. the blocks cannot all be resident): fall back to whole tiles
       }
     }
   }
-  kern<<<(unsigned)ntiles, Cf::NT, Cf::SMEM_BYTES, a.stream>>>(prm, sc);
+  kern<<<(unsigned)ntiles, Cf::NT, Cf::SMEM_BYTES, a.stream>>>(prm, sc, maps);
   return (int)cudaGetLastError();
 }
 
