@@ -228,8 +228,10 @@ int swila_selftest_tf32_mma(const float *A, const float *B, float *D, int N, int
  * The same self-test with BF16 operands (no counterpart in the paper): A and B are DEVICE fp32
  * row-major and are rounded to bf16 (nearest even) by the kernel; FP32 accumulation.  a_in_smem = 0:
  * A goes through tensor memory, two consecutive K elements per 32-bit column; a_in_smem = 1: A
- * goes through shared memory in the K-major layout of B.  (N, K, a_in_smem) in {(64,128,0),
- * (128,32,0), (32,32,0), (64,64,1)}; anything else returns SWILA_ERR_UNSUPPORTED.
+ * goes through shared memory in the K-major layout of B; a_in_smem = 2: both operands in shared
+ * memory in the 128-byte-swizzle K-major layout (what a tensor copy with that swizzle mode
+ * writes).  (N, K, a_in_smem) in {(64,128,0), (128,32,0), (32,32,0), (64,64,1), (64,64,2),
+ * (32,64,2)}; anything else returns SWILA_ERR_UNSUPPORTED.
  */
 int swila_selftest_bf16_mma(const float *A, const float *B, float *D, int N, int K, int a_in_smem, int *status,
                             void *stream);

@@ -168,6 +168,19 @@ __device__ __forceinline__ uint64_t smem_desc_kmajor(uint32_t smem_addr, uint32_
   d |= (uint64_t)1 << 46;  // descriptor version of this architecture
   return d;                // base offset 0, layout type 0 (no swizzle)
 }
+// Shared-memory operand, K-major, 128-byte swizzle: a row (the M or N index) is 128 bytes = 64 16-bit elements of K;
+// 8 rows form a 1024-byte atom inside which the 16-byte units of row r are stored at unit index u ^ (r & 7) (the layout
+// a tensor copy with the 128-byte swizzle mode produces); `sbo` = byte distance between 8-row atoms.  The tile must be
+// 1024-byte aligned; a K step of 16 elements advances the start address by 32 bytes.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t smem_addr, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr >> 4) & 0x3fffu);
+  d |= (uint64_t)1 << 16;  // leading-dimension offset: not used by this layout
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
+  d |= (uint64_t)1 << 46;  // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;  // layout type: 128-byte swizzle
+  return d;
+}
 // Instruction descriptor: TF32 x TF32 -> FP32, both operands K-major, dense.
 __host__ __device__ constexpr uint32_t idesc_tf32(int M, int N) {
   return (1u << 4) /*D = f32*/ | (2u << 7) /*A = tf32*/ | (2u << 10) /*B = tf32*/ | ((uint32_t)(N >> 3) << 17) |

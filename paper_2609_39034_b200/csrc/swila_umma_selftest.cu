@@ -162,6 +162,64 @@ __global__ void __launch_bounds__(128) umma_selftest_bf16_kernel(const float *A,
   __syncthreads();
   if (warp == 0) tmem_dealloc(tbase, TM_COLS);
 }
+
+// Both operands in shared memory in the 128-byte-swizzle K-major layout (K = 64 per tile): D[128 x N] = A B^T.
+template <int N>
+__global__ void __launch_bounds__(128) umma_selftest_sw128_kernel(const float *A, const float *B, float *D, int *status) {
+  constexpr int K = 64;
+  __shared__ __align__(1024) uint16_t sA[128 * K];
+  __shared__ __align__(1024) uint16_t sB[N * K];
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ uint32_t tmem_base_s;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  constexpr uint32_t TM_COLS = 256;
+
+  if (warp == 0) tmem_alloc(&tmem_base_s, TM_COLS);
+  if (tid == 0) {
+    mbar_init(&bar, 1);
+    mbar_fence_init();
+  }
+  // element (row, k) -> row*64 + ((k/8) ^ (row & 7))*8 + k%8
+  for (int i = tid; i < N * K; i += 128) {
+    const int n = i / K, k = i % K;
+    sB[n * K + (((k >> 3) ^ (n & 7)) << 3) + (k & 7)] = (uint16_t)bf16_bits(B[(size_t)n * K + k]);
+  }
+  for (int i = tid; i < 128 * K; i += 128) {
+    const int m = i / K, k = i % K;
+    sA[m * K + (((k >> 3) ^ (m & 7)) << 3) + (k & 7)] = (uint16_t)bf16_bits(A[(size_t)m * K + k]);
+  }
+  fence_async_smem();
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tbase = tmem_base_s;
+  const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+  if (tid == 0) {
+    constexpr uint32_t idesc = idesc_bf16(128, N);
+#pragma unroll
+    for (int ks = 0; ks < K / 16; ++ks)
+      mma_bf16_ss(tbase + 128, smem_desc_sw128(smem_u32(sA) + ks * 32, 1024), smem_desc_sw128(smem_u32(sB) + ks * 32, 1024),
+                  idesc, ks > 0);
+    mma_commit(&bar);
+  }
+  const bool ok = mbar_wait(&bar, 0);
+  tc_fence_after_sync();
+  if (ok) {
+#pragma unroll
+    for (int c = 0; c < N / 16; ++c) {
+      float v[16];
+      tmem_ld16(tbase + lane_base + 128 + c * 16, v);
+      tmem_ld_wait();
+#pragma unroll
+      for (int i = 0; i < 16; ++i) D[(size_t)tid * N + c * 16 + i] = v[i];
+    }
+  } else if (tid == 0) {
+    *status = 1;
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tbase, TM_COLS);
+}
 }  // namespace
 
 extern "C" int swila_selftest_tf32_mma(const float *A, const float *B, float *D, int N, int K, int *status,
@@ -183,7 +241,9 @@ extern "C" int swila_selftest_bf16_mma(const float *A, const float *B, float *D,
   if (N == 64 && K == 128 && !a_in_smem) umma_selftest_bf16_kernel<64, 128, 0><<<1, 128, 0, st>>>(A, B, D, status);
   else if (N == 128 && K == 32 && !a_in_smem) umma_selftest_bf16_kernel<128, 32, 0><<<1, 128, 0, st>>>(A, B, D, status);
   else if (N == 32 && K == 32 && !a_in_smem) umma_selftest_bf16_kernel<32, 32, 0><<<1, 128, 0, st>>>(A, B, D, status);
-  else if (N == 64 && K == 64 && a_in_smem) umma_selftest_bf16_kernel<64, 64, 1><<<1, 128, 0, st>>>(A, B, D, status);
+  else if (N == 64 && K == 64 && a_in_smem == 1) umma_selftest_bf16_kernel<64, 64, 1><<<1, 128, 0, st>>>(A, B, D, status);
+  else if (N == 64 && K == 64 && a_in_smem == 2) umma_selftest_sw128_kernel<64><<<1, 128, 0, st>>>(A, B, D, status);
+  else if (N == 32 && K == 64 && a_in_smem == 2) umma_selftest_sw128_kernel<32><<<1, 128, 0, st>>>(A, B, D, status);
   else return SWILA_ERR_UNSUPPORTED;
   return cudaGetLastError() == cudaSuccess ? SWILA_OK : SWILA_ERR_CUDA;
 }
