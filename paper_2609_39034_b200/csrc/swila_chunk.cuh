@@ -104,13 +104,14 @@ struct ChunkCfg {
   static constexpr int TM_ALLOC = 512;
   static_assert(TM_USED <= TM_ALLOC, "tensor memory budget");
   static_assert(J == 4 || J == 8, "the output transposition assumes that J divides 8");
-  // K/Q operand tile (bf16, K-major, no swizzle): 16-byte unit (row, c) = 8 key dims 8c..8c+7 of one
-  // token at c*TILE_LBO + row*16, rows [K_even ; Q_even ; K_odd ; Q_odd]: the chunks of both parities
-  // side by side, so that one 128-row A operand covers the keys of two consecutive chunks.  cp.async
-  // writes it directly from global memory.
-  static constexpr int TILE_LBO = 4 * C * 16 + 16;  // + 16: consecutive columns start 4 banks apart (conflict-free
-                                                    // cp.async stores and transposing reads)
-  static constexpr int TILE_BYTES = (DK / 8) * TILE_LBO;
+  // K/Q operand tile (bf16, K-major, 128-byte swizzle): per half of 64 key dims, 128 rows of 128 bytes, rows
+  // [K_even ; Q_even ; K_odd ; Q_odd]: the chunks of both parities side by side, so that one 128-row A operand
+  // covers the keys of two consecutive chunks.  Key dim d of row r sits at
+  //   (d / 64) * TILE_HALF + r * 128 + (((d / 8) % 8) ^ (r % 8)) * 16 + (d % 8) * 2,
+  // which is what a tensor copy with the 128-byte swizzle mode writes: k and q go straight from global memory
+  // into the tile, 4 KB per copy.
+  static constexpr int TILE_HALF = 4 * C * 128;
+  static constexpr int TILE_BYTES = (DK / 64) * TILE_HALF;
   // raw stages (2-deep ring): v [C][COLS] bf16; beta logits [C][J][COLS] bf16, overwritten in place by the
   // helpers with beta = sigmoid(.) as fp32 [C][NROW] (hence the fp32-sized slot); pik logits [C][J][COLS]
   // bf16.  The query-prior logits piq [C][J][COLS] live in their own 4-deep ring because the outputs of
@@ -123,8 +124,8 @@ struct ChunkCfg {
   static constexpr int R_PK = R_B + C * NROW * 4;
   static constexpr int RAW_BYTES = R_PK + C * J * GROW * ES;
   static constexpr int RPQ_BYTES = C * J * GROW * ES;
-  // bytes one chunk's tensor copies deliver: v and three gate tensors (k and q come by cp.async)
-  static constexpr int STAGE_TX_BYTES = C * COLS * ES + 3 * C * J * GROW * ES;
+  // bytes one chunk's tensor copies deliver: k and q into the operand tile, v, three gate tensors
+  static constexpr int STAGE_TX_BYTES = 2 * C * DK * ES + C * COLS * ES + 3 * C * J * GROW * ES;
   static_assert(C * J * GROW * ES <= C * NROW * 4, "the beta logits must fit the slot their gates overwrite");
   static constexpr int C_K = DK * ES / 16, C_V = COLS * ES / 16;  // 16-byte units per token row / column slice
   // operand tiles written by the helpers (bf16, same unit layout, 8 tokens per unit)
@@ -145,9 +146,9 @@ struct ChunkCfg {
   static constexpr int OFF_OST = OFF_GX + 2 * GX_TILE;        // 2 x [C][COLS] bf16 output staging
   static constexpr int OFF_P0 = OFF_OST + 2 * C * COLS * ES;  // [C/4][NROW] float4: a chunk's P0 rows, kept for the rare redo
   static constexpr int OFF_BAR = OFF_P0 + C * NROW * 4;
-  static constexpr int SMEM_BYTES = OFF_BAR + 128;
+  static constexpr int SMEM_BYTES = OFF_BAR + 128 + 1024;  // + 1024: the kernel aligns its window to 1024 bytes
   static_assert(RAW_BYTES % 128 == 0 && RPQ_BYTES % 128 == 0 && R_B % 128 == 0 && R_PK % 128 == 0 && OFF_RAW % 128 == 0 &&
-                    OFF_RPQ % 128 == 0 && TILE_LBO % 16 == 0 && (COLS * ES) % 16 == 0 && (GROW * ES) % 16 == 0,
+                    OFF_RPQ % 128 == 0 && OFF_TILE % 1024 == 0 && DK % 64 == 0 && (COLS * ES) % 16 == 0 && (GROW * ES) % 16 == 0,
                 "destinations of the tensor copies are 128-byte aligned, their rows multiples of 16 bytes");
   static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 };
@@ -174,42 +175,26 @@ struct ChunkMaps {
   CUtensorMap k, q, v, be, pk, pq;
 };
 
-// Staging of chunk m of a piece.  v and the gate logits: tiled bulk tensor copies (TMA) issued by ONE thread straight
-// into the raw stage; tokens past the end of the sequence and columns past Dv are filled with zeros by the copy
-// engine, and the bytes land on `bar`.  k and q: 16-byte cp.async by all 128 helper threads (h = 0..127) into the
-// operand tile, whose 16-byte columns are too narrow for efficient tensor copies; the threads arrive on `bar`
-// themselves once their copies have landed.
+// Staging of chunk m of a piece by ONE thread: tiled bulk tensor copies (TMA) straight into the operand tile (k, q:
+// 64 key dims x 32 tokens per copy, 128-byte swizzle) and into the raw stage (v, gate logits).  Tokens past the end
+// of the sequence and columns past Dv are filled with zeros by the copy engine.  Everything lands on `bar`.
 template <class Cf>
-__device__ __forceinline__ void chunk_stage(const ScanParams &p, const ChunkMaps &maps, unsigned char *tile,
-                                            unsigned char *raw, unsigned char *rawpq, int bh, int tok, int T_end, int col0,
-                                            int m, int h, uint64_t *bar) {
+__device__ __forceinline__ void chunk_stage(const ChunkMaps &maps, unsigned char *tile, unsigned char *raw,
+                                            unsigned char *rawpq, int bh, int tok, int col0, int m, uint64_t *bar) {
   using namespace umma;
-  constexpr int DK = Cf::DK, C = Cf::C, ES = Cf::ES, C_K = Cf::C_K;
-  if (h == 0) {
-    fence_async_smem();  // the buffers were last read through ordinary loads
-    mbar_arrive_expect_tx(bar, Cf::STAGE_TX_BYTES);
-    tma_load_3d(raw + Cf::R_V, &maps.v, col0, tok, bh, bar);
-    tma_load_4d(raw + Cf::R_B, &maps.be, col0, 0, tok, bh, bar);
-    tma_load_4d(raw + Cf::R_PK, &maps.pk, col0, 0, tok, bh, bar);
-    tma_load_4d(rawpq, &maps.pq, col0, 0, tok, bh, bar);
-  }
-  const int nvalid = min(C, T_end - tok);
-  const size_t tokb = (size_t)bh * p.T + (size_t)tok;
-  const char *kb = (const char *)p.k + tokb * DK * ES;
-  const char *qb = (const char *)p.q + tokb * DK * ES;
-  unsigned char *trow = tile + (m & 1) * 2 * C * 16;  // this chunk's 2C rows of the operand tile
-  // One warp instruction copies 8 columns x 4 tokens: each quarter-warp reads 128 contiguous bytes of one token
-  // and writes 8 columns of the tile, which the padded column stride puts into 8 different bank groups.
-  static_assert(C_K % 8 == 0, "key dims come in groups of 64");
-  constexpr int NINSTR = (C_K / 8) * (C / 4);  // per tensor and chunk
+  constexpr int DK = Cf::DK, C = Cf::C;
+  fence_async_smem();  // the buffers were last read through ordinary loads
+  mbar_arrive_expect_tx(bar, Cf::STAGE_TX_BYTES);
+  unsigned char *trow = tile + (m & 1) * 2 * C * 128;  // this chunk's 2C rows of the operand tile
 #pragma unroll
-  for (int id = h >> 5; id < NINSTR; id += 4) {
-    const int c = (id % (C_K / 8)) * 8 + (h & 7), t = (id / (C_K / 8)) * 4 + ((h >> 3) & 3);
-    const bool valid = t < nvalid;
-    cp_async16(trow + c * Cf::TILE_LBO + t * 16, valid ? kb + (t * C_K + c) * 16 : (const char *)p.k, valid ? 16 : 0);
-    cp_async16(trow + c * Cf::TILE_LBO + (C + t) * 16, valid ? qb + (t * C_K + c) * 16 : (const char *)p.k, valid ? 16 : 0);
+  for (int hf = 0; hf < DK / 64; ++hf) {
+    tma_load_3d(trow + hf * Cf::TILE_HALF, &maps.k, hf * 64, tok, bh, bar);
+    tma_load_3d(trow + hf * Cf::TILE_HALF + C * 128, &maps.q, hf * 64, tok, bh, bar);
   }
-  cp_async_commit();
+  tma_load_3d(raw + Cf::R_V, &maps.v, col0, tok, bh, bar);
+  tma_load_4d(raw + Cf::R_B, &maps.be, col0, 0, tok, bh, bar);
+  tma_load_4d(raw + Cf::R_PK, &maps.pk, col0, 0, tok, bh, bar);
+  tma_load_4d(rawpq, &maps.pq, col0, 0, tok, bh, bar);
 }
 
 template <class Cf, bool RDEBUG>
@@ -218,7 +203,9 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
                                                                      const __grid_constant__ ChunkMaps maps) {
   using namespace umma;
   constexpr int J = Cf::J, DK = Cf::DK, C = Cf::C, NROW = Cf::NROW, COLS = Cf::COLS;
-  extern __shared__ __align__(128) unsigned char smem[];
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  // the swizzled operand tile needs a 1024-byte aligned shared-memory address
+  unsigned char *smem = smem_raw + ((1024u - (umma::smem_u32(smem_raw) & 1023u)) & 1023u);
   unsigned char *tile = smem + Cf::OFF_TILE;
   unsigned char *Kt = smem + Cf::OFF_KT;
   float *G_all = reinterpret_cast<float *>(smem + Cf::OFF_G);
@@ -299,8 +286,8 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     mbar_init(&bars[B_G], 1);
     mbar_init(&bars[B_U], 1);
     mbar_init(&bars[B_QD], 1);
-    mbar_init(&bars[B_KQ0], 129);  // the tensor copies' issuer + 128 helpers (their cp.async of k and q)
-    mbar_init(&bars[B_KQ1], 129);
+    mbar_init(&bars[B_KQ0], 1);  // the thread that issues the tensor copies
+    mbar_init(&bars[B_KQ1], 1);
     mbar_init(&bars[B_KT], 128);
     mbar_init(&bars[B_WP], 128);
     mbar_init(&bars[B_GS], 64);
@@ -565,16 +552,17 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     const int h = r;
     // K of a chunk, transposed: unit (row d', c) holds K[8c .. 8c+7][d'], read from the operand tile
     auto cook_kt = [&](int m) {
-      const unsigned char *trow = tile + (m & 1) * 2 * C * 16;
+      const unsigned char *trow = tile + (m & 1) * 2 * C * 128;
 #pragma unroll 1
       for (int e = h; e < (C / 8) * DK; e += 128) {
         const int dd = e % DK, c = e / DK;
-        const unsigned char *src = trow + (dd >> 3) * Cf::TILE_LBO + (8 * c) * 16 + (dd & 7) * 2;
+        const unsigned char *src = trow + (dd >> 6) * Cf::TILE_HALF + (8 * c) * 128 + (dd & 7) * 2;
+        const int cu = (dd >> 3) & 7;  // 16-byte unit of the row before the swizzle; token 8c+i sits in row ... + i
         uint32_t w[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-          w[i] = (uint32_t)*reinterpret_cast<const unsigned short *>(src + (2 * i) * 16) |
-                 ((uint32_t)*reinterpret_cast<const unsigned short *>(src + (2 * i + 1) * 16) << 16);
+          w[i] = (uint32_t)*reinterpret_cast<const unsigned short *>(src + (2 * i) * 128 + ((cu ^ (2 * i)) << 4)) |
+                 ((uint32_t)*reinterpret_cast<const unsigned short *>(src + (2 * i + 1) * 128 + ((cu ^ (2 * i + 1)) << 4)) << 16);
         *reinterpret_cast<uint4 *>(Kt + c * Cf::KT_LBO + dd * 16) = make_uint4(w[0], w[1], w[2], w[3]);
       }
     };
@@ -655,21 +643,15 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     // stage chunk m of this piece (one thread; the buffers it overwrites were last read through ordinary loads,
     // hence the proxy fence)
     auto stage = [&](int m) {
-      chunk_stage<Cf>(p, maps, tile, smem + Cf::OFF_RAW + (m & 1) * Cf::RAW_BYTES, smem + Cf::OFF_RPQ + (m & 3) * Cf::RPQ_BYTES,
-                      bh, tseg0 + m * C, tseg0 + Tseg, col0, m, h, &bars[B_KQ0 + (m & 1)]);
+      chunk_stage<Cf>(maps, tile, smem + Cf::OFF_RAW + (m & 1) * Cf::RAW_BYTES, smem + Cf::OFF_RPQ + (m & 3) * Cf::RPQ_BYTES, bh,
+                      tseg0 + m * C, col0, m, &bars[B_KQ0 + (m & 1)]);
     };
-    // this thread's cp.async of chunk m (all but the `pending` most recent groups) have landed: tell the barrier
-    // of m's parity, then wait until everything staged for the chunk is there (the barrier completes once per
-    // chunk of that parity)
-    auto staged = [&](int m, auto pending) {
-      cp_async_wait<decltype(pending)::value>();
-      fence_async_smem();
-      mbar_arrive(&bars[B_KQ0 + (m & 1)]);
-      return mbar_wait(&bars[B_KQ0 + (m & 1)], (m >> 1) & 1);
-    };
-    stage(0);
-    if (nchunks > 1) stage(1);
-    else cp_async_commit();
+    // everything staged for chunk m has landed (the barrier of m's parity completes once per chunk of that parity)
+    auto staged = [&](int m) { return mbar_wait(&bars[B_KQ0 + (m & 1)], (m >> 1) & 1); };
+    if (h == 0) {
+      stage(0);
+      if (nchunks > 1) stage(1);
+    }
     if (from_flag) {  // the head of this tile was processed by another block: wait for its state
       if (h == 0) {
         bool seen = false;
@@ -710,10 +692,10 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       mbar_arrive(&bars[B_WP]);
     }
     if (nchunks == 1) {  // the odd half of the operand tile is read (as don't-care rows) by the Gram batch: make it finite
-      for (int e = h; e < (DK / 8) * 2 * C; e += 128)
-        *reinterpret_cast<uint4 *>(tile + (e / (2 * C)) * Cf::TILE_LBO + (2 * C + e % (2 * C)) * 16) = make_uint4(0, 0, 0, 0);
+      for (int e = h; e < (DK / 64) * 2 * C * 8; e += 128)
+        *reinterpret_cast<uint4 *>(tile + (e / (2 * C * 8)) * Cf::TILE_HALF + 2 * C * 128 + (e % (2 * C * 8)) * 16) = make_uint4(0, 0, 0, 0);
     }
-    if (!staged(0, std::integral_constant<int, 1>{})) failed = true;
+    if (!staged(0)) failed = true;
     cook_be(smem + Cf::OFF_RAW);
     mbar_arrive(&bars[B_BE]);
     cook_kt(0);
@@ -733,7 +715,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       PROF_ADD(0);
       if (more) {
         // (1) gates of chunk n+1 for the row warps, then its Gram batch
-        if (!staged(n + 1, std::integral_constant<int, 0>{})) { failed = true; break; }
+        if (!staged(n + 1)) { failed = true; break; }
         cook_be(smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES);
         mbar_arrive(&bars[B_BE]);
         PROF_ADD(1);
@@ -755,7 +737,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       // (3) chunk n is finished by the row warps: stage chunk n+2 into the buffers chunk n used
       if (!mbar_wait(&bars[B_C], n & 1)) { failed = true; break; }
       PROF_ADD(4);
-      if (n + 2 < nchunks) stage(n + 2);
+      if (n + 2 < nchunks && h == 0) stage(n + 2);
       // (4) W has been updated with chunk n: split it into operand parts again
       if (!mbar_wait(&bars[B_U], n & 1)) { failed = true; break; }
       PROF_ADD(5);
@@ -780,22 +762,24 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     constexpr uint32_t idE = idesc_bf16(128, 2 * C);  // N = 2C: [P0 | Q0], Gram batch, cross-chunk term
     constexpr uint32_t idU = idesc_bf16(128, DK);
     constexpr uint32_t idQ = idesc_bf16(128, C);
-    const uint64_t tile_a = smem_desc_kmajor(smem_u32(tile), Cf::TILE_LBO, 128);  // all 128 rows, as an A operand
-    const uint64_t kq_b[2] = {smem_desc_kmajor(smem_u32(tile), Cf::TILE_LBO, 128),
-                              smem_desc_kmajor(smem_u32(tile) + 2 * C * 16, Cf::TILE_LBO, 128)};  // [K;Q] (or K) of a parity
+    // operand of the tile starting at row `row0`, K step ks (16 key dims = 32 bytes inside a 128-byte row; four
+    // steps per half of 64 key dims)
+    const uint32_t tile_addr = smem_u32(tile);
+    auto tile_desc = [&](int row0, int ks) {
+      return smem_desc_sw128(tile_addr + (ks >> 2) * Cf::TILE_HALF + row0 * 128 + (ks & 3) * 32, 1024);
+    };
     const uint64_t kt0 = smem_desc_kmajor(smem_u32(Kt), Cf::KT_LBO, 128);
     const uint64_t gx_hi = smem_desc_kmajor(smem_u32(GX_all), Cf::GX_LBO, 128);
     const uint64_t gx_lo = smem_desc_kmajor(smem_u32(GX_all + Cf::GX_TILE), Cf::GX_LBO, 128);
-    constexpr uint64_t TILE_ADV = 2 * (Cf::TILE_LBO / 16);  // start-address advance per 16 key dims, 16-byte units
     // Gram batch of chunk m: every row of the tile against [K;Q] of chunk m and against K of chunk m-1
     auto gram = [&](int m) {
 #pragma unroll 1
       for (int ks = 0; ks < DK / 16; ++ks)
-        mma_bf16_ss(tb0 + Cf::TM_G, tile_a + ks * TILE_ADV, kq_b[m & 1] + ks * TILE_ADV, idE, ks > 0);
+        mma_bf16_ss(tb0 + Cf::TM_G, tile_desc(0, ks), tile_desc((m & 1) * 2 * C, ks), idE, ks > 0);
       if (m > 0) {
 #pragma unroll 1
         for (int ks = 0; ks < DK / 16; ++ks)
-          mma_bf16_ss(tb0 + Cf::TM_G + 2 * C, tile_a + ks * TILE_ADV, kq_b[(m - 1) & 1] + ks * TILE_ADV, idQ, ks > 0);
+          mma_bf16_ss(tb0 + Cf::TM_G + 2 * C, tile_desc(0, ks), tile_desc(((m - 1) & 1) * 2 * C, ks), idQ, ks > 0);
       }
       mma_commit(&bars[B_G]);
     };
@@ -803,10 +787,10 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     auto w_times_kq = [&](int m) {
 #pragma unroll 1
       for (int ks = 0; ks < DK / 16; ++ks)
-        mma_bf16_ts(tb0 + Cf::TM_PQ, tb0 + Cf::TM_WHI + ks * 8, kq_b[m & 1] + ks * TILE_ADV, idE, ks > 0);
+        mma_bf16_ts(tb0 + Cf::TM_PQ, tb0 + Cf::TM_WHI + ks * 8, tile_desc((m & 1) * 2 * C, ks), idE, ks > 0);
 #pragma unroll 1
       for (int ks = 0; ks < DK / 16; ++ks)
-        mma_bf16_ts(tb0 + Cf::TM_PQ, tb0 + Cf::TM_WLO + ks * 8, kq_b[m & 1] + ks * TILE_ADV, idE, true);
+        mma_bf16_ts(tb0 + Cf::TM_PQ, tb0 + Cf::TM_WLO + ks * 8, tile_desc((m & 1) * 2 * C, ks), idE, true);
     };
     // + Cmat (K_prev [K;Q]^T): the update of the chunk that just finished, seen by the next chunk's products
     auto cross = [&]() {
@@ -911,26 +895,28 @@ inline ChunkEncodeTiledFn chunk_encode_fn() {
 // One bf16 tensor map: `rank` dimensions (innermost first) of sizes `dims` with byte strides `strides` (for dimensions
 // 1 .. rank-1) and a copy box of `box` elements; no swizzle, out-of-range elements read as zero.
 inline bool chunk_encode(CUtensorMap *map, const void *base, int rank, const cuuint64_t *dims, const cuuint64_t *strides,
-                         const cuuint32_t *box) {
+                         const cuuint32_t *box, CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_NONE) {
   ChunkEncodeTiledFn fn = chunk_encode_fn();
   if (!fn) return false;
   const cuuint32_t ones[4] = {1, 1, 1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void *>(base), dims, strides, box, ones,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Tensor maps of one launch.  k, q [BH][T][DK] are seen as (8 key dims, DK/8, T, BH) so that one box is the
-// 16-byte column c of 32 tokens, which is how the operand tile stores them; v [BH][T][Dv] as (Dv, T, BH); the gate
+// Tensor maps of one launch.  k, q [BH][T][DK] as (DK, T, BH) with a box of 64 key dims x 32 tokens and the 128-byte
+// swizzle, which is how the operand tile stores them; v [BH][T][Dv] as (Dv, T, BH); the gate
 // logits [BH][T][J][Dv] as (Dv, J, T, BH) with a box of GROW columns, all J components, 32 tokens.
 template <class Cf>
 bool chunk_make_maps(const ScanParams &p, ChunkMaps *m) {
   const cuuint64_t BH = (cuuint64_t)p.B * p.H, T = (cuuint64_t)p.T, Dv = (cuuint64_t)p.Dv, J = Cf::J, DK = Cf::DK;
   {
-    const cuuint64_t dims[4] = {8, DK / 8, T, BH};
-    const cuuint64_t strides[3] = {16, DK * 2, T * DK * 2};
-    const cuuint32_t box[4] = {8, 1, (cuuint32_t)Cf::C, 1};
-    if (!chunk_encode(&m->k, p.k, 4, dims, strides, box) || !chunk_encode(&m->q, p.q, 4, dims, strides, box)) return false;
+    const cuuint64_t dims[3] = {DK, T, BH};
+    const cuuint64_t strides[2] = {DK * 2, T * DK * 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)Cf::C, 1};
+    if (!chunk_encode(&m->k, p.k, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !chunk_encode(&m->q, p.q, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
+      return false;
   }
   {
     const cuuint64_t dims[3] = {Dv, T, BH};
