@@ -230,8 +230,9 @@ int swila_selftest_tf32_mma(const float *A, const float *B, float *D, int N, int
  * A goes through tensor memory, two consecutive K elements per 32-bit column; a_in_smem = 1: A
  * goes through shared memory in the K-major layout of B; a_in_smem = 2: both operands in shared
  * memory in the 128-byte-swizzle K-major layout (what a tensor copy with that swizzle mode
- * writes).  (N, K, a_in_smem) in {(64,128,0), (128,32,0), (32,32,0), (64,64,1), (64,64,2),
- * (32,64,2)}; anything else returns SWILA_ERR_UNSUPPORTED.
+ * writes); a_in_smem = 3: A through tensor memory, B stored MN-major (N contiguous) with the
+ * 128-byte swizzle.  (N, K, a_in_smem) in {(64,128,0), (128,32,0), (32,32,0), (64,64,1),
+ * (64,64,2), (32,64,2), (128,32,3)}; anything else returns SWILA_ERR_UNSUPPORTED.
  */
 int swila_selftest_bf16_mma(const float *A, const float *B, float *D, int N, int K, int a_in_smem, int *status,
                             void *stream);

@@ -243,7 +243,7 @@ def selftest_tf32_mma(A: torch.Tensor, B: torch.Tensor) -> torch.Tensor:
 def selftest_bf16_mma(A: torch.Tensor, B: torch.Tensor, a_in_smem: int = 0) -> torch.Tensor:
     """D = bf16(A) @ bf16(B).T on the tcgen05 path (A [128,K], B [N,K], fp32 on the device).
     a_in_smem: 0 = A through tensor memory, 1 = A through shared memory, 2 = both operands in
-    the 128-byte-swizzle shared-memory layout."""
+    the 128-byte-swizzle shared-memory layout, 3 = A through tensor memory and B MN-major with that swizzle."""
     N, K = B.shape
     D = torch.zeros((128, N), device=A.device, dtype=torch.float32)
     status = torch.zeros(1, device=A.device, dtype=torch.int32)

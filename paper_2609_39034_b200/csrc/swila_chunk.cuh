@@ -112,6 +112,10 @@ struct ChunkCfg {
   // into the tile, 4 KB per copy.
   static constexpr int TILE_HALF = 4 * C * 128;
   static constexpr int TILE_BYTES = (DK / 64) * TILE_HALF;
+  // A second copy of a chunk's keys for the update MMA, which reads them MN-major (tokens = K index) after the
+  // chunk, when the tile rows are already being refilled: 3-deep ring of [DK/64][C rows][128 bytes], same swizzle.
+  static constexpr int KU_HALF = C * 128;
+  static constexpr int KU_BYTES = (DK / 64) * KU_HALF;
   // raw stages (2-deep ring): v [C][COLS] bf16; beta logits [C][J][COLS] bf16, overwritten in place by the
   // helpers with beta = sigmoid(.) as fp32 [C][NROW] (hence the fp32-sized slot); pik logits [C][J][COLS]
   // bf16.  The query-prior logits piq [C][J][COLS] live in their own 4-deep ring because the outputs of
@@ -125,22 +129,20 @@ struct ChunkCfg {
   static constexpr int RAW_BYTES = R_PK + C * J * GROW * ES;
   static constexpr int RPQ_BYTES = C * J * GROW * ES;
   // bytes one chunk's tensor copies deliver: k and q into the operand tile, v, three gate tensors
-  static constexpr int STAGE_TX_BYTES = 2 * C * DK * ES + C * COLS * ES + 3 * C * J * GROW * ES;
+  static constexpr int STAGE_TX_BYTES = 3 * C * DK * ES + C * COLS * ES + 3 * C * J * GROW * ES;
   static_assert(C * J * GROW * ES <= C * NROW * 4, "the beta logits must fit the slot their gates overwrite");
   static constexpr int C_K = DK * ES / 16, C_V = COLS * ES / 16;  // 16-byte units per token row / column slice
   // operand tiles written by the helpers (bf16, same unit layout, 8 tokens per unit)
-  static constexpr int KT_LBO = DK * 16;           // K transposed: rows = key dims, K index = tokens
-  static constexpr int KT_BYTES = (C / 8) * KT_LBO;
   static constexpr int BQ_LBO = C * 16;            // masked (K Q^T)^T: rows = later token, K index = earlier token
   static constexpr int BQ_TILE = (C / 8) * BQ_LBO;
   static constexpr int GX_LBO = 2 * C * 16;        // ([K;Q]_{n+1} K_n^T): rows = token of the next chunk
   static constexpr int GX_TILE = (C / 8) * GX_LBO;
   // shared memory map (bytes)
   static constexpr int OFF_TILE = 0;
-  static constexpr int OFF_RAW = OFF_TILE + TILE_BYTES;
+  static constexpr int OFF_KU = OFF_TILE + TILE_BYTES;
+  static constexpr int OFF_RAW = OFF_KU + 3 * KU_BYTES;
   static constexpr int OFF_RPQ = OFF_RAW + 2 * RAW_BYTES;
-  static constexpr int OFF_KT = OFF_RPQ + 4 * RPQ_BYTES;
-  static constexpr int OFF_G = OFF_KT + KT_BYTES;             // 2 x Gkk [C][C] fp32 (K K^T, for the row warps)
+  static constexpr int OFF_G = OFF_RPQ + 4 * RPQ_BYTES;             // 2 x Gkk [C][C] fp32 (K K^T, for the row warps)
   static constexpr int OFF_BQ = OFF_G + 2 * C * C * 4;        // 2 x { hi, lo } readout operand tiles
   static constexpr int OFF_GX = OFF_BQ + 2 * 2 * BQ_TILE;     // { hi, lo } cross-chunk operand tiles
   static constexpr int OFF_OST = OFF_GX + 2 * GX_TILE;        // 2 x [C][COLS] bf16 output staging
@@ -148,7 +150,7 @@ struct ChunkCfg {
   static constexpr int OFF_BAR = OFF_P0 + C * NROW * 4;
   static constexpr int SMEM_BYTES = OFF_BAR + 128 + 1024;  // + 1024: the kernel aligns its window to 1024 bytes
   static_assert(RAW_BYTES % 128 == 0 && RPQ_BYTES % 128 == 0 && R_B % 128 == 0 && R_PK % 128 == 0 && OFF_RAW % 128 == 0 &&
-                    OFF_RPQ % 128 == 0 && OFF_TILE % 1024 == 0 && DK % 64 == 0 && (COLS * ES) % 16 == 0 && (GROW * ES) % 16 == 0,
+                    OFF_RPQ % 128 == 0 && OFF_TILE % 1024 == 0 && OFF_KU % 1024 == 0 && KU_BYTES % 1024 == 0 && DK % 64 == 0 && (COLS * ES) % 16 == 0 && (GROW * ES) % 16 == 0,
                 "destinations of the tensor copies are 128-byte aligned, their rows multiples of 16 bytes");
   static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 };
@@ -158,7 +160,7 @@ struct ChunkCfg {
 // odd chunk has landed).  Arrived by threads: KT (transposed keys ready, 128 helpers), WP (operand parts of W refreshed, 128 helpers), GS
 // (Gram batch spilled, 2 helper warps), C (chunk finished, 128 rows), PQF ([P0|Q0] taken out of tensor
 // memory, 128 rows), BE (gates of a chunk ready, 128 helpers), OD (outputs of a chunk formed, 128 helpers).
-enum { B_E = 0, B_G, B_U, B_QD, B_KQ0, B_KQ1, B_KT, B_WP, B_GS, B_C, B_PQF, B_BE, B_OD, B_COUNT };
+enum { B_E = 0, B_G, B_U, B_QD, B_KQ0, B_KQ1, B_WP, B_GS, B_C, B_PQF, B_BE, B_OD, B_COUNT };
 
 // bf16 split of FP32 values: hi = bf16(x) (nearest), lo = bf16(x - hi); pairs packed with the first
 // value in the low half, which is where the tensor cores expect the even K index.
@@ -179,7 +181,7 @@ struct ChunkMaps {
 // 64 key dims x 32 tokens per copy, 128-byte swizzle) and into the raw stage (v, gate logits).  Tokens past the end
 // of the sequence and columns past Dv are filled with zeros by the copy engine.  Everything lands on `bar`.
 template <class Cf>
-__device__ __forceinline__ void chunk_stage(const ChunkMaps &maps, unsigned char *tile, unsigned char *raw,
+__device__ __forceinline__ void chunk_stage(const ChunkMaps &maps, unsigned char *tile, unsigned char *ku, unsigned char *raw,
                                             unsigned char *rawpq, int bh, int tok, int col0, int m, uint64_t *bar) {
   using namespace umma;
   constexpr int DK = Cf::DK, C = Cf::C;
@@ -190,6 +192,7 @@ __device__ __forceinline__ void chunk_stage(const ChunkMaps &maps, unsigned char
   for (int hf = 0; hf < DK / 64; ++hf) {
     tma_load_3d(trow + hf * Cf::TILE_HALF, &maps.k, hf * 64, tok, bh, bar);
     tma_load_3d(trow + hf * Cf::TILE_HALF + C * 128, &maps.q, hf * 64, tok, bh, bar);
+    tma_load_3d(ku + hf * Cf::KU_HALF, &maps.k, hf * 64, tok, bh, bar);
   }
   tma_load_3d(raw + Cf::R_V, &maps.v, col0, tok, bh, bar);
   tma_load_4d(raw + Cf::R_B, &maps.be, col0, 0, tok, bh, bar);
@@ -207,7 +210,6 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   // the swizzled operand tile needs a 1024-byte aligned shared-memory address
   unsigned char *smem = smem_raw + ((1024u - (umma::smem_u32(smem_raw) & 1023u)) & 1023u);
   unsigned char *tile = smem + Cf::OFF_TILE;
-  unsigned char *Kt = smem + Cf::OFF_KT;
   float *G_all = reinterpret_cast<float *>(smem + Cf::OFF_G);
   unsigned char *BQ_all = smem + Cf::OFF_BQ;
   unsigned char *GX_all = smem + Cf::OFF_GX;
@@ -288,7 +290,6 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     mbar_init(&bars[B_QD], 1);
     mbar_init(&bars[B_KQ0], 1);  // the thread that issues the tensor copies
     mbar_init(&bars[B_KQ1], 1);
-    mbar_init(&bars[B_KT], 128);
     mbar_init(&bars[B_WP], 128);
     mbar_init(&bars[B_GS], 64);
     mbar_init(&bars[B_C], 128);
@@ -550,22 +551,6 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   } else if (warp < 8) {
     // =============================== helper warps ============================================
     const int h = r;
-    // K of a chunk, transposed: unit (row d', c) holds K[8c .. 8c+7][d'], read from the operand tile
-    auto cook_kt = [&](int m) {
-      const unsigned char *trow = tile + (m & 1) * 2 * C * 128;
-#pragma unroll 1
-      for (int e = h; e < (C / 8) * DK; e += 128) {
-        const int dd = e % DK, c = e / DK;
-        const unsigned char *src = trow + (dd >> 6) * Cf::TILE_HALF + (8 * c) * 128 + (dd & 7) * 2;
-        const int cu = (dd >> 3) & 7;  // 16-byte unit of the row before the swizzle; token 8c+i sits in row ... + i
-        uint32_t w[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-          w[i] = (uint32_t)*reinterpret_cast<const unsigned short *>(src + (2 * i) * 128 + ((cu ^ (2 * i)) << 4)) |
-                 ((uint32_t)*reinterpret_cast<const unsigned short *>(src + (2 * i + 1) * 128 + ((cu ^ (2 * i + 1)) << 4)) << 16);
-        *reinterpret_cast<uint4 *>(Kt + c * Cf::KT_LBO + dd * 16) = make_uint4(w[0], w[1], w[2], w[3]);
-      }
-    };
     // beta = sigmoid(logit) of this helper's row for every token of a raw stage (App. B.2), written over the
     // logits: all helpers read their logits first, then all write
     auto cook_be = [&](unsigned char *raw) {
@@ -643,7 +628,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     // stage chunk m of this piece (one thread; the buffers it overwrites were last read through ordinary loads,
     // hence the proxy fence)
     auto stage = [&](int m) {
-      chunk_stage<Cf>(maps, tile, smem + Cf::OFF_RAW + (m & 1) * Cf::RAW_BYTES, smem + Cf::OFF_RPQ + (m & 3) * Cf::RPQ_BYTES, bh,
+      chunk_stage<Cf>(maps, tile, smem + Cf::OFF_KU + (m % 3) * Cf::KU_BYTES, smem + Cf::OFF_RAW + (m & 1) * Cf::RAW_BYTES, smem + Cf::OFF_RPQ + (m & 3) * Cf::RPQ_BYTES, bh,
                       tseg0 + m * C, col0, m, &bars[B_KQ0 + (m & 1)]);
     };
     // everything staged for chunk m has landed (the barrier of m's parity completes once per chunk of that parity)
@@ -698,9 +683,6 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     if (!staged(0)) failed = true;
     cook_be(smem + Cf::OFF_RAW);
     mbar_arrive(&bars[B_BE]);
-    cook_kt(0);
-    fence_async_smem();
-    mbar_arrive(&bars[B_KT]);
     if (spill_mine[0]) {
       if (!mbar_wait(&bars[B_G], 0)) failed = true;
       tc_fence_after_sync();
@@ -747,12 +729,6 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         mbar_arrive(&bars[B_WP]);
       }
       PROF_ADD(6);
-      // (5) transposed K of chunk n+1 (the update of chunk n has released the tile)
-      if (more) {
-        cook_kt(n + 1);
-        fence_async_smem();
-        mbar_arrive(&bars[B_KT]);
-      }
       PROF_ADD(7);
     }
     if (!failed && !mbar_wait(&bars[B_QD], (nchunks - 1) & 1)) failed = true;
@@ -760,7 +736,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   } else if (lane == 0) {
     // =============================== MMA issuer ==============================================
     constexpr uint32_t idE = idesc_bf16(128, 2 * C);  // N = 2C: [P0 | Q0], Gram batch, cross-chunk term
-    constexpr uint32_t idU = idesc_bf16(128, DK);
+    constexpr uint32_t idU = idesc_bf16_bmn(128, DK);  // B (the keys) is read MN-major
     constexpr uint32_t idQ = idesc_bf16(128, C);
     // operand of the tile starting at row `row0`, K step ks (16 key dims = 32 bytes inside a 128-byte row; four
     // steps per half of 64 key dims)
@@ -768,7 +744,6 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     auto tile_desc = [&](int row0, int ks) {
       return smem_desc_sw128(tile_addr + (ks >> 2) * Cf::TILE_HALF + row0 * 128 + (ks & 3) * 32, 1024);
     };
-    const uint64_t kt0 = smem_desc_kmajor(smem_u32(Kt), Cf::KT_LBO, 128);
     const uint64_t gx_hi = smem_desc_kmajor(smem_u32(GX_all), Cf::GX_LBO, 128);
     const uint64_t gx_lo = smem_desc_kmajor(smem_u32(GX_all + Cf::GX_TILE), Cf::GX_LBO, 128);
     // Gram batch of chunk m: every row of the tile against [K;Q] of chunk m and against K of chunk m-1
@@ -839,6 +814,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         PROF_ADD(1);
       }
       if (!mbar_wait(&bars[B_C], n & 1)) { failed = true; break; }
+      tc_fence_after_sync();
       PROF_ADD(2);
       if (more) {
         if (!mbar_wait(&bars[B_GS], (n + 1) & 1)) { failed = true; break; }
@@ -846,12 +822,12 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         cross();  // -> E(n+1): the only tensor work between two chunks of the row warps
       }
       PROF_ADD(3);
-      if (!mbar_wait(&bars[B_KT], n & 1)) { failed = true; break; }
-      tc_fence_after_sync();
       PROF_ADD(4);
 #pragma unroll 1
       for (int ks = 0; ks < C / 16; ++ks) {  // W += Cmat K (Eq. 3.3 summed over the chunk)
-        const uint64_t bt = kt0 + (uint64_t)(ks * 2 * (Cf::KT_LBO / 16));
+        // B = the second copy of the chunk's keys, read MN-major: 16 tokens per step = 16 rows of 128 bytes, the
+        // halves of 64 key dims KU_HALF apart
+        const uint64_t bt = smem_desc_sw128_mn(smem_u32(smem + Cf::OFF_KU + (n % 3) * Cf::KU_BYTES) + ks * 16 * 128, Cf::KU_HALF, 1024);
         mma_bf16_ts(tb0 + Cf::TM_W, tb0 + Cf::TM_CHI + ks * 8, bt, idU, true);
         mma_bf16_ts(tb0 + Cf::TM_W, tb0 + Cf::TM_CLO + ks * 8, bt, idU, true);
       }

@@ -181,6 +181,19 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t smem_addr, uint32_t
   d |= (uint64_t)2 << 61;  // layout type: 128-byte swizzle
   return d;
 }
+// The same swizzle for an operand stored MN-major (the M or N index contiguous): a row is 128 bytes = 64 consecutive
+// M/N indices of one K index, 8 K indices form a 1024-byte atom; `lbo` = byte distance between the atoms of
+// consecutive blocks of 64 M/N indices, `sbo` = byte distance between atoms of consecutive groups of 8 K indices.
+// To be used with the matching major-ness bit of the instruction descriptor.
+__device__ __forceinline__ uint64_t smem_desc_sw128_mn(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((smem_addr >> 4) & 0x3fffu);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
 // Instruction descriptor: TF32 x TF32 -> FP32, both operands K-major, dense.
 __host__ __device__ constexpr uint32_t idesc_tf32(int M, int N) {
   return (1u << 4) /*D = f32*/ | (2u << 7) /*A = tf32*/ | (2u << 10) /*B = tf32*/ | ((uint32_t)(N >> 3) << 17) |
@@ -216,6 +229,8 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int M, int N) {
   return (1u << 4) /*D = f32*/ | (1u << 7) /*A = bf16*/ | (1u << 10) /*B = bf16*/ | ((uint32_t)(N >> 3) << 17) |
          ((uint32_t)(M >> 4) << 24);
 }
+// The same with B stored MN-major in shared memory (bit 16 of the descriptor).
+__host__ __device__ constexpr uint32_t idesc_bf16_bmn(int M, int N) { return idesc_bf16(M, N) | (1u << 16); }
 // D[tmem] (+)= A[tmem] * B[smem] with 16-bit operands: the A tile holds two consecutive K elements per
 // 32-bit tensor-memory column (even k in the low half), 8 columns per instruction.
 __device__ __forceinline__ void mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,

@@ -220,6 +220,72 @@ __global__ void __launch_bounds__(128) umma_selftest_sw128_kernel(const float *A
   __syncthreads();
   if (warp == 0) tmem_dealloc(tbase, TM_COLS);
 }
+
+// A through tensor memory (two K elements per column), B [N = 128][K = 32] stored MN-major with the 128-byte
+// swizzle: rows = K index, 128 bytes = 64 consecutive N per row, two blocks of 64 N.
+__global__ void __launch_bounds__(128) umma_selftest_bmn_kernel(const float *A, const float *B, float *D, int *status) {
+  constexpr int N = 128, K = 32, BLOCK = K * 128;  // bytes of one block of 64 N
+  __shared__ __align__(1024) unsigned char sB[2 * BLOCK];
+  __shared__ __align__(8) uint64_t bar;
+  __shared__ uint32_t tmem_base_s;
+  const int tid = threadIdx.x, warp = tid >> 5;
+  constexpr uint32_t TM_COLS = 256;
+
+  if (warp == 0) tmem_alloc(&tmem_base_s, TM_COLS);
+  if (tid == 0) {
+    mbar_init(&bar, 1);
+    mbar_fence_init();
+  }
+  for (int i = tid; i < N * K; i += 128) {
+    const int n = i / K, k = i % K;
+    const int off = (n >> 6) * BLOCK + k * 128 + ((((n & 63) >> 3) ^ (k & 7)) << 4) + (n & 7) * 2;
+    *reinterpret_cast<uint16_t *>(sB + off) = (uint16_t)bf16_bits(B[(size_t)n * K + k]);
+  }
+  fence_async_smem();
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tbase = tmem_base_s;
+  const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+#pragma unroll
+  for (int c = 0; c < K / 8; ++c) {
+    uint32_t v[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      v[i] = bf16_bits(A[(size_t)tid * K + c * 8 + 2 * i]) | (bf16_bits(A[(size_t)tid * K + c * 8 + 2 * i + 1]) << 16);
+    tmem_st4(tbase + lane_base + c * 4, v);
+  }
+  tmem_st_wait();
+  tc_fence_before_sync();
+  __syncthreads();
+  if (tid == 0) {
+    tc_fence_after_sync();
+    constexpr uint32_t idesc = idesc_bf16_bmn(128, N);
+#pragma unroll
+    for (int ks = 0; ks < K / 16; ++ks) {  // 16 K indices = 16 rows of 128 bytes
+      const uint64_t bdesc = smem_desc_sw128_mn(smem_u32(sB) + ks * 16 * 128, BLOCK, 1024);
+      mma_bf16_ts(tbase + 128, tbase + ks * 8, bdesc, idesc, ks > 0);
+    }
+    mma_commit(&bar);
+  }
+  const bool ok = mbar_wait(&bar, 0);
+  tc_fence_after_sync();
+  if (ok) {
+#pragma unroll
+    for (int c = 0; c < N / 16; ++c) {
+      float v[16];
+      tmem_ld16(tbase + lane_base + 128 + c * 16, v);
+      tmem_ld_wait();
+#pragma unroll
+      for (int i = 0; i < 16; ++i) D[(size_t)tid * N + c * 16 + i] = v[i];
+    }
+  } else if (tid == 0) {
+    *status = 1;
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tbase, TM_COLS);
+}
 }  // namespace
 
 extern "C" int swila_selftest_tf32_mma(const float *A, const float *B, float *D, int N, int K, int *status,
@@ -244,6 +310,7 @@ extern "C" int swila_selftest_bf16_mma(const float *A, const float *B, float *D,
   else if (N == 64 && K == 64 && a_in_smem == 1) umma_selftest_bf16_kernel<64, 64, 1><<<1, 128, 0, st>>>(A, B, D, status);
   else if (N == 64 && K == 64 && a_in_smem == 2) umma_selftest_sw128_kernel<64><<<1, 128, 0, st>>>(A, B, D, status);
   else if (N == 32 && K == 64 && a_in_smem == 2) umma_selftest_sw128_kernel<32><<<1, 128, 0, st>>>(A, B, D, status);
+  else if (N == 128 && K == 32 && a_in_smem == 3) umma_selftest_bmn_kernel<<<1, 128, 0, st>>>(A, B, D, status);
   else return SWILA_ERR_UNSUPPORTED;
   return cudaGetLastError() == cudaSuccess ? SWILA_OK : SWILA_ERR_CUDA;
 }

@@ -26,7 +26,7 @@ def test_tf32_mma_matches_matmul(N, K):
     assert err < 1e-5, err
 
 
-@pytest.mark.parametrize("N,K,a_in_smem", [(64, 128, 0), (128, 32, 0), (32, 32, 0), (64, 64, 1), (64, 64, 2), (32, 64, 2)])
+@pytest.mark.parametrize("N,K,a_in_smem", [(64, 128, 0), (128, 32, 0), (32, 32, 0), (64, 64, 1), (64, 64, 2), (32, 64, 2), (128, 32, 3)])
 def test_bf16_mma_matches_matmul(N, K, a_in_smem):
     assert torch.cuda.is_available()
     from paper_2609_39034_b200 import binding
