@@ -565,7 +565,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     };
     // operand parts of W after an update, this helper's tensor-memory lane
     auto refresh_parts = [&]() {
-#pragma unroll
+#pragma unroll 2
       for (int cc = 0; cc < DK / 16; ++cc) {
         float w[16];
         uint32_t hi[8], lo[8];

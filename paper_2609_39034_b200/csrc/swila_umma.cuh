@@ -39,14 +39,27 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
-  if (mbar_try_wait(bar, parity)) return true;
+// The polling loop is kept out of line (one copy per translation unit) so that the many wait sites of a kernel
+// cost the instruction cache one test and one call each.
+static __device__ __noinline__ bool mbar_wait_poll(uint32_t bar_addr, uint32_t parity) {
   const unsigned long long t0 = global_timer_ns();
 #pragma unroll 1
   for (uint32_t i = 1;; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar_addr), "r"(parity)
+        : "memory");
+    if (ok) return true;
     if ((i & 255u) == 0 && global_timer_ns() - t0 > 2000000000ull) return false;
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;  // the common case: the phase is already complete
+  return mbar_wait_poll(smem_u32(bar), parity);
 }
 
 // Arrive on a barrier and announce `bytes` of asynchronous copies that will complete on it.
