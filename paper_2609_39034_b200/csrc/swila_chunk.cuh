@@ -31,14 +31,17 @@
 // three roles that run concurrently and meet on mbarriers:
 //   row warps 0-3    thread r serves row (d = r / J, j = r % J), which is also its tensor-memory
 //                    lane; the J components of a column sit in adjacent lanes, so the E-step
-//                    normalisation is a few shuffles.  They run the sequential part of a chunk
-//                    and, while the tensor cores finish the hand-over to the next chunk, form the
-//                    outputs of the previous one.
-//   helper warps 4-7 stage chunks (cp.async straight into the tensor cores' operand layout for k
-//                    and q), turn gate logits into gates, move Gram matrices from tensor memory to
-//                    shared memory (plain rows for the row warps, hi / lo operand tiles for the
-//                    MMAs), split the state into its operand parts after each update.
+//                    normalisation is a few shuffles.  They run the sequential part of a chunk.
+//   helper warps 4-7 turn gate logits into gates, move Gram matrices from tensor memory to shared
+//                    memory (plain rows for the row warps, hi / lo operand tiles for the MMAs),
+//                    split the state into its operand parts after each update, and form the
+//                    outputs of the previous chunk.  One of their threads issues the tensor copies
+//                    (TMA) that stage a chunk: k and q straight into the tensor cores' swizzled
+//                    operand tile, v and the gate logits into a raw stage.
 //   warp 8, lane 0   issues every tcgen05.mma and commits them to the barriers.
+//
+// When the tiles of a launch do not fill a whole number of waves, the chunk sequence is cut into
+// equal runs per gang of blocks and split tiles hand their state over between blocks (ChunkSched).
 #pragma once
 
 #include <cuda.h>  // CUtensorMap and its enums (types only; the encoder is fetched through the runtime)
