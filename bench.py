@@ -286,6 +286,59 @@ def paper_shapes_leg(binding, stream):
     return out
 
 
+def variants_leg(binding, stream, fma_peak_tflops: float):
+    """The Temporal and Gated variants (App. B.3, Eqs. 3.7-3.8) on all five configurations: prefill time per
+    variant for configs 0-3, decode time per step for config 4 (after a 256-token prefill).  Every variant runs in
+    the scan kernel; the vanilla line is there for comparison (AUTO: the chunked kernel where it applies)."""
+    names = [("vanilla", {}), ("temporal", dict(temporal=True)), ("gated_pre_per_key", dict(gated=True)),
+             ("gated_post_per_key", dict(gated=True, post_decay=True)),
+             ("gated_pre_per_out", dict(gated=True, granularity=wl.GRAN_PER_OUT)),
+             ("gated_temporal", dict(temporal=True, gated=True))]
+    peaks = _peaks()
+    out = {}
+    for cfg in (0, 1, 2, 3):
+        rows = {}
+        for name, kw in names:
+            w = wl.CONFIGS[cfg].variant(**kw)
+            inp = wl.make_inputs(w, device="cuda")
+            st = binding.state_alloc(w)
+            o = torch.empty((w.B, w.H, w.T, w.Dv), device="cuda", dtype=w.torch_io_dtype)
+            f = lambda: binding.swila_forward(w, inp, state_in=None, state_out=st, o=o)
+            for _ in range(3):
+                f()
+            torch.cuda.synchronize()
+            ms = time_steps(f, 10, stream) / 10
+            tfl = algorithmic_flops(w) / (ms * 1e-3) / 1e12
+            rows[name] = {"ms": ms, "tokens_per_s": w.B * w.T / (ms * 1e-3), "alu_frac": tfl / fma_peak_tflops,
+                          "hbm_frac": algorithmic_bytes(w) / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+            del inp, st, o
+        out[wl.CONFIGS[cfg].name] = rows
+    rows = {}
+    for name, kw in names:
+        w = wl.CONFIGS[4].variant(**kw).with_(T=256)
+        st = binding.state_alloc(w)
+        pre = wl.make_inputs(w, device="cuda", seed_offset=1)
+        binding.swila_forward(w, pre, state_in=st, state_out=st)
+        del pre
+        steps = [wl.decode_step_inputs(w, s, device="cuda") for s in range(8)]
+        o1 = torch.empty((w.B, w.H, 1, w.Dv), device="cuda", dtype=w.torch_io_dtype)
+        k = [0]
+
+        def step():
+            binding.swila_decode_step(w, steps[k[0] % 8], st, o=o1)
+            k[0] += 1
+
+        for _ in range(8):
+            step()
+        torch.cuda.synchronize()
+        ms = time_steps(step, 64, stream) / 64
+        rows[name] = {"ms_per_step": ms, "steps_per_s": 1e3 / ms,
+                      "hbm_frac": algorithmic_bytes(w.with_(T=1)) / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        del st, steps, o1
+    out[wl.CONFIGS[4].name + "_decode"] = rows
+    return out
+
+
 def _peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -307,6 +360,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     ap.add_argument("--no-scan", action="store_true", help="skip the scan-kernel comparison leg")
     ap.add_argument("--paper-shapes", action="store_true", help="also time the shapes the paper itself quotes")
+    ap.add_argument("--variants", action="store_true", help="also time the Temporal / Gated variants on all five configs")
     ap.add_argument("--decode-steps", type=int, default=wl.DECODE_STEPS)
     ap.add_argument("--decode-prefill", type=int, default=4096)
     ap.add_argument("--decode-batch", type=int, default=0, help="override B of the decode leg (0 = 256)")
@@ -455,6 +509,7 @@ def main():
         torch.cuda.empty_cache()
 
     paper = paper_shapes_leg(binding, stream) if args.paper_shapes else None
+    variants = variants_leg(binding, stream, fma_peak_nominal) if args.variants else None
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -474,7 +529,7 @@ def main():
                        "l2": "inputs (2.1 GB) larger than L2; no flush needed",
                        "multi_gpu": "independent replicas, no collective"},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": args.steps,
-            "clocks": clocks, "decode": decode, "scan": scan, "paper_shapes": paper,
+            "clocks": clocks, "decode": decode, "scan": scan, "paper_shapes": paper, "variants": variants,
         }
         print(json.dumps(line))
     if world > 1:

@@ -237,6 +237,23 @@ int swila_selftest_tf32_mma(const float *A, const float *B, float *D, int N, int
 int swila_selftest_bf16_mma(const float *A, const float *B, float *D, int N, int K, int a_in_smem, int *status,
                             void *stream);
 
+/*
+ * Host-only probes of how SWILA_ALGO_CHUNK distributes work (no counterpart in the paper; no GPU call).
+ * A launch has B*H*ceil(Dv / (128/J)) tiles of 128 state rows, each a sequence of ceil(T/32) chunks.
+ *
+ * swila_chunk_plan: the layout chosen for a device with `sm_count` SMs.  out[0] = 1 if the chunk sequence
+ * is cut into equal runs (taken when the tiles do not fill a whole number of waves and a state output is
+ * given), else 0 (one tile per block); out[1] = blocks per gang (column slices of one (batch, head));
+ * out[2] = chunks per unit; out[3] = chunks per run; out[4] = units (tiles, or (batch, head) pairs when
+ * split); out[5] = blocks launched.  Returns SWILA_OK or an error code (J must be 4 or 8).
+ *
+ * swila_chunk_run_pieces: the pieces of run `run` in the order a block processes them, as triples
+ * (unit, first chunk, end chunk) written to `pieces` (HOST int[3 * capacity]).  Returns the number of pieces
+ * (0 for a run past the end of the work) or a negative error code.
+ */
+int swila_chunk_plan(int B, int H, int T, int Dv, int J, int sm_count, int has_state_out, long long out[6]);
+int swila_chunk_run_pieces(long long units, int nch, int per, long long run, int *pieces, int capacity);
+
 #ifdef __cplusplus
 }
 #endif

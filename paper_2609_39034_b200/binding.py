@@ -24,7 +24,7 @@ ALGO_AUTO, ALGO_SCAN, ALGO_SCAN_WIDE, ALGO_SCAN_NARROW, ALGO_CHUNK = 0, 1, 2, 3,
 EXPORTS = ("swila_version", "swila_strerror", "swila_last_cuda_error", "swila_state_w_bytes",
            "swila_state_r_bytes", "swila_state_init", "swila_forward", "swila_decode_step",
            "swila_bench_fma_chain", "swila_forward_host", "swila_forward_host_workspace_bytes",
-           "swila_forward_host_static", "swila_forward_host_static_capacity", "swila_selftest_tf32_mma", "swila_selftest_bf16_mma", "swila_device_status")
+           "swila_forward_host_static", "swila_forward_host_static_capacity", "swila_selftest_tf32_mma", "swila_selftest_bf16_mma", "swila_device_status", "swila_chunk_plan", "swila_chunk_run_pieces")
 
 
 class Shape(ctypes.Structure):
@@ -89,6 +89,11 @@ def _load() -> ctypes.CDLL:
     L.swila_selftest_tf32_mma.restype = ctypes.c_int
     L.swila_selftest_tf32_mma.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
                                           ctypes.c_void_p, ctypes.c_void_p]
+    L.swila_chunk_plan.restype = ctypes.c_int
+    L.swila_chunk_plan.argtypes = [ctypes.c_int] * 7 + [ctypes.POINTER(ctypes.c_longlong)]
+    L.swila_chunk_run_pieces.restype = ctypes.c_int
+    L.swila_chunk_run_pieces.argtypes = [ctypes.c_longlong, ctypes.c_int, ctypes.c_int, ctypes.c_longlong,
+                                         ctypes.POINTER(ctypes.c_int), ctypes.c_int]
     L.swila_device_status.restype = ctypes.c_int
     L.swila_bench_fma_chain.restype = ctypes.c_int
     L.swila_bench_fma_chain.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
@@ -252,6 +257,23 @@ def selftest_bf16_mma(A: torch.Tensor, B: torch.Tensor, a_in_smem: int = 0) -> t
     if int(status.item()) != 0:
         raise RuntimeError("tcgen05 self-test: the MMA did not signal completion")
     return D
+
+
+def chunk_plan(B: int, H: int, T: int, Dv: int, J: int, sm_count: int, has_state_out: bool = True) -> dict:
+    """Work layout SWILA_ALGO_CHUNK would choose (host arithmetic only)."""
+    out = (ctypes.c_longlong * 6)()
+    check(lib.swila_chunk_plan(B, H, T, Dv, J, sm_count, int(has_state_out), out))
+    return dict(zip(("split", "gang", "nch", "per", "units", "grid"), (int(x) for x in out)))
+
+
+def chunk_run_pieces(units: int, nch: int, per: int, run: int) -> list:
+    """Pieces (unit, first chunk, end chunk) of one run, in processing order (host arithmetic only)."""
+    cap = 16 + per // max(nch, 1)
+    buf = (ctypes.c_int * (3 * cap))()
+    n = lib.swila_chunk_run_pieces(units, nch, per, run, buf, cap)
+    if n < 0:
+        check(n)
+    return [(buf[3 * i], buf[3 * i + 1], buf[3 * i + 2]) for i in range(n)]
 
 
 def device_status() -> None:

@@ -50,6 +50,7 @@
 #include <atomic>
 #include <type_traits>
 
+#include "swila_chunk_sched.h"
 #include "swila_common.cuh"
 #include "swila_umma.cuh"
 
@@ -226,10 +227,8 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   uint32_t *fail_s = tmem_base_s + 1;  // set by any thread whose bounded wait expired: no further piece is started
   // this block's run of chunks and the pieces (tile, first chunk, end chunk) it falls into
   const int gang_slice = (int)(blockIdx.x % sched.gang);
-  const long long run0 = (long long)(blockIdx.x / sched.gang) * sched.per;
-  const long long run1 = min((long long)sched.ntiles * sched.nch, run0 + sched.per);
-  const int tile_first = (int)(run0 / sched.nch), chunk_first = (int)(run0 % sched.nch);
-  const int npieces = run1 > run0 ? (int)((run1 - 1) / sched.nch) - tile_first + 1 : 0;
+  const long long run = blockIdx.x / sched.gang;
+  const int npieces = chunk_run_pieces(sched.ntiles, sched.nch, sched.per, run);
   if (warp == 8) tmem_alloc(tmem_base_s, Cf::TM_ALLOC);
   if (tid == 0) *fail_s = 0;
   const uint32_t tb_lane = ((uint32_t)((warp & 3) * 32) << 16);  // this warp's lane quarter
@@ -252,23 +251,9 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
 
 #pragma unroll 1
   for (int pi = 0; pi < npieces; ++pi) {
-    // the piece being processed (uniform over the block).  Order: a trailing piece that ends inside a tile
-    // (a head, whose state another block waits for) first, whole tiles next, a leading piece that starts
-    // inside a tile (a tail, which waits for another block's head) last.  A head is shorter than a run, so
-    // it is finished before the block that owns the tail gets there.
-    const bool has_tail = chunk_first > 0;
-    const bool has_head = run1 % sched.nch != 0 && !(npieces == 1 && has_tail);
-    int ps;
-    if (has_head && pi == 0) {
-      ps = npieces - 1;
-    } else {
-      const int k = pi - (has_head ? 1 : 0);
-      const int mid = npieces - (has_head ? 1 : 0) - (has_tail ? 1 : 0);
-      ps = k < mid ? k + (has_tail ? 1 : 0) : 0;
-    }
-    const int tl = tile_first + ps;
-    const int cb = ps == 0 ? chunk_first : 0;
-    const int ce = (int)min((long long)sched.nch, run1 - (long long)tl * sched.nch);
+    // the piece being processed (uniform over the block); the order of a run's pieces is chunk_run_piece's
+    const ChunkPiece piece = chunk_run_piece(sched.ntiles, sched.nch, sched.per, run, pi);
+    const int tl = piece.unit, cb = piece.cb, ce = piece.ce;
     const int bh = sched.gang > 1 ? tl : tl / nslice;
     const int col0 = (sched.gang > 1 ? gang_slice : tl - bh * nslice) * COLS;
     const int nchunks = ce - cb;
@@ -947,29 +932,19 @@ int launch_chunk(const LaunchArgs &a) {
   if (!chunk_make_maps<Cf>(a.p, &maps)) return (int)cudaErrorInvalidValue;
 
   // More tiles than SMs, not a whole number of waves: cut the chunk sequence into equal runs instead of whole
-  // tiles, so that the last wave is not half empty.  The runs are laid over (batch, head) units and walked by
-  // gangs of nslice blocks (one column slice each, see ChunkSched).  The state of a split tile travels through
-  // the state output, hence only when that is given; blocks of such a launch wait for each other, hence the
+  // tiles, so that the last wave is not half empty (chunk_plan).  The state of a split tile travels through the
+  // state output, hence only when that is given; blocks of such a launch wait for each other, hence the
   // cooperative launch (all blocks resident or no launch at all).
-  const int nsm = chunk_sm_count();
-  const long long nbh = (long long)a.p.B * a.p.H;
-  const long long gangs = nslice > 0 ? nsm / nslice : 0;
-  if (gangs > 0 && a.p.W_out && nbh > gangs && ntiles <= kChunkFlagTiles && nch >= 16) {
-    const long long total = nbh * nch;
-    const long long per = (total + gangs - 1) / gangs;
-    const long long plain = ((ntiles + nsm - 1) / nsm) * nch;
-    if (per >= nch && per * 100 <= plain * 97) {
-      unsigned *flags = nullptr;
-      if (cudaGetSymbolAddress((void **)&flags, g_chunk_flags) == cudaSuccess) {
-        const unsigned epoch = chunk_next_epoch();
-        ChunkSched ss{(int)nbh, (int)nch, (int)per, (int)nslice, epoch,
-                      flags + (size_t)(epoch % kChunkFlagSlots) * kChunkFlagTiles};
-        const long long grid = ((total + per - 1) / per) * nslice;
-        void *args[] = {(void *)&prm, (void *)&ss, (void *)&maps};
-        e = cudaLaunchCooperativeKernel((const void *)kern, dim3((unsigned)grid), dim3(Cf::NT), args, Cf::SMEM_BYTES, a.stream);
-        if (e == cudaSuccess) return (int)cudaGetLastError();
-        (void)cudaGetLastError();  // not launched (e.g. the blocks cannot all be resident): fall back to whole tiles
-      }
+  const ChunkPlan pl = chunk_plan((long long)a.p.B * a.p.H, nslice, nch, chunk_sm_count(), a.p.W_out != nullptr, kChunkFlagTiles);
+  if (pl.split) {
+    unsigned *flags = nullptr;
+    if (cudaGetSymbolAddress((void **)&flags, g_chunk_flags) == cudaSuccess) {
+      const unsigned epoch = chunk_next_epoch();
+      ChunkSched ss{(int)pl.units, pl.nch, pl.per, pl.gang, epoch, flags + (size_t)(epoch % kChunkFlagSlots) * kChunkFlagTiles};
+      void *args[] = {(void *)&prm, (void *)&ss, (void *)&maps};
+      e = cudaLaunchCooperativeKernel((const void *)kern, dim3((unsigned)pl.grid), dim3(Cf::NT), args, Cf::SMEM_BYTES, a.stream);
+      if (e == cudaSuccess) return (int)cudaGetLastError();
+      (void)cudaGetLastError();  // not launched (e.g. the blocks cannot all be resident): fall back to whole tiles
     }
   }
   kern<<<(unsigned)ntiles, Cf::NT, Cf::SMEM_BYTES, a.stream>>>(prm, sc, maps);

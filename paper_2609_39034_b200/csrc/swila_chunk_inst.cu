@@ -1,5 +1,6 @@
 // Instantiations and dispatch of the chunked tensor-core kernel (bf16 io, ungated, non-temporal,
 // J in {4, 8}: with fewer components a block covers more columns and its shared-memory tiles do not fit).
+#include "../../include/swila.h"
 #include "swila_chunk.cuh"
 
 namespace swila {
@@ -28,6 +29,30 @@ int chunk_error_fetch(int *flag) {
 }
 
 }  // namespace swila
+
+// Host-only probes of the chunked kernel's work distribution (no GPU call): what the CPU tests check.
+extern "C" int swila_chunk_plan(int B, int H, int T, int Dv, int J, int sm_count, int has_state_out, long long out[6]) {
+  if (!out) return SWILA_ERR_NULL;
+  if (B <= 0 || H <= 0 || T <= 0 || Dv <= 0 || sm_count <= 0) return SWILA_ERR_SHAPE;
+  if (J != 4 && J != 8) return SWILA_ERR_UNSUPPORTED;
+  const long long cols = 128 / J, nslice = (Dv + cols - 1) / cols, nch = (T + 31) / 32;
+  const swila::ChunkPlan pl =
+      swila::chunk_plan((long long)B * H, nslice, nch, sm_count, has_state_out != 0, swila::kChunkFlagTiles);
+  out[0] = pl.split; out[1] = pl.gang; out[2] = pl.nch; out[3] = pl.per; out[4] = pl.units; out[5] = pl.grid;
+  return SWILA_OK;
+}
+
+extern "C" int swila_chunk_run_pieces(long long units, int nch, int per, long long run, int *pieces, int capacity) {
+  if (units <= 0 || nch <= 0 || per <= 0 || run < 0) return SWILA_ERR_SHAPE;
+  const int n = swila::chunk_run_pieces(units, nch, per, run);
+  if (n > capacity) return SWILA_ERR_SIZE;
+  if (n > 0 && !pieces) return SWILA_ERR_NULL;
+  for (int i = 0; i < n; ++i) {
+    const swila::ChunkPiece pc = swila::chunk_run_piece(units, nch, per, run, i);
+    pieces[3 * i] = pc.unit; pieces[3 * i + 1] = pc.cb; pieces[3 * i + 2] = pc.ce;
+  }
+  return n;
+}
 
 #ifdef SWILA_CHUNK_PROFILE
 // Developer build only: per-phase cycle counters of block 0, 8 per warp role (rows, helpers, ...).
