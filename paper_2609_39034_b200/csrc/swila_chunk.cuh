@@ -94,6 +94,8 @@ template <int J_, int DK_>
 struct ChunkCfg {
   static constexpr int J = J_, DK = DK_;
   static constexpr int C = 32;            // tokens per chunk
+  static constexpr int WIN = 24;          // tokens ahead (incl. its own trip) that a token's pushes reach on the ALUs;
+                                          // the pushes of tokens 0-7 into tokens 24-31 go through the tensor cores
   static constexpr int GT = 8;            // tokens per trip of the rolled loops (keeps the hot code inside the instruction cache)
   static constexpr int NROW = 128;        // row threads = rows of the tile
   static constexpr int NT = 288;          // 4 row warps + 4 helper warps + 1 MMA warp
@@ -101,10 +103,12 @@ struct ChunkCfg {
   static constexpr int ES = 2;            // bf16 io
   // tensor-memory columns.  W: the state (FP32 accumulator); WHI / WLO: its bf16 operand parts, two key
   // dims per column; PQ: [P0 | Q0] = state x [K;Q] of the next chunk to run; QD: the query-side readouts
-  // of a chunk (double-buffered); G: Gram matrices as they leave the tensor cores; CHI / CLO: the bf16
-  // parts of the chunk's update coefficients, two tokens per column
+  // of a chunk (double-buffered); G: Gram matrices as they leave the tensor cores; FAR: what the first 8 tokens of
+  // the chunk add to the predictions of its last 16 (only the last 8 are non-zero); CHI / CLO: the bf16 parts of the
+  // chunk's update coefficients, two tokens per column
   static constexpr int TM_W = 0, TM_WHI = DK, TM_WLO = DK + DK / 2, TM_PQ = 2 * DK, TM_QD = TM_PQ + 2 * C,
-                       TM_G = TM_QD + 2 * C, TM_CHI = TM_G + 3 * C, TM_CLO = TM_CHI + C / 2, TM_USED = TM_CLO + C / 2;
+                       TM_G = TM_QD + 2 * C, TM_FAR = TM_G + 2 * C, TM_CHI = TM_FAR + C / 2, TM_CLO = TM_CHI + C / 2,
+                       TM_USED = TM_CLO + C / 2;
   static constexpr int TM_ALLOC = 512;
   static_assert(TM_USED <= TM_ALLOC, "tensor memory budget");
   static_assert(J == 4 || J == 8, "the output transposition assumes that J divides 8");
@@ -150,7 +154,10 @@ struct ChunkCfg {
   static constexpr int OFF_BQ = OFF_G + 2 * C * C * 4;        // 2 x { hi, lo } readout operand tiles
   static constexpr int OFF_GX = OFF_BQ + 2 * 2 * BQ_TILE;     // { hi, lo } cross-chunk operand tiles
   static constexpr int OFF_OST = OFF_GX + 2 * GX_TILE;        // 2 x [C][COLS] bf16 output staging
-  static constexpr int OFF_P0 = OFF_OST + 2 * C * COLS * ES;  // [C/4][NROW] float4: a chunk's P0 rows, kept for the rare redo
+  static constexpr int FAR_LBO = (C / 2) * 16;     // far-push operand: rows = tokens 16..31, K index = tokens 0..15
+  static constexpr int FAR_TILE = 2 * FAR_LBO;
+  static constexpr int OFF_FAR = OFF_OST + 2 * C * COLS * ES;  // 2 x { hi, lo }
+  static constexpr int OFF_P0 = OFF_FAR + 2 * 2 * FAR_TILE;  // [C/4][NROW] float4: a chunk's P0 rows, kept for the rare redo
   static constexpr int OFF_BAR = OFF_P0 + C * NROW * 4;
   static constexpr int SMEM_BYTES = OFF_BAR + 128 + 1024;  // + 1024: the kernel aligns its window to 1024 bytes
   static_assert(RAW_BYTES % 128 == 0 && RPQ_BYTES % 128 == 0 && R_B % 128 == 0 && R_PK % 128 == 0 && OFF_RAW % 128 == 0 &&
@@ -163,8 +170,9 @@ struct ChunkCfg {
 // U (update of W), QD (readouts).  Completed by the tensor copies: KQ0 / KQ1 (everything staged for an even /
 // odd chunk has landed).  Arrived by threads: KT (transposed keys ready, 128 helpers), WP (operand parts of W refreshed, 128 helpers), GS
 // (Gram batch spilled, 2 helper warps), C (chunk finished, 128 rows), PQF ([P0|Q0] taken out of tensor
-// memory, 128 rows), BE (gates of a chunk ready, 128 helpers), OD (outputs of a chunk formed, 128 helpers).
-enum { B_E = 0, B_G, B_U, B_QD, B_KQ0, B_KQ1, B_WP, B_GS, B_C, B_PQF, B_BE, B_OD, B_COUNT };
+// memory, 128 rows), BE (gates of a chunk ready, 128 helpers), OD (outputs of a chunk formed, 128 helpers), T0 (update
+// coefficients of a chunk's first 8 tokens stored, 128 rows); committed by the MMA thread: FAR (far pushes of those).
+enum { B_E = 0, B_G, B_U, B_QD, B_KQ0, B_KQ1, B_WP, B_GS, B_C, B_PQF, B_BE, B_OD, B_T0, B_FAR, B_COUNT };
 
 // bf16 split of FP32 values: hi = bf16(x) (nearest), lo = bf16(x - hi); pairs packed with the first
 // value in the low half, which is where the tensor cores expect the even K index.
@@ -284,6 +292,8 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     mbar_init(&bars[B_PQF], 128);
     mbar_init(&bars[B_BE], 128);
     mbar_init(&bars[B_OD], 128);
+    mbar_init(&bars[B_T0], 128);
+    mbar_init(&bars[B_FAR], 1);
     mbar_fence_init();
   }
   tc_fence_before_sync();
@@ -415,15 +425,33 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         constexpr bool EXACT = decltype(exact_tag)::value;
         constexpr int GT = Cf::GT;
         bool bad = false;
-        // pred[i]: prediction of token tg + i of the current trip (slots past the chunk end are dead weight that
-        // keeps the trip's code independent of tg); slot C takes the last token's push
-        float pred[C + 1];
+        // pred[i]: prediction of token tg + i of the current trip, for the WINS tokens that the pushes of a token reach
+        // on the ALUs (slots past the chunk end are dead weight that keeps the trip's code independent of tg).  The fast
+        // pass reaches WIN = 24 tokens: the pushes of tokens 0-7 into tokens 24-31 come from the tensor cores (FAR)
+        // when token 24 is reached.  The redo pass does everything itself.
+        constexpr int WINS = EXACT ? C : Cf::WIN;
+        float pred[WINS];
 #pragma unroll
-        for (int t = 0; t < C; ++t) pred[t] = pred0[t];
-        pred[C] = 0.f;
+        for (int t = 0; t < WINS; ++t) pred[t] = pred0[t];
+        [[maybe_unused]] float p0late[C - Cf::WIN];
+        if constexpr (!EXACT) {
+#pragma unroll
+          for (int t = 0; t < C - Cf::WIN; ++t) p0late[t] = pred0[Cf::WIN + t];
+        }
         float c_prev = 0.f;
 #pragma unroll 1
         for (int tg = 0; tg < C; tg += GT) {
+          if constexpr (!EXACT) {
+            if (tg == Cf::WIN) {  // far pushes of tokens 0-6 into tokens 24-31
+              if (!mbar_wait(&bars[B_FAR], n & 1)) failed = true;
+              tc_fence_after_sync();
+              float far[8];
+              tmem_ld8(tb + Cf::TM_FAR + Cf::WIN - C / 2, far);
+              tmem_ld_wait();
+#pragma unroll
+              for (int i = 0; i < 8; ++i) pred[i] += far[i];
+            }
+          }
           float cs[GT];
 #pragma unroll
           for (int i = 0; i < GT; ++i) {
@@ -455,7 +483,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
             {  // deferred push of token t-1 into the predictions of tokens t+1 .. (slots i+1 ..)
               const float4 *gp = reinterpret_cast<const float4 *>(Gkk + max(t - 1, 0) * C + tg);
 #pragma unroll
-              for (int u4 = (i + 1) / 4; u4 < C / 4; ++u4) {
+              for (int u4 = (i + 1) / 4; u4 < WINS / 4; ++u4) {
                 const float4 g = gp[u4];
                 if (4 * u4 + 0 > i) pred[4 * u4 + 0] = fmaf(c_prev, g.x, pred[4 * u4 + 0]);
                 if (4 * u4 + 1 > i) pred[4 * u4 + 1] = fmaf(c_prev, g.y, pred[4 * u4 + 1]);
@@ -487,10 +515,24 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
             tmem_st4(tb + Cf::TM_CHI + tg / 2, hi);
             tmem_st4(tb + Cf::TM_CLO + tg / 2, lo);
           }
+          if constexpr (!EXACT) {
+            if (tg == 0) {  // the coefficients of tokens 0-7 are in place: the far pushes may be issued
+              tmem_st_wait();
+              tc_fence_before_sync();
+              mbar_arrive(&bars[B_T0]);
+            }
+          }
 #pragma unroll
-          for (int i = 0; i + GT <= C; ++i) pred[i] = pred[i + GT];
+          for (int i = 0; i + GT < WINS; ++i) pred[i] = pred[i + GT];
 #pragma unroll
-          for (int i = C - GT + 1; i <= C; ++i) pred[i] = 0.f;
+          for (int i = 0; i < GT; ++i) {  // the slots that enter the window: tokens 24-31 after the first trip, dead later
+            if constexpr (EXACT) {
+              pred[WINS - GT + i] = 0.f;
+            } else {
+              pred[WINS - GT + i] = p0late[i];
+              p0late[i] = 0.f;
+            }
+          }
         }
         return bad;
       };
@@ -594,6 +636,21 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
 #pragma unroll
         for (int i = 0; i < C / 4; ++i)
           *reinterpret_cast<float4 *>(Gkk + lane * C + i * 4) = make_float4(a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
+        // far-push operand: row = token u = lane (16..31), K index = tokens 0..7 (K K^T is symmetric, so this lane's
+        // row holds k_s.k_u).  Through the tensor cores go the pushes of tokens s = 0..6 into tokens u >= WIN: the row
+        // warps push token s into tokens s+1 .. 23 while they are in the first trip, and token 7, whose deferred push
+        // runs in the second trip, reaches token 31 there.  Everything else in the operand is zero.
+        if (lane >= C / 2) {
+          uint32_t hi[4], lo[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const bool use = lane >= Cf::WIN;
+            bf16_split2(use ? a[2 * i] : 0.f, (use && 2 * i + 1 < Cf::GT - 1) ? a[2 * i + 1] : 0.f, hi[i], lo[i]);
+          }
+          unsigned char *ft = smem + Cf::OFF_FAR + (m & 1) * 2 * Cf::FAR_TILE;
+          *reinterpret_cast<uint4 *>(ft + (lane - C / 2) * 16) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+          *reinterpret_cast<uint4 *>(ft + Cf::FAR_TILE + (lane - C / 2) * 16) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        }
       } else {
 #pragma unroll
         for (int s = 0; s < C; ++s) a[s] = (s <= lane) ? a[s] : 0.f;
@@ -603,7 +660,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       if (m > 0) {
 #pragma unroll
         for (int cc = 0; cc < C / 16; ++cc)
-          tmem_ld16(tb + Cf::TM_G + 2 * C + cc * 16, reinterpret_cast<float(&)[16]>(a[cc * 16]));
+          tmem_ld16(tb + Cf::TM_G + C + cc * 16, reinterpret_cast<float(&)[16]>(a[cc * 16]));
         tmem_ld_wait();
         store_parts(a, GX_all, GX_all + Cf::GX_TILE, Cf::GX_LBO, (qrows ? C : 0) + lane);
       }
@@ -660,10 +717,22 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         tmem_st8(tb + Cf::TM_WHI + cc * 8, reinterpret_cast<const float(&)[8]>(hi));
         tmem_st8(tb + Cf::TM_WLO + cc * 8, reinterpret_cast<const float(&)[8]>(lo));
       }
+      {  // coefficient columns: finite from the start (see below); ordered before the row warps' first store by WP -> E
+        const uint32_t z[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+        for (int cc = 0; cc < C / 8; ++cc) {
+          tmem_st4(tb + Cf::TM_CHI + cc * 4, z);
+          tmem_st4(tb + Cf::TM_CLO + cc * 4, z);
+        }
+      }
       tmem_st_wait();
       tc_fence_before_sync();
       mbar_arrive(&bars[B_WP]);
     }
+    // the far-push MMA spans 16 tokens of coefficients and of its operand, of which only the first 8 count: the
+    // operand's other half stays zero, and the coefficient columns must at least be finite from the start
+    for (int e = h; e < 4 * (C / 2); e += 128)
+      *reinterpret_cast<uint4 *>(smem + Cf::OFF_FAR + (e / (C / 2)) * Cf::FAR_TILE + Cf::FAR_LBO + (e % (C / 2)) * 16) = make_uint4(0, 0, 0, 0);
     if (nchunks == 1) {  // the odd half of the operand tile is read (as don't-care rows) by the Gram batch: make it finite
       for (int e = h; e < (DK / 64) * 2 * C * 8; e += 128)
         *reinterpret_cast<uint4 *>(tile + (e / (2 * C * 8)) * Cf::TILE_HALF + 2 * C * 128 + (e % (2 * C * 8)) * 16) = make_uint4(0, 0, 0, 0);
@@ -734,15 +803,15 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     };
     const uint64_t gx_hi = smem_desc_kmajor(smem_u32(GX_all), Cf::GX_LBO, 128);
     const uint64_t gx_lo = smem_desc_kmajor(smem_u32(GX_all + Cf::GX_TILE), Cf::GX_LBO, 128);
-    // Gram batch of chunk m: every row of the tile against [K;Q] of chunk m and against K of chunk m-1
+    // Gram batch of chunk m: every row of the tile against the keys of chunk m and against the keys of chunk m-1
     auto gram = [&](int m) {
 #pragma unroll 1
       for (int ks = 0; ks < DK / 16; ++ks)
-        mma_bf16_ss(tb0 + Cf::TM_G, tile_desc(0, ks), tile_desc((m & 1) * 2 * C, ks), idE, ks > 0);
+        mma_bf16_ss(tb0 + Cf::TM_G, tile_desc(0, ks), tile_desc((m & 1) * 2 * C, ks), idQ, ks > 0);
       if (m > 0) {
 #pragma unroll 1
         for (int ks = 0; ks < DK / 16; ++ks)
-          mma_bf16_ss(tb0 + Cf::TM_G + 2 * C, tile_desc(0, ks), tile_desc(((m - 1) & 1) * 2 * C, ks), idQ, ks > 0);
+          mma_bf16_ss(tb0 + Cf::TM_G + C, tile_desc(0, ks), tile_desc(((m - 1) & 1) * 2 * C, ks), idQ, ks > 0);
       }
       mma_commit(&bars[B_G]);
     };
@@ -798,6 +867,22 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         tc_fence_after_sync();
         PROF_ADD(0);
         gram(n + 1);
+      }
+      {
+        // far pushes of chunk n: what its first 8 tokens add to the predictions of its last 8, needed when the row
+        // warps reach token 24.  A = the coefficient columns of tokens 0..15 (8..15 are stale but finite and meet
+        // zero rows of the operand), B = rows 16..31 of K K^T against tokens 0..7.
+        if (!mbar_wait(&bars[B_T0], n & 1)) { failed = true; break; }
+        tc_fence_after_sync();
+        const uint32_t fa = smem_u32(smem + Cf::OFF_FAR + (n & 1) * 2 * Cf::FAR_TILE);
+        const uint64_t f_hi = smem_desc_kmajor(fa, Cf::FAR_LBO, 128), f_lo = smem_desc_kmajor(fa + Cf::FAR_TILE, Cf::FAR_LBO, 128);
+        constexpr uint32_t idF = idesc_bf16(128, C / 2);
+        mma_bf16_ts(tb0 + Cf::TM_FAR, tb0 + Cf::TM_CHI, f_hi, idF, false);
+        mma_bf16_ts(tb0 + Cf::TM_FAR, tb0 + Cf::TM_CLO, f_hi, idF, true);
+        mma_bf16_ts(tb0 + Cf::TM_FAR, tb0 + Cf::TM_CHI, f_lo, idF, true);
+        mma_commit(&bars[B_FAR]);
+      }
+      if (more) {
         w_times_kq(n + 1);
         PROF_ADD(1);
       }
