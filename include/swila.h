@@ -161,11 +161,16 @@ int swila_decode_step(const swila_shape_t *shape, const void *q, const void *k, 
  * whose tensors live in host memory.  q, k, v, every pointer inside `gates`, `state_in`,
  * `state_out` and o are HOST pointers (pinned memory makes the copies asynchronous);
  * `workspace` is a DEVICE buffer of at least swila_forward_host_workspace_bytes(shape)
- * bytes, owned by the caller and reusable across calls.  On `stream` the call enqueues the
- * host-to-device copies, the kernel, and the device-to-host copies of o and of the final
- * state; it returns without synchronising.  state_in == NULL starts from the initial
- * state; state_out == NULL discards the final state.  Errors as swila_forward, plus
- * SWILA_ERR_SIZE when the workspace is too small.
+ * bytes, owned by the caller and reusable across calls.  The call enqueues the host-to-device
+ * copies, the kernel(s), and the device-to-host copies of o and of the final state, and returns
+ * without synchronising; everything is complete once `stream` has been synchronised.  Problems
+ * of 64 MB and more go through in up to 8 slabs of (batch, head) pairs -- which are independent
+ * -- with the copies on two internal streams (created on the first such call on a device and
+ * kept) beside the kernels on `stream`, so that transfers in both directions overlap the
+ * compute; `stream` waits for the internal streams at the end.  Smaller problems use `stream`
+ * alone.  Calls from several host threads on one device share those copy streams.
+ * state_in == NULL starts from the initial state; state_out == NULL discards the final state.
+ * Errors as swila_forward, plus SWILA_ERR_SIZE when the workspace is too small.
  */
 size_t swila_forward_host_workspace_bytes(const swila_shape_t *shape);
 int swila_forward_host(const swila_shape_t *shape, const void *q, const void *k, const void *v,

@@ -1,6 +1,9 @@
 // C-ABI entry points of the SwiLA library: host-side validation and kernel dispatch.
-// No device memory is allocated here and no state is kept between calls.
+// No device memory is allocated here; the only state kept between calls is the pair of copy streams (and their
+// events) that the host-buffer front end creates on first use for problems of 64 MB and more.
 #include <string.h>
+
+#include <mutex>
 
 #include "swila_common.cuh"
 
@@ -269,6 +272,43 @@ size_t swila_forward_host_workspace_bytes(const swila_shape_t *s) {
   return host_plan(s).total;
 }
 
+}  // extern "C"
+
+// Streams and events of the pipelined host path, one set per device, created on first use and kept.
+namespace swila {
+constexpr int kHostSlabs = 8;
+struct HostPipe {
+  bool ready = false;
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t start = nullptr, done = nullptr, landed[kHostSlabs] = {}, computed[kHostSlabs] = {};
+};
+static HostPipe *host_pipe() {
+  static std::mutex mu;
+  static HostPipe pipes[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  HostPipe &hp = pipes[dev];
+  if (!hp.ready) {
+    bool ok = cudaStreamCreateWithFlags(&hp.in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&hp.out, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&hp.done, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; ok && i < kHostSlabs; ++i)
+      ok = cudaEventCreateWithFlags(&hp.landed[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&hp.computed[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
+      (void)cudaGetLastError();
+      return nullptr;
+    }
+    hp.ready = true;
+  }
+  return &hp;
+}
+}  // namespace swila
+
+extern "C" {
+
 int swila_forward_host(const swila_shape_t *s, const void *q, const void *k, const void *v, const swila_gates_t *g,
                        const swila_state_t *state_in, swila_state_t *state_out, void *o, void *workspace,
                        size_t workspace_bytes, void *stream) {
@@ -287,32 +327,78 @@ int swila_forward_host(const swila_shape_t *s, const void *q, const void *k, con
   char *ws = (char *)workspace;
   cudaStream_t cs = (cudaStream_t)stream;
   cudaError_t e = cudaSuccess;
-  auto up = [&](size_t off, const void *src, size_t n) {
-    if (e == cudaSuccess && n) e = cudaMemcpyAsync(ws + off, src, n, cudaMemcpyHostToDevice, cs);
-  };
-  up(h.q, q, h.n_qk); up(h.k, k, h.n_qk); up(h.v, v, h.n_v);
-  up(h.beta, g->beta_logit, h.n_gate); up(h.pik, g->pik_logit, h.n_gate); up(h.piq, g->piq_logit, h.n_gate);
-  if (temporal) { up(h.gk, g->gk_logit, h.n_tg); up(h.gq, g->gq_logit, h.n_tg); }
-  if (gated) up(h.alpha, g->alpha, h.n_alpha);
-  swila_state_t dstate = {(float *)(ws + h.W), temporal ? (float *)(ws + h.r) : nullptr,
-                          temporal ? (float *)(ws + h.rho) : nullptr};
-  if (state_in) {
-    up(h.W, state_in->W, h.n_W);
-    if (temporal) { up(h.r, state_in->r_prev, h.n_r); up(h.rho, state_in->rho_prev, h.n_r); }
+
+  // Every tensor is [B*H, ...] with the (batch, head) index outermost, and (batch, head) pairs are independent: large
+  // problems go through in slabs of (batch, head) pairs, the host-to-device copies of slab i+1 and the device-to-host
+  // copies of slab i-1 running on two internal streams beside the kernel of slab i on `stream`.  The call still
+  // returns without synchronising and `stream` is complete when everything is (it waits for the internal streams).
+  const long long nbh = (long long)s->B * s->H;
+  auto slab_ok = [&](size_t total) { return (total / (size_t)nbh) % 16 == 0; };  // slab bases stay 16-byte aligned
+  const bool sliceable = slab_ok(h.n_qk) && slab_ok(h.n_v) && slab_ok(h.n_gate) && slab_ok(h.n_tg) && slab_ok(h.n_alpha) &&
+                         slab_ok(h.n_W) && slab_ok(h.n_r);
+  HostPipe *hp = (h.total >= (64u << 20) && nbh >= 2 && sliceable) ? host_pipe() : nullptr;
+  const int nslab = hp ? (int)(nbh < kHostSlabs ? nbh : kHostSlabs) : 1;
+  cudaStream_t s_in = hp ? hp->in : cs, s_out = hp ? hp->out : cs;
+  if (hp) {
+    e = cudaEventRecord(hp->start, cs);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(s_in, hp->start, 0);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(s_out, hp->start, 0);
   }
-  if (e != cudaSuccess) return cuda_fail(e);
-  swila_gates_t dg = {ws + h.beta, ws + h.pik, ws + h.piq, temporal ? ws + h.gk : nullptr,
-                      temporal ? ws + h.gq : nullptr, gated ? (const float *)(ws + h.alpha) : nullptr};
-  rc = swila_forward(s, ws + h.q, ws + h.k, ws + h.v, &dg, state_in ? &dstate : nullptr,
-                     state_out ? &dstate : nullptr, ws + h.o, nullptr, stream);
-  if (rc) return rc;
-  auto down = [&](void *dst, size_t off, size_t n) {
-    if (e == cudaSuccess && n) e = cudaMemcpyAsync(dst, ws + off, n, cudaMemcpyDeviceToHost, cs);
-  };
-  down(o, h.o, h.n_v);
-  if (state_out) {
-    down(state_out->W, h.W, h.n_W);
-    if (temporal) { down(state_out->r_prev, h.r, h.n_r); down(state_out->rho_prev, h.rho, h.n_r); }
+  swila_shape_t sub = *s;
+  sub.B = 1;
+  for (int i = 0; i < nslab && e == cudaSuccess; ++i) {
+    const long long bh0 = nbh * i / nslab, bh1 = nbh * (i + 1) / nslab, cnt = bh1 - bh0;
+    if (cnt == 0) continue;
+    sub.H = (int32_t)cnt;
+    // byte range of this slab inside a tensor of `total` bytes
+    auto lo = [&](size_t total) { return (size_t)(total / (size_t)nbh) * (size_t)bh0; };
+    auto len = [&](size_t total) { return (size_t)(total / (size_t)nbh) * (size_t)cnt; };
+    auto up = [&](size_t off, const void *src, size_t total) {
+      if (e == cudaSuccess && total)
+        e = cudaMemcpyAsync(ws + off + lo(total), (const char *)src + lo(total), len(total), cudaMemcpyHostToDevice, s_in);
+    };
+    up(h.q, q, h.n_qk); up(h.k, k, h.n_qk); up(h.v, v, h.n_v);
+    up(h.beta, g->beta_logit, h.n_gate); up(h.pik, g->pik_logit, h.n_gate); up(h.piq, g->piq_logit, h.n_gate);
+    if (temporal) { up(h.gk, g->gk_logit, h.n_tg); up(h.gq, g->gq_logit, h.n_tg); }
+    if (gated) up(h.alpha, g->alpha, h.n_alpha);
+    if (state_in) {
+      up(h.W, state_in->W, h.n_W);
+      if (temporal) { up(h.r, state_in->r_prev, h.n_r); up(h.rho, state_in->rho_prev, h.n_r); }
+    }
+    if (e != cudaSuccess) break;
+    if (hp) {
+      e = cudaEventRecord(hp->landed[i], s_in);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(cs, hp->landed[i], 0);
+      if (e != cudaSuccess) break;
+    }
+    swila_state_t dstate = {(float *)(ws + h.W + lo(h.n_W)), temporal ? (float *)(ws + h.r + lo(h.n_r)) : nullptr,
+                            temporal ? (float *)(ws + h.rho + lo(h.n_r)) : nullptr};
+    swila_gates_t dg = {ws + h.beta + lo(h.n_gate), ws + h.pik + lo(h.n_gate), ws + h.piq + lo(h.n_gate),
+                        temporal ? ws + h.gk + lo(h.n_tg) : nullptr, temporal ? ws + h.gq + lo(h.n_tg) : nullptr,
+                        gated ? (const float *)(ws + h.alpha + lo(h.n_alpha)) : nullptr};
+    rc = swila_forward(&sub, ws + h.q + lo(h.n_qk), ws + h.k + lo(h.n_qk), ws + h.v + lo(h.n_v), &dg,
+                       state_in ? &dstate : nullptr, state_out ? &dstate : nullptr, ws + h.o + lo(h.n_v), nullptr, stream);
+    if (rc) return rc;
+    if (hp) {
+      e = cudaEventRecord(hp->computed[i], cs);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(s_out, hp->computed[i], 0);
+      if (e != cudaSuccess) break;
+    }
+    auto down = [&](void *dst, size_t off, size_t total) {
+      if (e == cudaSuccess && total)
+        e = cudaMemcpyAsync((char *)dst + lo(total), ws + off + lo(total), len(total), cudaMemcpyDeviceToHost, s_out);
+    };
+    down(o, h.o, h.n_v);
+    if (state_out) {
+      down(state_out->W, h.W, h.n_W);
+      if (temporal) { down(state_out->r_prev, h.r, h.n_r); down(state_out->rho_prev, h.rho, h.n_r); }
+    }
+  }
+  if (hp && e == cudaSuccess) {  // `stream` ends when the last copies have: the caller synchronises on it as before
+    e = cudaEventRecord(hp->done, s_out);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(cs, hp->done, 0);
+    if (e == cudaSuccess) e = cudaEventRecord(hp->done, s_in);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(cs, hp->done, 0);
   }
   return e == cudaSuccess ? SWILA_OK : cuda_fail(e);
 }

@@ -48,3 +48,25 @@ def test_host_entry_rejects_a_small_workspace(binding):
     with pytest.raises(binding.SwilaError) as e:
         binding.swila_forward_host(w, host, ws)
     assert e.value.status == binding.ERR_SIZE
+
+
+@pytest.mark.parametrize("var,T", [(dict(), 2304), (dict(temporal=True, gated=True), 1400)], ids=["vanilla", "gated_temporal"])
+def test_host_entry_in_slabs_equals_device_entry(binding, var, T):
+    """Problems of 64 MB and more go through in slabs of (batch, head) pairs over internal copy streams; with 15
+    pairs the 8 slabs are uneven.  The results must be those of one call on device tensors."""
+    w = wl.CONFIGS[1].with_(B=3, H=5, T=T).variant(**var)
+    assert binding.host_workspace_bytes(w) >= 64 << 20
+    inp = wl.make_inputs(w, stress=True)
+    dev = gpu_forward(binding, w, to_dev(inp))
+    host = _pin(inp)
+    ws = torch.empty(binding.host_workspace_bytes(w), device="cuda", dtype=torch.uint8)
+    sin = {"W": host["W0"], "r_prev": host["r0"], "rho_prev": host["rho0"]}
+    sout = {"W": torch.empty_like(inp["W0"]).pin_memory(),
+            "r_prev": torch.empty_like(inp["r0"]).pin_memory() if w.temporal else None,
+            "rho_prev": torch.empty_like(inp["rho0"]).pin_memory() if w.temporal else None}
+    for _ in range(2):  # twice in a row: the second call reuses the streams and events of the first
+        o = binding.swila_forward_host(w, host, ws, state_in=sin, state_out=sout)
+        torch.cuda.synchronize()
+        assert torch.equal(o, dev["o"]) and torch.equal(sout["W"], dev["W"])
+        if w.temporal:
+            assert torch.equal(sout["r_prev"], dev["r_prev"]) and torch.equal(sout["rho_prev"], dev["rho_prev"])
