@@ -263,6 +263,19 @@ def paper_shapes_leg(binding, stream):
     out["lm374m_layer_prefill"] = {"B": lm.B, "H": lm.H, "T": lm.T, "D": lm.Dk, "J": lm.J, "ms": ms,
                                    "tokens_per_s": lm.B * lm.T / (ms * 1e-3)}
     del inp, o, st
+    # the component-count ablation of Sec. 5: the same layer with J = 16 (scan kernel)
+    lm16 = lm.with_(name="lm374m_layer_j16", J=16)
+    inp = wl.make_inputs(lm16, device="cuda")
+    st = binding.state_alloc(lm16, init=False)
+    o = torch.empty((lm16.B, lm16.H, lm16.T, lm16.Dv), device="cuda", dtype=lm16.torch_io_dtype)
+    f16 = lambda: binding.swila_forward(lm16, inp, state_in=None, state_out=st, o=o)
+    for _ in range(3):
+        f16()
+    torch.cuda.synchronize()
+    ms = time_steps(f16, 10, stream) / 10
+    out["lm374m_layer_prefill_j16"] = {"B": lm16.B, "H": lm16.H, "T": lm16.T, "D": lm16.Dk, "J": lm16.J, "ms": ms,
+                                       "tokens_per_s": lm16.B * lm16.T / (ms * 1e-3)}
+    del inp, o, st
     gen_out = []
     for B in (1, 8, 128):
         g = wl.CONFIGS[1].with_(name="generation", B=B, H=8, T=2048)

@@ -84,7 +84,7 @@ enum {
 typedef struct {
   int32_t B, H, T;          /* batch, heads, tokens (T >= 0; ignored by swila_decode_step) */
   int32_t Dk, Dv;           /* key / value head dimension; Dk in {16, 64, 128}; Dv % 8 == 0 */
-  int32_t J;                /* mixture components, in {1, 2, 4, 8} */
+  int32_t J;                /* mixture components, in {1, 2, 4, 8, 16} */
   int32_t io_dtype;         /* SWILA_IO_*: dtype of q, k, v, o and of every *_logit tensor */
   int32_t flags;            /* SWILA_TEMPORAL | SWILA_GATED | SWILA_POST_DECAY */
   int32_t gate_granularity; /* SWILA_GATE_*; must be NONE iff GATED is clear */

@@ -34,7 +34,7 @@ static int check_shape(const swila_shape_t *s, bool need_T) {
   if (need_T && s->T < 0) return SWILA_ERR_SHAPE;
   if (s->Dv % 8 != 0) return SWILA_ERR_SHAPE;
   if (s->Dk != 16 && s->Dk != 64 && s->Dk != 128) return SWILA_ERR_UNSUPPORTED;
-  if (s->J != 1 && s->J != 2 && s->J != 4 && s->J != 8) return SWILA_ERR_UNSUPPORTED;
+  if (s->J != 1 && s->J != 2 && s->J != 4 && s->J != 8 && s->J != 16) return SWILA_ERR_UNSUPPORTED;
   if (s->io_dtype != SWILA_IO_FP32 && s->io_dtype != SWILA_IO_BF16) return SWILA_ERR_UNSUPPORTED;
   if (s->flags & ~(SWILA_TEMPORAL | SWILA_GATED | SWILA_POST_DECAY)) return SWILA_ERR_UNSUPPORTED;
   const bool gated = (s->flags & SWILA_GATED) != 0;

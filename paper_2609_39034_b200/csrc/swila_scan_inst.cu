@@ -38,6 +38,7 @@ int pick_j(const LaunchArgs &a) {
     case 2: return pick<IO, 2>(a);
     case 4: return pick<IO, 4>(a);
     case 8: return pick<IO, 8>(a);
+    case 16: return pick<IO, 16>(a);
     default: return -1000;
   }
 }

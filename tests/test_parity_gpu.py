@@ -40,6 +40,9 @@ SMALL = [
     _case("j2_d64", 1, B=1, H=2, T=50, J=2),
     _case("j4_d16_bf16", 0, T=45, J=4, io_dtype="bf16"),
     _case("j8_d16", 0, T=45, J=8),
+    _case("j16_d64", 1, B=1, H=2, T=70, J=16),          # the component-count ablation of Sec. 5 (J = 16 at D = 64)
+    _case("j16_d128_fp32", 2, B=1, H=1, T=40, J=16, recipe="gauss", io_dtype="fp32"),
+    _case("j16_d16", 0, T=45, J=16),
 ]
 
 
@@ -61,7 +64,7 @@ VARIANTS = [
     dict(gated=True, granularity=wl.GRAN_SCALAR, post_decay=True),
     dict(temporal=True, gated=True, granularity=wl.GRAN_SCALAR),
 ]
-VAR_SHAPES = [SMALL[0], SMALL[2], SMALL[3], SMALL[4], SMALL[6], SMALL[10]]
+VAR_SHAPES = [SMALL[0], SMALL[2], SMALL[3], SMALL[4], SMALL[6], SMALL[10], SMALL[15]]
 
 
 @pytest.mark.parametrize("w0", VAR_SHAPES, ids=lambda w: w.name)
@@ -82,7 +85,7 @@ def test_wide_blocks_match_oracle(binding, oracle, w):
     assert_close(w, got, ref, w.name)
 
 
-CHUNK_SHAPES = [w for w in SMALL if w.io_dtype == "bf16" and w.Dk in (64, 128) and w.J >= 4] + [
+CHUNK_SHAPES = [w for w in SMALL if w.io_dtype == "bf16" and w.Dk in (64, 128) and w.J in (4, 8)] + [
     _case("c2_one_chunk", 2, B=1, H=1, T=32, recipe="gauss"),
     _case("c2_short", 2, B=1, H=1, T=5, recipe="gauss"),
     _case("c2_long", 2, B=1, H=2, T=1000, recipe="gauss"),
