@@ -66,7 +66,8 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-// Tiled bulk tensor copies global -> shared (TMA), no multicast; completion (the box's bytes) lands on `bar`.
+// Tiled bulk tensor copies global -> shared (TMA), each into this block's own shared memory only; completion (the
+// box's bytes) lands on `bar`.
 // The innermost coordinate times the element size must be a multiple of 16 bytes, `dst` 128-byte aligned.
 __device__ __forceinline__ void tma_load_3d(void *dst, const void *tensor_map, int c0, int c1, int c2, uint64_t *bar) {
   asm volatile(
