@@ -15,8 +15,9 @@ int pick(const LaunchArgs &a) {
   constexpr int DK = SWILA_DK;
   constexpr int GATE = SWILA_GATE;
   constexpr bool POST = SWILA_POST != 0;
-  // tokens per staged block: fp32 rows are twice as wide, keep two blocks per SM resident
-  constexpr int TB = sizeof(IO) == 2 ? 8 : 4;
+  // tokens per staged block: fp32 rows are twice as wide, and per-key gates at Dk = 128 add 2 KB of fp32 per token;
+  // keep two blocks per SM resident (8-token blocks of gates would leave room for one only)
+  constexpr int TB = (sizeof(IO) == 2 && !(GATE == 1 && DK == 128)) ? 8 : 4;
   if constexpr (DK == 16) {
     return launch_scan<ScanCfg<IO, J, DK, 32, TB, GATE>, POST>(a);
   } else {
