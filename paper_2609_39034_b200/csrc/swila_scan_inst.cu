@@ -29,6 +29,9 @@ int pick(const LaunchArgs &a) {
       if constexpr (GATE == 0 && DK == 128 && J >= 4) return launch_scan<ScanCfg<IO, J, DK, 128, TB, GATE, 16>, POST>(a);
       return -1000;
     }
+    // a decode step stages and prepares one token: blocks of one token (same arithmetic per token, so the bits
+    // of a prefill and of the decode steps that continue it still agree)
+    if (a.p.T == 1) return launch_scan<ScanCfg<IO, J, DK, 128, 1, GATE>, POST>(a);
     return launch_scan<ScanCfg<IO, J, DK, 128, TB, GATE>, POST>(a);
   }
 }
