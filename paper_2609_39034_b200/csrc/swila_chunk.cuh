@@ -18,8 +18,12 @@
 // operand (the state, the update coefficients, Gram matrices used as operands) is split as
 // x = hi + lo with hi = bf16(x), lo = bf16(x - hi) and both parts are multiplied (lo x lo is
 // dropped), which keeps 16 significant bits of the operand: a relative error of 4e-6 per product,
-// unbiased, against a parity tolerance of 1e-4.  The triangular part (the sums over s inside the
-// chunk) and the E-step stay on the FP32 ALUs, one thread per row.
+// unbiased, against a parity tolerance of 1e-4.  The update coefficients of W += Cmat K alone get
+// a third part (24 bits): their rounding is the one error that is added to the state and carried
+// along the sequence, and from a zero state with near-uniform gates, where the components separate
+// only through the E-step's feedback, 16 bits left the state 2e-4 off after 8192 tokens.  The
+// triangular part (the sums over s inside the chunk) and the E-step stay on the FP32 ALUs, one
+// thread per row.
 //
 // Across chunks the products of the state with the next chunk's keys and queries are taken off
 // the serial path: with W_{n+1} = W_n + Cmat_n K_n,
@@ -104,11 +108,11 @@ struct ChunkCfg {
   // tensor-memory columns.  W: the state (FP32 accumulator); WHI / WLO: its bf16 operand parts, two key
   // dims per column; PQ: [P0 | Q0] = state x [K;Q] of the next chunk to run; QD: the query-side readouts
   // of a chunk (double-buffered); G: Gram matrices as they leave the tensor cores; FAR: what the first 8 tokens of
-  // the chunk add to the predictions of its last 16 (only the last 8 are non-zero); CHI / CLO: the bf16 parts of the
-  // chunk's update coefficients, two tokens per column
+  // the chunk add to the predictions of its last 16 (only the last 8 are non-zero); CHI / CLO / CL3: the bf16 parts of the
+  // chunk's update coefficients, two tokens per column (the third part is an operand of the state update only)
   static constexpr int TM_W = 0, TM_WHI = DK, TM_WLO = DK + DK / 2, TM_PQ = 2 * DK, TM_QD = TM_PQ + 2 * C,
                        TM_G = TM_QD + 2 * C, TM_FAR = TM_G + 2 * C, TM_CHI = TM_FAR + C / 2, TM_CLO = TM_CHI + C / 2,
-                       TM_USED = TM_CLO + C / 2;
+                       TM_CL3 = TM_CLO + C / 2, TM_USED = TM_CL3 + C / 2;
   static constexpr int TM_ALLOC = 512;
   static_assert(TM_USED <= TM_ALLOC, "tensor memory budget");
   static_assert(J == 4 || J == 8, "the output transposition assumes that J divides 8");
@@ -181,6 +185,17 @@ __device__ __forceinline__ void bf16_split2(float x0, float x1, uint32_t &hi, ui
   hi = *reinterpret_cast<const uint32_t *>(&h);
   const float r0 = x0 - __uint_as_float(hi << 16), r1 = x1 - __uint_as_float(hi & 0xffff0000u);
   const __nv_bfloat162 l = __floats2bfloat162_rn(r0, r1);
+  lo = *reinterpret_cast<const uint32_t *>(&l);
+}
+// Three parts (24 bits of the value): for operands whose rounding would otherwise accumulate in the state.
+__device__ __forceinline__ void bf16_split3(float x0, float x1, uint32_t &hi, uint32_t &mid, uint32_t &lo) {
+  const __nv_bfloat162 h = __floats2bfloat162_rn(x0, x1);
+  hi = *reinterpret_cast<const uint32_t *>(&h);
+  const float r0 = x0 - __uint_as_float(hi << 16), r1 = x1 - __uint_as_float(hi & 0xffff0000u);
+  const __nv_bfloat162 m = __floats2bfloat162_rn(r0, r1);
+  mid = *reinterpret_cast<const uint32_t *>(&m);
+  const float s0 = r0 - __uint_as_float(mid << 16), s1 = r1 - __uint_as_float(mid & 0xffff0000u);
+  const __nv_bfloat162 l = __floats2bfloat162_rn(s0, s1);
   lo = *reinterpret_cast<const uint32_t *>(&l);
 }
 
@@ -509,11 +524,12 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
             PROF_ADD(7);
           }
           {  // GT update coefficients complete: park their bf16 parts in tensor memory, two tokens per column
-            uint32_t hi[GT / 2], lo[GT / 2];
+            uint32_t hi[GT / 2], lo[GT / 2], l3[GT / 2];
 #pragma unroll
-            for (int i = 0; i < GT / 2; ++i) bf16_split2(cs[2 * i], cs[2 * i + 1], hi[i], lo[i]);
+            for (int i = 0; i < GT / 2; ++i) bf16_split3(cs[2 * i], cs[2 * i + 1], hi[i], lo[i], l3[i]);
             tmem_st4(tb + Cf::TM_CHI + tg / 2, hi);
             tmem_st4(tb + Cf::TM_CLO + tg / 2, lo);
+            tmem_st4(tb + Cf::TM_CL3 + tg / 2, l3);
           }
           if constexpr (!EXACT) {
             if (tg == 0) {  // the coefficients of tokens 0-7 are in place: the far pushes may be issued
@@ -903,6 +919,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         const uint64_t bt = smem_desc_sw128_mn(smem_u32(smem + Cf::OFF_KU + (n % 3) * Cf::KU_BYTES) + ks * 16 * 128, Cf::KU_HALF, 1024);
         mma_bf16_ts(tb0 + Cf::TM_W, tb0 + Cf::TM_CHI + ks * 8, bt, idU, true);
         mma_bf16_ts(tb0 + Cf::TM_W, tb0 + Cf::TM_CLO + ks * 8, bt, idU, true);
+        mma_bf16_ts(tb0 + Cf::TM_W, tb0 + Cf::TM_CL3 + ks * 8, bt, idU, true);
       }
       mma_commit(&bars[B_U]);
       readout(n);
