@@ -154,7 +154,7 @@ struct ChunkCfg {
   static constexpr int OFF_KU = OFF_TILE + TILE_BYTES;
   static constexpr int OFF_RAW = OFF_KU + 3 * KU_BYTES;
   static constexpr int OFF_RPQ = OFF_RAW + 2 * RAW_BYTES;
-  static constexpr int OFF_G = OFF_RPQ + 4 * RPQ_BYTES;             // 2 x Gkk [C][C] fp32 (K K^T, for the row warps)
+  static constexpr int OFF_G = OFF_RPQ + 4 * RPQ_BYTES;             // 2 x Gkk [C][C] fp32 (-K K^T, for the row warps)
   static constexpr int OFF_BQ = OFF_G + 2 * C * C * 4;        // 2 x { hi, lo } readout operand tiles
   static constexpr int OFF_GX = OFF_BQ + 2 * 2 * BQ_TILE;     // { hi, lo } cross-chunk operand tiles
   static constexpr int OFF_OST = OFF_GX + 2 * GX_TILE;        // 2 x [C][COLS] bf16 output staging
@@ -440,18 +440,20 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         constexpr bool EXACT = decltype(exact_tag)::value;
         constexpr int GT = Cf::GT;
         bool bad = false;
-        // pred[i]: prediction of token tg + i of the current trip, for the WINS tokens that the pushes of a token reach
-        // on the ALUs (slots past the chunk end are dead weight that keeps the trip's code independent of tg).  The fast
-        // pass reaches WIN = 24 tokens: the pushes of tokens 0-7 into tokens 24-31 come from the tensor cores (FAR)
-        // when token 24 is reached.  The redo pass does everything itself.
+        // pred[i]: v - prediction (the prediction error so far) of token tg + i of the current trip, for the WINS
+        // tokens that the pushes of a token reach on the ALUs (slots past the chunk end are dead weight that keeps the
+        // trip's code independent of tg); the Gram rows are stored negated, so a push is one FMA and the error of
+        // the next token is ready without a subtraction on the serial chain.  The fast pass reaches WIN = 24 tokens:
+        // the pushes of tokens 0-7 into tokens 24-31 come from the tensor cores (FAR) when token 24 is reached.
+        // The redo pass does everything itself.
         constexpr int WINS = EXACT ? C : Cf::WIN;
         float pred[WINS];
 #pragma unroll
-        for (int t = 0; t < WINS; ++t) pred[t] = pred0[t];
+        for (int t = 0; t < WINS; ++t) pred[t] = __bfloat162float(rv[t * COLS + dl]) - pred0[t];
         [[maybe_unused]] float p0late[C - Cf::WIN];
         if constexpr (!EXACT) {
 #pragma unroll
-          for (int t = 0; t < C - Cf::WIN; ++t) p0late[t] = pred0[Cf::WIN + t];
+          for (int t = 0; t < C - Cf::WIN; ++t) p0late[t] = __bfloat162float(rv[(Cf::WIN + t) * COLS + dl]) - pred0[Cf::WIN + t];
         }
         float c_prev = 0.f;
 #pragma unroll 1
@@ -464,17 +466,16 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
               tmem_ld8(tb + Cf::TM_FAR + Cf::WIN - C / 2, far);
               tmem_ld_wait();
 #pragma unroll
-              for (int i = 0; i < 8; ++i) pred[i] += far[i];
+              for (int i = 0; i < 8; ++i) pred[i] -= far[i];
             }
           }
           float cs[GT];
 #pragma unroll
           for (int i = 0; i < GT; ++i) {
             const int t = tg + i;
-            const float v = __bfloat162float(rv[t * COLS + dl]);
             const float be = bes[t * NROW + r];
             // serial chain: prediction error -> responsibilities (Eq. 3.4) -> update coefficient (Eq. 3.3)
-            const float delta = v - pred[i];
+            const float delta = pred[i];
             const float a = fmaf(-kHalfLog2e * delta, delta, __bfloat162float(rpk[(t * J + j) * Cf::GROW + dl]) * kLog2e);
             float e, sum;
             if constexpr (EXACT) {
@@ -490,9 +491,16 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
               e = ex2_approx(a - m);
             } else {
               e = ex2_approx(a);
-              sum = e;
+              float part[J];  // the other components' terms arrive together: add them as a tree
+              part[0] = e;
 #pragma unroll
-              for (int jj = 1; jj < J; ++jj) sum += __shfl_sync(0xffffffffu, e, jbase + ((j + jj) & (J - 1)));
+              for (int jj = 1; jj < J; ++jj) part[jj] = __shfl_sync(0xffffffffu, e, jbase + ((j + jj) & (J - 1)));
+#pragma unroll
+              for (int w = J / 2; w >= 1; w /= 2) {
+#pragma unroll
+                for (int jj = 0; jj < w; ++jj) part[jj] += part[jj + w];
+              }
+              sum = part[0];
               bad = bad || !(sum > 1e-30f && sum < 1e30f);
             }
             {  // deferred push of token t-1 into the predictions of tokens t+1 .. (slots i+1 ..)
@@ -506,12 +514,12 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
                 if (4 * u4 + 3 > i) pred[4 * u4 + 3] = fmaf(c_prev, g.w, pred[4 * u4 + 3]);
               }
             }
-            const float rr = e * rcp_approx(sum);
-            float c = (be * delta) * rr;
+            const float rs = rcp_approx(sum);
+            float c = ((be * delta) * e) * rs;  // beta r delta with one multiplication after the reciprocal
             if (t >= nvalid) c = 0.f;  // padding tokens of the last chunk leave the state alone
             cs[i] = c;
             if constexpr (RDEBUG) {
-              if (col_ok && t < nvalid) p.r_debug[((tok0 + (size_t)(t0 + t)) * J + j) * p.Dv + col] = rr;
+              if (col_ok && t < nvalid) p.r_debug[((tok0 + (size_t)(t0 + t)) * J + j) * p.Dv + col] = e * rs;
             }
             pred[i + 1] = fmaf(c, Gkk[t * C + t + 1], pred[i + 1]);  // the push the next token waits for
             c_prev = c;
@@ -638,7 +646,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     };
     // The Gram batch of chunk m is [K_e;Q_e;K_o;Q_o] x [K_m;Q_m | K_{m-1}]^T; the two helper warps whose
     // tensor-memory lanes hold the rows of chunk m's keys and queries spill it:
-    //   key rows   (lane s):  K_m K_m^T as plain FP32 rows for the row warps;
+    //   key rows   (lane s):  -K_m K_m^T as plain FP32 rows for the row warps (negated: they track v - prediction);
     //   query rows (lane t):  Q_m K_m^T, causally masked (s <= t), as the hi / lo operand of the readout MMA;
     //   both:                 [K_m;Q_m] K_{m-1}^T as the hi / lo operand of the cross-chunk MMA.
     auto spill_gram = [&](int m) {
@@ -651,7 +659,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         float *Gkk = G_all + (m & 1) * C * C;
 #pragma unroll
         for (int i = 0; i < C / 4; ++i)
-          *reinterpret_cast<float4 *>(Gkk + lane * C + i * 4) = make_float4(a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
+          *reinterpret_cast<float4 *>(Gkk + lane * C + i * 4) = make_float4(-a[4 * i], -a[4 * i + 1], -a[4 * i + 2], -a[4 * i + 3]);
         // far-push operand: row = token u = lane (16..31), K index = tokens 0..7 (K K^T is symmetric, so this lane's
         // row holds k_s.k_u).  Through the tensor cores go the pushes of tokens s = 0..6 into tokens u >= WIN: the row
         // warps push token s into tokens s+1 .. 23 while they are in the first trip, and token 7, whose deferred push
