@@ -52,7 +52,11 @@ enum { SWILA_IO_FP32 = 0, SWILA_IO_BF16 = 1 };
 enum {
   SWILA_TEMPORAL = 1,   /* Temporal SwiLA (Sec. 3.3, App. B.3) */
   SWILA_GATED = 2,      /* Gated SwiLA, pre-decay form (Eq. 3.8) unless POST_DECAY */
-  SWILA_POST_DECAY = 4  /* with GATED: post-decay form (Eq. 3.7) */
+  SWILA_POST_DECAY = 4, /* with GATED: post-decay form (Eq. 3.7) */
+  SWILA_QKV_ACT = 8     /* q, k, v are the raw projections: the kernel applies SiLU to all three and then
+                           divides q and k by sqrt(sum over Dk of squares + 1e-6), as the paper's models do
+                           (App. B.2, App. D.1).  The activated values stay in FP32 (no rounding to the io
+                           dtype).  Scan kernels only: with SWILA_ALGO_CHUNK -> SWILA_ERR_UNSUPPORTED */
 };
 
 /* gate_granularity (App. B.4): which indices the decay alpha depends on */
@@ -86,7 +90,7 @@ typedef struct {
   int32_t Dk, Dv;           /* key / value head dimension; Dk in {16, 64, 128}; Dv % 8 == 0 */
   int32_t J;                /* mixture components, in {1, 2, 4, 8, 16} */
   int32_t io_dtype;         /* SWILA_IO_*: dtype of q, k, v, o and of every *_logit tensor */
-  int32_t flags;            /* SWILA_TEMPORAL | SWILA_GATED | SWILA_POST_DECAY */
+  int32_t flags;            /* SWILA_TEMPORAL | SWILA_GATED | SWILA_POST_DECAY | SWILA_QKV_ACT */
   int32_t gate_granularity; /* SWILA_GATE_*; must be NONE iff GATED is clear */
   int32_t algo;             /* SWILA_ALGO_* */
 } swila_shape_t;
@@ -145,6 +149,39 @@ int swila_state_init(const swila_shape_t *shape, swila_state_t *state, void *str
 int swila_forward(const swila_shape_t *shape, const void *q, const void *k, const void *v,
                   const swila_gates_t *gates, const swila_state_t *state_in,
                   swila_state_t *state_out, void *o, float *r_debug, void *stream);
+
+/*
+ * Sums over time of the mixture weights, for the mutual-information load-balancing loss (Sec. 3.5: entropy
+ * of the time-averaged responsibilities minus the mean per-token entropy, key side and query side) and the
+ * router diagnostics of App. D.5.  Every pointer is a DEVICE pointer to fp32 or NULL (that sum is not
+ * formed).  The sums of a call are ADDED to the buffers, so a sequence fed in several calls accumulates;
+ * the caller zeroes them first.
+ */
+typedef struct {
+  float *r_sum;    /* [B,H,J,Dv] += sum over t of the responsibilities r_tjd of Eq. 3.4             */
+  float *r_ent;    /* [B,H,Dv]   += sum over t of -sum_j r_tjd ln r_tjd (nats; 0 ln 0 = 0)          */
+  float *rho_sum;  /* [B,H,J,Dv] += sum over t of the readout weights of Eq. 3.5: pi^q_tjd, or the  */
+                   /*               running average rho-bar_tjd when TEMPORAL (App. B.3)            */
+  float *rho_ent;  /* [B,H,Dv]   += sum over t of their entropy over j (nats)                       */
+} swila_stats_t;
+
+/*
+ * swila_forward that also forms the sums of `stats` (which must not be NULL; any of its members may be).
+ * Runs the scan kernel (SWILA_ALGO_CHUNK -> SWILA_ERR_UNSUPPORTED); outputs and state are those of
+ * swila_forward with SWILA_ALGO_SCAN, bit for bit.
+ */
+int swila_forward_stats(const swila_shape_t *shape, const void *q, const void *k, const void *v,
+                        const swila_gates_t *gates, const swila_state_t *state_in,
+                        swila_state_t *state_out, void *o, float *r_debug, const swila_stats_t *stats,
+                        void *stream);
+
+/*
+ * RMSNorm of the layer output (App. D.1), in place: for every (batch, head, token) row of o [B,H,T,Dv]
+ * (io dtype), o_d <- o_d / sqrt(mean over d of o_d^2 + eps) * weight_d.  weight: DEVICE fp32 [Dv], or NULL
+ * for all ones.  A separate memory-bound pass over o (the rows of o are spread over several thread blocks
+ * of the recurrence, so the mean is not available there).  Uses shape->B, H, T, Dv and io_dtype.
+ */
+int swila_output_norm(const swila_shape_t *shape, void *o, const float *weight, float eps, void *stream);
 
 /*
  * Decode: one token of the same recurrence on a carried state, updated in place

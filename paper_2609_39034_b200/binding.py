@@ -24,7 +24,8 @@ ALGO_AUTO, ALGO_SCAN, ALGO_SCAN_WIDE, ALGO_SCAN_NARROW, ALGO_CHUNK = 0, 1, 2, 3,
 EXPORTS = ("swila_version", "swila_strerror", "swila_last_cuda_error", "swila_state_w_bytes",
            "swila_state_r_bytes", "swila_state_init", "swila_forward", "swila_decode_step",
            "swila_bench_fma_chain", "swila_forward_host", "swila_forward_host_workspace_bytes",
-           "swila_forward_host_static", "swila_forward_host_static_capacity", "swila_selftest_tf32_mma", "swila_selftest_bf16_mma", "swila_device_status", "swila_chunk_plan", "swila_chunk_run_pieces")
+           "swila_forward_host_static", "swila_forward_host_static_capacity", "swila_selftest_tf32_mma", "swila_selftest_bf16_mma", "swila_device_status", "swila_chunk_plan", "swila_chunk_run_pieces",
+           "swila_forward_stats", "swila_output_norm")
 
 
 class Shape(ctypes.Structure):
@@ -39,6 +40,11 @@ class Gates(ctypes.Structure):
 
 class State(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in ("W", "r_prev", "rho_prev")]
+
+
+class Stats(ctypes.Structure):
+    _fields_ = [("r_sum", ctypes.c_void_p), ("r_ent", ctypes.c_void_p), ("rho_sum", ctypes.c_void_p),
+                ("rho_ent", ctypes.c_void_p)]
 
 
 class SwilaError(RuntimeError):
@@ -69,6 +75,13 @@ def _load() -> ctypes.CDLL:
     L.swila_forward.argtypes = [ctypes.POINTER(Shape), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                 ctypes.POINTER(Gates), ctypes.POINTER(State), ctypes.POINTER(State),
                                 ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+    L.swila_forward_stats.restype = ctypes.c_int
+    L.swila_forward_stats.argtypes = [ctypes.POINTER(Shape), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                      ctypes.POINTER(Gates), ctypes.POINTER(State), ctypes.POINTER(State),
+                                      ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(Stats), ctypes.c_void_p]
+    L.swila_output_norm.restype = ctypes.c_int
+    L.swila_output_norm.argtypes = [ctypes.POINTER(Shape), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_float,
+                                    ctypes.c_void_p]
     L.swila_decode_step.restype = ctypes.c_int
     L.swila_decode_step.argtypes = [ctypes.POINTER(Shape), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                     ctypes.POINTER(Gates), ctypes.POINTER(State), ctypes.c_void_p, ctypes.c_void_p]
@@ -165,6 +178,41 @@ def swila_forward(w: Workload, inp: dict, *, state_in: Optional[dict] = None, st
     check(lib.swila_forward(ctypes.byref(sh), _p(inp["q"]), _p(inp["k"]), _p(inp["v"]), ctypes.byref(g),
                             ctypes.byref(sin) if sin else None, ctypes.byref(sout) if sout else None,
                             _p(o), _p(r_debug), _stream(stream)))
+    return o
+
+
+def stats_alloc(w: Workload, device="cuda") -> dict:
+    """Zeroed buffers for swila_forward_stats: r_sum, rho_sum [B,H,J,Dv]; r_ent, rho_ent [B,H,Dv]."""
+    z = lambda *shape: torch.zeros(shape, device=device, dtype=torch.float32)  # noqa: E731
+    return {"r_sum": z(w.B, w.H, w.J, w.Dv), "r_ent": z(w.B, w.H, w.Dv),
+            "rho_sum": z(w.B, w.H, w.J, w.Dv), "rho_ent": z(w.B, w.H, w.Dv)}
+
+
+def swila_forward_stats(w: Workload, inp: dict, stats: dict, *, state_in: Optional[dict] = None,
+                        state_out: Optional[dict] = None, o: Optional[torch.Tensor] = None,
+                        r_debug: Optional[torch.Tensor] = None, algo: int = ALGO_AUTO, stream=None,
+                        T: Optional[int] = None) -> torch.Tensor:
+    """swila_forward that also ADDS the sums over time of the mixture weights (Sec. 3.5) to the
+    buffers in ``stats`` (keys r_sum, r_ent, rho_sum, rho_ent; a missing key or None skips that sum)."""
+    T = inp["q"].shape[2] if T is None else T
+    sh = make_shape(w, T=T, algo=algo)
+    if o is None:
+        o = torch.empty((w.B, w.H, T, w.Dv), device=inp["q"].device, dtype=w.torch_io_dtype)
+    g = _gates(inp)
+    sin = _state(state_in["W"], state_in.get("r_prev"), state_in.get("rho_prev")) if state_in else None
+    sout = _state(state_out["W"], state_out.get("r_prev"), state_out.get("rho_prev")) if state_out else None
+    st = Stats(*[(_p(stats.get(n)) or ctypes.c_void_p(None)).value for n in ("r_sum", "r_ent", "rho_sum", "rho_ent")])
+    check(lib.swila_forward_stats(ctypes.byref(sh), _p(inp["q"]), _p(inp["k"]), _p(inp["v"]), ctypes.byref(g),
+                                  ctypes.byref(sin) if sin else None, ctypes.byref(sout) if sout else None,
+                                  _p(o), _p(r_debug), ctypes.byref(st), _stream(stream)))
+    return o
+
+
+def swila_output_norm(w: Workload, o: torch.Tensor, weight: Optional[torch.Tensor] = None, eps: float = 1e-6,
+                      stream=None) -> torch.Tensor:
+    """RMSNorm of o [B,H,T,Dv] over its last axis, in place (App. D.1); weight fp32 [Dv] or None."""
+    sh = make_shape(w, T=o.shape[2])
+    check(lib.swila_output_norm(ctypes.byref(sh), _p(o), _p(weight), ctypes.c_float(eps), _stream(stream)))
     return o
 
 

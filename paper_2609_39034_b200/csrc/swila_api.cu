@@ -36,7 +36,7 @@ static int check_shape(const swila_shape_t *s, bool need_T) {
   if (s->Dk != 16 && s->Dk != 64 && s->Dk != 128) return SWILA_ERR_UNSUPPORTED;
   if (s->J != 1 && s->J != 2 && s->J != 4 && s->J != 8 && s->J != 16) return SWILA_ERR_UNSUPPORTED;
   if (s->io_dtype != SWILA_IO_FP32 && s->io_dtype != SWILA_IO_BF16) return SWILA_ERR_UNSUPPORTED;
-  if (s->flags & ~(SWILA_TEMPORAL | SWILA_GATED | SWILA_POST_DECAY)) return SWILA_ERR_UNSUPPORTED;
+  if (s->flags & ~(SWILA_TEMPORAL | SWILA_GATED | SWILA_POST_DECAY | SWILA_QKV_ACT)) return SWILA_ERR_UNSUPPORTED;
   const bool gated = (s->flags & SWILA_GATED) != 0;
   if (!gated && (s->flags & SWILA_POST_DECAY)) return SWILA_ERR_UNSUPPORTED;
   if (gated != (s->gate_granularity != SWILA_GATE_NONE)) return SWILA_ERR_UNSUPPORTED;
@@ -57,7 +57,8 @@ static bool overlaps(const void *a, size_t na, const void *b, size_t nb) {
 }
 
 static int run(const swila_shape_t *s, int T, const void *q, const void *k, const void *v, const swila_gates_t *g,
-               const swila_state_t *sin, swila_state_t *sout, void *o, float *r_debug, void *stream) {
+               const swila_state_t *sin, swila_state_t *sout, void *o, float *r_debug, void *stream,
+               const swila_stats_t *stats = nullptr) {
   const bool temporal = (s->flags & SWILA_TEMPORAL) != 0;
   const bool gated = (s->flags & SWILA_GATED) != 0;
   if (!q || !k || !v || !g || !o) return SWILA_ERR_NULL;
@@ -100,6 +101,12 @@ static int run(const swila_shape_t *s, int T, const void *q, const void *k, cons
   a.p.rho_out = (sout && temporal) ? sout->rho_prev : nullptr;
   a.p.o = o;
   a.p.r_debug = r_debug;
+  a.p.qkv_act = (s->flags & SWILA_QKV_ACT) ? 1 : 0;
+  if (stats) {
+    a.p.r_sum = stats->r_sum; a.p.r_ent = stats->r_ent;
+    a.p.rho_sum = stats->rho_sum; a.p.rho_ent = stats->rho_ent;
+  }
+  const bool want_stats = a.p.r_sum || a.p.r_ent || a.p.rho_sum || a.p.rho_ent;
   a.Dk = s->Dk; a.J = s->J; a.io_dtype = s->io_dtype;
   a.gate_mode = !gated ? 0 : (s->gate_granularity == SWILA_GATE_PER_KEY ? 1 : 2);
   a.post = (s->flags & SWILA_POST_DECAY) ? 1 : 0;
@@ -110,7 +117,7 @@ static int run(const swila_shape_t *s, int T, const void *q, const void *k, cons
   // AUTO: the chunked tensor-core kernel whenever it applies and the sequence is long enough to
   // amortise its per-chunk set-up; the scan otherwise (fp32 io, TEMPORAL / GATED, decode).
   const bool chunk_ok = s->io_dtype == SWILA_IO_BF16 && s->flags == 0 && (s->Dk == 64 || s->Dk == 128) &&
-                        (s->J == 4 || s->J == 8);
+                        (s->J == 4 || s->J == 8) && !want_stats;
   if (s->algo == SWILA_ALGO_CHUNK || (s->algo == SWILA_ALGO_AUTO && chunk_ok && T >= 64)) {
     rc = chunk_dispatch(a);
     if (rc == -1000 && s->algo == SWILA_ALGO_CHUNK) return SWILA_ERR_UNSUPPORTED;
@@ -220,6 +227,17 @@ int swila_forward(const swila_shape_t *s, const void *q, const void *k, const vo
     return e == cudaSuccess ? SWILA_OK : cuda_fail(e);
   }
   return run(s, s->T, q, k, v, g, state_in, state_out, o, r_debug, stream);
+}
+
+int swila_forward_stats(const swila_shape_t *s, const void *q, const void *k, const void *v, const swila_gates_t *g,
+                        const swila_state_t *state_in, swila_state_t *state_out, void *o, float *r_debug,
+                        const swila_stats_t *stats, void *stream) {
+  int rc = check_shape(s, true);
+  if (rc) return rc;
+  if (!stats) return SWILA_ERR_NULL;
+  if (s->algo == SWILA_ALGO_CHUNK) return SWILA_ERR_UNSUPPORTED;
+  if (s->T == 0) return swila_forward(s, q, k, v, g, state_in, state_out, o, r_debug, stream);  // nothing to add
+  return run(s, s->T, q, k, v, g, state_in, state_out, o, r_debug, stream, stats);
 }
 
 int swila_decode_step(const swila_shape_t *s, const void *q, const void *k, const void *v, const swila_gates_t *g,

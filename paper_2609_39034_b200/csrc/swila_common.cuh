@@ -23,7 +23,12 @@ struct ScanParams {
   float *W_out, *r_out, *rho_out;     // may be null: state discarded
   void *o;
   float *r_debug;                     // may be null
+  int qkv_act;                        // 0/1: SiLU on q, k, v and L2 normalisation of q, k inside the kernel
+  float *r_sum, *r_ent, *rho_sum, *rho_ent;  // sums over time of the mixture weights; each may be null
 };
+
+// epsilon under the root of the in-kernel L2 normalisation of q and k
+constexpr float kL2Eps = 1e-6f;
 
 struct LaunchArgs {
   ScanParams p;
@@ -58,6 +63,9 @@ __device__ __forceinline__ float rcp_approx(float x) {
 __device__ __forceinline__ float sigmoid_approx(float x) {
   return rcp_approx(1.0f + ex2_approx(-kLog2e * x));
 }
+
+// SiLU(x) = x sigmoid(x) (App. B.2)
+__device__ __forceinline__ float silu_approx(float x) { return x * sigmoid_approx(x); }
 
 __device__ __forceinline__ float to_f32(float x) { return x; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }

@@ -1,0 +1,99 @@
+// RMSNorm of the layer output (App. D.1), in place: a memory-bound pass over o [B,H,T,Dv].
+//
+// One warp per (batch, head, token) row; a lane holds one 16-byte vector of the row at a time (8 bf16 or 4 fp32
+// values), rows up to 32 vectors wide are read once and kept in registers between the mean and the scaling
+// (Dv <= 256 in bf16, <= 128 in fp32), wider rows are read twice (the second time from L1/L2).  Traffic is one
+// read and one write of o: the roofline is the HBM copy bandwidth.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/swila.h"
+
+namespace swila {
+
+template <bool BF16>
+__device__ __forceinline__ void unpack(const uint4 &u, float (&x)[8]) {
+  if constexpr (BF16) {
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      x[2 * i] = __uint_as_float(w[i] << 16);
+      x[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  } else {
+    x[0] = __uint_as_float(u.x); x[1] = __uint_as_float(u.y); x[2] = __uint_as_float(u.z); x[3] = __uint_as_float(u.w);
+    x[4] = x[5] = x[6] = x[7] = 0.f;
+  }
+}
+
+template <bool BF16>
+__device__ __forceinline__ uint4 pack(const float (&x)[8]) {
+  uint4 u;
+  if constexpr (BF16) {
+    const __nv_bfloat162 a = __floats2bfloat162_rn(x[0], x[1]), b = __floats2bfloat162_rn(x[2], x[3]);
+    const __nv_bfloat162 c = __floats2bfloat162_rn(x[4], x[5]), d = __floats2bfloat162_rn(x[6], x[7]);
+    u.x = *reinterpret_cast<const uint32_t *>(&a); u.y = *reinterpret_cast<const uint32_t *>(&b);
+    u.z = *reinterpret_cast<const uint32_t *>(&c); u.w = *reinterpret_cast<const uint32_t *>(&d);
+  } else {
+    u.x = __float_as_uint(x[0]); u.y = __float_as_uint(x[1]); u.z = __float_as_uint(x[2]); u.w = __float_as_uint(x[3]);
+  }
+  return u;
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(256) rmsnorm_kernel(uint4 *o, const float *weight, size_t rows, int Dv, float eps) {
+  constexpr int EPV = BF16 ? 8 : 4;  // elements per 16-byte vector
+  const int lane = threadIdx.x & 31;
+  const size_t warp0 = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const size_t nwarps = ((size_t)gridDim.x * blockDim.x) >> 5;
+  const int nvec = Dv / EPV;
+  const float inv_dv = 1.0f / (float)Dv;
+  for (size_t row = warp0; row < rows; row += nwarps) {
+    uint4 *base = o + row * nvec;
+    uint4 held = make_uint4(0, 0, 0, 0);
+    float ss = 0.f;
+    for (int c = lane; c < nvec; c += 32) {
+      const uint4 u = __ldcs(base + c);
+      if (c == lane) held = u;
+      float x[8];
+      unpack<BF16>(u, x);
+#pragma unroll
+      for (int i = 0; i < EPV; ++i) ss = fmaf(x[i], x[i], ss);
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+    const float scale = rsqrtf(fmaf(ss, inv_dv, eps));
+    for (int c = lane; c < nvec; c += 32) {
+      const uint4 u = (c == lane) ? held : base[c];
+      float x[8];
+      unpack<BF16>(u, x);
+#pragma unroll
+      for (int i = 0; i < EPV; ++i) x[i] *= weight ? scale * __ldg(weight + c * EPV + i) : scale;
+      __stcs(base + c, pack<BF16>(x));
+    }
+  }
+}
+
+}  // namespace swila
+
+extern "C" int swila_output_norm(const swila_shape_t *s, void *o, const float *weight, float eps, void *stream) {
+  if (!s || !o) return SWILA_ERR_NULL;
+  if (s->B <= 0 || s->H <= 0 || s->T < 0 || s->Dv <= 0 || s->Dv % 8 != 0 || !(eps >= 0.f)) return SWILA_ERR_SHAPE;
+  if (s->io_dtype != SWILA_IO_FP32 && s->io_dtype != SWILA_IO_BF16) return SWILA_ERR_UNSUPPORTED;
+  if (reinterpret_cast<uintptr_t>(o) & 15u) return SWILA_ERR_ALIGN;
+  const size_t rows = (size_t)s->B * s->H * (size_t)s->T;
+  if (rows == 0) return SWILA_OK;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return SWILA_ERR_CUDA;
+  // 8 warps per block, 8 blocks per SM: enough loads in flight to cover the memory latency
+  const size_t want = (rows + 7) / 8;
+  const unsigned grid = (unsigned)(want < (size_t)sms * 8 ? want : (size_t)sms * 8);
+  if (s->io_dtype == SWILA_IO_BF16)
+    swila::rmsnorm_kernel<true><<<grid, 256, 0, (cudaStream_t)stream>>>((uint4 *)o, weight, rows, s->Dv, eps);
+  else
+    swila::rmsnorm_kernel<false><<<grid, 256, 0, (cudaStream_t)stream>>>((uint4 *)o, weight, rows, s->Dv, eps);
+  return cudaGetLastError() == cudaSuccess ? SWILA_OK : SWILA_ERR_CUDA;
+}

@@ -154,15 +154,45 @@ __device__ __forceinline__ void cook_block(const ScanParams &p, const unsigned c
   (void)J; (void)DK; (void)NT; (void)TB; (void)GATE;
   constexpr int COLS = C::COLS;
   const int nvalid = min(TB, p.T - t0);
-  // k, q: straight conversion
   const IO *rk = reinterpret_cast<const IO *>(raw + C::R_K);
   const IO *rq = reinterpret_cast<const IO *>(raw + C::R_Q);
-  for (int i = tid; i < nvalid * DK / 4; i += NT) {
-    float4 a, b;
-    a.x = to_f32(rk[4 * i]); a.y = to_f32(rk[4 * i + 1]); a.z = to_f32(rk[4 * i + 2]); a.w = to_f32(rk[4 * i + 3]);
-    b.x = to_f32(rq[4 * i]); b.y = to_f32(rq[4 * i + 1]); b.z = to_f32(rq[4 * i + 2]); b.w = to_f32(rq[4 * i + 3]);
-    reinterpret_cast<float4 *>(ck + C::K_K)[i] = a;
-    reinterpret_cast<float4 *>(ck + C::K_Q)[i] = b;
+  if (!p.qkv_act) {
+    // k, q: straight conversion
+    for (int i = tid; i < nvalid * DK / 4; i += NT) {
+      float4 a, b;
+      a.x = to_f32(rk[4 * i]); a.y = to_f32(rk[4 * i + 1]); a.z = to_f32(rk[4 * i + 2]); a.w = to_f32(rk[4 * i + 3]);
+      b.x = to_f32(rq[4 * i]); b.y = to_f32(rq[4 * i + 1]); b.z = to_f32(rq[4 * i + 2]); b.w = to_f32(rq[4 * i + 3]);
+      reinterpret_cast<float4 *>(ck + C::K_K)[i] = a;
+      reinterpret_cast<float4 *>(ck + C::K_Q)[i] = b;
+    }
+  } else {
+    // raw projections: SiLU, then division by the L2 norm over the key dimension (App. B.2, App. D.1).  A token's
+    // DK / 4 work items sit in adjacent lanes of one warp (DK / 4 divides 32 and NT is a multiple of 32), so the
+    // sums of squares are xor-shuffles; every thread runs every trip of the loop.
+    constexpr int LPT = DK / 4;
+    static_assert(LPT <= 32 && 32 % LPT == 0 && NT % 32 == 0, "a token's lanes must share a warp");
+    const int items = nvalid * LPT;
+    for (int i0 = 0; i0 < items; i0 += NT) {
+      const int i = i0 + tid;
+      const bool on = i < items;
+      float a[4] = {0.f, 0.f, 0.f, 0.f}, b[4] = {0.f, 0.f, 0.f, 0.f};
+      if (on) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { a[e] = silu_approx(to_f32(rk[4 * i + e])); b[e] = silu_approx(to_f32(rq[4 * i + e])); }
+      }
+      float sa = a[0] * a[0] + a[1] * a[1] + a[2] * a[2] + a[3] * a[3];
+      float sb = b[0] * b[0] + b[1] * b[1] + b[2] * b[2] + b[3] * b[3];
+#pragma unroll
+      for (int off = 1; off < LPT; off <<= 1) {
+        sa += __shfl_xor_sync(0xffffffffu, sa, off);
+        sb += __shfl_xor_sync(0xffffffffu, sb, off);
+      }
+      const float ia = rsqrtf(sa + kL2Eps), ib = rsqrtf(sb + kL2Eps);
+      if (on) {
+        reinterpret_cast<float4 *>(ck + C::K_K)[i] = make_float4(a[0] * ia, a[1] * ia, a[2] * ia, a[3] * ia);
+        reinterpret_cast<float4 *>(ck + C::K_Q)[i] = make_float4(b[0] * ib, b[1] * ib, b[2] * ib, b[3] * ib);
+      }
+    }
   }
   // per (token, column): v and the gate activations
   const IO *rv = reinterpret_cast<const IO *>(raw + C::R_V);
@@ -173,7 +203,7 @@ __device__ __forceinline__ void cook_block(const ScanParams &p, const unsigned c
   const IO *rgq = reinterpret_cast<const IO *>(raw + C::R_GQ);
   for (int i = tid; i < nvalid * COLS; i += NT) {
     const int s = i / COLS, c = i - s * COLS;
-    ck[C::K_V + i] = to_f32(rv[i]);
+    ck[C::K_V + i] = p.qkv_act ? silu_approx(to_f32(rv[i])) : to_f32(rv[i]);
     float be[J], lk[J], pq[J];
 #pragma unroll
     for (int j = 0; j < J; ++j) {
@@ -246,7 +276,9 @@ __device__ __forceinline__ void flush_o(const ScanParams &p, const unsigned char
 }
 
 // ---- the kernel ---------------------------------------------------------------------------
-template <class C, bool POST, bool RDEBUG>
+// AUX: the instantiation that also writes the responsibilities (r_debug) and / or forms the sums over time of the
+// mixture weights (Sec. 3.5); run-time tests of those pointers stay out of the plain instantiation's serial chain.
+template <class C, bool POST, bool AUX>
 __global__ void __launch_bounds__(C::NT, C::MIN_BLOCKS) swila_scan_kernel(const __grid_constant__ ScanParams p) {
   using IO = typename C::IO;
   constexpr int J = C::J, DK = C::DK, NT = C::NT, TB = C::TB, GATE = C::GATE;
@@ -269,6 +301,9 @@ __global__ void __launch_bounds__(C::NT, C::MIN_BLOCKS) swila_scan_kernel(const 
   // ---- state slice -> registers: lane g holds key dims (i*G + g)*4 .. +3, i = 0..L/4-1 ----
   float2 w[J][L / 2];
   float rprev[J], rho[J];
+  [[maybe_unused]] float st_r[J], st_q[J], st_re = 0.f, st_qe = 0.f;  // AUX: sums over time, entropies in bits
+#pragma unroll
+  for (int j = 0; j < J; ++j) st_r[j] = st_q[j] = 0.f;
 #pragma unroll
   for (int j = 0; j < J; ++j) {
     const float *src = p.W_in ? p.W_in + (((size_t)bh * J + j) * p.Dv + col) * DK : nullptr;
@@ -393,11 +428,23 @@ __global__ void __launch_bounds__(C::NT, C::MIN_BLOCKS) swila_scan_kernel(const 
           pq[j] = rho[j];
         }
       }
-      if constexpr (RDEBUG) {  // compile-time: a run-time test here would sit on every token's serial chain
-        if (g == 0 && col_ok) {
+      if constexpr (AUX) {  // compile-time: a run-time test here would sit on every token's serial chain
+        if (p.r_debug && g == 0 && col_ok) {
 #pragma unroll
           for (int j = 0; j < J; ++j) p.r_debug[((tok0 + (size_t)(t0 + s)) * J + j) * p.Dv + col] = rr[j];
         }
+        // sums over time (Sec. 3.5).  log2 r_j = a_j - m - log2(sum) and sum_j r_j = 1, so the entropy in bits is
+        // log2(sum) - sum_j r_j (a_j - m); a component whose responsibility underflowed adds nothing
+        float hk = 0.f, hq = 0.f;
+#pragma unroll
+        for (int j = 0; j < J; ++j) {
+          st_r[j] += rr[j];
+          st_q[j] += pq[j];
+          if (rr[j] > 0.f) hk = fmaf(rr[j], a[j] - m, hk);
+          if (pq[j] > 0.f) hq = fmaf(pq[j], lg2_approx(pq[j]), hq);
+        }
+        st_re += lg2_approx(sum) - hk;
+        st_qe -= hq;
       }
 
       // ---- pass B: M-step (Eq. 3.3 / 3.7) and readout on the updated state (Eq. 3.5) ----
@@ -449,6 +496,18 @@ __global__ void __launch_bounds__(C::NT, C::MIN_BLOCKS) swila_scan_kernel(const 
                make_float4(w[j][2 * i].x, w[j][2 * i].y, w[j][2 * i + 1].x, w[j][2 * i + 1].y));
     }
   }
+  if constexpr (AUX) {
+    if (col_ok && g == 0) {  // each element belongs to one thread of one block: plain read-modify-write
+      constexpr float kLn2 = 0.6931471805599453f;
+#pragma unroll
+      for (int j = 0; j < J; ++j) {
+        if (p.r_sum) p.r_sum[((size_t)bh * J + j) * p.Dv + col] += st_r[j];
+        if (p.rho_sum) p.rho_sum[((size_t)bh * J + j) * p.Dv + col] += st_q[j];
+      }
+      if (p.r_ent) p.r_ent[(size_t)bh * p.Dv + col] += st_re * kLn2;
+      if (p.rho_ent) p.rho_ent[(size_t)bh * p.Dv + col] += st_qe * kLn2;
+    }
+  }
   if (temporal && col_ok && g == 0) {
 #pragma unroll
     for (int j = 0; j < J; ++j) {
@@ -464,7 +523,8 @@ int launch_scan(const LaunchArgs &a) {
   using IO = typename C::IO;
   constexpr int J = C::J, DK = C::DK, NT = C::NT, TB = C::TB, GATE = C::GATE;
   (void)J; (void)DK; (void)NT; (void)TB; (void)GATE;
-  auto kern = a.p.r_debug ? swila_scan_kernel<C, POST, true> : swila_scan_kernel<C, POST, false>;
+  const bool aux = a.p.r_debug || a.p.r_sum || a.p.r_ent || a.p.rho_sum || a.p.rho_ent;
+  auto kern = aux ? swila_scan_kernel<C, POST, true> : swila_scan_kernel<C, POST, false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES);
   if (e != cudaSuccess) return (int)e;
   const long long nslice = (a.p.Dv + C::COLS - 1) / C::COLS;

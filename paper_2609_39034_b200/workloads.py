@@ -24,6 +24,7 @@ import torch
 FLAG_TEMPORAL = 1
 FLAG_GATED = 2
 FLAG_POST_DECAY = 4
+FLAG_QKV_ACT = 8  # q, k, v are raw projections: SiLU + L2 normalisation inside the kernel (App. B.2, App. D.1)
 
 GRAN_NONE = 0
 GRAN_PER_KEY = 1

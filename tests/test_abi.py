@@ -55,7 +55,7 @@ def test_state_bytes(binding):
 @pytest.mark.parametrize("change,status", [
     (dict(B=0), -2), (dict(Dv=12), -2), (dict(T=-1), -2), (dict(Dk=48), -3), (dict(J=3), -3),
     (dict(flags=wl.FLAG_POST_DECAY), -3), (dict(flags=wl.FLAG_GATED), -3),
-    (dict(gate_granularity=wl.GRAN_PER_KEY), -3), (dict(flags=8), -3),
+    (dict(gate_granularity=wl.GRAN_PER_KEY), -3), (dict(flags=16), -3),
 ])
 def test_forward_rejects_bad_shapes_on_the_host(binding, change, status):
     w = wl.CONFIGS[0].with_(**change)
