@@ -352,6 +352,39 @@ def variants_leg(binding, stream, fma_peak_tflops: float):
     return out
 
 
+def fusions_leg(binding, stream):
+    """The steps either side of the recurrence (App. B.2, App. D.1, Sec. 3.5) on the LM-shaped prefill: what the
+    in-kernel q/k/v activation and the sums over time cost the scan kernel, and the output RMSNorm pass against
+    the copy bandwidth (it reads and writes o once)."""
+    peaks = _peaks()
+    w = wl.CONFIGS[HEADLINE]
+    inp = wl.make_inputs(w, device="cuda")
+    st = binding.state_alloc(w)
+    o = torch.empty((w.B, w.H, w.T, w.Dv), device="cuda", dtype=w.torch_io_dtype)
+    stats = binding.stats_alloc(w)
+    wa = w.with_(flags=w.flags | wl.FLAG_QKV_ACT)
+    wgt = torch.ones(w.Dv, device="cuda")
+    w4 = w.with_(B=4 * w.B)  # 537 MB of outputs: four times the L2, so the pass runs from HBM
+    o4 = torch.randn((w4.B, w4.H, w4.T, w4.Dv), device="cuda").to(w.torch_io_dtype)
+    calls = {
+        "scan_plain": lambda: binding.swila_forward(w, inp, state_in=None, state_out=st, o=o, algo=binding.ALGO_SCAN),
+        "scan_qkv_act": lambda: binding.swila_forward(wa, inp, state_in=None, state_out=st, o=o, algo=binding.ALGO_SCAN),
+        "scan_stats": lambda: binding.swila_forward_stats(w, inp, stats, state_in=None, state_out=st, o=o),
+        "output_norm": lambda: binding.swila_output_norm(w4, o4, wgt),
+    }
+    out = {}
+    for name, f in calls.items():
+        for _ in range(3):
+            f()
+        torch.cuda.synchronize()
+        out[name] = {"ms": time_steps(f, 10, stream) / 10}
+    norm_bytes = 2 * o4.numel() * o4.element_size()
+    out["output_norm"].update({"bytes": norm_bytes, "gbs": norm_bytes / (out["output_norm"]["ms"] * 1e-3) / 1e9,
+                               "hbm_frac": norm_bytes / (out["output_norm"]["ms"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                               "note": "o of four LM-shaped prefills (537 MB, larger than L2), read and written once"})
+    return out
+
+
 def _peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -374,6 +407,7 @@ def main():
     ap.add_argument("--no-scan", action="store_true", help="skip the scan-kernel comparison leg")
     ap.add_argument("--paper-shapes", action="store_true", help="also time the shapes the paper itself quotes")
     ap.add_argument("--variants", action="store_true", help="also time the Temporal / Gated variants on all five configs")
+    ap.add_argument("--fusions", action="store_true", help="also time the q/k/v activation, the statistics and the output norm")
     ap.add_argument("--decode-steps", type=int, default=wl.DECODE_STEPS)
     ap.add_argument("--decode-prefill", type=int, default=4096)
     ap.add_argument("--decode-batch", type=int, default=0, help="override B of the decode leg (0 = 256)")
@@ -523,6 +557,7 @@ def main():
 
     paper = paper_shapes_leg(binding, stream) if args.paper_shapes else None
     variants = variants_leg(binding, stream, fma_peak_nominal) if args.variants else None
+    fusions = fusions_leg(binding, stream) if args.fusions else None
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
@@ -542,7 +577,7 @@ def main():
                        "l2": "inputs (2.1 GB) larger than L2; no flush needed",
                        "multi_gpu": "independent replicas, no collective"},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": args.steps,
-            "clocks": clocks, "decode": decode, "scan": scan, "paper_shapes": paper, "variants": variants,
+            "clocks": clocks, "decode": decode, "scan": scan, "paper_shapes": paper, "variants": variants, "fusions": fusions,
         }
         print(json.dumps(line))
     if world > 1:

@@ -1,9 +1,9 @@
 // RMSNorm of the layer output (App. D.1), in place: a memory-bound pass over o [B,H,T,Dv].
 //
-// One warp per (batch, head, token) row; a lane holds one 16-byte vector of the row at a time (8 bf16 or 4 fp32
-// values), rows up to 32 vectors wide are read once and kept in registers between the mean and the scaling
-// (Dv <= 256 in bf16, <= 128 in fp32), wider rows are read twice (the second time from L1/L2).  Traffic is one
-// read and one write of o: the roofline is the HBM copy bandwidth.
+// A lane holds 16-byte vectors of a row (8 bf16 or 4 fp32 values).  Rows up to 32 vectors wide (Dv <= 256 in bf16,
+// <= 128 in fp32) are shared by the lanes of a warp, several rows per warp in flight, read once and kept in
+// registers between the mean and the scaling; wider rows take one warp each and are read twice (the second time
+// from L1/L2).  Traffic is one read and one write of o: the roofline is the HBM copy bandwidth.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -41,6 +41,48 @@ __device__ __forceinline__ uint4 pack(const float (&x)[8]) {
   return u;
 }
 
+// Rows of at most 32 vectors: LPR lanes per row (the power of two that covers the row), 32 / LPR rows per warp at
+// a time and U such groups in flight per warp, so that enough bytes are outstanding to cover the memory latency
+// (one 256-byte row per warp at a time reached a third of the copy bandwidth).
+template <bool BF16, int LPR>
+__global__ void __launch_bounds__(256) rmsnorm_rows_kernel(uint4 *o, const float *weight, size_t rows, int Dv, float eps) {
+  constexpr int EPV = BF16 ? 8 : 4, RPW = 32 / LPR, U = 4;
+  const int lane = threadIdx.x & 31, c = lane % LPR, sub = lane / LPR;
+  const size_t warp0 = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const size_t nwarps = ((size_t)gridDim.x * blockDim.x) >> 5;
+  const int nvec = Dv / EPV;
+  const bool c_ok = c < nvec;
+  const float inv_dv = 1.0f / (float)Dv;
+  float wv[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) wv[i] = (weight && c_ok && i < EPV) ? __ldg(weight + c * EPV + i) : 1.0f;
+  for (size_t row0 = warp0 * (RPW * U); row0 < rows; row0 += nwarps * (RPW * U)) {
+    uint4 u[U];
+    bool ok[U];
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+      const size_t row = row0 + k * RPW + sub;
+      ok[k] = c_ok && row < rows;
+      u[k] = ok[k] ? __ldcs(o + row * nvec + c) : make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int k = 0; k < U; ++k) {
+      float x[8];
+      unpack<BF16>(u[k], x);
+      float ss = 0.f;
+#pragma unroll
+      for (int i = 0; i < EPV; ++i) ss = fmaf(x[i], x[i], ss);
+#pragma unroll
+      for (int off = 1; off < LPR; off <<= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+      const float scale = rsqrtf(fmaf(ss, inv_dv, eps));
+#pragma unroll
+      for (int i = 0; i < EPV; ++i) x[i] *= scale * wv[i];
+      if (ok[k]) __stcs(o + (row0 + k * RPW + sub) * nvec + c, pack<BF16>(x));
+    }
+  }
+}
+
+// Any row width: one warp per row, the row read twice when it is wider than 32 vectors.
 template <bool BF16>
 __global__ void __launch_bounds__(256) rmsnorm_kernel(uint4 *o, const float *weight, size_t rows, int Dv, float eps) {
   constexpr int EPV = BF16 ? 8 : 4;  // elements per 16-byte vector
@@ -75,6 +117,24 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(uint4 *o, const float *wei
   }
 }
 
+template <bool BF16>
+static void launch_rmsnorm(uint4 *o, const float *weight, size_t rows, int Dv, float eps, int sms, cudaStream_t st) {
+  const int nvec = Dv / (BF16 ? 8 : 4);
+  // 8 warps per block, up to 8 blocks per SM
+  auto grid_for = [&](size_t rows_per_warp) {
+    const size_t want = (rows + 8 * rows_per_warp - 1) / (8 * rows_per_warp);
+    return (unsigned)(want < (size_t)sms * 8 ? want : (size_t)sms * 8);
+  };
+#define SWILA_NORM_CASE(LPR)                                                                                   \
+  if (nvec <= LPR) {                                                                                           \
+    rmsnorm_rows_kernel<BF16, LPR><<<grid_for(4 * 32 / LPR), 256, 0, st>>>(o, weight, rows, Dv, eps);           \
+    return;                                                                                                    \
+  }
+  SWILA_NORM_CASE(2) SWILA_NORM_CASE(4) SWILA_NORM_CASE(8) SWILA_NORM_CASE(16) SWILA_NORM_CASE(32)
+#undef SWILA_NORM_CASE
+  rmsnorm_kernel<BF16><<<grid_for(1), 256, 0, st>>>(o, weight, rows, Dv, eps);
+}
+
 }  // namespace swila
 
 extern "C" int swila_output_norm(const swila_shape_t *s, void *o, const float *weight, float eps, void *stream) {
@@ -88,12 +148,9 @@ extern "C" int swila_output_norm(const swila_shape_t *s, void *o, const float *w
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return SWILA_ERR_CUDA;
-  // 8 warps per block, 8 blocks per SM: enough loads in flight to cover the memory latency
-  const size_t want = (rows + 7) / 8;
-  const unsigned grid = (unsigned)(want < (size_t)sms * 8 ? want : (size_t)sms * 8);
   if (s->io_dtype == SWILA_IO_BF16)
-    swila::rmsnorm_kernel<true><<<grid, 256, 0, (cudaStream_t)stream>>>((uint4 *)o, weight, rows, s->Dv, eps);
+    swila::launch_rmsnorm<true>((uint4 *)o, weight, rows, s->Dv, eps, sms, (cudaStream_t)stream);
   else
-    swila::rmsnorm_kernel<false><<<grid, 256, 0, (cudaStream_t)stream>>>((uint4 *)o, weight, rows, s->Dv, eps);
+    swila::launch_rmsnorm<false>((uint4 *)o, weight, rows, s->Dv, eps, sms, (cudaStream_t)stream);
   return cudaGetLastError() == cudaSuccess ? SWILA_OK : SWILA_ERR_CUDA;
 }
