@@ -120,19 +120,23 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(uint4 *o, const float *wei
 template <bool BF16>
 static void launch_rmsnorm(uint4 *o, const float *weight, size_t rows, int Dv, float eps, int sms, cudaStream_t st) {
   const int nvec = Dv / (BF16 ? 8 : 4);
-  // 8 warps per block, up to 8 blocks per SM
-  auto grid_for = [&](size_t rows_per_warp) {
-    const size_t want = (rows + 8 * rows_per_warp - 1) / (8 * rows_per_warp);
-    return (unsigned)(want < (size_t)sms * 8 ? want : (size_t)sms * 8);
+  // 8 warps per block; as many blocks as are resident at once (the kernels stride over the rows), fewer for few rows
+  auto grid_for = [&](auto kern, size_t rows_per_warp) {
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, 256, 0) != cudaSuccess || per_sm < 1) per_sm = 1;
+    const size_t want = (rows + 8 * rows_per_warp - 1) / (8 * rows_per_warp), cap = (size_t)sms * per_sm;
+    return (unsigned)(want < cap ? want : cap);
   };
 #define SWILA_NORM_CASE(LPR)                                                                                   \
   if (nvec <= LPR) {                                                                                           \
-    rmsnorm_rows_kernel<BF16, LPR><<<grid_for(4 * 32 / LPR), 256, 0, st>>>(o, weight, rows, Dv, eps);           \
+    auto kern = rmsnorm_rows_kernel<BF16, LPR>;                                                                \
+    kern<<<grid_for(kern, 4 * 32 / LPR), 256, 0, st>>>(o, weight, rows, Dv, eps);                               \
     return;                                                                                                    \
   }
   SWILA_NORM_CASE(2) SWILA_NORM_CASE(4) SWILA_NORM_CASE(8) SWILA_NORM_CASE(16) SWILA_NORM_CASE(32)
 #undef SWILA_NORM_CASE
-  rmsnorm_kernel<BF16><<<grid_for(1), 256, 0, st>>>(o, weight, rows, Dv, eps);
+  auto kern = rmsnorm_kernel<BF16>;
+  kern<<<grid_for(kern, 1), 256, 0, st>>>(o, weight, rows, Dv, eps);
 }
 
 }  // namespace swila
