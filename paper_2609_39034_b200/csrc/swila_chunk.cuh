@@ -606,16 +606,22 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     // =============================== helper warps ============================================
     const int h = r;
     // beta = sigmoid(logit) of this helper's row for every token of a raw stage (App. B.2), written over the
-    // logits: all helpers read their logits first, then all write
+    // logits, 8 tokens per pass (rolled: less code in the instruction cache), last tokens first: a token's FP32
+    // row (512 bytes) lies further into the region than its logits (at most 384 bytes), so a pass overwrites only
+    // logits of its own tokens -- which every helper has read by the barrier -- and of later, finished ones
     auto cook_be = [&](unsigned char *raw) {
       const __nv_bfloat16 *rb = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_B);
       float *bes = reinterpret_cast<float *>(raw + Cf::R_B);
-      float be[C];
+      static_assert(J * Cf::GROW * Cf::ES <= NROW * 4, "a token's logits end before its FP32 row does");
+#pragma unroll 1
+      for (int t8 = C - 8; t8 >= 0; t8 -= 8) {
+        float be[8];
 #pragma unroll
-      for (int t = 0; t < C; ++t) be[t] = sigmoid_approx(__bfloat162float(rb[(t * J + j) * Cf::GROW + dl]));
-      named_bar_sync(3, 128);
+        for (int i = 0; i < 8; ++i) be[i] = sigmoid_approx(__bfloat162float(rb[((t8 + i) * J + j) * Cf::GROW + dl]));
+        named_bar_sync(3, 128);
 #pragma unroll
-      for (int t = 0; t < C; ++t) bes[t * NROW + h] = be[t];
+        for (int i = 0; i < 8; ++i) bes[(t8 + i) * NROW + h] = be[i];
+      }
     };
     // operand parts of W after an update, this helper's tensor-memory lane
     auto refresh_parts = [&]() {
