@@ -369,7 +369,11 @@ def fusions_leg(binding, stream):
     calls = {
         "scan_plain": lambda: binding.swila_forward(w, inp, state_in=None, state_out=st, o=o, algo=binding.ALGO_SCAN),
         "scan_qkv_act": lambda: binding.swila_forward(wa, inp, state_in=None, state_out=st, o=o, algo=binding.ALGO_SCAN),
-        "scan_stats": lambda: binding.swila_forward_stats(w, inp, stats, state_in=None, state_out=st, o=o),
+        "scan_stats": lambda: binding.swila_forward_stats(w, inp, stats, state_in=None, state_out=st, o=o,
+                                                          algo=binding.ALGO_SCAN),
+        "chunk_plain": lambda: binding.swila_forward(w, inp, state_in=None, state_out=st, o=o, algo=binding.ALGO_CHUNK),
+        "chunk_stats": lambda: binding.swila_forward_stats(w, inp, stats, state_in=None, state_out=st, o=o,
+                                                           algo=binding.ALGO_CHUNK),
         "output_norm": lambda: binding.swila_output_norm(w4, o4, wgt),
     }
     out = {}

@@ -167,8 +167,9 @@ typedef struct {
 
 /*
  * swila_forward that also forms the sums of `stats` (which must not be NULL; any of its members may be).
- * Runs the scan kernel (SWILA_ALGO_CHUNK -> SWILA_ERR_UNSUPPORTED); outputs and state are those of
- * swila_forward with SWILA_ALGO_SCAN, bit for bit.
+ * The kernel is chosen as in swila_forward; outputs and state are those of swila_forward with the same
+ * shape->algo, bit for bit.  The chunked kernel adds its sums with atomic operations (the pieces of a sequence
+ * may run in different thread blocks), so their last bits can differ from run to run; the scan kernel's do not.
  */
 int swila_forward_stats(const swila_shape_t *shape, const void *q, const void *k, const void *v,
                         const swila_gates_t *gates, const swila_state_t *state_in,

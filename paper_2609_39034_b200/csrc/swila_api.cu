@@ -106,7 +106,6 @@ static int run(const swila_shape_t *s, int T, const void *q, const void *k, cons
     a.p.r_sum = stats->r_sum; a.p.r_ent = stats->r_ent;
     a.p.rho_sum = stats->rho_sum; a.p.rho_ent = stats->rho_ent;
   }
-  const bool want_stats = a.p.r_sum || a.p.r_ent || a.p.rho_sum || a.p.rho_ent;
   a.Dk = s->Dk; a.J = s->J; a.io_dtype = s->io_dtype;
   a.gate_mode = !gated ? 0 : (s->gate_granularity == SWILA_GATE_PER_KEY ? 1 : 2);
   a.post = (s->flags & SWILA_POST_DECAY) ? 1 : 0;
@@ -117,7 +116,7 @@ static int run(const swila_shape_t *s, int T, const void *q, const void *k, cons
   // AUTO: the chunked tensor-core kernel whenever it applies and the sequence is long enough to
   // amortise its per-chunk set-up; the scan otherwise (fp32 io, TEMPORAL / GATED, decode).
   const bool chunk_ok = s->io_dtype == SWILA_IO_BF16 && s->flags == 0 && (s->Dk == 64 || s->Dk == 128) &&
-                        (s->J == 4 || s->J == 8) && !want_stats;
+                        (s->J == 4 || s->J == 8);
   if (s->algo == SWILA_ALGO_CHUNK || (s->algo == SWILA_ALGO_AUTO && chunk_ok && T >= 64)) {
     rc = chunk_dispatch(a);
     if (rc == -1000 && s->algo == SWILA_ALGO_CHUNK) return SWILA_ERR_UNSUPPORTED;
@@ -235,7 +234,6 @@ int swila_forward_stats(const swila_shape_t *s, const void *q, const void *k, co
   int rc = check_shape(s, true);
   if (rc) return rc;
   if (!stats) return SWILA_ERR_NULL;
-  if (s->algo == SWILA_ALGO_CHUNK) return SWILA_ERR_UNSUPPORTED;
   if (s->T == 0) return swila_forward(s, q, k, v, g, state_in, state_out, o, r_debug, stream);  // nothing to add
   return run(s, s->T, q, k, v, g, state_in, state_out, o, r_debug, stream, stats);
 }

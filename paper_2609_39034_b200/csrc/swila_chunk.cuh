@@ -227,6 +227,9 @@ __device__ __forceinline__ void chunk_stage(const ChunkMaps &maps, unsigned char
   tma_load_4d(rawpq, &maps.pq, col0, 0, tok, bh, bar);
 }
 
+// RDEBUG: the auxiliary instantiation, which also writes the responsibilities (p.r_debug) and / or adds the sums
+// over time of the mixture weights (Sec. 3.5) to p.r_sum, p.r_ent, p.rho_sum, p.rho_ent; each pointer is tested at
+// run time there, none of it is in the plain instantiation.
 template <class Cf, bool RDEBUG>
 __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_constant__ ScanParams p,
                                                                      const __grid_constant__ ChunkSched sched,
@@ -320,6 +323,9 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
 
   // outputs of one chunk (Eq. 3.5): o_td = sum_j pi^q_j (w_t.q_t)_j, pi^q = softmax over the J
   // components of a column
+  [[maybe_unused]] float sq_sum[J], sq_ent = 0.f;  // helper lanes, auxiliary instantiation: slot c = component j ^ pattern(c)
+#pragma unroll
+  for (int c = 0; c < J; ++c) sq_sum[c] = 0.f;
   auto write_outputs = [&](int n) {
     const int t0 = n * C;
     const int nvalid = min(C, Tseg - t0);
@@ -361,6 +367,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       for (int rest = 0; rest < (8 >> LJ); ++rest) {
         const int tl = tg + (j << (3 - LJ)) + rest;
         float x[J];
+        [[maybe_unused]] float ex[J];
         float mx = -3.0e38f;
 #pragma unroll
         for (int c = 0; c < J; ++c) {
@@ -374,10 +381,25 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
 #pragma unroll
         for (int c = 0; c < J; ++c) {
           const float e = ex2_approx(x[c] - mx);
+          if constexpr (RDEBUG) ex[c] = e;
           se += e;
           so = fmaf(e, hq[(c << (3 - LJ)) | rest], so);
         }
-        ost[tl * COLS + dl] = __float2bfloat16_rn(so * rcp_approx(se));
+        const float ise = rcp_approx(se);
+        ost[tl * COLS + dl] = __float2bfloat16_rn(so * ise);
+        if constexpr (RDEBUG) {
+          // sums over time of the readout weights and of their entropy (bits): log2 p_c = x_c - mx - log2(se)
+          if (tl < nvalid) {
+            float hb = 0.f;
+#pragma unroll
+            for (int c = 0; c < J; ++c) {
+              const float pc = ex[c] * ise;
+              sq_sum[c] += pc;
+              if (pc > 0.f) hb = fmaf(pc, x[c] - mx, hb);
+            }
+            sq_ent += lg2_approx(se) - hb;
+          }
+        }
       }
     }
     tc_fence_before_sync();
@@ -394,6 +416,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   if (warp < 4) {
     // =============================== row warps ===============================================
     const int jbase = lane - j;
+    [[maybe_unused]] float st_r = 0.f, st_h = 0.f;  // auxiliary instantiation: this piece's sums over time
     if (!mbar_wait(&bars[B_BE], 0) || !mbar_wait(&bars[B_GS], 0)) failed = true;
 #pragma unroll 1
     for (int n = 0; n < nchunks && !failed; ++n) {
@@ -436,10 +459,12 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       //      FAST: exponentials are taken without subtracting the per-token maximum; the pass reports whether
       //      any normaliser left the safe range (all components > ~13 standard deviations off, or extreme
       //      prior logits), in which case the chunk is redone with the maximum subtracted. ----
+      [[maybe_unused]] float chunk_r = 0.f, chunk_h = 0.f;  // written by the pass whose results stand
       auto sequential = [&](auto exact_tag) -> bool {
         constexpr bool EXACT = decltype(exact_tag)::value;
         constexpr int GT = Cf::GT;
         bool bad = false;
+        [[maybe_unused]] float cr = 0.f, ch = 0.f;  // auxiliary instantiation: this chunk's sums of r and of r log2 r
         // pred[i]: v - prediction (the prediction error so far) of token tg + i of the current trip, for the WINS
         // tokens that the pushes of a token reach on the ALUs (slots past the chunk end are dead weight that keeps the
         // trip's code independent of tg); the Gram rows are stored negated, so a push is one FMA and the error of
@@ -519,7 +544,12 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
             if (t >= nvalid) c = 0.f;  // padding tokens of the last chunk leave the state alone
             cs[i] = c;
             if constexpr (RDEBUG) {
-              if (col_ok && t < nvalid) p.r_debug[((tok0 + (size_t)(t0 + t)) * J + j) * p.Dv + col] = e * rs;
+              const float rr = e * rs;
+              if (p.r_debug && col_ok && t < nvalid) p.r_debug[((tok0 + (size_t)(t0 + t)) * J + j) * p.Dv + col] = rr;
+              if (t < nvalid) {  // log2 r = log2 e - log2(sum); a component whose responsibility underflowed adds nothing
+                cr += rr;
+                if (rr > 0.f) ch = fmaf(rr, lg2_approx(e) - lg2_approx(sum), ch);
+              }
             }
             pred[i + 1] = fmaf(c, Gkk[t * C + t + 1], pred[i + 1]);  // the push the next token waits for
             c_prev = c;
@@ -558,6 +588,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
             }
           }
         }
+        if constexpr (RDEBUG) { chunk_r = cr; chunk_h = ch; }
         return bad;
       };
       const bool unsafe = sequential(std::false_type{});
@@ -571,6 +602,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         }
         sequential(std::true_type{});
       }
+      if constexpr (RDEBUG) { st_r += chunk_r; st_h += chunk_h; }
       tmem_st_wait();
       tc_fence_before_sync();
       PROF_ADD(2);
@@ -595,6 +627,13 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
 #pragma unroll
         for (int i = 0; i < 4; ++i)
           __stcs(reinterpret_cast<float4 *>(dst + cc * 16 + i * 4), make_float4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]));
+      }
+    }
+    if constexpr (RDEBUG) {
+      if (!failed && col_ok) {  // other pieces of the tile may run in other blocks: atomic additions
+        constexpr float kLn2 = 0.6931471805599453f;
+        if (p.r_sum) atomicAdd(p.r_sum + ((size_t)bh * J + j) * p.Dv + col, st_r);
+        if (p.r_ent) atomicAdd(p.r_ent + (size_t)bh * p.Dv + col, -st_h * kLn2);
       }
     }
     if (to_flag) {  // the rest of this tile belongs to another block: publish the state
@@ -820,6 +859,22 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     }
     if (!failed && !mbar_wait(&bars[B_QD], (nchunks - 1) & 1)) failed = true;
     if (!failed) write_outputs(nchunks - 1);
+    if constexpr (RDEBUG) {
+      // this piece's sums of the readout weights: the J lanes of a column hold disjoint tokens, and other pieces of
+      // the tile may run in other blocks, hence atomic additions
+      if (!failed && col_ok) {
+        constexpr int LJ = (J == 4) ? 2 : 3;
+        constexpr float kLn2 = 0.6931471805599453f;
+#pragma unroll
+        for (int c = 0; c < J; ++c) {
+          int pat = 0;
+#pragma unroll
+          for (int rd = 0; rd < LJ; ++rd) pat |= ((c >> (LJ - 1 - rd)) & 1) ? (J >> (rd + 1)) : 0;
+          if (p.rho_sum) atomicAdd(p.rho_sum + ((size_t)bh * J + (j ^ pat)) * p.Dv + col, sq_sum[c]);
+        }
+        if (p.rho_ent) atomicAdd(p.rho_ent + (size_t)bh * p.Dv + col, sq_ent * kLn2);
+      }
+    }
   } else if (lane == 0) {
     // =============================== MMA issuer ==============================================
     constexpr uint32_t idE = idesc_bf16(128, 2 * C);  // N = 2C: [P0 | Q0], Gram batch, cross-chunk term
@@ -1035,7 +1090,8 @@ inline unsigned chunk_next_epoch() {
 template <int J, int DK>
 int launch_chunk(const LaunchArgs &a) {
   using Cf = ChunkCfg<J, DK>;
-  auto kern = a.p.r_debug ? swila_chunk_kernel<Cf, true> : swila_chunk_kernel<Cf, false>;
+  const bool aux = a.p.r_debug || a.p.r_sum || a.p.r_ent || a.p.rho_sum || a.p.rho_ent;
+  auto kern = aux ? swila_chunk_kernel<Cf, true> : swila_chunk_kernel<Cf, false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cf::SMEM_BYTES);
   if (e != cudaSuccess) return (int)e;
   const long long nslice = (a.p.Dv + Cf::COLS - 1) / Cf::COLS;

@@ -8,7 +8,6 @@ namespace swila {
 // Returns a cudaError_t value (>= 0), or -1000 when the combination is not compiled.
 int chunk_dispatch(const LaunchArgs &a) {
   if (a.io_dtype != SWILA_IO_BF16 || a.gate_mode != 0 || a.p.temporal || a.p.qkv_act) return -1000;
-  if (a.p.r_sum || a.p.r_ent || a.p.rho_sum || a.p.rho_ent) return -1000;
 #define SWILA_CHUNK_CASE(JJ)                         \
   case JJ:                                           \
     if (a.Dk == 128) return launch_chunk<JJ, 128>(a); \

@@ -84,8 +84,11 @@ def test_qkv_activation_is_refused_by_the_chunked_kernel(binding):
 
 
 @pytest.mark.parametrize("w", SHAPES)
-@pytest.mark.parametrize("temporal", [False, True], ids=["vanilla", "temporal"])
-def test_statistics_match_the_oracle(binding, oracle, fus, w, temporal):
+@pytest.mark.parametrize("temporal,algo", [(False, "scan"), (True, "scan"), (False, "auto")],
+                         ids=["vanilla_scan", "temporal_scan", "vanilla_auto"])
+def test_statistics_match_the_oracle(binding, oracle, fus, w, temporal, algo):
+    """`auto` takes the chunked tensor-core kernel for the bf16 shapes of 64 tokens and more."""
+    algo = getattr(binding, "ALGO_" + algo.upper())
     wv = w.variant(temporal=temporal)
     inp = wl.make_inputs(wv, stress=True)
     ref = oracle.forward_inputs(inp, flags=wv.flags, want_r=True)
@@ -95,14 +98,14 @@ def test_statistics_match_the_oracle(binding, oracle, fus, w, temporal):
     stats = binding.stats_alloc(wv)
     st_out = binding.state_alloc(wv, init=False)
     sin = {"W": dev["W0"], "r_prev": dev.get("r0"), "rho_prev": dev.get("rho0")}
-    o = binding.swila_forward_stats(wv, dev, stats, state_in=sin, state_out=st_out)
+    o = binding.swila_forward_stats(wv, dev, stats, state_in=sin, state_out=st_out, algo=algo)
     torch.cuda.synchronize()
     # sums of T values in [0, 1] (entropies in [0, ln J]) accumulated in FP32 from FP32 responsibilities
     for name in ("r_sum", "r_ent", "rho_sum", "rho_ent"):
         assert wl.rel_err(stats[name].cpu(), torch.from_numpy(want[name])) < 1e-4, name
-    # outputs and state are those of the plain scan call, bit for bit
+    # outputs and state are those of the plain call, bit for bit
     st2 = binding.state_alloc(wv, init=False)
-    o2 = binding.swila_forward(wv, dev, state_in=sin, state_out=st2, algo=binding.ALGO_SCAN)
+    o2 = binding.swila_forward(wv, dev, state_in=sin, state_out=st2, algo=algo)
     torch.cuda.synchronize()
     assert torch.equal(o, o2) and torch.equal(st_out["W"], st2["W"])
     # a second call ADDS to the buffers; a sequence fed in two pieces accumulates to the same sums
@@ -111,29 +114,56 @@ def test_statistics_match_the_oracle(binding, oracle, fus, w, temporal):
     first = {k: (v[:, :, :half].contiguous() if v is not None and k not in ("W0", "r0", "rho0") else v) for k, v in dev.items()}
     second = {k: (v[:, :, half:].contiguous() if v is not None and k not in ("W0", "r0", "rho0") else v) for k, v in dev.items()}
     carry = binding.state_alloc(wv, init=False)
-    binding.swila_forward_stats(wv, first, stats2, state_in=sin, state_out=carry)
-    binding.swila_forward_stats(wv, second, stats2, state_in=carry, state_out=carry)
+    binding.swila_forward_stats(wv, first, stats2, state_in=sin, state_out=carry, algo=algo)
+    binding.swila_forward_stats(wv, second, stats2, state_in=carry, state_out=carry, algo=algo)
     torch.cuda.synchronize()
     for name in ("r_sum", "r_ent", "rho_sum", "rho_ent"):
-        assert wl.rel_err(stats2[name].cpu(), stats[name].cpu()) < 1e-5, name
+        assert wl.rel_err(stats2[name].cpu(), stats[name].cpu()) < 2e-5, name
     # mutual information of Sec. 3.5 from the sums: the quantity the loss is built from
     mi = fus.mutual_information(stats["r_sum"].cpu().numpy(), stats["r_ent"].cpu().numpy(), wv.T)
     mi_ref = fus.mutual_information(want["r_sum"], want["r_ent"], wv.T)
     assert np.max(np.abs(mi - mi_ref)) < 1e-4
 
 
-def test_statistics_members_are_optional_and_chunk_is_refused(binding):
+@pytest.mark.parametrize("algo", ["scan", "chunk"])
+def test_statistics_members_are_optional(binding, algo):
+    algo = getattr(binding, "ALGO_" + algo.upper())
     w = wl.CONFIGS[1].with_(B=1, H=1, T=96)
     inp = wl.make_inputs(w, device="cuda")
     full = binding.stats_alloc(w)
-    binding.swila_forward_stats(w, inp, full)
+    binding.swila_forward_stats(w, inp, full, algo=algo)
     only = {"r_sum": torch.zeros_like(full["r_sum"])}
-    binding.swila_forward_stats(w, inp, only)
+    binding.swila_forward_stats(w, inp, only, algo=algo)
     torch.cuda.synchronize()
-    assert torch.equal(only["r_sum"], full["r_sum"])
-    with pytest.raises(binding.SwilaError) as e:
-        binding.swila_forward_stats(w, inp, full, algo=binding.ALGO_CHUNK)
-    assert e.value.status == binding.ERR_UNSUPPORTED
+    assert torch.equal(only["r_sum"], full["r_sum"])  # one piece per tile here: a single addition per element
+
+
+def test_statistics_on_the_balanced_schedule(binding, oracle, fus):
+    """More tiles than SMs: the chunked kernel cuts sequences into pieces that run in different blocks, whose sums
+    meet in the caller's buffers through atomic additions.  Checked against the scan kernel's sums and, on sampled
+    rows, against the oracle."""
+    w = wl.CONFIGS[2].with_(B=2, H=20, T=1024)
+    inp = wl.make_inputs(w, device="cuda", stress=True)
+    sin = {"W": inp["W0"]}
+    got, ref = binding.stats_alloc(w), binding.stats_alloc(w)
+    st = binding.state_alloc(w, init=False)
+    binding.swila_forward_stats(w, inp, got, state_in=sin, state_out=st, algo=binding.ALGO_CHUNK)
+    binding.swila_forward_stats(w, inp, ref, state_in=sin, state_out=st, algo=binding.ALGO_SCAN)
+    torch.cuda.synchronize()
+    binding.device_status()
+    for name in ("r_sum", "r_ent", "rho_sum", "rho_ent"):
+        assert wl.rel_err(got[name].cpu(), ref[name].cpu()) < 1e-4, name
+    bh = torch.tensor([3, 17, 38])
+    cols = torch.tensor([0, 31, 32, 77, 127])
+    rows = wl.slice_rows(inp, bh.cuda(), cols.cuda())
+    o_ref = oracle.forward_inputs({k: (v.cpu() if v is not None else None) for k, v in rows.items()}, want_r=True)
+    want = fus.responsibility_stats(o_ref["r"], fus.readout_weights(rows["piq_logit"].cpu()))
+    for name in ("r_sum", "rho_sum"):
+        g = got[name].reshape(w.B * w.H, w.J, w.Dv)[bh.cuda()][:, :, cols.cuda()].unsqueeze(1).cpu()
+        assert wl.rel_err(g, torch.from_numpy(want[name])) < 1e-4, name
+    for name in ("r_ent", "rho_ent"):
+        g = got[name].reshape(w.B * w.H, w.Dv)[bh.cuda()][:, cols.cuda()].unsqueeze(1).cpu()
+        assert wl.rel_err(g, torch.from_numpy(want[name])) < 1e-4, name
 
 
 @pytest.mark.parametrize("io,Dv,T", [("bf16", 128, 1000), ("bf16", 64, 77), ("fp32", 16, 50), ("fp32", 256, 33), ("bf16", 512, 9)])
