@@ -145,6 +145,8 @@ int swila_state_init(const swila_shape_t *shape, swila_state_t *state, void *str
  *               (each thread block reads its slice completely before writing it).
  *   r_debug   : NULL, or fp32 [B,H,T,J,Dv] receiving the responsibilities r of Eq. 3.4.
  * T == 0 copies state_in to state_out and touches nothing else.
+ * The call only enqueues kernels on `stream`; it (and swila_decode_step) may be captured into a CUDA graph
+ * and replayed, after one ordinary call of the same shape on the device.
  */
 int swila_forward(const swila_shape_t *shape, const void *q, const void *k, const void *v,
                   const swila_gates_t *gates, const swila_state_t *state_in,

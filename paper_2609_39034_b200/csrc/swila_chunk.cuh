@@ -763,6 +763,9 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
           }
         }
         if (!seen) *fail_s = 1;
+        // A flag has one producer and one consumer per launch.  The consumer clears it, so that a launch that is
+        // replayed with the SAME epoch (a captured CUDA graph) waits again instead of finding last time's value.
+        else st_release_gpu(flag, 0u);
       }
       named_bar_sync(1, 128);
       if (*fail_s) failed = true;
