@@ -94,9 +94,12 @@ struct ChunkSched {
 constexpr int kChunkFlagSlots = 8, kChunkFlagTiles = 4096;
 static __device__ unsigned g_chunk_flags[kChunkFlagSlots][kChunkFlagTiles];
 
-template <int J_, int DK_>
+// TEMPORAL_: Temporal SwiLA (App. B.3): two more streamed inputs (the temporal gate logits), the key-side prior
+// normalised by the helpers (it enters a convex combination), and two carried distributions per row.
+template <int J_, int DK_, bool TEMPORAL_ = false>
 struct ChunkCfg {
   static constexpr int J = J_, DK = DK_;
+  static constexpr bool TEMPORAL = TEMPORAL_;
   static constexpr int C = 32;            // tokens per chunk
   static constexpr int WIN = 24;          // tokens ahead (incl. its own trip) that a token's pushes reach on the ALUs;
                                           // the pushes of tokens 0-7 into tokens 24-31 go through the tensor cores
@@ -138,10 +141,15 @@ struct ChunkCfg {
   static constexpr int R_V = 0;
   static constexpr int R_B = R_V + C * COLS * ES;
   static constexpr int R_PK = R_B + C * NROW * 4;
-  static constexpr int RAW_BYTES = R_PK + C * J * GROW * ES;
-  static constexpr int RPQ_BYTES = C * J * GROW * ES;
-  // bytes one chunk's tensor copies deliver: k and q into the operand tile, v, three gate tensors
-  static constexpr int STAGE_TX_BYTES = 3 * C * DK * ES + C * COLS * ES + 3 * C * J * GROW * ES;
+  // Temporal: the pik logits are overwritten in place by the normalised prior as fp32 [C][NROW] (like beta), and
+  // the key-side temporal gate logits gk [C][COLS] bf16 follow; the query-side ones gq [C][COLS] follow the piq
+  // logits in their ring.
+  static constexpr int R_GK = R_PK + (TEMPORAL ? C * NROW * 4 : C * J * GROW * ES);
+  static constexpr int RAW_BYTES = R_GK + (TEMPORAL ? C * COLS * ES : 0);
+  static constexpr int RQ_GQ = C * J * GROW * ES;
+  static constexpr int RPQ_BYTES = RQ_GQ + (TEMPORAL ? C * COLS * ES : 0);
+  // bytes one chunk's tensor copies deliver: k and q into the operand tile, v, three gate tensors (+ gk, gq)
+  static constexpr int STAGE_TX_BYTES = 3 * C * DK * ES + C * COLS * ES + 3 * C * J * GROW * ES + (TEMPORAL ? 2 * C * COLS * ES : 0);
   static_assert(C * J * GROW * ES <= C * NROW * 4, "the beta logits must fit the slot their gates overwrite");
   static constexpr int C_K = DK * ES / 16, C_V = COLS * ES / 16;  // 16-byte units per token row / column slice
   // operand tiles written by the helpers (bf16, same unit layout, 8 tokens per unit)
@@ -162,8 +170,10 @@ struct ChunkCfg {
   static constexpr int FAR_TILE = 2 * FAR_LBO;
   static constexpr int OFF_FAR = OFF_OST + 2 * C * COLS * ES;  // 2 x { hi, lo }
   static constexpr int OFF_P0 = OFF_FAR + 2 * 2 * FAR_TILE;  // [C/4][NROW] float4: a chunk's P0 rows, kept for the rare redo
-  static constexpr int OFF_BAR = OFF_P0 + C * NROW * 4;
+  static constexpr int OFF_RP = OFF_P0 + C * NROW * 4;  // Temporal: [NROW] fp32, a piece's initial r_prev, helpers -> row warps
+  static constexpr int OFF_BAR = OFF_RP + (TEMPORAL ? NROW * 4 : 0);
   static constexpr int SMEM_BYTES = OFF_BAR + 128 + 1024;  // + 1024: the kernel aligns its window to 1024 bytes
+  static_assert(R_GK % 128 == 0 && RQ_GQ % 128 == 0, "temporal gate rows start 128-byte aligned");
   static_assert(RAW_BYTES % 128 == 0 && RPQ_BYTES % 128 == 0 && R_B % 128 == 0 && R_PK % 128 == 0 && OFF_RAW % 128 == 0 &&
                     OFF_RPQ % 128 == 0 && OFF_TILE % 1024 == 0 && OFF_KU % 1024 == 0 && KU_BYTES % 1024 == 0 && DK % 64 == 0 && (COLS * ES) % 16 == 0 && (GROW * ES) % 16 == 0,
                 "destinations of the tensor copies are 128-byte aligned, their rows multiples of 16 bytes");
@@ -202,6 +212,7 @@ __device__ __forceinline__ void bf16_split3(float x0, float x1, uint32_t &hi, ui
 // Tensor maps of the six streamed inputs (built by the host for every launch), see chunk_make_maps.
 struct ChunkMaps {
   CUtensorMap k, q, v, be, pk, pq;
+  CUtensorMap gk, gq;  // Temporal only
 };
 
 // Staging of chunk m of a piece by ONE thread: tiled bulk tensor copies (TMA) straight into the operand tile (k, q:
@@ -225,6 +236,10 @@ __device__ __forceinline__ void chunk_stage(const ChunkMaps &maps, unsigned char
   tma_load_4d(raw + Cf::R_B, &maps.be, col0, 0, tok, bh, bar);
   tma_load_4d(raw + Cf::R_PK, &maps.pk, col0, 0, tok, bh, bar);
   tma_load_4d(rawpq, &maps.pq, col0, 0, tok, bh, bar);
+  if constexpr (Cf::TEMPORAL) {
+    tma_load_3d(raw + Cf::R_GK, &maps.gk, col0, tok, bh, bar);
+    tma_load_3d(rawpq + Cf::RQ_GQ, &maps.gq, col0, tok, bh, bar);
+  }
 }
 
 // RDEBUG: the auxiliary instantiation, which also writes the responsibilities (p.r_debug) and / or adds the sums
@@ -236,6 +251,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
                                                                      const __grid_constant__ ChunkMaps maps) {
   using namespace umma;
   constexpr int J = Cf::J, DK = Cf::DK, C = Cf::C, NROW = Cf::NROW, COLS = Cf::COLS;
+  static_assert(!(RDEBUG && Cf::TEMPORAL), "the auxiliary outputs of the Temporal variant come from the scan kernel");
   extern __shared__ __align__(128) unsigned char smem_raw[];
   // the swizzled operand tile needs a 1024-byte aligned shared-memory address
   unsigned char *smem = smem_raw + ((1024u - (umma::smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -323,6 +339,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
 
   // outputs of one chunk (Eq. 3.5): o_td = sum_j pi^q_j (w_t.q_t)_j, pi^q = softmax over the J
   // components of a column
+  [[maybe_unused]] float rho_run = 1.0f / J;  // helper lanes, Temporal: running average of the query-side prior (App. B.3)
   [[maybe_unused]] float sq_sum[J], sq_ent = 0.f;  // helper lanes, auxiliary instantiation: slot c = component j ^ pattern(c)
 #pragma unroll
   for (int c = 0; c < J; ++c) sq_sum[c] = 0.f;
@@ -341,6 +358,29 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       float hq[8];
       tmem_ld8(tb + Cf::TM_QD + (n & 1) * C + tg, hq);
       tmem_ld_wait();
+      if constexpr (Cf::TEMPORAL) {
+        // readout weight of this lane's own component: rho_t = (1 - g) rho_{t-1} + g pi^q_t, g = sigmoid(gq logit),
+        // a running average along the tokens, so it is applied before the transposition
+        const __nv_bfloat16 *rgq = reinterpret_cast<const __nv_bfloat16 *>(reinterpret_cast<const unsigned char *>(rpq) + Cf::RQ_GQ);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int t = tg + i;
+          float x[J], mx = -3.0e38f;
+#pragma unroll
+          for (int jj = 0; jj < J; ++jj) {
+            x[jj] = __bfloat162float(rpq[(t * J + jj) * Cf::GROW + dl]) * kLog2e;
+            mx = fmaxf(mx, x[jj]);
+          }
+          float se = 0.f;
+#pragma unroll
+          for (int jj = 0; jj < J; ++jj) se += ex2_approx(x[jj] - mx);
+          const float own = __bfloat162float(rpq[(t * J + j) * Cf::GROW + dl]) * kLog2e;
+          const float pq = ex2_approx(own - mx) * rcp_approx(se);
+          const float gq = sigmoid_approx(__bfloat162float(rgq[t * COLS + dl]));
+          if (t < nvalid) rho_run = fmaf(gq, pq - rho_run, rho_run);
+          hq[i] *= rho_run;
+        }
+      }
 #pragma unroll
       for (int rd = 0; rd < LJ; ++rd) {
         const int nrem = 3 - rd;              // token bits still in the index
@@ -366,6 +406,13 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
 #pragma unroll
       for (int rest = 0; rest < (8 >> LJ); ++rest) {
         const int tl = tg + (j << (3 - LJ)) + rest;
+        if constexpr (Cf::TEMPORAL) {  // the readouts arrive weighted: the output is their plain sum over the components
+          float so = 0.f;
+#pragma unroll
+          for (int c = 0; c < J; ++c) so += hq[(c << (3 - LJ)) | rest];
+          ost[tl * COLS + dl] = __float2bfloat16_rn(so);
+          continue;
+        }
         float x[J];
         [[maybe_unused]] float ex[J];
         float mx = -3.0e38f;
@@ -418,6 +465,8 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     const int jbase = lane - j;
     [[maybe_unused]] float st_r = 0.f, st_h = 0.f;  // auxiliary instantiation: this piece's sums over time
     if (!mbar_wait(&bars[B_BE], 0) || !mbar_wait(&bars[B_GS], 0)) failed = true;
+    [[maybe_unused]] float rprev = 1.0f / J;  // Temporal: this row's previous responsibility r_{t-1} (App. B.3)
+    if constexpr (Cf::TEMPORAL) rprev = reinterpret_cast<const float *>(smem + Cf::OFF_RP)[r];
 #pragma unroll 1
     for (int n = 0; n < nchunks && !failed; ++n) {
       const int t0 = n * C;
@@ -426,6 +475,8 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       const __nv_bfloat16 *rv = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_V);
       const float *bes = reinterpret_cast<const float *>(raw + Cf::R_B);
       const __nv_bfloat16 *rpk = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_PK);
+      [[maybe_unused]] const float *pks = reinterpret_cast<const float *>(raw + Cf::R_PK);            // Temporal: normalised prior
+      [[maybe_unused]] const __nv_bfloat16 *rgk = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_GK);  // Temporal: gate logits
       const float *Gkk = G_all + (n & 1) * C * C;
 
       PROF_ADD(0);
@@ -460,8 +511,10 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       //      any normaliser left the safe range (all components > ~13 standard deviations off, or extreme
       //      prior logits), in which case the chunk is redone with the maximum subtracted. ----
       [[maybe_unused]] float chunk_r = 0.f, chunk_h = 0.f;  // written by the pass whose results stand
-      auto sequential = [&](auto exact_tag) -> bool {
+      [[maybe_unused]] float chunk_rp = 0.f;                 // Temporal: r of the chunk's last token, likewise
+      auto sequential = [&](auto exact_tag, [[maybe_unused]] const float rp_in) -> bool {
         constexpr bool EXACT = decltype(exact_tag)::value;
+        [[maybe_unused]] float rp = rp_in;
         constexpr int GT = Cf::GT;
         bool bad = false;
         [[maybe_unused]] float cr = 0.f, ch = 0.f;  // auxiliary instantiation: this chunk's sums of r and of r log2 r
@@ -501,7 +554,16 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
             const float be = bes[t * NROW + r];
             // serial chain: prediction error -> responsibilities (Eq. 3.4) -> update coefficient (Eq. 3.3)
             const float delta = pred[i];
-            const float a = fmaf(-kHalfLog2e * delta, delta, __bfloat162float(rpk[(t * J + j) * Cf::GROW + dl]) * kLog2e);
+            float a;
+            if constexpr (Cf::TEMPORAL) {
+              // key-side prior (1 - g) r_{t-1} + g pi^k with g = sigmoid(gk logit) (App. B.3): a convex combination of
+              // two distributions over j, so it needs no further normalisation
+              const float gk = sigmoid_approx(__bfloat162float(rgk[t * COLS + dl]));
+              const float prior = fmaf(gk, pks[t * NROW + r] - rp, rp);
+              a = fmaf(-kHalfLog2e * delta, delta, lg2_approx(prior));
+            } else {
+              a = fmaf(-kHalfLog2e * delta, delta, __bfloat162float(rpk[(t * J + j) * Cf::GROW + dl]) * kLog2e);
+            }
             float e, sum;
             if constexpr (EXACT) {
               float all[J];
@@ -541,6 +603,9 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
             }
             const float rs = rcp_approx(sum);
             float c = ((be * delta) * e) * rs;  // beta r delta with one multiplication after the reciprocal
+            if constexpr (Cf::TEMPORAL) {
+              if (t < nvalid) rp = e * rs;
+            }
             if (t >= nvalid) c = 0.f;  // padding tokens of the last chunk leave the state alone
             cs[i] = c;
             if constexpr (RDEBUG) {
@@ -589,9 +654,10 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
           }
         }
         if constexpr (RDEBUG) { chunk_r = cr; chunk_h = ch; }
+        if constexpr (Cf::TEMPORAL) chunk_rp = rp;
         return bad;
       };
-      const bool unsafe = sequential(std::false_type{});
+      const bool unsafe = sequential(std::false_type{}, rprev);
       PROF_ADD(5);
       if (__any_sync(0xffffffffu, unsafe)) {
         tmem_st_wait();
@@ -600,8 +666,9 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
           const float4 v4 = p0s[i * NROW + r];
           pred0[4 * i] = v4.x; pred0[4 * i + 1] = v4.y; pred0[4 * i + 2] = v4.z; pred0[4 * i + 3] = v4.w;
         }
-        sequential(std::true_type{});
+        sequential(std::true_type{}, rprev);
       }
+      if constexpr (Cf::TEMPORAL) rprev = chunk_rp;
       if constexpr (RDEBUG) { st_r += chunk_r; st_h += chunk_h; }
       tmem_st_wait();
       tc_fence_before_sync();
@@ -636,9 +703,13 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         if (p.r_ent) atomicAdd(p.r_ent + (size_t)bh * p.Dv + col, -st_h * kLn2);
       }
     }
+    if constexpr (Cf::TEMPORAL) {
+      if (!failed && p.r_out && col_ok) p.r_out[((size_t)bh * J + j) * p.Dv + col] = rprev;
+    }
     if (to_flag) {  // the rest of this tile belongs to another block: publish the state
       __threadfence();
-      named_bar_sync(4, 128);
+      if constexpr (Cf::TEMPORAL) named_bar_sync(5, 256);  // ... the helpers' part of it included
+      else named_bar_sync(4, 128);
       if (r == 0 && !failed) st_release_gpu(flag, sched.epoch);
     }
   } else if (warp < 8) {
@@ -660,6 +731,33 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         named_bar_sync(3, 128);
 #pragma unroll
         for (int i = 0; i < 8; ++i) bes[(t8 + i) * NROW + h] = be[i];
+      }
+    };
+    // Temporal: the key-side prior pi^k = softmax over the J components (App. B.2) of this helper's row for every token
+    // of a raw stage, written over the logits as fp32 [C][NROW] in the same rolled, last-tokens-first passes as beta
+    [[maybe_unused]] auto cook_pk = [&](unsigned char *raw) {
+      const __nv_bfloat16 *rk = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_PK);
+      float *pks = reinterpret_cast<float *>(raw + Cf::R_PK);
+#pragma unroll 1
+      for (int t8 = C - 8; t8 >= 0; t8 -= 8) {
+        float pk[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          float x[J], mx = -3.0e38f;
+#pragma unroll
+          for (int jj = 0; jj < J; ++jj) {
+            x[jj] = __bfloat162float(rk[((t8 + i) * J + jj) * Cf::GROW + dl]) * kLog2e;
+            mx = fmaxf(mx, x[jj]);
+          }
+          float se = 0.f;
+#pragma unroll
+          for (int jj = 0; jj < J; ++jj) se += ex2_approx(x[jj] - mx);
+          const float own = __bfloat162float(rk[((t8 + i) * J + j) * Cf::GROW + dl]) * kLog2e;
+          pk[i] = ex2_approx(own - mx) * rcp_approx(se);
+        }
+        named_bar_sync(3, 128);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) pks[(t8 + i) * NROW + h] = pk[i];
       }
     };
     // operand parts of W after an update, this helper's tensor-memory lane
@@ -770,6 +868,19 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       named_bar_sync(1, 128);
       if (*fail_s) failed = true;
     }
+    if constexpr (Cf::TEMPORAL) {
+      // carried distributions of this helper's row (App. B.3): r_prev goes to the row warps through shared memory
+      // (published with the first gates, barrier BE), rho_prev stays here
+      const float *r_src = from_flag ? p.r_out : p.r_in, *q_src = from_flag ? p.rho_out : p.rho_in;
+      float rp = 1.0f / J;
+      rho_run = 1.0f / J;
+      if (col_ok && !failed) {
+        const size_t idx = ((size_t)bh * J + j) * p.Dv + col;
+        if (r_src) rp = __ldcg(r_src + idx);
+        if (q_src) rho_run = __ldcg(q_src + idx);
+      }
+      reinterpret_cast<float *>(smem + Cf::OFF_RP)[h] = rp;
+    }
     {
       const float *w_src = from_flag ? p.W_out : p.W_in;
       const float *src = (w_src && col_ok && !failed) ? w_src + (((size_t)bh * J + j) * p.Dv + col) * DK : nullptr;
@@ -811,6 +922,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     }
     if (!staged(0)) failed = true;
     cook_be(smem + Cf::OFF_RAW);
+    if constexpr (Cf::TEMPORAL) cook_pk(smem + Cf::OFF_RAW);
     mbar_arrive(&bars[B_BE]);
     if (spill_mine[0]) {
       if (!mbar_wait(&bars[B_G], 0)) failed = true;
@@ -828,6 +940,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         // (1) gates of chunk n+1 for the row warps, then its Gram batch
         if (!staged(n + 1)) { failed = true; break; }
         cook_be(smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES);
+        if constexpr (Cf::TEMPORAL) cook_pk(smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES);
         mbar_arrive(&bars[B_BE]);
         PROF_ADD(1);
         if (spill_mine[(n + 1) & 1]) {
@@ -862,6 +975,13 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     }
     if (!failed && !mbar_wait(&bars[B_QD], (nchunks - 1) & 1)) failed = true;
     if (!failed) write_outputs(nchunks - 1);
+    if constexpr (Cf::TEMPORAL) {
+      if (!failed && p.rho_out && col_ok) p.rho_out[((size_t)bh * J + j) * p.Dv + col] = rho_run;
+      if (to_flag) {  // the row warps publish the hand-over flag once both roles have stored their carried state
+        __threadfence();
+        named_bar_sync(5, 256);
+      }
+    }
     if constexpr (RDEBUG) {
       // this piece's sums of the readout weights: the J lanes of a column hold disjoint tokens, and other pieces of
       // the tile may run in other blocks, hence atomic additions
@@ -1061,6 +1181,10 @@ bool chunk_make_maps(const ScanParams &p, ChunkMaps *m) {
     const cuuint64_t strides[2] = {Dv * 2, T * Dv * 2};
     const cuuint32_t box[3] = {(cuuint32_t)Cf::COLS, (cuuint32_t)Cf::C, 1};
     if (!chunk_encode(&m->v, p.v, 3, dims, strides, box)) return false;
+    if constexpr (Cf::TEMPORAL) {
+      if (!chunk_encode(&m->gk, p.gk_logit, 3, dims, strides, box) || !chunk_encode(&m->gq, p.gq_logit, 3, dims, strides, box))
+        return false;
+    }
   }
   {
     const cuuint64_t dims[4] = {Dv, J, T, BH};
@@ -1090,11 +1214,15 @@ inline unsigned chunk_next_epoch() {
   return e;
 }
 
-template <int J, int DK>
+template <int J, int DK, bool TEMPORAL = false>
 int launch_chunk(const LaunchArgs &a) {
-  using Cf = ChunkCfg<J, DK>;
+  using Cf = ChunkCfg<J, DK, TEMPORAL>;
   const bool aux = a.p.r_debug || a.p.r_sum || a.p.r_ent || a.p.rho_sum || a.p.rho_ent;
-  auto kern = aux ? swila_chunk_kernel<Cf, true> : swila_chunk_kernel<Cf, false>;
+  if (TEMPORAL && aux) return -1000;  // the Temporal variant's auxiliary outputs come from the scan kernel
+  auto kern = swila_chunk_kernel<Cf, false>;
+  if constexpr (!TEMPORAL) {
+    if (aux) kern = swila_chunk_kernel<Cf, true>;
+  }
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cf::SMEM_BYTES);
   if (e != cudaSuccess) return (int)e;
   const long long nslice = (a.p.Dv + Cf::COLS - 1) / Cf::COLS;
@@ -1110,7 +1238,8 @@ int launch_chunk(const LaunchArgs &a) {
   // tiles, so that the last wave is not half empty (chunk_plan).  The state of a split tile travels through the
   // state output, hence only when that is given; blocks of such a launch wait for each other, hence the
   // cooperative launch (all blocks resident or no launch at all).
-  const ChunkPlan pl = chunk_plan((long long)a.p.B * a.p.H, nslice, nch, chunk_sm_count(), a.p.W_out != nullptr, kChunkFlagTiles);
+  const ChunkPlan pl = chunk_plan((long long)a.p.B * a.p.H, nslice, nch, chunk_sm_count(),
+                                   a.p.W_out != nullptr && (!TEMPORAL || (a.p.r_out && a.p.rho_out)), kChunkFlagTiles);
   if (pl.split) {
     unsigned *flags = nullptr;
     if (cudaGetSymbolAddress((void **)&flags, g_chunk_flags) == cudaSuccess) {

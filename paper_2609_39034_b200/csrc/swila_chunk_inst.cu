@@ -1,4 +1,4 @@
-// Instantiations and dispatch of the chunked tensor-core kernel (bf16 io, ungated, non-temporal,
+// Instantiations and dispatch of the chunked tensor-core kernel (bf16 io, ungated, plain or Temporal,
 // J in {4, 8}: with fewer components a block covers more columns and its shared-memory tiles do not fit).
 #include "../../include/swila.h"
 #include "swila_chunk.cuh"
@@ -7,11 +7,11 @@ namespace swila {
 
 // Returns a cudaError_t value (>= 0), or -1000 when the combination is not compiled.
 int chunk_dispatch(const LaunchArgs &a) {
-  if (a.io_dtype != SWILA_IO_BF16 || a.gate_mode != 0 || a.p.temporal || a.p.qkv_act) return -1000;
-#define SWILA_CHUNK_CASE(JJ)                         \
-  case JJ:                                           \
-    if (a.Dk == 128) return launch_chunk<JJ, 128>(a); \
-    if (a.Dk == 64) return launch_chunk<JJ, 64>(a);   \
+  if (a.io_dtype != SWILA_IO_BF16 || a.gate_mode != 0 || a.p.qkv_act) return -1000;
+#define SWILA_CHUNK_CASE(JJ)                                                                   \
+  case JJ:                                                                                     \
+    if (a.Dk == 128) return a.p.temporal ? launch_chunk<JJ, 128, true>(a) : launch_chunk<JJ, 128>(a); \
+    if (a.Dk == 64) return a.p.temporal ? launch_chunk<JJ, 64, true>(a) : launch_chunk<JJ, 64>(a);   \
     return -1000;
   switch (a.J) {
     SWILA_CHUNK_CASE(4)

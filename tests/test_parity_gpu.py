@@ -5,7 +5,7 @@ import pytest
 import torch
 
 from paper_2609_39034_b200 import workloads as wl
-from tests._gpu_util import assert_close, gpu_forward, to_dev
+from tests._gpu_util import TOL_BF16_O, TOL_STATE, assert_close, gpu_forward, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -101,6 +101,45 @@ def test_chunked_tensor_core_kernel_matches_oracle(binding, oracle, w, stress):
     got = gpu_forward(binding, w, to_dev(inp), want_r=True, algo=binding.ALGO_CHUNK)
     binding.device_status()
     assert_close(w, got, ref, w.name)
+
+
+@pytest.mark.parametrize("w", CHUNK_SHAPES, ids=lambda w: w.name)
+@pytest.mark.parametrize("stress", [False, True], ids=["calm", "stress"])
+def test_chunked_kernel_temporal_matches_oracle(binding, oracle, w, stress):
+    """Temporal SwiLA (App. B.3) in the chunked kernel: the key-side prior mixes in the previous token's
+    responsibilities on the serial chain, the readout weights are a running average formed with the outputs;
+    both carried distributions enter and leave with the state."""
+    wt = w.variant(temporal=True)
+    inp = wl.make_inputs(wt, stress=stress)
+    ref = oracle.forward_inputs(inp, flags=wt.flags)
+    got = gpu_forward(binding, wt, to_dev(inp), algo=binding.ALGO_CHUNK)
+    binding.device_status()
+    assert_close(wt, got, ref, wt.name)
+
+
+def test_chunked_kernel_temporal_in_pieces_and_decode(binding, oracle):
+    """A Temporal sequence fed to the chunked kernel in two calls with the state carried (W, r_prev, rho_prev), then
+    decode steps (scan kernel) on that state: the whole must equal one oracle pass over all tokens."""
+    w = SMALL[4].variant(temporal=True).with_(T=200)
+    inp = wl.make_inputs(w, stress=True)
+    ref = oracle.forward_inputs(inp, flags=w.flags)
+    dev = to_dev(inp)
+    cut = 96
+    part = lambda a, b: {k: (v[:, :, a:b].contiguous() if v is not None and k not in ("W0", "r0", "rho0") else v)  # noqa: E731
+                         for k, v in dev.items()}
+    st = {"W": dev["W0"].clone(), "r_prev": dev["r0"].clone(), "rho_prev": dev["rho0"].clone()}
+    o1 = binding.swila_forward(w, part(0, cut), state_in=st, state_out=st, algo=binding.ALGO_CHUNK)
+    o2 = binding.swila_forward(w, part(cut, 190), state_in=st, state_out=st, algo=binding.ALGO_CHUNK)
+    outs = [o1, o2]
+    for t in range(190, 200):
+        outs.append(binding.swila_decode_step(w, part(t, t + 1), st))
+    torch.cuda.synchronize()
+    binding.device_status()
+    o = torch.cat(outs, dim=2).cpu()
+    assert wl.rel_err(o, torch.from_numpy(ref["o"])) < TOL_BF16_O
+    assert wl.rel_err(st["W"].cpu(), torch.from_numpy(ref["W"])) < TOL_STATE
+    assert wl.rel_err(st["r_prev"].cpu(), torch.from_numpy(ref["r_prev"])) < TOL_STATE
+    assert wl.rel_err(st["rho_prev"].cpu(), torch.from_numpy(ref["rho_prev"])) < TOL_STATE
 
 
 def test_chunked_kernel_extreme_prediction_errors(binding, oracle):
