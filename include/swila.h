@@ -79,7 +79,8 @@ enum {
                               on the tcgen05 tensor cores (bf16 hi/lo operand split, FP32
                               accumulation in tensor memory), the E-step and intra-chunk
                               corrections on the FP32 ALUs.  bf16 io, Dk in {64, 128}, J in {4, 8},
-                              no TEMPORAL / GATED.  When a state output is given and the tiles do
+                              plain or TEMPORAL (the latter without r_debug / statistics), no GATED,
+                              no QKV_ACT.  When a state output is given and the tiles do
                               not fill a whole number of waves, the launch is cooperative and
                               balances chunks over the SMs; up to 8 such launches may overlap on
                               one device */

@@ -204,3 +204,33 @@ def test_calls_replay_from_a_cuda_graph(binding):
         torch.cuda.synchronize()
         binding.device_status()
         assert torch.equal(got[0], o) and torch.equal(got[1], o1) and torch.equal(got[2], st["W"]), rep
+
+
+@pytest.mark.parametrize("shape", ["headline", "more_tiles_than_sms"])
+def test_temporal_prefill_sampled(binding, oracle, shape):
+    """Temporal SwiLA (App. B.3) at full size through the default dispatch (chunked kernel): the LM-shaped
+    configuration, and a shape whose tiles are split between blocks, so that W, r_prev and rho_prev of a split tile
+    travel through the state output and the hand-over flag.  Sampled rows are replayed by the oracle; the whole
+    state is compared with the scan kernel's."""
+    base = wl.CONFIGS[2] if shape == "headline" else wl.CONFIGS[2].with_(B=2, H=20, T=1024)
+    w = base.variant(temporal=True)
+    inp = wl.make_inputs(w, device="cuda", stress=True)
+    sin = {"W": inp["W0"], "r_prev": inp["r0"], "rho_prev": inp["rho0"]}
+    st = binding.state_alloc(w, init=False)
+    o = binding.swila_forward(w, inp, state_in=sin, state_out=st)
+    st_scan = binding.state_alloc(w, init=False)
+    o_scan = binding.swila_forward(w, inp, state_in=sin, state_out=st_scan, algo=binding.ALGO_SCAN)
+    torch.cuda.synchronize()
+    binding.device_status()
+    assert wl.rel_err(o.float().cpu(), o_scan.float().cpu()) < TOL_BF16_O
+    for name in ("W", "r_prev", "rho_prev"):
+        # two kernels, each held to the tolerance against the oracle below: against each other, twice that
+        assert wl.rel_err(st[name].cpu(), st_scan[name].cpu()) < 2 * TOL_STATE, name
+    bh, cols = _sample(w, 4, 8, seed=21)
+    sub = wl.slice_rows(inp, bh.cuda(), cols.cuda())
+    ref = oracle.forward_inputs({n: (x.cpu() if x is not None else None) for n, x in sub.items()}, flags=w.flags)
+    pick = lambda x: x.reshape((w.B * w.H,) + tuple(x.shape[2:]))[bh.cuda()]  # noqa: E731
+    assert wl.rel_err(pick(o)[..., cols.cuda()].unsqueeze(1).cpu(), torch.from_numpy(ref["o"])) < TOL_BF16_O
+    assert wl.rel_err(pick(st["W"])[:, :, cols.cuda()].unsqueeze(1).cpu(), torch.from_numpy(ref["W"])) < TOL_STATE
+    for name in ("r_prev", "rho_prev"):
+        assert wl.rel_err(pick(st[name])[..., cols.cuda()].unsqueeze(1).cpu(), torch.from_numpy(ref[name])) < TOL_STATE, name
