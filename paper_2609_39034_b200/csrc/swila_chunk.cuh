@@ -371,11 +371,12 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
             x[jj] = __bfloat162float(rpq[(t * J + jj) * Cf::GROW + dl]) * kLog2e;
             mx = fmaxf(mx, x[jj]);
           }
-          float se = 0.f;
-#pragma unroll
-          for (int jj = 0; jj < J; ++jj) se += ex2_approx(x[jj] - mx);
           const float own = __bfloat162float(rpq[(t * J + j) * Cf::GROW + dl]) * kLog2e;
-          const float pq = ex2_approx(own - mx) * rcp_approx(se);
+          const float eo = ex2_approx(own - mx);
+          float se = eo;
+#pragma unroll
+          for (int off = 1; off < J; off <<= 1) se += __shfl_xor_sync(0xffffffffu, se, off);
+          const float pq = eo * rcp_approx(se);
           const float gq = sigmoid_approx(__bfloat162float(rgq[t * COLS + dl]));
           if (t < nvalid) rho_run = fmaf(gq, pq - rho_run, rho_run);
           hq[i] *= rho_run;
@@ -749,11 +750,13 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
             x[jj] = __bfloat162float(rk[((t8 + i) * J + jj) * Cf::GROW + dl]) * kLog2e;
             mx = fmaxf(mx, x[jj]);
           }
-          float se = 0.f;
-#pragma unroll
-          for (int jj = 0; jj < J; ++jj) se += ex2_approx(x[jj] - mx);
+          // every lane of the column's J-lane group takes one exponential; the normaliser is their sum
           const float own = __bfloat162float(rk[((t8 + i) * J + j) * Cf::GROW + dl]) * kLog2e;
-          pk[i] = ex2_approx(own - mx) * rcp_approx(se);
+          const float eo = ex2_approx(own - mx);
+          float se = eo;
+#pragma unroll
+          for (int off = 1; off < J; off <<= 1) se += __shfl_xor_sync(0xffffffffu, se, off);
+          pk[i] = eo * rcp_approx(se);
         }
         named_bar_sync(3, 128);
 #pragma unroll
