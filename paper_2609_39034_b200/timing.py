@@ -20,8 +20,8 @@ from . import workloads as wl
 ALGOS = {"auto": binding.ALGO_AUTO, "scan": binding.ALGO_SCAN, "chunk": binding.ALGO_CHUNK}
 
 
-def time_config(index: int, algo: int, launches: int = 7, warmup: int = 3):
-    w = wl.CONFIGS[index]
+def time_config(index: int, algo: int, launches: int = 7, warmup: int = 3, temporal: bool = False):
+    w = wl.CONFIGS[index].variant(temporal=temporal)
     inp = wl.make_inputs(w, device="cuda")
     state = binding.state_alloc(w)
     o = torch.empty((w.B, w.H, w.T, w.Dv), device="cuda", dtype=w.torch_io_dtype)
@@ -71,6 +71,7 @@ def main():
     ap.add_argument("--algo", choices=sorted(ALGOS), default="auto")
     ap.add_argument("--launches", type=int, default=7)
     ap.add_argument("--norm", action="store_true", help="time swila_output_norm instead of swila_forward")
+    ap.add_argument("--temporal", action="store_true", help="the Temporal variant (App. B.3) of the configurations")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         raise SystemExit("a CUDA device is required")
@@ -79,8 +80,8 @@ def main():
         print(f"config {index} x4 ({w.B}x{w.H}x{w.T}x{w.Dv} {w.io_dtype}) output norm: min {t_min:.4f} ms, median "
               f"{t_med:.4f} ms, {nbytes / t_min * 1e3 / 1e9:.0f} GB/s (read + write)", flush=True)
     for index in [] if args.norm else args.configs:
-        w, t_min, t_med = time_config(index, ALGOS[args.algo], args.launches)
-        print(f"config {index} ({w.name}) {args.algo}: min {t_min:.3f} ms, median {t_med:.3f} ms, "
+        w, t_min, t_med = time_config(index, ALGOS[args.algo], args.launches, temporal=args.temporal)
+        print(f"config {index} ({w.name}{' temporal' if args.temporal else ''}) {args.algo}: min {t_min:.3f} ms, median {t_med:.3f} ms, "
               f"{w.B * w.T / t_min * 1e3 / 1e6:.2f} M tokens/s", flush=True)
 
 
