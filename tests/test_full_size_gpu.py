@@ -164,21 +164,23 @@ def test_long_sequence_from_zero_state(binding, oracle, algo):
     assert wl.rel_err(got["W"], torch.from_numpy(ref["W"])) < TOL_STATE
 
 
-def test_calls_replay_from_a_cuda_graph(binding):
+@pytest.mark.parametrize("temporal", [False, True], ids=["vanilla", "temporal"])
+def test_calls_replay_from_a_cuda_graph(binding, temporal):
     """A prefill on the balanced schedule (cooperative launch, state handed over between blocks through flags that
     carry the launch's epoch) and a decode step, captured once in a CUDA graph and replayed on fresh inputs: every
     replay must equal the eager call on the same inputs.  A replay reuses the captured epoch, so the hand-over flags
     must not keep last replay's value."""
-    w = wl.CONFIGS[2].with_(B=2, H=20, T=1024)
-    inp = wl.make_inputs(w, device="cuda")
+    w = wl.CONFIGS[2].with_(B=2, H=20, T=1024).variant(temporal=temporal)
+    inp = wl.make_inputs(w, device="cuda", stress=True)
     st = binding.state_alloc(w, init=False)
     o = torch.empty((w.B, w.H, w.T, w.Dv), device="cuda", dtype=w.torch_io_dtype)
     w1 = w.with_(T=1)
+    sin = {"W": inp["W0"], "r_prev": inp.get("r0"), "rho_prev": inp.get("rho0")}
     step = wl.decode_step_inputs(w, 0, device="cuda")
     o1 = torch.empty((w.B, w.H, 1, w.Dv), device="cuda", dtype=w.torch_io_dtype)
 
     def call():
-        binding.swila_forward(w, inp, state_in={"W": inp["W0"]}, state_out=st, o=o, algo=binding.ALGO_CHUNK)
+        binding.swila_forward(w, inp, state_in=sin, state_out=st, o=o, algo=binding.ALGO_CHUNK)
         binding.swila_decode_step(w1, step, st, o=o1)
 
     side = torch.cuda.Stream()
@@ -189,7 +191,7 @@ def test_calls_replay_from_a_cuda_graph(binding):
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph):
         call()
-    names = ("q", "k", "v", "beta_logit", "pik_logit", "piq_logit")
+    names = ("q", "k", "v", "beta_logit", "pik_logit", "piq_logit") + (("gk_logit", "gq_logit") if temporal else ())
     for rep in range(3):
         fresh = wl.make_inputs(w, device="cuda", seed_offset=rep + 1, stress=True)
         fresh_step = wl.decode_step_inputs(w, rep + 1, device="cuda")
@@ -197,13 +199,18 @@ def test_calls_replay_from_a_cuda_graph(binding):
             inp[n].copy_(fresh[n])
             step[n].copy_(fresh_step[n])
         inp["W0"].copy_(fresh["W0"])
+        if temporal:
+            inp["r0"].copy_(fresh["r0"])
+            inp["rho0"].copy_(fresh["rho0"])
         graph.replay()
         torch.cuda.synchronize()
-        got = (o.clone(), o1.clone(), st["W"].clone())
+        got = (o.clone(), o1.clone(), st["W"].clone()) + ((st["r_prev"].clone(), st["rho_prev"].clone()) if temporal else ())
         call()
         torch.cuda.synchronize()
         binding.device_status()
         assert torch.equal(got[0], o) and torch.equal(got[1], o1) and torch.equal(got[2], st["W"]), rep
+        if temporal:
+            assert torch.equal(got[3], st["r_prev"]) and torch.equal(got[4], st["rho_prev"]), rep
 
 
 @pytest.mark.parametrize("shape", ["headline", "more_tiles_than_sms"])
