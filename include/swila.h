@@ -78,7 +78,8 @@ enum {
   SWILA_ALGO_CHUNK = 4     /* chunked form: the state-times-token contractions of 32-token chunks
                               on the tcgen05 tensor cores (bf16 hi/lo operand split, FP32
                               accumulation in tensor memory), the E-step and intra-chunk
-                              corrections on the FP32 ALUs.  bf16 io, Dk in {64, 128}, J in {4, 8},
+                              corrections on the FP32 ALUs.  bf16 io, Dk in {64, 128}, J in {4, 8}
+                              (J = 16 at Dk = 64, without r_debug / statistics),
                               plain or TEMPORAL (the latter without r_debug / statistics), no GATED,
                               no QKV_ACT.  When a state output is given and the tiles do
                               not fill a whole number of waves, the launch is cooperative and

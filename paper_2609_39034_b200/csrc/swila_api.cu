@@ -116,7 +116,8 @@ static int run(const swila_shape_t *s, int T, const void *q, const void *k, cons
   // AUTO: the chunked tensor-core kernel whenever it applies and the sequence is long enough to
   // amortise its per-chunk set-up; the scan otherwise (fp32 io, GATED, decode, Temporal with auxiliary outputs).
   const bool chunk_ok = s->io_dtype == SWILA_IO_BF16 && (s->flags & ~SWILA_TEMPORAL) == 0 && (s->Dk == 64 || s->Dk == 128) &&
-                        (s->J == 4 || s->J == 8) &&
+                        (s->J == 4 || s->J == 8 || (s->J == 16 && s->Dk == 64 && !r_debug && !a.p.r_sum && !a.p.r_ent &&
+                                                     !a.p.rho_sum && !a.p.rho_ent)) &&
                         !(temporal && (r_debug || a.p.r_sum || a.p.r_ent || a.p.rho_sum || a.p.rho_ent));
   if (s->algo == SWILA_ALGO_CHUNK || (s->algo == SWILA_ALGO_AUTO && chunk_ok && T >= 64)) {
     rc = chunk_dispatch(a);

@@ -118,7 +118,8 @@ struct ChunkCfg {
                        TM_CL3 = TM_CLO + C / 2, TM_USED = TM_CL3 + C / 2;
   static constexpr int TM_ALLOC = 512;
   static_assert(TM_USED <= TM_ALLOC, "tensor memory budget");
-  static_assert(J == 4 || J == 8, "the output transposition assumes that J divides 8");
+  static_assert(J == 4 || J == 8 || (J == 16 && DK == 64),
+                "J = 4, 8: outputs by in-group transposition; J = 16: by shuffle sums, and only Dk = 64 fits shared memory");
   // K/Q operand tile (bf16, K-major, 128-byte swizzle): per half of 64 key dims, 128 rows of 128 bytes, rows
   // [K_even ; Q_even ; K_odd ; Q_odd]: the chunks of both parities side by side, so that one 128-row A operand
   // covers the keys of two consecutive chunks.  Key dim d of row r sits at
@@ -171,7 +172,8 @@ struct ChunkCfg {
   static constexpr int OFF_FAR = OFF_OST + 2 * C * COLS * ES;  // 2 x { hi, lo }
   static constexpr int OFF_P0 = OFF_FAR + 2 * 2 * FAR_TILE;  // [C/4][NROW] float4: a chunk's P0 rows, kept for the rare redo
   static constexpr int OFF_RP = OFF_P0 + C * NROW * 4;  // Temporal: [NROW] fp32, a piece's initial r_prev, helpers -> row warps
-  static constexpr int OFF_BAR = OFF_RP + (TEMPORAL ? NROW * 4 : 0);
+  static constexpr int OFF_OS = OFF_RP + (TEMPORAL ? NROW * 4 : 0);  // J = 16: [C][COLS][J] fp32, a chunk's readouts regrouped by output
+  static constexpr int OFF_BAR = OFF_OS + (J > 8 ? C * NROW * 4 : 0);
   static constexpr int SMEM_BYTES = OFF_BAR + 128 + 1024;  // + 1024: the kernel aligns its window to 1024 bytes
   static_assert(R_GK % 128 == 0 && RQ_GQ % 128 == 0, "temporal gate rows start 128-byte aligned");
   static_assert(RAW_BYTES % 128 == 0 && RPQ_BYTES % 128 == 0 && R_B % 128 == 0 && R_PK % 128 == 0 && OFF_RAW % 128 == 0 &&
@@ -252,6 +254,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   using namespace umma;
   constexpr int J = Cf::J, DK = Cf::DK, C = Cf::C, NROW = Cf::NROW, COLS = Cf::COLS;
   static_assert(!(RDEBUG && Cf::TEMPORAL), "the auxiliary outputs of the Temporal variant come from the scan kernel");
+  static_assert(!(RDEBUG && J > 8), "the auxiliary outputs for J = 16 come from the scan kernel");
   extern __shared__ __align__(128) unsigned char smem_raw[];
   // the swizzled operand tile needs a 1024-byte aligned shared-memory address
   unsigned char *smem = smem_raw + ((1024u - (umma::smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -382,6 +385,15 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
           hq[i] *= rho_run;
         }
       }
+      if constexpr (J > 8) {
+        // More components than tokens in a trip: no transposition inside the lane group.  The readouts (Temporal:
+        // already weighted) go to shared memory grouped by output, [token][column][component]: a warp's 32 lanes
+        // (2 columns x 16 components) write 32 consecutive floats per token; the outputs are formed below.
+        float *os = reinterpret_cast<float *>(smem + Cf::OFF_OS);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) os[((tg + i) * COLS + dl) * J + j] = hq[i];
+        continue;
+      }
 #pragma unroll
       for (int rd = 0; rd < LJ; ++rd) {
         const int nrem = 3 - rd;              // token bits still in the index
@@ -448,6 +460,42 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
             sq_ent += lg2_approx(se) - hb;
           }
         }
+      }
+    }
+    if constexpr (J > 8) {
+      // one thread per output (C x COLS = 256 of them): its J readouts are 4 vector loads, the softmax over the
+      // components of Eq. 3.5 is local (shuffle sums over 16 lanes cost several times as much)
+      named_bar_sync(2, 128);
+      const float *os = reinterpret_cast<const float *>(smem + Cf::OFF_OS);
+      for (int e = r; e < C * COLS; e += 128) {
+        const int t = e / COLS, d = e - t * COLS;
+        float val[J];
+#pragma unroll
+        for (int c4 = 0; c4 < J / 4; ++c4) {
+          const float4 v4 = *reinterpret_cast<const float4 *>(os + e * J + c4 * 4);
+          val[4 * c4] = v4.x; val[4 * c4 + 1] = v4.y; val[4 * c4 + 2] = v4.z; val[4 * c4 + 3] = v4.w;
+        }
+        float out = 0.f;
+        if constexpr (Cf::TEMPORAL) {
+#pragma unroll
+          for (int jj = 0; jj < J; ++jj) out += val[jj];
+        } else {
+          float x[J], mx = -3.0e38f;
+#pragma unroll
+          for (int jj = 0; jj < J; ++jj) {
+            x[jj] = __bfloat162float(rpq[(t * J + jj) * Cf::GROW + d]) * kLog2e;
+            mx = fmaxf(mx, x[jj]);
+          }
+          float se = 0.f;
+#pragma unroll
+          for (int jj = 0; jj < J; ++jj) {
+            const float ex = ex2_approx(x[jj] - mx);
+            se += ex;
+            out = fmaf(ex, val[jj], out);
+          }
+          out *= rcp_approx(se);
+        }
+        ost[t * COLS + d] = __float2bfloat16_rn(out);
       }
     }
     tc_fence_before_sync();
@@ -579,16 +627,22 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
               e = ex2_approx(a - m);
             } else {
               e = ex2_approx(a);
-              float part[J];  // the other components' terms arrive together: add them as a tree
-              part[0] = e;
+              if constexpr (J <= 8) {
+                float part[J];  // the other components' terms arrive together: add them as a tree
+                part[0] = e;
 #pragma unroll
-              for (int jj = 1; jj < J; ++jj) part[jj] = __shfl_sync(0xffffffffu, e, jbase + ((j + jj) & (J - 1)));
+                for (int jj = 1; jj < J; ++jj) part[jj] = __shfl_sync(0xffffffffu, e, jbase + ((j + jj) & (J - 1)));
 #pragma unroll
-              for (int w = J / 2; w >= 1; w /= 2) {
+                for (int w = J / 2; w >= 1; w /= 2) {
 #pragma unroll
-                for (int jj = 0; jj < w; ++jj) part[jj] += part[jj + w];
+                  for (int jj = 0; jj < w; ++jj) part[jj] += part[jj + w];
+                }
+                sum = part[0];
+              } else {  // 15 shuffles per token cost more than the latency of 4 dependent rounds
+                sum = e;
+#pragma unroll
+                for (int off = 1; off < J; off <<= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
               }
-              sum = part[0];
               bad = bad || !(sum > 1e-30f && sum < 1e30f);
             }
             {  // deferred push of token t-1 into the predictions of tokens t+1 .. (slots i+1 ..)
@@ -1222,8 +1276,9 @@ int launch_chunk(const LaunchArgs &a) {
   using Cf = ChunkCfg<J, DK, TEMPORAL>;
   const bool aux = a.p.r_debug || a.p.r_sum || a.p.r_ent || a.p.rho_sum || a.p.rho_ent;
   if (TEMPORAL && aux) return -1000;  // the Temporal variant's auxiliary outputs come from the scan kernel
+  if (J > 8 && aux) return -1000;     // likewise for J = 16
   auto kern = swila_chunk_kernel<Cf, false>;
-  if constexpr (!TEMPORAL) {
+  if constexpr (!TEMPORAL && J <= 8) {
     if (aux) kern = swila_chunk_kernel<Cf, true>;
   }
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cf::SMEM_BYTES);

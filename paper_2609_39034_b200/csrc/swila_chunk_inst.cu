@@ -1,5 +1,6 @@
 // Instantiations and dispatch of the chunked tensor-core kernel (bf16 io, ungated, plain or Temporal,
-// J in {4, 8}: with fewer components a block covers more columns and its shared-memory tiles do not fit).
+// J in {4, 8}, and 16 at Dk = 64: with fewer components a block covers more columns and its shared-memory tiles do
+// not fit).
 #include "../../include/swila.h"
 #include "swila_chunk.cuh"
 
@@ -16,6 +17,9 @@ int chunk_dispatch(const LaunchArgs &a) {
   switch (a.J) {
     SWILA_CHUNK_CASE(4)
     SWILA_CHUNK_CASE(8)
+    case 16:  // the component-count ablation of Sec. 5; only Dk = 64 fits shared memory
+      if (a.Dk == 64) return a.p.temporal ? launch_chunk<16, 64, true>(a) : launch_chunk<16, 64>(a);
+      return -1000;
     default: return -1000;
   }
 }
@@ -34,7 +38,7 @@ int chunk_error_fetch(int *flag) {
 extern "C" int swila_chunk_plan(int B, int H, int T, int Dv, int J, int sm_count, int has_state_out, long long out[6]) {
   if (!out) return SWILA_ERR_NULL;
   if (B <= 0 || H <= 0 || T <= 0 || Dv <= 0 || sm_count <= 0) return SWILA_ERR_SHAPE;
-  if (J != 4 && J != 8) return SWILA_ERR_UNSUPPORTED;
+  if (J != 4 && J != 8 && J != 16) return SWILA_ERR_UNSUPPORTED;
   const long long cols = 128 / J, nslice = (Dv + cols - 1) / cols, nch = (T + 31) / 32;
   const swila::ChunkPlan pl =
       swila::chunk_plan((long long)B * H, nslice, nch, sm_count, has_state_out != 0, swila::kChunkFlagTiles);

@@ -109,6 +109,17 @@ def test_paper_native_shapes(binding, oracle):
     bh, cols = _sample(lm, 8, 16, seed=11)
     _check_sample(lm, oracle, inp, o, st["W"], bh, cols, lm.name)
 
+    # the component-count ablation of Sec. 5: the same layer with J = 16 (chunked kernel, outputs formed per thread)
+    abl = lm.with_(name="lm374m_layer_j16", J=16)
+    inp = wl.make_inputs(abl, device="cuda", stress=True)
+    st = binding.state_alloc(abl, init=False)
+    o = binding.swila_forward(abl, inp, state_in={"W": inp["W0"]}, state_out=st)
+    torch.cuda.synchronize()
+    binding.device_status()
+    bh, cols = _sample(abl, 6, 12, seed=13)
+    _check_sample(abl, oracle, inp, o, st["W"], bh, cols, abl.name)
+    del inp, st, o
+
     gen = wl.CONFIGS[1].with_(name="generation", B=8, H=8, T=2048)
     bh, cols = _sample(gen, 8, 8, seed=12)
     prompt = wl.make_inputs(gen, device="cuda")
