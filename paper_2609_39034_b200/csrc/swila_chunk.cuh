@@ -661,7 +661,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
             if constexpr (Cf::TEMPORAL) {
               if (t < nvalid) rp = e * rs;
             }
-            if (t >= nvalid) c = 0.f;  // padding tokens of the last chunk leave the state alone
+            // (padding tokens of the last chunk have beta = 0 and leave the state alone)
             cs[i] = c;
             if constexpr (RDEBUG) {
               const float rr = e * rs;
@@ -774,7 +774,9 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     // logits, 8 tokens per pass (rolled: less code in the instruction cache), last tokens first: a token's FP32
     // row (512 bytes) lies further into the region than its logits (at most 384 bytes), so a pass overwrites only
     // logits of its own tokens -- which every helper has read by the barrier -- and of later, finished ones
-    auto cook_be = [&](unsigned char *raw) {
+    // Tokens past the end of the sequence (the last chunk's padding) get beta = 0: their update coefficient is then
+    // zero by itself and the row warps need no test on their serial chain.
+    auto cook_be = [&](unsigned char *raw, const int nvalid) {
       const __nv_bfloat16 *rb = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_B);
       float *bes = reinterpret_cast<float *>(raw + Cf::R_B);
       static_assert(J * Cf::GROW * Cf::ES <= NROW * 4, "a token's logits end before its FP32 row does");
@@ -782,7 +784,10 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       for (int t8 = C - 8; t8 >= 0; t8 -= 8) {
         float be[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) be[i] = sigmoid_approx(__bfloat162float(rb[((t8 + i) * J + j) * Cf::GROW + dl]));
+        for (int i = 0; i < 8; ++i) {
+          be[i] = sigmoid_approx(__bfloat162float(rb[((t8 + i) * J + j) * Cf::GROW + dl]));
+          if (t8 + i >= nvalid) be[i] = 0.f;
+        }
         named_bar_sync(3, 128);
 #pragma unroll
         for (int i = 0; i < 8; ++i) bes[(t8 + i) * NROW + h] = be[i];
@@ -978,7 +983,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         *reinterpret_cast<uint4 *>(tile + (e / (2 * C * 8)) * Cf::TILE_HALF + 2 * C * 128 + (e % (2 * C * 8)) * 16) = make_uint4(0, 0, 0, 0);
     }
     if (!staged(0)) failed = true;
-    cook_be(smem + Cf::OFF_RAW);
+    cook_be(smem + Cf::OFF_RAW, min(C, Tseg));
     if constexpr (Cf::TEMPORAL) cook_pk(smem + Cf::OFF_RAW);
     mbar_arrive(&bars[B_BE]);
     if (spill_mine[0]) {
@@ -996,7 +1001,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       if (more) {
         // (1) gates of chunk n+1 for the row warps, then its Gram batch
         if (!staged(n + 1)) { failed = true; break; }
-        cook_be(smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES);
+        cook_be(smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES, min(C, Tseg - (n + 1) * C));
         if constexpr (Cf::TEMPORAL) cook_pk(smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES);
         mbar_arrive(&bars[B_BE]);
         PROF_ADD(1);
