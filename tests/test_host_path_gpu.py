@@ -21,7 +21,8 @@ def _pin(inp):
     return {n: (x.pin_memory() if x is not None else None) for n, x in inp.items()}
 
 
-@pytest.mark.parametrize("var", [dict(), dict(temporal=True, gated=True)], ids=["vanilla", "gated_temporal"])
+@pytest.mark.parametrize("var", [dict(), dict(temporal=True), dict(temporal=True, gated=True)],
+                         ids=["vanilla", "temporal", "gated_temporal"])
 def test_host_entry_equals_device_entry(binding, oracle, var):
     w = wl.CONFIGS[1].with_(B=2, H=3, T=75).variant(**var)
     inp = wl.make_inputs(w, stress=True)
@@ -50,7 +51,8 @@ def test_host_entry_rejects_a_small_workspace(binding):
     assert e.value.status == binding.ERR_SIZE
 
 
-@pytest.mark.parametrize("var,T", [(dict(), 2304), (dict(temporal=True, gated=True), 1400)], ids=["vanilla", "gated_temporal"])
+@pytest.mark.parametrize("var,T", [(dict(), 2304), (dict(temporal=True), 2304), (dict(temporal=True, gated=True), 1400)],
+                         ids=["vanilla", "temporal", "gated_temporal"])
 def test_host_entry_in_slabs_equals_device_entry(binding, var, T):
     """Problems of 64 MB and more go through in slabs of (batch, head) pairs over internal copy streams; with 15
     pairs the 8 slabs are uneven.  The results must be those of one call on device tensors."""
