@@ -793,33 +793,47 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         for (int i = 0; i < 8; ++i) bes[(t8 + i) * NROW + h] = be[i];
       }
     };
-    // Temporal: the key-side prior pi^k = softmax over the J components (App. B.2) of this helper's row for every token
-    // of a raw stage, written over the logits as fp32 [C][NROW] in the same rolled, last-tokens-first passes as beta
+    // Temporal: the key-side prior pi^k = softmax over the J components (App. B.2), written over the logits as fp32
+    // [C][NROW] in the same rolled, last-tokens-first passes as beta.  The J lanes of a column share the work by
+    // token: a lane takes the whole softmax of 8 / J tokens of the pass and writes all J values of each (one or two
+    // 16-byte stores), instead of every lane taking one exponential of every token plus a shuffle sum.
     [[maybe_unused]] auto cook_pk = [&](unsigned char *raw) {
       const __nv_bfloat16 *rk = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_PK);
       float *pks = reinterpret_cast<float *>(raw + Cf::R_PK);
+      constexpr int TPL = (J <= 8) ? 8 / J : 1;  // tokens per lane and pass (J = 16: lanes 8..15 of a column idle)
 #pragma unroll 1
       for (int t8 = C - 8; t8 >= 0; t8 -= 8) {
-        float pk[8];
+        float pk[TPL][J];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          float x[J], mx = -3.0e38f;
+        for (int i = 0; i < TPL; ++i) {
+          const int t = t8 + (j * TPL + i) % 8;
+          float mx = -3.0e38f;
 #pragma unroll
           for (int jj = 0; jj < J; ++jj) {
-            x[jj] = __bfloat162float(rk[((t8 + i) * J + jj) * Cf::GROW + dl]) * kLog2e;
-            mx = fmaxf(mx, x[jj]);
+            pk[i][jj] = __bfloat162float(rk[(t * J + jj) * Cf::GROW + dl]) * kLog2e;
+            mx = fmaxf(mx, pk[i][jj]);
           }
-          // every lane of the column's J-lane group takes one exponential; the normaliser is their sum
-          const float own = __bfloat162float(rk[((t8 + i) * J + j) * Cf::GROW + dl]) * kLog2e;
-          const float eo = ex2_approx(own - mx);
-          float se = eo;
+          float se = 0.f;
 #pragma unroll
-          for (int off = 1; off < J; off <<= 1) se += __shfl_xor_sync(0xffffffffu, se, off);
-          pk[i] = eo * rcp_approx(se);
+          for (int jj = 0; jj < J; ++jj) {
+            pk[i][jj] = ex2_approx(pk[i][jj] - mx);
+            se += pk[i][jj];
+          }
+          const float inv = rcp_approx(se);
+#pragma unroll
+          for (int jj = 0; jj < J; ++jj) pk[i][jj] *= inv;
         }
         named_bar_sync(3, 128);
+        if (J <= 8 || j < 8) {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) pks[(t8 + i) * NROW + h] = pk[i];
+          for (int i = 0; i < TPL; ++i) {
+            const int t = t8 + (j * TPL + i) % 8;
+#pragma unroll
+            for (int c4 = 0; c4 < J / 4; ++c4)
+              *reinterpret_cast<float4 *>(pks + t * NROW + dl * J + c4 * 4) =
+                  make_float4(pk[i][4 * c4], pk[i][4 * c4 + 1], pk[i][4 * c4 + 2], pk[i][4 * c4 + 3]);
+          }
+        }
       }
     };
     // operand parts of W after an update, this helper's tensor-memory lane
