@@ -46,6 +46,11 @@
 //
 // When the tiles of a launch do not fill a whole number of waves, the chunk sequence is cut into
 // equal runs per gang of blocks and split tiles hand their state over between blocks (ChunkSched).
+//
+// Instantiations: J = 4, 8 at Dk = 64, 128 and J = 16 at Dk = 64; plain, Temporal (App. B.3: the key-side prior
+// mixes in the row's previous responsibility on the serial chain, the readout weights are a running average the
+// helper warps form with the outputs), and an auxiliary one (plain, J <= 8) that also writes the responsibilities
+// and the sums over time behind the load-balancing loss of Sec. 3.5.
 #pragma once
 
 #include <cuda.h>  // CUtensorMap and its enums (types only; the encoder is fetched through the runtime)
@@ -182,12 +187,12 @@ struct ChunkCfg {
   static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 };
 
-// barrier slots.  Committed by the MMA thread: E (state x [K;Q] of a chunk complete), G (Gram batch),
-// U (update of W), QD (readouts).  Completed by the tensor copies: KQ0 / KQ1 (everything staged for an even /
-// odd chunk has landed).  Arrived by threads: KT (transposed keys ready, 128 helpers), WP (operand parts of W refreshed, 128 helpers), GS
-// (Gram batch spilled, 2 helper warps), C (chunk finished, 128 rows), PQF ([P0|Q0] taken out of tensor
-// memory, 128 rows), BE (gates of a chunk ready, 128 helpers), OD (outputs of a chunk formed, 128 helpers), T0 (update
-// coefficients of a chunk's first 8 tokens stored, 128 rows); committed by the MMA thread: FAR (far pushes of those).
+// barrier slots.  Committed by the MMA thread: E (state x [K;Q] of a chunk complete), G (Gram batch), U (update of W),
+// QD (readouts), FAR (far pushes of a chunk's first 8 tokens).  Completed by the tensor copies: KQ0 / KQ1 (everything
+// staged for an even / odd chunk has landed).  Arrived by threads: WP (operand parts of W refreshed, 128 helpers), GS
+// (Gram batch spilled, 2 helper warps), C (chunk finished, 128 rows), PQF ([P0|Q0] taken out of tensor memory, 128
+// rows), BE (gates of a chunk ready, 128 helpers), OD (outputs of a chunk formed, 128 helpers), T0 (update
+// coefficients of a chunk's first 8 tokens stored, 128 rows).
 enum { B_E = 0, B_G, B_U, B_QD, B_KQ0, B_KQ1, B_WP, B_GS, B_C, B_PQF, B_BE, B_OD, B_T0, B_FAR, B_COUNT };
 
 // bf16 split of FP32 values: hi = bf16(x) (nearest), lo = bf16(x - hi); pairs packed with the first
