@@ -537,6 +537,9 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       if (!mbar_wait(&bars[B_E], n & 1)) { failed = true; break; }
       tc_fence_after_sync();
       PROF_ADD(1);
+      // the readout buffer this chunk seeds below was last read by the helpers for the outputs of chunk n-2: they
+      // finish those about when chunk n-1 ends, so the wait belongs here, where it has long been met, not there
+      if (n >= 2 && !mbar_wait(&bars[B_OD], n & 1)) { failed = true; break; }
       // [P0 | Q0] out of tensor memory: P0 to registers, Q0 seeds the readout accumulator of this chunk;
       // then the tensor cores may overwrite the region with the next chunk's products
       float pred0[C];
@@ -734,10 +737,8 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       tc_fence_before_sync();
       PROF_ADD(2);
       // what the next steps rely on must be in place before this chunk is handed over (this also keeps every
-      // barrier at most one phase ahead of its waiters): operands, gates and Gram rows of chunk n+1
-      // gates and Gram rows of chunk n+1, and the helpers done with the readout buffer that chunk n+1 will seed
+      // barrier at most one phase ahead of its waiters): gates and Gram rows of chunk n+1
       if (n + 1 < nchunks && (!mbar_wait(&bars[B_BE], (n + 1) & 1) || !mbar_wait(&bars[B_GS], (n + 1) & 1))) failed = true;
-      if (n > 0 && !mbar_wait(&bars[B_OD], (n - 1) & 1)) failed = true;
       mbar_arrive(&bars[B_C]);
       PROF_ADD(3);
     }
@@ -1032,8 +1033,12 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         }
       }
       PROF_ADD(2);
-      // (2) outputs of chunk n-1, whose readouts completed shortly after chunk n started
+      // (2) outputs of chunk n-1, whose readouts completed shortly after chunk n started.  The row warps wait for
+      // OD(n-2) at the top of chunk n, and OD must not complete another phase before they have: in every iteration
+      // but the last the Gram batch spilled above was issued after the row warps passed that point (PQF(n)); in the
+      // last one the same barrier is waited for here.
       if (n > 0) {
+        if (!more && !mbar_wait(&bars[B_PQF], n & 1)) { failed = true; break; }
         if (!mbar_wait(&bars[B_QD], (n - 1) & 1)) { failed = true; break; }
         write_outputs(n - 1);
         mbar_arrive(&bars[B_OD]);
