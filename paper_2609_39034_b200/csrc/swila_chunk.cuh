@@ -260,6 +260,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   constexpr int J = Cf::J, DK = Cf::DK, C = Cf::C, NROW = Cf::NROW, COLS = Cf::COLS;
   static_assert(!(RDEBUG && Cf::TEMPORAL), "the auxiliary outputs of the Temporal variant come from the scan kernel");
   static_assert(!(RDEBUG && J > 8), "the auxiliary outputs for J = 16 come from the scan kernel");
+  constexpr bool kOdWaitAtTop = DK == 128;  // where the row warps wait for the helpers' outputs of an earlier chunk
   extern __shared__ __align__(128) unsigned char smem_raw[];
   // the swizzled operand tile needs a 1024-byte aligned shared-memory address
   unsigned char *smem = smem_raw + ((1024u - (umma::smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -537,9 +538,12 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       if (!mbar_wait(&bars[B_E], n & 1)) { failed = true; break; }
       tc_fence_after_sync();
       PROF_ADD(1);
-      // the readout buffer this chunk seeds below was last read by the helpers for the outputs of chunk n-2: they
-      // finish those about when chunk n-1 ends, so the wait belongs here, where it has long been met, not there
-      if (n >= 2 && !mbar_wait(&bars[B_OD], n & 1)) { failed = true; break; }
+      // the readout buffer this chunk seeds below was last read by the helpers for the outputs of chunk n-2.  At
+      // Dk = 128 they finish those about when chunk n-1 ends, so the wait sits here, where it has long been met; at
+      // Dk = 64 they are early and the wait is cheaper at the hand-over below (both placements measured)
+      if constexpr (kOdWaitAtTop) {
+        if (n >= 2 && !mbar_wait(&bars[B_OD], n & 1)) { failed = true; break; }
+      }
       // [P0 | Q0] out of tensor memory: P0 to registers, Q0 seeds the readout accumulator of this chunk;
       // then the tensor cores may overwrite the region with the next chunk's products
       float pred0[C];
@@ -739,6 +743,9 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       // what the next steps rely on must be in place before this chunk is handed over (this also keeps every
       // barrier at most one phase ahead of its waiters): gates and Gram rows of chunk n+1
       if (n + 1 < nchunks && (!mbar_wait(&bars[B_BE], (n + 1) & 1) || !mbar_wait(&bars[B_GS], (n + 1) & 1))) failed = true;
+      if constexpr (!kOdWaitAtTop) {
+        if (n > 0 && !mbar_wait(&bars[B_OD], (n - 1) & 1)) failed = true;
+      }
       mbar_arrive(&bars[B_C]);
       PROF_ADD(3);
     }
