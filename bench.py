@@ -494,7 +494,7 @@ def main():
                              "frac": flops / sec / 1e12 / bf16_peak,
                              "peak_source": "measured bf16 peak (the kernel's MMAs take bf16 operands)"},
             "note": "latency-bound: the T tokens of a row are a serial dependency chain "
-                    "(~180 cycles per token for a row warp running alone, ~260 beside the helper warps)",
+                    "(~180 cycles per token for a row warp running alone, ~210 beside the helper warps)",
         }
     else:
         ach_tflops = flops / sec / 1e12
