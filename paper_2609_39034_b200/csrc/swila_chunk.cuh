@@ -29,7 +29,8 @@
 // the serial path: with W_{n+1} = W_n + Cmat_n K_n,
 //   W_{n+1} [K;Q]_{n+1}^T = W_n [K;Q]_{n+1}^T  +  Cmat_n (K_n [K;Q]_{n+1}^T),
 // the first term only needs the state BEFORE chunk n's update, so it runs while chunk n is still
-// being processed; after chunk n only the small second term (K = 32) remains.
+// being processed; of the small second term (K = 32) the half of the chunk's first 16 tokens is
+// issued as soon as their coefficients are final, the other half remains after the chunk.
 //
 // One block owns 128 rows = COLS = 128/J output columns of one (batch, head) and is split into
 // three roles that run concurrently and meet on mbarriers:
@@ -276,12 +277,15 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int nslice = (p.Dv + COLS - 1) / COLS;
   uint32_t *fail_s = tmem_base_s + 1;  // set by any thread whose bounded wait expired: no further piece is started
+  // set by a row warp that redid a chunk with the exact E-step: the part of the cross-chunk term that was issued
+  // while the chunk still ran used the fast pass's coefficients and is issued again (read and cleared by the MMA thread)
+  volatile uint32_t *redo_s = tmem_base_s + 2;
   // this block's run of chunks and the pieces (tile, first chunk, end chunk) it falls into
   const int gang_slice = (int)(blockIdx.x % sched.gang);
   const long long run = blockIdx.x / sched.gang;
   const int npieces = chunk_run_pieces(sched.ntiles, sched.nch, sched.per, run);
   if (warp == 8) tmem_alloc(tmem_base_s, Cf::TM_ALLOC);
-  if (tid == 0) *fail_s = 0;
+  if (tid == 0) { *fail_s = 0; *redo_s = 0; }
   const uint32_t tb_lane = ((uint32_t)((warp & 3) * 32) << 16);  // this warp's lane quarter
   // row served by this thread in either 128-thread role
   const int r = tid & 127;
@@ -702,7 +706,9 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
             tmem_st4(tb + Cf::TM_CL3 + tg / 2, l3);
           }
           if constexpr (!EXACT) {
-            if (tg == 0) {  // the coefficients of tokens 0-7 are in place: the far pushes may be issued
+            // the coefficients of tokens 0-15 are in place: the far pushes (of tokens 0-7, needed at token 24) and the
+            // first half of the cross-chunk term may be issued
+            if (tg == GT) {
               tmem_st_wait();
               tc_fence_before_sync();
               mbar_arrive(&bars[B_T0]);
@@ -727,6 +733,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       const bool unsafe = sequential(std::false_type{}, rprev);
       PROF_ADD(5);
       if (__any_sync(0xffffffffu, unsafe)) {
+        if (lane == 0) *redo_s = 1;
         tmem_st_wait();
 #pragma unroll
         for (int i = 0; i < C / 4; ++i) {  // P0 again, from the copy in shared memory
@@ -1126,15 +1133,12 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         mma_bf16_ts(tb0 + Cf::TM_PQ, tb0 + Cf::TM_WLO + ks * 8, tile_desc((m & 1) * 2 * C, ks), idE, true);
     };
     // + Cmat (K_prev [K;Q]^T): the update of the chunk that just finished, seen by the next chunk's products
-    auto cross = [&]() {
-#pragma unroll 1
-      for (int ks = 0; ks < C / 16; ++ks) {
-        const uint64_t adv = (uint64_t)(ks * 2 * (Cf::GX_LBO / 16));
-        mma_bf16_ts(tb0 + Cf::TM_PQ, tb0 + Cf::TM_CHI + ks * 8, gx_hi + adv, idE, true);
-        mma_bf16_ts(tb0 + Cf::TM_PQ, tb0 + Cf::TM_CLO + ks * 8, gx_hi + adv, idE, true);
-        mma_bf16_ts(tb0 + Cf::TM_PQ, tb0 + Cf::TM_CHI + ks * 8, gx_lo + adv, idE, true);
-      }
-      mma_commit(&bars[B_E]);
+    // (16 tokens of the chunk per call)
+    auto cross = [&](int ks) {
+      const uint64_t adv = (uint64_t)(ks * 2 * (Cf::GX_LBO / 16));
+      mma_bf16_ts(tb0 + Cf::TM_PQ, tb0 + Cf::TM_CHI + ks * 8, gx_hi + adv, idE, true);
+      mma_bf16_ts(tb0 + Cf::TM_PQ, tb0 + Cf::TM_CLO + ks * 8, gx_hi + adv, idE, true);
+      mma_bf16_ts(tb0 + Cf::TM_PQ, tb0 + Cf::TM_CHI + ks * 8, gx_lo + adv, idE, true);
     };
     // readouts of chunk n: QD += Cmat (K Q^T masked)  -- c_hi B_hi + c_lo B_hi + c_hi B_lo
     auto readout = [&](int n) {
@@ -1186,14 +1190,24 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       if (more) {
         w_times_kq(n + 1);
         PROF_ADD(1);
+        // first half of the cross-chunk term (tokens 0-15 of chunk n, whose coefficients T0 released), while the
+        // chunk still runs
+        if (!mbar_wait(&bars[B_GS], (n + 1) & 1)) { failed = true; break; }
+        tc_fence_after_sync();
+        cross(0);
       }
       if (!mbar_wait(&bars[B_C], n & 1)) { failed = true; break; }
       tc_fence_after_sync();
       PROF_ADD(2);
+      const bool redone = *redo_s != 0;  // ordered by the barrier: set before the row warps arrived
+      if (redone) *redo_s = 0;
       if (more) {
-        if (!mbar_wait(&bars[B_GS], (n + 1) & 1)) { failed = true; break; }
-        tc_fence_after_sync();
-        cross();  // -> E(n+1): the only tensor work between two chunks of the row warps
+        if (redone) {  // rare: a row warp replaced the coefficients that the first half was formed from
+          w_times_kq(n + 1);
+          cross(0);
+        }
+        cross(1);  // -> E(n+1): the only tensor work left between two chunks of the row warps
+        mma_commit(&bars[B_E]);
       }
       PROF_ADD(3);
       PROF_ADD(4);
