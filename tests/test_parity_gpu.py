@@ -145,16 +145,20 @@ def test_chunked_kernel_temporal_in_pieces_and_decode(binding, oracle):
     assert wl.rel_err(st["rho_prev"].cpu(), torch.from_numpy(ref["rho_prev"])) < TOL_STATE
 
 
-def test_chunked_kernel_extreme_prediction_errors(binding, oracle):
+@pytest.mark.parametrize("temporal", [False, True], ids=["vanilla", "temporal"])
+def test_chunked_kernel_extreme_prediction_errors(binding, oracle, temporal):
     """Values far outside the model's noise scale make every Gaussian factor underflow in fp32; the
-    chunked kernel must then fall back to its max-subtracted E-step and still match the oracle."""
-    w = SMALL[4].with_(T=100)
+    chunked kernel must then fall back to its max-subtracted E-step and still match the oracle.  The first
+    outlier sits in the first 16 tokens of a chunk, whose part of the cross-chunk term has been issued from the
+    fast pass's coefficients by then and must be formed again; the second in the last trip of a chunk."""
+    w = SMALL[4].with_(T=100).variant(temporal=temporal)
     inp = wl.make_inputs(w, stress=True)
     v = inp["v"].float()
     v[:, :, 10:13] *= 40.0   # |delta| ~ 40: exp(-delta^2/2) = 0 in fp32 for every component
     v[:, :, 70] = 55.0
+    v[:, :, 95] = -48.0
     inp["v"] = v.to(inp["q"].dtype)
-    ref = oracle.forward_inputs(inp)
+    ref = oracle.forward_inputs(inp, flags=w.flags)
     got = gpu_forward(binding, w, to_dev(inp), algo=binding.ALGO_CHUNK)
     binding.device_status()
     scan = gpu_forward(binding, w, to_dev(inp), algo=binding.ALGO_SCAN)
