@@ -136,7 +136,10 @@ struct ChunkCfg {
   static constexpr int TILE_BYTES = (DK / 64) * TILE_HALF;
   // A second copy of a chunk's keys for the update MMA, which reads them MN-major (tokens = K index) after the
   // chunk, when the tile rows are already being refilled: 3-deep ring of [DK/64][C rows][128 bytes], same swizzle.
-  static constexpr int KU_HALF = C * 128;
+  // The ring is laid out [half of 64 key dims][slot][token row]: the slots of two consecutive chunks are then
+  // adjacent rows of one K-major operand (except when the ring wraps), which is what the Gram batch reads.
+  static constexpr int KU_HALF = C * 128;        // one slot of one half
+  static constexpr int KU_HSTRIDE = 3 * KU_HALF; // distance between the halves
   static constexpr int KU_BYTES = (DK / 64) * KU_HALF;
   // raw stages (2-deep ring): v [C][COLS] bf16; beta logits [C][J][COLS] bf16, overwritten in place by the
   // helpers with beta = sigmoid(.) as fp32 [C][NROW] (hence the fp32-sized slot); pik logits [C][J][COLS]
@@ -238,7 +241,7 @@ __device__ __forceinline__ void chunk_stage(const ChunkMaps &maps, unsigned char
   for (int hf = 0; hf < DK / 64; ++hf) {
     tma_load_3d(trow + hf * Cf::TILE_HALF, &maps.k, hf * 64, tok, bh, bar);
     tma_load_3d(trow + hf * Cf::TILE_HALF + C * 128, &maps.q, hf * 64, tok, bh, bar);
-    tma_load_3d(ku + hf * Cf::KU_HALF, &maps.k, hf * 64, tok, bh, bar);
+    tma_load_3d(ku + hf * Cf::KU_HSTRIDE, &maps.k, hf * 64, tok, bh, bar);
   }
   tma_load_3d(raw + Cf::R_V, &maps.v, col0, tok, bh, bar);
   tma_load_4d(raw + Cf::R_B, &maps.be, col0, 0, tok, bh, bar);
@@ -883,7 +886,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         *reinterpret_cast<uint4 *>(tlo + c * lbo + row * 16) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
       }
     };
-    // The Gram batch of chunk m is [K_e;Q_e;K_o;Q_o] x [K_m;Q_m | K_{m-1}]^T; the two helper warps whose
+    // The Gram batch of chunk m is [K_e;Q_e;K_o;Q_o] x [K_{m-1} | K_m]^T (in that order in tensor memory); the two helper warps whose
     // tensor-memory lanes hold the rows of chunk m's keys and queries spill it:
     //   key rows   (lane s):  -K_m K_m^T as plain FP32 rows for the row warps (negated: they track v - prediction);
     //   query rows (lane t):  Q_m K_m^T, causally masked (s <= t), as the hi / lo operand of the readout MMA;
@@ -892,7 +895,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       const bool qrows = (warp & 1) != 0;
       float a[C];
 #pragma unroll
-      for (int cc = 0; cc < C / 16; ++cc) tmem_ld16(tb + Cf::TM_G + cc * 16, reinterpret_cast<float(&)[16]>(a[cc * 16]));
+      for (int cc = 0; cc < C / 16; ++cc) tmem_ld16(tb + Cf::TM_G + C + cc * 16, reinterpret_cast<float(&)[16]>(a[cc * 16]));
       tmem_ld_wait();
       if (!qrows) {
         float *Gkk = G_all + (m & 1) * C * C;
@@ -923,7 +926,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       if (m > 0) {
 #pragma unroll
         for (int cc = 0; cc < C / 16; ++cc)
-          tmem_ld16(tb + Cf::TM_G + C + cc * 16, reinterpret_cast<float(&)[16]>(a[cc * 16]));
+          tmem_ld16(tb + Cf::TM_G + cc * 16, reinterpret_cast<float(&)[16]>(a[cc * 16]));
         tmem_ld_wait();
         store_parts(a, GX_all, GX_all + Cf::GX_TILE, Cf::GX_LBO, (qrows ? C : 0) + lane);
       }
@@ -936,7 +939,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     // stage chunk m of this piece (one thread; the buffers it overwrites were last read through ordinary loads,
     // hence the proxy fence)
     auto stage = [&](int m) {
-      chunk_stage<Cf>(maps, tile, smem + Cf::OFF_KU + (m % 3) * Cf::KU_BYTES, smem + Cf::OFF_RAW + (m & 1) * Cf::RAW_BYTES, smem + Cf::OFF_RPQ + (m & 3) * Cf::RPQ_BYTES, bh,
+      chunk_stage<Cf>(maps, tile, smem + Cf::OFF_KU + (m % 3) * Cf::KU_HALF, smem + Cf::OFF_RAW + (m & 1) * Cf::RAW_BYTES, smem + Cf::OFF_RPQ + (m & 3) * Cf::RPQ_BYTES, bh,
                       tseg0 + m * C, col0, m, &bars[B_KQ0 + (m & 1)]);
     };
     // everything staged for chunk m has landed (the barrier of m's parity completes once per chunk of that parity)
@@ -1112,14 +1115,24 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     const uint64_t gx_hi = smem_desc_kmajor(smem_u32(GX_all), Cf::GX_LBO, 128);
     const uint64_t gx_lo = smem_desc_kmajor(smem_u32(GX_all + Cf::GX_TILE), Cf::GX_LBO, 128);
     // Gram batch of chunk m: every row of the tile against the keys of chunk m and against the keys of chunk m-1
+    // The keys come from the ring of key copies: when the slots of chunks m-1 and m are adjacent (two times out of
+    // three) they are one operand of 64 rows and one MMA per K step gives [Tile K_{m-1}^T | Tile K_m^T].
+    const uint32_t ku_addr = smem_u32(smem + Cf::OFF_KU);
+    auto ku_desc = [&](int slot, int ks) {
+      return smem_desc_sw128(ku_addr + (ks >> 2) * Cf::KU_HSTRIDE + slot * Cf::KU_HALF + (ks & 3) * 32, 1024);
+    };
     auto gram = [&](int m) {
+      const int so = m % 3, sp = (m + 2) % 3;
+      if (m > 0 && sp + 1 == so) {
 #pragma unroll 1
-      for (int ks = 0; ks < DK / 16; ++ks)
-        mma_bf16_ss(tb0 + Cf::TM_G, tile_desc(0, ks), tile_desc((m & 1) * 2 * C, ks), idQ, ks > 0);
-      if (m > 0) {
+        for (int ks = 0; ks < DK / 16; ++ks) mma_bf16_ss(tb0 + Cf::TM_G, tile_desc(0, ks), ku_desc(sp, ks), idE, ks > 0);
+      } else {
 #pragma unroll 1
-        for (int ks = 0; ks < DK / 16; ++ks)
-          mma_bf16_ss(tb0 + Cf::TM_G + C, tile_desc(0, ks), tile_desc(((m - 1) & 1) * 2 * C, ks), idQ, ks > 0);
+        for (int ks = 0; ks < DK / 16; ++ks) mma_bf16_ss(tb0 + Cf::TM_G + C, tile_desc(0, ks), ku_desc(so, ks), idQ, ks > 0);
+        if (m > 0) {
+#pragma unroll 1
+          for (int ks = 0; ks < DK / 16; ++ks) mma_bf16_ss(tb0 + Cf::TM_G, tile_desc(0, ks), ku_desc(sp, ks), idQ, ks > 0);
+        }
       }
       mma_commit(&bars[B_G]);
     };
@@ -1214,8 +1227,8 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
 #pragma unroll 1
       for (int ks = 0; ks < C / 16; ++ks) {  // W += Cmat K (Eq. 3.3 summed over the chunk)
         // B = the second copy of the chunk's keys, read MN-major: 16 tokens per step = 16 rows of 128 bytes, the
-        // halves of 64 key dims KU_HALF apart
-        const uint64_t bt = smem_desc_sw128_mn(smem_u32(smem + Cf::OFF_KU + (n % 3) * Cf::KU_BYTES) + ks * 16 * 128, Cf::KU_HALF, 1024);
+        // halves of 64 key dims KU_HSTRIDE apart
+        const uint64_t bt = smem_desc_sw128_mn(smem_u32(smem + Cf::OFF_KU + (n % 3) * Cf::KU_HALF) + ks * 16 * 128, Cf::KU_HSTRIDE, 1024);
         mma_bf16_ts(tb0 + Cf::TM_W, tb0 + Cf::TM_CHI + ks * 8, bt, idU, true);
         mma_bf16_ts(tb0 + Cf::TM_W, tb0 + Cf::TM_CLO + ks * 8, bt, idU, true);
         mma_bf16_ts(tb0 + Cf::TM_W, tb0 + Cf::TM_CL3 + ks * 8, bt, idU, true);
