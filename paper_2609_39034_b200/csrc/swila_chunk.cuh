@@ -138,8 +138,12 @@ struct ChunkCfg {
   // chunk, when the tile rows are already being refilled: 3-deep ring of [DK/64][C rows][128 bytes], same swizzle.
   // The ring is laid out [half of 64 key dims][slot][token row]: the slots of two consecutive chunks are then
   // adjacent rows of one K-major operand (except when the ring wraps), which is what the Gram batch reads.
+  // A fourth slot mirrors slot 0 (a chunk that goes to slot 0 is copied there too), so that the pair is adjacent
+  // also when the ring wraps: (slot 2, slot 3).  The Temporal kernel at Dk = 128 has no room for it and issues two
+  // MMAs per K step on those chunks.
+  static constexpr bool KU_MIRROR = !(TEMPORAL && DK == 128);
   static constexpr int KU_HALF = C * 128;        // one slot of one half
-  static constexpr int KU_HSTRIDE = 3 * KU_HALF; // distance between the halves
+  static constexpr int KU_HSTRIDE = (KU_MIRROR ? 4 : 3) * KU_HALF;  // distance between the halves
   static constexpr int KU_BYTES = (DK / 64) * KU_HALF;
   // raw stages (2-deep ring): v [C][COLS] bf16; beta logits [C][J][COLS] bf16, overwritten in place by the
   // helpers with beta = sigmoid(.) as fp32 [C][NROW] (hence the fp32-sized slot); pik logits [C][J][COLS]
@@ -170,7 +174,7 @@ struct ChunkCfg {
   // shared memory map (bytes)
   static constexpr int OFF_TILE = 0;
   static constexpr int OFF_KU = OFF_TILE + TILE_BYTES;
-  static constexpr int OFF_RAW = OFF_KU + 3 * KU_BYTES;
+  static constexpr int OFF_RAW = OFF_KU + (DK / 64) * KU_HSTRIDE;
   static constexpr int OFF_RPQ = OFF_RAW + 2 * RAW_BYTES;
   static constexpr int OFF_G = OFF_RPQ + 4 * RPQ_BYTES;             // 2 x Gkk [C][C] fp32 (-K K^T, for the row warps)
   static constexpr int OFF_BQ = OFF_G + 2 * C * C * 4;        // 2 x { hi, lo } readout operand tiles
@@ -231,17 +235,19 @@ struct ChunkMaps {
 // of the sequence and columns past Dv are filled with zeros by the copy engine.  Everything lands on `bar`.
 template <class Cf>
 __device__ __forceinline__ void chunk_stage(const ChunkMaps &maps, unsigned char *tile, unsigned char *ku, unsigned char *raw,
-                                            unsigned char *rawpq, int bh, int tok, int col0, int m, uint64_t *bar) {
+                                            unsigned char *rawpq, int bh, int tok, int col0, int m, uint64_t *bar,
+                                            unsigned char *ku_mirror) {
   using namespace umma;
   constexpr int DK = Cf::DK, C = Cf::C;
   fence_async_smem();  // the buffers were last read through ordinary loads
-  mbar_arrive_expect_tx(bar, Cf::STAGE_TX_BYTES);
+  mbar_arrive_expect_tx(bar, Cf::STAGE_TX_BYTES + (ku_mirror ? C * DK * Cf::ES : 0));
   unsigned char *trow = tile + (m & 1) * 2 * C * 128;  // this chunk's 2C rows of the operand tile
 #pragma unroll
   for (int hf = 0; hf < DK / 64; ++hf) {
     tma_load_3d(trow + hf * Cf::TILE_HALF, &maps.k, hf * 64, tok, bh, bar);
     tma_load_3d(trow + hf * Cf::TILE_HALF + C * 128, &maps.q, hf * 64, tok, bh, bar);
     tma_load_3d(ku + hf * Cf::KU_HSTRIDE, &maps.k, hf * 64, tok, bh, bar);
+    if (ku_mirror) tma_load_3d(ku_mirror + hf * Cf::KU_HSTRIDE, &maps.k, hf * 64, tok, bh, bar);
   }
   tma_load_3d(raw + Cf::R_V, &maps.v, col0, tok, bh, bar);
   tma_load_4d(raw + Cf::R_B, &maps.be, col0, 0, tok, bh, bar);
@@ -940,7 +946,8 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     // hence the proxy fence)
     auto stage = [&](int m) {
       chunk_stage<Cf>(maps, tile, smem + Cf::OFF_KU + (m % 3) * Cf::KU_HALF, smem + Cf::OFF_RAW + (m & 1) * Cf::RAW_BYTES, smem + Cf::OFF_RPQ + (m & 3) * Cf::RPQ_BYTES, bh,
-                      tseg0 + m * C, col0, m, &bars[B_KQ0 + (m & 1)]);
+                      tseg0 + m * C, col0, m, &bars[B_KQ0 + (m & 1)],
+                      (Cf::KU_MIRROR && m > 0 && m % 3 == 0) ? smem + Cf::OFF_KU + 3 * Cf::KU_HALF : nullptr);
     };
     // everything staged for chunk m has landed (the barrier of m's parity completes once per chunk of that parity)
     auto staged = [&](int m) { return mbar_wait(&bars[B_KQ0 + (m & 1)], (m >> 1) & 1); };
@@ -1115,15 +1122,16 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     const uint64_t gx_hi = smem_desc_kmajor(smem_u32(GX_all), Cf::GX_LBO, 128);
     const uint64_t gx_lo = smem_desc_kmajor(smem_u32(GX_all + Cf::GX_TILE), Cf::GX_LBO, 128);
     // Gram batch of chunk m: every row of the tile against the keys of chunk m and against the keys of chunk m-1
-    // The keys come from the ring of key copies: when the slots of chunks m-1 and m are adjacent (two times out of
-    // three) they are one operand of 64 rows and one MMA per K step gives [Tile K_{m-1}^T | Tile K_m^T].
+    // The keys come from the ring of key copies: when the slots of chunks m-1 and m are adjacent (always with the
+    // mirror slot, else two times out of three) they are one operand of 64 rows and one MMA per K step gives
+    // [Tile K_{m-1}^T | Tile K_m^T].
     const uint32_t ku_addr = smem_u32(smem + Cf::OFF_KU);
     auto ku_desc = [&](int slot, int ks) {
       return smem_desc_sw128(ku_addr + (ks >> 2) * Cf::KU_HSTRIDE + slot * Cf::KU_HALF + (ks & 3) * 32, 1024);
     };
     auto gram = [&](int m) {
       const int so = m % 3, sp = (m + 2) % 3;
-      if (m > 0 && sp + 1 == so) {
+      if (m > 0 && (sp + 1 == so || Cf::KU_MIRROR)) {  // (slot 2, mirror of slot 0) when the ring wraps
 #pragma unroll 1
         for (int ks = 0; ks < DK / 16; ++ks) mma_bf16_ss(tb0 + Cf::TM_G, tile_desc(0, ks), ku_desc(sp, ks), idE, ks > 0);
       } else {
