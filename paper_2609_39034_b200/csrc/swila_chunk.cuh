@@ -139,16 +139,17 @@ struct ChunkCfg {
   // The ring is laid out [half of 64 key dims][slot][token row]: the slots of two consecutive chunks are then
   // adjacent rows of one K-major operand (except when the ring wraps), which is what the Gram batch reads.
   // A fourth slot mirrors slot 0 (a chunk that goes to slot 0 is copied there too), so that the pair is adjacent
-  // also when the ring wraps: (slot 2, slot 3).  The Temporal kernel at Dk = 128 has no room for it and issues two
-  // MMAs per K step on those chunks.
+  // also when the ring wraps: (slot 2, slot 3).  Not in the Temporal kernel at Dk = 128, which is not bound by its
+  // MMA count and measured 1 % slower with the extra copies (two MMAs per K step on those chunks there).
   static constexpr bool KU_MIRROR = !(TEMPORAL && DK == 128);
   static constexpr int KU_HALF = C * 128;        // one slot of one half
   static constexpr int KU_HSTRIDE = (KU_MIRROR ? 4 : 3) * KU_HALF;  // distance between the halves
   static constexpr int KU_BYTES = (DK / 64) * KU_HALF;
   // raw stages (2-deep ring): v [C][COLS] bf16; beta logits [C][J][COLS] bf16, overwritten in place by the
   // helpers with beta = sigmoid(.) as fp32 [C][NROW] (hence the fp32-sized slot); pik logits [C][J][COLS]
-  // bf16.  The query-prior logits piq [C][J][COLS] live in their own 4-deep ring because the outputs of
-  // chunk n are formed while chunk n+2 is being fetched.
+  // bf16.  The query-prior logits piq [C][J][COLS] live in their own 3-deep ring because the outputs of
+  // chunk n are formed while chunk n+2 is being fetched; chunk n+3 is staged into the slot of chunk n by the helper
+  // thread that has just passed the barrier that ends the forming of chunk n's outputs.
   // Gate rows are fetched 8 columns wider than the slice (GROW = COLS + 8, the extra columns are never read):
   // the 16-byte skew between rows spreads the J lanes of a column over different banks.
   static constexpr int GROW = COLS + 8;
@@ -176,7 +177,7 @@ struct ChunkCfg {
   static constexpr int OFF_KU = OFF_TILE + TILE_BYTES;
   static constexpr int OFF_RAW = OFF_KU + (DK / 64) * KU_HSTRIDE;
   static constexpr int OFF_RPQ = OFF_RAW + 2 * RAW_BYTES;
-  static constexpr int OFF_G = OFF_RPQ + 4 * RPQ_BYTES;             // 2 x Gkk [C][C] fp32 (-K K^T, for the row warps)
+  static constexpr int OFF_G = OFF_RPQ + 3 * RPQ_BYTES;             // 2 x Gkk [C][C] fp32 (-K K^T, for the row warps)
   static constexpr int OFF_BQ = OFF_G + 2 * C * C * 4;        // 2 x { hi, lo } readout operand tiles
   static constexpr int OFF_GX = OFF_BQ + 2 * 2 * BQ_TILE;     // { hi, lo } cross-chunk operand tiles
   static constexpr int OFF_OST = OFF_GX + 2 * GX_TILE;        // 2 x [C][COLS] bf16 output staging
@@ -368,7 +369,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   auto write_outputs = [&](int n) {
     const int t0 = n * C;
     const int nvalid = min(C, Tseg - t0);
-    const __nv_bfloat16 *rpq = reinterpret_cast<const __nv_bfloat16 *>(smem + Cf::OFF_RPQ + (n & 3) * Cf::RPQ_BYTES);
+    const __nv_bfloat16 *rpq = reinterpret_cast<const __nv_bfloat16 *>(smem + Cf::OFF_RPQ + (n % 3) * Cf::RPQ_BYTES);
     __nv_bfloat16 *ost = ostage + (n & 1) * C * COLS;
     tc_fence_after_sync();
 #pragma unroll 1
@@ -945,7 +946,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     // stage chunk m of this piece (one thread; the buffers it overwrites were last read through ordinary loads,
     // hence the proxy fence)
     auto stage = [&](int m) {
-      chunk_stage<Cf>(maps, tile, smem + Cf::OFF_KU + (m % 3) * Cf::KU_HALF, smem + Cf::OFF_RAW + (m & 1) * Cf::RAW_BYTES, smem + Cf::OFF_RPQ + (m & 3) * Cf::RPQ_BYTES, bh,
+      chunk_stage<Cf>(maps, tile, smem + Cf::OFF_KU + (m % 3) * Cf::KU_HALF, smem + Cf::OFF_RAW + (m & 1) * Cf::RAW_BYTES, smem + Cf::OFF_RPQ + (m % 3) * Cf::RPQ_BYTES, bh,
                       tseg0 + m * C, col0, m, &bars[B_KQ0 + (m & 1)],
                       (Cf::KU_MIRROR && m > 0 && m % 3 == 0) ? smem + Cf::OFF_KU + 3 * Cf::KU_HALF : nullptr);
     };
