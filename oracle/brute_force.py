@@ -21,7 +21,7 @@ def swila_one_head(q, k, v, beta_logit, pik_logit, piq_logit, W0, *, gk_logit=No
                    r0=None, rho0=None, alpha=None, gran: int = 0, post_decay: bool = False):
     """One (batch, head).  q,k: T x Dk; v: T x Dv; logits: T x J x Dv; W0: J x Dv x Dk;
     gk/gq logits: T x Dv; r0, rho0: J x Dv; alpha: by granularity (1: T x J x Dk,
-    2: T x J x Dv, 3: T x J).  Returns (o [T][Dv], W [J][Dv][Dk], r [T][J][Dv], r_prev, rho_prev)."""
+    2: T x J x Dv, 3: T x J, 4: T x J x Dv x Dk).  Returns (o [T][Dv], W [J][Dv][Dk], r [T][J][Dv], r_prev, rho_prev)."""
     T, Dk, Dv, J = len(q), len(q[0]) if len(q) else 0, len(v[0]) if len(v) else 0, len(W0)
     W = [[[float(x) for x in row] for row in comp] for comp in W0]
     temporal = gk_logit is not None
@@ -36,6 +36,8 @@ def swila_one_head(q, k, v, beta_logit, pik_logit, piq_logit, W0, *, gk_logit=No
             return float(alpha[t][j][c])
         if gran == 2:
             return float(alpha[t][j][d])
+        if gran == 4:  # one value per state element (App. B.4, the general form)
+            return float(alpha[t][j][d][c])
         return float(alpha[t][j])
 
     for t in range(T):

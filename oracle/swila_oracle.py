@@ -75,7 +75,7 @@ def forward(q, k, v, beta_logit, pik_logit, piq_logit, *, gk_logit=None, gq_logi
         rh = np.full((B, H, J, Dv), 1.0 / J) if rho0 is None else _f64(rho0).copy()
     if gated:
         al = _f64(alpha)
-        want = {1: (B, H, T, J, Dk), 2: (B, H, T, J, Dv), 3: (B, H, T, J)}[gran]
+        want = {1: (B, H, T, J, Dk), 2: (B, H, T, J, Dv), 3: (B, H, T, J), 4: (B, H, T, J, Dv, Dk)}[gran]
         assert al.shape == want, (al.shape, want)
     o = np.zeros((B, H, T, Dv))
     r = np.zeros((B, H, T, J, Dv)) if want_r else None

@@ -27,7 +27,8 @@
  *     delta, r and the update all use the decayed state; post-decay (Eq. 3.7): delta and r
  *     from the undecayed state, then w = alpha*w + beta r delta k.  Granularity of
  *     alpha (App. B.4): 1 = one gate per key dimension [B,H,T,J,Dk], 2 = per output
- *     dimension [B,H,T,J,Dv], 3 = scalar per component [B,H,T,J].
+ *     dimension [B,H,T,J,Dv], 3 = scalar per component [B,H,T,J], 4 = one gate per state
+ *     element [B,H,T,J,Dv,Dk] (the general form, of which 1-3 are restrictions).
  *
  * Layouts (row-major, last index fastest): q,k [B,H,T,Dk]; v,o [B,H,T,Dv];
  * gate logits [B,H,T,J,Dv]; temporal gate logits [B,H,T,Dv]; W [B,H,J,Dv,Dk] (rows =
@@ -61,6 +62,18 @@ static void softmax_(int J, const double *x, size_t stride, double *out) {
   for (int j = 0; j < J; ++j) out[j] /= s;
 }
 
+/* decay alpha_{t,j,d,c} of state element (component j, output dim d, key dim c) at token `tok`, by granularity
+ * (App. B.4, "Granularity of the gate"): 4 = one value per element (the general form), 1 = per key dimension
+ * (W Diag(a_tj)), 2 = per output dimension (Diag(alpha_tj) W), 3 = one scalar per component */
+static double decay_(const double *alpha, int gran, size_t tok, int j, int d, int c, int J, int Dv, int Dk) {
+  switch (gran) {
+    case 1: return alpha[(tok * J + j) * (size_t)Dk + c];
+    case 2: return alpha[(tok * J + j) * (size_t)Dv + d];
+    case 3: return alpha[tok * J + j];
+    default: return alpha[((tok * J + j) * (size_t)Dv + d) * (size_t)Dk + c];
+  }
+}
+
 int swila_ref_threads(void) {
 #ifdef _OPENMP
   return omp_get_max_threads();
@@ -81,7 +94,7 @@ int swila_ref_forward(int B, int H, int T, int Dk, int Dv, int J, int flags, int
   const int gated = (flags & REF_GATED) != 0;
   const int post = (flags & REF_POST_DECAY) != 0;
   if (temporal && (!gk_logit || !gq_logit || !r_prev || !rho_prev)) return -1;
-  if (gated && (!alpha || gran < 1 || gran > 3)) return -1;
+  if (gated && (!alpha || gran < 1 || gran > 4)) return -1;
   if (J > 64) return -1;
 
   const long rows = (long)B * H * Dv;
@@ -102,10 +115,7 @@ int swila_ref_forward(int B, int H, int T, int Dk, int Dv, int J, int flags, int
         for (int j = 0; j < J; ++j) {
           double *w = W + ((bh * J + j) * (size_t)Dv + d) * Dk;
           for (int c = 0; c < Dk; ++c) {
-            double al = gran == 1   ? alpha[(tok * J + j) * (size_t)Dk + c]
-                        : gran == 2 ? alpha[(tok * J + j) * (size_t)Dv + d]
-                                    : alpha[tok * J + j];
-            w[c] *= al;
+            w[c] *= decay_(alpha, gran, tok, j, d, c, J, Dv, Dk);
           }
         }
       }
@@ -153,10 +163,7 @@ int swila_ref_forward(int B, int H, int T, int Dk, int Dv, int J, int flags, int
         for (int c = 0; c < Dk; ++c) {
           double wc = w[c];
           if (gated && post) {
-            double al = gran == 1   ? alpha[(tok * J + j) * (size_t)Dk + c]
-                        : gran == 2 ? alpha[(tok * J + j) * (size_t)Dv + d]
-                                    : alpha[tok * J + j];
-            wc *= al;
+            wc *= decay_(alpha, gran, tok, j, d, c, J, Dv, Dk);
           }
           w[c] = wc + coef * kt[c];
         }

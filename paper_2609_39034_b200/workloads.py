@@ -30,6 +30,7 @@ GRAN_NONE = 0
 GRAN_PER_KEY = 1
 GRAN_PER_OUT = 2
 GRAN_SCALAR = 3
+GRAN_ELEMENTWISE = 4  # alpha [B,H,T,J,Dv,Dk]: one decay per state element (App. B.4, the general form)
 
 
 @dataclass(frozen=True)
@@ -173,10 +174,14 @@ def make_inputs(w: Workload, *, device="cpu", stress: bool = False, seed_offset:
 
     if w.gated:
         # Decay values in (0,1), mostly near 1 (sigmoid(3) ~ 0.95), key-dependent.
-        m = {GRAN_PER_KEY: Dk, GRAN_PER_OUT: Dv, GRAN_SCALAR: 1}[w.gate_granularity]
+        m = {GRAN_PER_KEY: Dk, GRAN_PER_OUT: Dv, GRAN_SCALAR: 1, GRAN_ELEMENTWISE: Dv * Dk}[w.gate_granularity]
         th_a = _randn((H, J * m, Dk), base + 9, device, pstd)
         a = torch.sigmoid(3.0 + _head_proj(th_a, k_for_alpha)).view(B, H, T, J, m)
-        out["alpha"] = (a.view(B, H, T, J) if w.gate_granularity == GRAN_SCALAR else a).contiguous()
+        if w.gate_granularity == GRAN_SCALAR:
+            a = a.view(B, H, T, J)
+        elif w.gate_granularity == GRAN_ELEMENTWISE:
+            a = a.view(B, H, T, J, Dv, Dk)
+        out["alpha"] = a.contiguous()
     else:
         out["alpha"] = None
 
@@ -251,10 +256,14 @@ def decode_step_inputs(w: Workload, step: int, *, device="cpu", stress: bool = F
         out["gk_logit"] = _head_proj(_randn((H, Dv, Dk), base + 7, device, pstd), k).to(io)
         out["gq_logit"] = _head_proj(_randn((H, Dv, Dk), base + 8, device, pstd), q).to(io)
     if w1.gated:
-        m = {GRAN_PER_KEY: Dk, GRAN_PER_OUT: Dv, GRAN_SCALAR: 1}[w.gate_granularity]
+        m = {GRAN_PER_KEY: Dk, GRAN_PER_OUT: Dv, GRAN_SCALAR: 1, GRAN_ELEMENTWISE: Dv * Dk}[w.gate_granularity]
         th_a = _randn((H, J * m, Dk), base + 9, device, pstd)
         a = torch.sigmoid(3.0 + _head_proj(th_a, k)).view(B, H, 1, J, m)
-        out["alpha"] = (a.view(B, H, 1, J) if w.gate_granularity == GRAN_SCALAR else a).contiguous()
+        if w.gate_granularity == GRAN_SCALAR:
+            a = a.view(B, H, 1, J)
+        elif w.gate_granularity == GRAN_ELEMENTWISE:
+            a = a.view(B, H, 1, J, Dv, Dk)
+        out["alpha"] = a.contiguous()
     return out
 
 
@@ -290,6 +299,8 @@ def slice_rows(inp: Dict[str, Optional[torch.Tensor]], bh_index: torch.Tensor,
             flat = flat[:, :, cols, :]
         elif name == "alpha" and gran == GRAN_PER_OUT:
             flat = flat[..., cols]
+        elif name == "alpha" and gran == GRAN_ELEMENTWISE:
+            flat = flat[..., cols, :]
         out[name] = flat.unsqueeze(1).contiguous()
     return out
 

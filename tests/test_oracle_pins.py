@@ -30,7 +30,7 @@ def _rand_problem(seed, B=2, H=2, T=12, Dk=8, Dv=6, J=3, temporal=False, gran=0,
         r0 = g.random((B, H, J, Dv)); p["r0"] = r0 / r0.sum(2, keepdims=True)
         rho0 = g.random((B, H, J, Dv)); p["rho0"] = rho0 / rho0.sum(2, keepdims=True)
     if gran:
-        shape = {1: (B, H, T, J, Dk), 2: (B, H, T, J, Dv), 3: (B, H, T, J)}[gran]
+        shape = {1: (B, H, T, J, Dk), 2: (B, H, T, J, Dv), 3: (B, H, T, J), 4: (B, H, T, J, Dv, Dk)}[gran]
         p["alpha"] = 0.5 + 0.5 * g.random(shape)
     return p
 
@@ -228,7 +228,7 @@ def test_split_sequence_continuity(oracle, flags, gran):
 
 
 # ---- brute force on tiny inputs -------------------------------------------------------------
-@pytest.mark.parametrize("flags,gran", [(0, 0), (1, 0), (2, 1), (2, 2), (2, 3), (6, 1), (6, 2), (3, 1), (7, 3)])
+@pytest.mark.parametrize("flags,gran", [(0, 0), (1, 0), (2, 1), (2, 2), (2, 3), (6, 1), (6, 2), (3, 1), (7, 3), (2, 4), (6, 4), (3, 4)])
 def test_brute_force(oracle, flags, gran):
     from oracle import brute_force
 
@@ -287,8 +287,27 @@ def test_decay_granularities_agree_when_tied(oracle):
         s = _run(oracle, p, fl, 3)
         pk = dict(p, alpha=np.broadcast_to(p["alpha"][..., None], (B, H, T, J, Dk)).copy())
         po = dict(p, alpha=np.broadcast_to(p["alpha"][..., None], (B, H, T, J, Dv)).copy())
+        pe = dict(p, alpha=np.broadcast_to(p["alpha"][..., None, None], (B, H, T, J, Dv, Dk)).copy())
         np.testing.assert_array_equal(_run(oracle, pk, fl, 1)["o"], s["o"])
         np.testing.assert_array_equal(_run(oracle, po, fl, 2)["o"], s["o"])
+        np.testing.assert_array_equal(_run(oracle, pe, fl, 4)["o"], s["o"])
+
+
+@pytest.mark.parametrize("gran", [1, 2])
+def test_elementwise_gate_restricts_to_the_coarser_ones(oracle, gran):
+    # Eq. (gate-elementwise) of App. B.4 with alpha_{tjdd'} constant along the output index d is W Diag(a_tj)
+    # (one gate per key dimension); constant along the key index d' it is Diag(alpha_tj) W (one per output
+    # dimension).  Dk != Dv here, so an elementwise gate indexed [d'][d] instead of [d][d'] cannot pass.
+    p = _rand_problem(15, gran=gran, J=3, temporal=True)
+    B, H, T, J = p["alpha"].shape[:4]
+    Dk, Dv = p["q"].shape[-1], p["v"].shape[-1]
+    assert Dk != Dv
+    full = p["alpha"][..., None, :] if gran == 1 else p["alpha"][..., :, None]
+    pe = dict(p, alpha=np.broadcast_to(full, (B, H, T, J, Dv, Dk)).copy())
+    for fl in (2, 6, 3):
+        a, b = _run(oracle, p, fl, gran), _run(oracle, pe, fl, 4)
+        np.testing.assert_array_equal(a["o"], b["o"])
+        np.testing.assert_array_equal(a["W"], b["W"])
 
 
 # ---- own-block Jacobian of the update (Eqs. C.4-C.5) by finite differences ---------------
