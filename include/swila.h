@@ -16,7 +16,11 @@
  *
  * Conventions
  *  - Every pointer is a DEVICE pointer owned by the caller unless a function says HOST.
- *    The library allocates no device memory and keeps no per-call state.
+ *    The library never allocates device memory at run time and keeps no per-call state.  What it
+ *    holds per device for as long as it is loaded: three file-scope device arrays (the 16 MiB
+ *    staging array of swila_forward_host_static, 128 KB of hand-over flags and one error word of
+ *    the chunked kernel) and, after the first pipelined swila_forward_host call on a device, two
+ *    internal copy streams with their events.
  *  - All tensors are contiguous, last index fastest.  Base addresses must be 16-byte
  *    aligned.  Dv must be a multiple of 8.
  *  - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default
@@ -64,27 +68,19 @@ enum {
   SWILA_GATE_NONE = 0,
   SWILA_GATE_PER_KEY = 1, /* alpha [B,H,T,J,Dk]: one gate per key dimension (the LM setting, App. D.3) */
   SWILA_GATE_PER_OUT = 2, /* alpha [B,H,T,J,Dv]: one gate per output dimension (Eq. 3.7 as printed) */
-  SWILA_GATE_SCALAR = 3   /* alpha [B,H,T,J]:    one gate per component */
+  SWILA_GATE_SCALAR = 3,  /* alpha [B,H,T,J]:    one gate per component */
+  SWILA_GATE_ELEMENTWISE = 4 /* alpha [B,H,T,J,Dv,Dk]: one gate per state element, the general form of App. B.4 of which
+                                the other three are restrictions (J*Dv*Dk values per token: small problems only) */
 };
 
-/* algo: which kernel evaluates the recurrence.  Every choice computes the same function. */
+/* algo: which kernel evaluates the recurrence.  Every choice computes the same function; what each
+ * kernel covers and what AUTO picks is part of the contract of swila_forward below. */
 enum {
-  SWILA_ALGO_AUTO = 0,     /* CHUNK where it applies and T >= 64, else SCAN */
-  SWILA_ALGO_SCAN = 1,     /* sequential scan, state resident in registers, FP32 FMA pipe */
-  SWILA_ALGO_SCAN_WIDE = 2, /* the same scan with 256-thread blocks (twice the columns per
-                              block); ungated shapes with Dk = 128 only */
-  SWILA_ALGO_SCAN_NARROW = 3, /* the same scan with 16 key dimensions per lane (more, lighter
-                              warps); ungated shapes with Dk = 128, J >= 4 only */
-  SWILA_ALGO_CHUNK = 4     /* chunked form: the state-times-token contractions of 32-token chunks
-                              on the tcgen05 tensor cores (bf16 hi/lo operand split, FP32
-                              accumulation in tensor memory), the E-step and intra-chunk
-                              corrections on the FP32 ALUs.  bf16 io, Dk in {64, 128}, J in {4, 8}
-                              (J = 16 at Dk = 64, without r_debug / statistics),
-                              plain or TEMPORAL (the latter without r_debug / statistics), no GATED,
-                              no QKV_ACT.  When a state output is given and the tiles do
-                              not fill a whole number of waves, the launch is cooperative and
-                              balances chunks over the SMs; up to 8 such launches may overlap on
-                              one device */
+  SWILA_ALGO_AUTO = 0,        /* the library chooses (see swila_forward) */
+  SWILA_ALGO_SCAN = 1,        /* sequential scan, state resident in registers, FP32 FMA pipe; every shape */
+  SWILA_ALGO_SCAN_WIDE = 2,   /* the same scan with 256-thread blocks; ungated shapes with Dk = 128 only */
+  SWILA_ALGO_SCAN_NARROW = 3, /* the same scan with 16 key dimensions per lane; ungated, Dk = 128, J >= 4 only */
+  SWILA_ALGO_CHUNK = 4        /* chunked form on the tcgen05 tensor cores (see swila_forward) */
 };
 
 typedef struct {
@@ -147,8 +143,35 @@ int swila_state_init(const swila_shape_t *shape, swila_state_t *state, void *str
  *               (each thread block reads its slice completely before writing it).
  *   r_debug   : NULL, or fp32 [B,H,T,J,Dv] receiving the responsibilities r of Eq. 3.4.
  * T == 0 copies state_in to state_out and touches nothing else.
- * The call only enqueues kernels on `stream`; it (and swila_decode_step) may be captured into a CUDA graph
- * and replayed, after one ordinary call of the same shape on the device.
+ * SWILA_ERR_ALIAS: o, r_debug or a tensor of state_out overlaps a streamed input (q, k, v, a gate tensor),
+ * or o overlaps r_debug or the state; state_out may alias state_in only tensor for tensor, exactly.
+ *
+ * Which kernel runs (shape->algo).  Two kernels evaluate the same recurrence and agree to rounding
+ * (1e-4 on the state):
+ *   SCAN   the sequential scan on the FP32 ALUs: every shape, dtype, flag and output.
+ *   CHUNK  32-token chunks whose state-times-token contractions run on the tcgen05 tensor cores (bf16
+ *          hi/lo operand split, FP32 accumulation in tensor memory), the E-step and the corrections
+ *          inside a chunk on the FP32 ALUs; several times faster.  It covers: bf16 io; Dk in {64, 128};
+ *          J in {4, 8}, and J = 16 at Dk = 64; plain or SWILA_TEMPORAL; not SWILA_GATED, not
+ *          SWILA_QKV_ACT.  r_debug and the sums of swila_forward_stats come from it only for plain
+ *          (non-Temporal) shapes with J <= 8.  Requested for anything else: SWILA_ERR_UNSUPPORTED.
+ *   AUTO   CHUNK when the call is inside that coverage and T >= 64, else SCAN.  So the following send an
+ *          AUTO call to the scan kernel, at 3-6 times the cost per token: fp32 io, SWILA_GATED,
+ *          SWILA_QKV_ACT, Dk = 16, J in {1, 2}, T < 64, and r_debug or statistics together with
+ *          SWILA_TEMPORAL or J = 16.
+ * Inside CHUNK the work distribution depends on state_out: with a state output, when the 128-row tiles
+ * of the launch do not fill a whole number of waves of SMs, the chunk sequence is cut into equal runs
+ * per SM and a tile that falls into two runs hands its state over through state_out (a cooperative
+ * launch; hand-over flags live in a library array indexed by a launch counter modulo 8).  With
+ * state_out == NULL every block takes whole tiles, which can cost up to one partly empty wave more.
+ * Results are the same to rounding.
+ *
+ * The call only enqueues work on `stream`; it (and swila_decode_step) may be captured into a CUDA graph
+ * and replayed, after one ordinary call of the same shape on the device.  Limits of a replayed CHUNK
+ * launch with hand-over: a replay reuses the counter value of its capture, so it must not overlap on the
+ * GPU another hand-over launch whose counter is congruent modulo 8 (in practice: do not overlap replays
+ * with each other or with more than 7 live calls), and swila_device_status must be clean before a replay
+ * (an expired wait leaves the launch incomplete).
  */
 int swila_forward(const swila_shape_t *shape, const void *q, const void *k, const void *v,
                   const swila_gates_t *gates, const swila_state_t *state_in,
@@ -191,9 +214,10 @@ int swila_output_norm(const swila_shape_t *shape, void *o, const float *weight, 
 /*
  * Decode: one token of the same recurrence on a carried state, updated in place
  * (generation, App. D.4).  q,k [B,H,1,Dk]; v, o [B,H,1,Dv]; gate tensors with T = 1.
- * shape->T is ignored.  Decode always runs the scan kernel with T = 1: its arithmetic and order
- * are those of a scan prefill (SWILA_ALGO_SCAN), so a scan prefill of T tokens equals, bit for
- * bit, T decode steps; against a chunked prefill the two agree to rounding (1e-4 on the state).
+ * shape->T is ignored.  Decode always runs the scan kernel with T = 1 whatever shape->algo says
+ * (SWILA_ALGO_CHUNK is read as SWILA_ALGO_SCAN): its arithmetic and order are those of a scan prefill,
+ * so a scan prefill of T tokens equals, bit for bit, T decode steps; against a chunked prefill the two
+ * agree to rounding (1e-4 on the state).
  */
 int swila_decode_step(const swila_shape_t *shape, const void *q, const void *k, const void *v,
                       const swila_gates_t *gates, swila_state_t *state, void *o, void *stream);
@@ -210,7 +234,8 @@ int swila_decode_step(const swila_shape_t *shape, const void *q, const void *k, 
  * -- with the copies on two internal streams (created on the first such call on a device and
  * kept) beside the kernels on `stream`, so that transfers in both directions overlap the
  * compute; `stream` waits for the internal streams at the end.  Smaller problems use `stream`
- * alone.  Calls from several host threads on one device share those copy streams.
+ * alone.  Calls from several host threads on one device are allowed (each with its own workspace):
+ * they share those copy streams, and the library serialises their enqueue phases with a per-device lock.
  * state_in == NULL starts from the initial state; state_out == NULL discards the final state.
  * Errors as swila_forward, plus SWILA_ERR_SIZE when the workspace is too small.
  */
@@ -249,57 +274,6 @@ size_t swila_forward_host_static_capacity(void);
 int swila_forward_host_static(const swila_shape_t *shape, const void *q, const void *k, const void *v,
                               const swila_gates_t *gates, const swila_state_t *state_in,
                               swila_state_t *state_out, void *o, void *stream);
-
-/*
- * Measurement helper (no counterpart in the paper): launches an FP32 FMA-chain
- * microbenchmark whose rate is the denominator of the scan kernel's roofline (the
- * recurrence costs 3*J*Dk*Dv FP32 FMAs per token and head, Sec. 3.2).  Every thread of
- * `blocks` blocks of 256 threads runs `iters` rounds of 2*`chains` independent register
- * FMAs; packed != 0 uses the packed f32x2 form.  chains in {4, 8, 16}.  scratch_out: device
- * pointer to >= 4 bytes (practically never written).  *fma_per_launch (HOST pointer) receives
- * the number of FMAs one launch performs; time the launch with CUDA events on `stream`.
- */
-int swila_bench_fma_chain(int packed, int chains, int blocks, int iters, float *scratch_out,
-                          double *fma_per_launch, void *stream);
-
-/*
- * Self-test of the tensor-core plumbing (no counterpart in the paper): one block computes
- * D[128 x N] = A[128 x K] * B[N x K]^T with TF32 operands and FP32 accumulation on the tcgen05
- * path (A through tensor memory, B through shared memory).  A [128,K], B [N,K], D [128,N] are
- * DEVICE fp32 row-major; *status (DEVICE int, zeroed by the caller) is set non-zero if the MMA
- * never completed.  (N, K) in {(32,32), (128,32), (32,128), (64,128)}.
- */
-int swila_selftest_tf32_mma(const float *A, const float *B, float *D, int N, int K, int *status, void *stream);
-
-/*
- * The same self-test with BF16 operands (no counterpart in the paper): A and B are DEVICE fp32
- * row-major and are rounded to bf16 (nearest even) by the kernel; FP32 accumulation.  a_in_smem = 0:
- * A goes through tensor memory, two consecutive K elements per 32-bit column; a_in_smem = 1: A
- * goes through shared memory in the K-major layout of B; a_in_smem = 2: both operands in shared
- * memory in the 128-byte-swizzle K-major layout (what a tensor copy with that swizzle mode
- * writes); a_in_smem = 3: A through tensor memory, B stored MN-major (N contiguous) with the
- * 128-byte swizzle.  (N, K, a_in_smem) in {(64,128,0), (128,32,0), (32,32,0), (64,64,1),
- * (64,64,2), (32,64,2), (128,32,3)}; anything else returns SWILA_ERR_UNSUPPORTED.
- */
-int swila_selftest_bf16_mma(const float *A, const float *B, float *D, int N, int K, int a_in_smem, int *status,
-                            void *stream);
-
-/*
- * Host-only probes of how SWILA_ALGO_CHUNK distributes work (no counterpart in the paper; no GPU call).
- * A launch has B*H*ceil(Dv / (128/J)) tiles of 128 state rows, each a sequence of ceil(T/32) chunks.
- *
- * swila_chunk_plan: the layout chosen for a device with `sm_count` SMs.  out[0] = 1 if the chunk sequence
- * is cut into equal runs (taken when the tiles do not fill a whole number of waves and a state output is
- * given), else 0 (one tile per block); out[1] = blocks per gang (column slices of one (batch, head));
- * out[2] = chunks per unit; out[3] = chunks per run; out[4] = units (tiles, or (batch, head) pairs when
- * split); out[5] = blocks launched.  Returns SWILA_OK or an error code (J must be 4 or 8).
- *
- * swila_chunk_run_pieces: the pieces of run `run` in the order a block processes them, as triples
- * (unit, first chunk, end chunk) written to `pieces` (HOST int[3 * capacity]).  Returns the number of pieces
- * (0 for a run past the end of the work) or a negative error code.
- */
-int swila_chunk_plan(int B, int H, int T, int Dv, int J, int sm_count, int has_state_out, long long out[6]);
-int swila_chunk_run_pieces(long long units, int nch, int per, long long run, int *pieces, int capacity);
 
 #ifdef __cplusplus
 }

@@ -25,7 +25,7 @@ EXPORTS = ("swila_version", "swila_strerror", "swila_last_cuda_error", "swila_st
            "swila_state_r_bytes", "swila_state_init", "swila_forward", "swila_decode_step",
            "swila_bench_fma_chain", "swila_forward_host", "swila_forward_host_workspace_bytes",
            "swila_forward_host_static", "swila_forward_host_static_capacity", "swila_selftest_tf32_mma", "swila_selftest_bf16_mma", "swila_device_status", "swila_chunk_plan", "swila_chunk_run_pieces",
-           "swila_forward_stats", "swila_output_norm")
+           "swila_forward_stats", "swila_output_norm", "swila_auto_algo")
 
 
 class Shape(ctypes.Structure):
@@ -108,6 +108,8 @@ def _load() -> ctypes.CDLL:
     L.swila_chunk_run_pieces.argtypes = [ctypes.c_longlong, ctypes.c_int, ctypes.c_int, ctypes.c_longlong,
                                          ctypes.POINTER(ctypes.c_int), ctypes.c_int]
     L.swila_device_status.restype = ctypes.c_int
+    L.swila_auto_algo.restype = ctypes.c_int
+    L.swila_auto_algo.argtypes = [ctypes.POINTER(Shape), ctypes.c_int]
     L.swila_bench_fma_chain.restype = ctypes.c_int
     L.swila_bench_fma_chain.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
                                         ctypes.POINTER(ctypes.c_double), ctypes.c_void_p]
@@ -322,6 +324,15 @@ def chunk_run_pieces(units: int, nch: int, per: int, run: int) -> list:
     if n < 0:
         check(n)
     return [(buf[3 * i], buf[3 * i + 1], buf[3 * i + 2]) for i in range(n)]
+
+
+def auto_algo(w: Workload, aux_outputs: bool = False) -> int:
+    """The kernel ALGO_AUTO resolves to for this workload (ALGO_CHUNK or ALGO_SCAN)."""
+    sh = make_shape(w)
+    rc = int(lib.swila_auto_algo(ctypes.byref(sh), int(aux_outputs)))
+    if rc < 0:
+        check(rc)
+    return rc
 
 
 def device_status() -> None:

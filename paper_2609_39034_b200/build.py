@@ -19,13 +19,12 @@ LIB = os.path.join(HERE, "libswila.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
-NVCC_FLAGS += os.environ.get("SWILA_NVCC_EXTRA", "").split()  # developer experiments only
 DKS = (16, 64, 128)
-GATE_MODES = ((0, 0), (1, 0), (1, 1), (2, 0), (2, 1))  # (decay mode, post-decay)
+GATE_MODES = ((0, 0), (1, 0), (1, 1), (2, 0), (2, 1), (3, 0), (3, 1))  # (decay mode, post-decay)
 
 
 def _sources():
-    return sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC)) + [os.path.join(INC, "swila.h")]
+    return sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC)) + sorted(os.path.join(INC, f) for f in os.listdir(INC))
 
 
 def _stamp() -> str:

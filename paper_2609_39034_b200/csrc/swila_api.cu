@@ -1,16 +1,20 @@
 // C-ABI entry points of the SwiLA library: host-side validation and kernel dispatch.
-// No device memory is allocated here; the only state kept between calls is the pair of copy streams (and their
-// events) that the host-buffer front end creates on first use for problems of 64 MB and more.
+// No device memory is allocated here; the only host-side state kept between calls is the pair of copy streams (and
+// their events) that the host-buffer front end creates per device on first use for problems of 64 MB and more.  (The
+// library image itself carries three device arrays: the staging array of the allocation-free entry point, and the
+// hand-over flags and the error word of the chunked kernel.)
 #include <string.h>
 
 #include <mutex>
 
+#include "../../include/swila_dev.h"
 #include "swila_common.cuh"
 
 namespace swila {
 #define SWILA_DECL(DK, GATE, POST) template <> int scan_dispatch<DK, GATE, POST>(const LaunchArgs &);
 #define SWILA_DECL_DK(DK) \
-  SWILA_DECL(DK, 0, false) SWILA_DECL(DK, 1, false) SWILA_DECL(DK, 1, true) SWILA_DECL(DK, 2, false) SWILA_DECL(DK, 2, true)
+  SWILA_DECL(DK, 0, false) SWILA_DECL(DK, 1, false) SWILA_DECL(DK, 1, true) SWILA_DECL(DK, 2, false) SWILA_DECL(DK, 2, true) \
+      SWILA_DECL(DK, 3, false) SWILA_DECL(DK, 3, true)
 SWILA_DECL_DK(16)
 SWILA_DECL_DK(64)
 SWILA_DECL_DK(128)
@@ -40,7 +44,7 @@ static int check_shape(const swila_shape_t *s, bool need_T) {
   const bool gated = (s->flags & SWILA_GATED) != 0;
   if (!gated && (s->flags & SWILA_POST_DECAY)) return SWILA_ERR_UNSUPPORTED;
   if (gated != (s->gate_granularity != SWILA_GATE_NONE)) return SWILA_ERR_UNSUPPORTED;
-  if (s->gate_granularity < SWILA_GATE_NONE || s->gate_granularity > SWILA_GATE_SCALAR) return SWILA_ERR_UNSUPPORTED;
+  if (s->gate_granularity < SWILA_GATE_NONE || s->gate_granularity > SWILA_GATE_ELEMENTWISE) return SWILA_ERR_UNSUPPORTED;
   if (s->algo != SWILA_ALGO_AUTO && s->algo != SWILA_ALGO_SCAN && s->algo != SWILA_ALGO_SCAN_WIDE &&
       s->algo != SWILA_ALGO_SCAN_NARROW && s->algo != SWILA_ALGO_CHUNK)
     return SWILA_ERR_UNSUPPORTED;
@@ -50,10 +54,32 @@ static int check_shape(const swila_shape_t *s, bool need_T) {
 static size_t w_elems(const swila_shape_t *s) { return (size_t)s->B * s->H * s->J * s->Dv * s->Dk; }
 static size_t r_elems(const swila_shape_t *s) { return (size_t)s->B * s->H * s->J * s->Dv; }
 
+// elements of alpha for T tokens, by granularity
+static size_t alpha_elems(const swila_shape_t *s, int T) {
+  const size_t ntok = (size_t)s->B * s->H * (size_t)T;
+  switch (s->gate_granularity) {
+    case SWILA_GATE_PER_KEY: return ntok * s->J * s->Dk;
+    case SWILA_GATE_PER_OUT: return ntok * s->J * s->Dv;
+    case SWILA_GATE_SCALAR: return ntok * s->J;
+    case SWILA_GATE_ELEMENTWISE: return ntok * s->J * s->Dv * s->Dk;
+    default: return 0;
+  }
+}
+
 static bool overlaps(const void *a, size_t na, const void *b, size_t nb) {
   if (!a || !b || na == 0 || nb == 0) return false;
   const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
   return a0 < b0 + nb && b0 < a0 + na;
+}
+
+// What the chunked tensor-core kernel covers (the AUTO rule of swila_forward is this and T >= 64): bf16 io, Dk in
+// {64, 128}, J in {4, 8} or J = 16 at Dk = 64, plain or Temporal; auxiliary outputs (r_debug, statistics) only for
+// plain shapes with J <= 8.
+static bool chunk_covers(const swila_shape_t *s, bool aux) {
+  if (s->io_dtype != SWILA_IO_BF16 || (s->flags & ~SWILA_TEMPORAL) != 0 || (s->Dk != 64 && s->Dk != 128)) return false;
+  if (!(s->J == 4 || s->J == 8 || (s->J == 16 && s->Dk == 64))) return false;
+  if (aux && ((s->flags & SWILA_TEMPORAL) || s->J == 16)) return false;
+  return true;
 }
 
 static int run(const swila_shape_t *s, int T, const void *q, const void *k, const void *v, const swila_gates_t *g,
@@ -78,10 +104,33 @@ static int run(const swila_shape_t *s, int T, const void *q, const void *k, cons
   const size_t ntok = (size_t)s->B * s->H * (size_t)T;
   const size_t o_bytes = ntok * s->Dv * es;
   const size_t gate_bytes = ntok * s->J * s->Dv * es;
-  if (overlaps(o, o_bytes, q, ntok * s->Dk * es) || overlaps(o, o_bytes, k, ntok * s->Dk * es) ||
-      overlaps(o, o_bytes, v, ntok * s->Dv * es) || overlaps(o, o_bytes, g->beta_logit, gate_bytes) ||
-      overlaps(o, o_bytes, g->pik_logit, gate_bytes) || overlaps(o, o_bytes, g->piq_logit, gate_bytes))
-    return SWILA_ERR_ALIAS;
+  {
+    // Both kernels read the streamed inputs ahead of the tokens they write (cp.async ring, tensor copies), so
+    // nothing that is written may overlap them; the written tensors must not overlap one another either.
+    struct Range { const void *p; size_t n; };
+    const Range in[] = {{q, ntok * s->Dk * es}, {k, ntok * s->Dk * es}, {v, ntok * s->Dv * es},
+                        {g->beta_logit, gate_bytes}, {g->pik_logit, gate_bytes}, {g->piq_logit, gate_bytes},
+                        {temporal ? g->gk_logit : nullptr, ntok * s->Dv * es},
+                        {temporal ? g->gq_logit : nullptr, ntok * s->Dv * es},
+                        {gated ? (const void *)g->alpha : nullptr, alpha_elems(s, T) * 4}};
+    const Range out[] = {{o, o_bytes}, {r_debug, ntok * s->J * s->Dv * 4},
+                         {sout ? sout->W : nullptr, w_elems(s) * 4},
+                         {(sout && temporal) ? sout->r_prev : nullptr, r_elems(s) * 4},
+                         {(sout && temporal) ? sout->rho_prev : nullptr, r_elems(s) * 4}};
+    for (const Range &w : out)
+      for (const Range &r : in)
+        if (overlaps(w.p, w.n, r.p, r.n)) return SWILA_ERR_ALIAS;
+    for (size_t i = 0; i < sizeof(out) / sizeof(out[0]); ++i)
+      for (size_t j = i + 1; j < sizeof(out) / sizeof(out[0]); ++j)
+        if (overlaps(out[i].p, out[i].n, out[j].p, out[j].n)) return SWILA_ERR_ALIAS;
+    if (sin) {  // the initial state may be the output state itself (in place), nothing else that is written
+      const Range st[] = {{sin->W, w_elems(s) * 4}, {temporal ? sin->r_prev : nullptr, r_elems(s) * 4},
+                          {temporal ? sin->rho_prev : nullptr, r_elems(s) * 4}};
+      for (int i = 0; i < 3; ++i)
+        for (int j = 0; j < 5; ++j)
+          if (!(j == 2 + i && st[i].p == out[j].p) && overlaps(st[i].p, st[i].n, out[j].p, out[j].n)) return SWILA_ERR_ALIAS;
+    }
+  }
 
   LaunchArgs a;
   memset(&a, 0, sizeof(a));
@@ -107,18 +156,14 @@ static int run(const swila_shape_t *s, int T, const void *q, const void *k, cons
     a.p.rho_sum = stats->rho_sum; a.p.rho_ent = stats->rho_ent;
   }
   a.Dk = s->Dk; a.J = s->J; a.io_dtype = s->io_dtype;
-  a.gate_mode = !gated ? 0 : (s->gate_granularity == SWILA_GATE_PER_KEY ? 1 : 2);
+  a.gate_mode = !gated ? 0 : (s->gate_granularity == SWILA_GATE_PER_KEY ? 1 : s->gate_granularity == SWILA_GATE_ELEMENTWISE ? 3 : 2);
   a.post = (s->flags & SWILA_POST_DECAY) ? 1 : 0;
   a.algo = s->algo;
   a.stream = (cudaStream_t)stream;
 
   int rc = -1000;
-  // AUTO: the chunked tensor-core kernel whenever it applies and the sequence is long enough to
-  // amortise its per-chunk set-up; the scan otherwise (fp32 io, GATED, decode, Temporal with auxiliary outputs).
-  const bool chunk_ok = s->io_dtype == SWILA_IO_BF16 && (s->flags & ~SWILA_TEMPORAL) == 0 && (s->Dk == 64 || s->Dk == 128) &&
-                        (s->J == 4 || s->J == 8 || (s->J == 16 && s->Dk == 64 && !r_debug && !a.p.r_sum && !a.p.r_ent &&
-                                                     !a.p.rho_sum && !a.p.rho_ent)) &&
-                        !(temporal && (r_debug || a.p.r_sum || a.p.r_ent || a.p.rho_sum || a.p.rho_ent));
+  const bool aux = r_debug || a.p.r_sum || a.p.r_ent || a.p.rho_sum || a.p.rho_ent;
+  const bool chunk_ok = chunk_covers(s, aux);
   if (s->algo == SWILA_ALGO_CHUNK || (s->algo == SWILA_ALGO_AUTO && chunk_ok && T >= 64)) {
     rc = chunk_dispatch(a);
     if (rc == -1000 && s->algo == SWILA_ALGO_CHUNK) return SWILA_ERR_UNSUPPORTED;
@@ -131,6 +176,7 @@ static int run(const swila_shape_t *s, int T, const void *q, const void *k, cons
   case DK:                                                                                      \
     if (a.gate_mode == 0) rc = scan_dispatch<DK, 0, false>(a);                                  \
     else if (a.gate_mode == 1) rc = a.post ? scan_dispatch<DK, 1, true>(a) : scan_dispatch<DK, 1, false>(a); \
+    else if (a.gate_mode == 3) rc = a.post ? scan_dispatch<DK, 3, true>(a) : scan_dispatch<DK, 3, false>(a); \
     else rc = a.post ? scan_dispatch<DK, 2, true>(a) : scan_dispatch<DK, 2, false>(a);          \
     break;
   switch (s->Dk) {
@@ -154,7 +200,13 @@ using namespace swila;
 
 extern "C" {
 
-int swila_version(void) { return 100; }
+int swila_version(void) { return 200; }
+
+int swila_auto_algo(const swila_shape_t *s, int aux_outputs) {
+  int rc = check_shape(s, true);
+  if (rc) return rc;
+  return (chunk_covers(s, aux_outputs != 0) && s->T >= 64) ? SWILA_ALGO_CHUNK : SWILA_ALGO_SCAN;
+}
 
 const char *swila_strerror(int status) {
   switch (status) {
@@ -245,7 +297,9 @@ int swila_decode_step(const swila_shape_t *s, const void *q, const void *k, cons
   int rc = check_shape(s, false);
   if (rc) return rc;
   if (!state) return SWILA_ERR_NULL;
-  return run(s, 1, q, k, v, g, state, state, o, nullptr, stream);
+  swila_shape_t one = *s;  // a single token always goes through the scan kernel (bit-equal to a scan prefill)
+  if (one.algo == SWILA_ALGO_CHUNK) one.algo = SWILA_ALGO_SCAN;
+  return run(&one, 1, q, k, v, g, state, state, o, nullptr, stream);
 }
 
 }  // extern "C"
@@ -266,9 +320,7 @@ static HostPlan host_plan(const swila_shape_t *s) {
   h.n_v = ntok * s->Dv * es;
   h.n_gate = ntok * s->J * s->Dv * es;
   h.n_tg = temporal ? ntok * s->Dv * es : 0;
-  const size_t per = s->gate_granularity == SWILA_GATE_PER_KEY ? (size_t)s->Dk
-                     : s->gate_granularity == SWILA_GATE_PER_OUT ? (size_t)s->Dv : 1;
-  h.n_alpha = gated ? ntok * s->J * per * 4 : 0;
+  h.n_alpha = gated ? alpha_elems(s, s->T) * 4 : 0;
   h.n_W = w_elems(s) * 4;
   h.n_r = temporal ? r_elems(s) * 4 : 0;
   size_t off = 0;
@@ -299,6 +351,10 @@ struct HostPipe {
   bool ready = false;
   cudaStream_t in = nullptr, out = nullptr;
   cudaEvent_t start = nullptr, done = nullptr, landed[kHostSlabs] = {}, computed[kHostSlabs] = {};
+  // Held by a call for its whole enqueue phase: every event above is recorded on one stream and waited for on
+  // another, and a wait refers to the latest record at the time it is enqueued, so the record/wait pairs of two
+  // host threads must not interleave.  (Their GPU work may: each call has its own workspace.)
+  std::mutex enqueue;
 };
 static HostPipe *host_pipe() {
   static std::mutex mu;
@@ -357,6 +413,8 @@ int swila_forward_host(const swila_shape_t *s, const void *q, const void *k, con
   HostPipe *hp = (h.total >= (64u << 20) && nbh >= 2 && sliceable) ? host_pipe() : nullptr;
   const int nslab = hp ? (int)(nbh < kHostSlabs ? nbh : kHostSlabs) : 1;
   cudaStream_t s_in = hp ? hp->in : cs, s_out = hp ? hp->out : cs;
+  std::unique_lock<std::mutex> enqueue_lock;
+  if (hp) enqueue_lock = std::unique_lock<std::mutex>(hp->enqueue);
   if (hp) {
     e = cudaEventRecord(hp->start, cs);
     if (e == cudaSuccess) e = cudaStreamWaitEvent(s_in, hp->start, 0);

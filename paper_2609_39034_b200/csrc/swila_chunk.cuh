@@ -68,19 +68,6 @@ namespace swila {
 
 // Set when a bounded wait on a completion barrier expires (never expected).
 static __device__ int g_chunk_error = 0;
-#ifdef SWILA_CHUNK_PROFILE
-// Developer build only: cycle counters per phase, kept in registers by the first thread of each warp
-// role of block 0 and written out at the end; per-block totals for every block.
-static __device__ long long g_chunk_prof[4 * 8];
-static __device__ long long g_chunk_blk[3 * 1024];  // per block: cycles, SM id, start time (ns)
-#ifdef SWILA_CHUNK_PHASES
-#define PROF_ADD(i) do { long long now_ = clock64(); prof_acc[i] += now_ - prof_t; prof_t = now_; } while (0)
-#else
-#define PROF_ADD(i) do {} while (0)
-#endif
-#else
-#define PROF_ADD(i) do {} while (0)
-#endif
 
 // How the (tile, chunk) work items are spread over the blocks of a launch.  The ntiles * nch chunks, tile
 // after tile, are cut into equal runs of `per` chunks, one run per block; within a run the piece that
@@ -300,19 +287,6 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   // row served by this thread in either 128-thread role
   const int r = tid & 127;
   const int dl = r / J, j = r % J;
-#ifdef SWILA_CHUNK_PROFILE
-  long long prof_t = clock64();
-  const long long prof_t0 = prof_t;
-  long long prof_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-  if (tid == 0 && blockIdx.x < 1024) {
-    unsigned smid;
-    unsigned long long ns;
-    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns));
-    g_chunk_blk[1024 + blockIdx.x] = smid;
-    g_chunk_blk[2048 + blockIdx.x] = (long long)ns;
-  }
-#endif
 
 #pragma unroll 1
   for (int pi = 0; pi < npieces; ++pi) {
@@ -548,10 +522,8 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       [[maybe_unused]] const __nv_bfloat16 *rgk = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_GK);  // Temporal: gate logits
       const float *Gkk = G_all + (n & 1) * C * C;
 
-      PROF_ADD(0);
       if (!mbar_wait(&bars[B_E], n & 1)) { failed = true; break; }
       tc_fence_after_sync();
-      PROF_ADD(1);
       // the readout buffer this chunk seeds below was last read by the helpers for the outputs of chunk n-2.  At
       // Dk = 128 they finish those about when chunk n-1 ends, so the wait sits here, where it has long been met; at
       // Dk = 64 they are early and the wait is cheaper at the hand-over below (both placements measured)
@@ -577,7 +549,6 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       tmem_st_wait();
       tc_fence_before_sync();
       mbar_arrive(&bars[B_PQF]);
-      PROF_ADD(4);
 
       // ---- sequential part of the chunk: E-step and the triangular key-side corrections.  Only one FMA
       //      of a token's push (into the next token's prediction) sits on the serial chain; the rest is
@@ -703,9 +674,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
           // the coefficient columns are still operands of the previous chunk's update and readout MMAs until
           // those complete (normally long before the first trip ends)
           if (tg == 0 && n > 0) {
-            PROF_ADD(6);
             if (!mbar_wait(&bars[B_QD], (n - 1) & 1)) failed = true;
-            PROF_ADD(7);
           }
           {  // GT update coefficients complete: park their bf16 parts in tensor memory, two tokens per column
             uint32_t hi[GT / 2], lo[GT / 2], l3[GT / 2];
@@ -741,7 +710,6 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         return bad;
       };
       const bool unsafe = sequential(std::false_type{}, rprev);
-      PROF_ADD(5);
       if (__any_sync(0xffffffffu, unsafe)) {
         if (lane == 0) *redo_s = 1;
         tmem_st_wait();
@@ -756,7 +724,6 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       if constexpr (RDEBUG) { st_r += chunk_r; st_h += chunk_h; }
       tmem_st_wait();
       tc_fence_before_sync();
-      PROF_ADD(2);
       // what the next steps rely on must be in place before this chunk is handed over (this also keeps every
       // barrier at most one phase ahead of its waiters): gates and Gram rows of chunk n+1
       if (n + 1 < nchunks && (!mbar_wait(&bars[B_BE], (n + 1) & 1) || !mbar_wait(&bars[B_GS], (n + 1) & 1))) failed = true;
@@ -764,7 +731,6 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         if (n > 0 && !mbar_wait(&bars[B_OD], (n - 1) & 1)) failed = true;
       }
       mbar_arrive(&bars[B_C]);
-      PROF_ADD(3);
     }
     // ---- final state row -> global ----
     if (!failed && !mbar_wait(&bars[B_U], (nchunks - 1) & 1)) failed = true;
@@ -1042,14 +1008,12 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
 #pragma unroll 1
     for (int n = 0; n < nchunks && !failed; ++n) {
       const bool more = n + 1 < nchunks;
-      PROF_ADD(0);
       if (more) {
         // (1) gates of chunk n+1 for the row warps, then its Gram batch
         if (!staged(n + 1)) { failed = true; break; }
         cook_be(smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES, min(C, Tseg - (n + 1) * C));
         if constexpr (Cf::TEMPORAL) cook_pk(smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES);
         mbar_arrive(&bars[B_BE]);
-        PROF_ADD(1);
         if (spill_mine[(n + 1) & 1]) {
           if (!mbar_wait(&bars[B_G], (n + 1) & 1)) failed = true;
           tc_fence_after_sync();
@@ -1057,7 +1021,6 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
           mbar_arrive(&bars[B_GS]);
         }
       }
-      PROF_ADD(2);
       // (2) outputs of chunk n-1, whose readouts completed shortly after chunk n started.  The row warps wait for
       // OD(n-2) at the top of chunk n, and OD must not complete another phase before they have: in every iteration
       // but the last the Gram batch spilled above was issued after the row warps passed that point (PQF(n)); in the
@@ -1068,21 +1031,16 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         write_outputs(n - 1);
         mbar_arrive(&bars[B_OD]);
       }
-      PROF_ADD(3);
       // (3) chunk n is finished by the row warps: stage chunk n+2 into the buffers chunk n used
       if (!mbar_wait(&bars[B_C], n & 1)) { failed = true; break; }
-      PROF_ADD(4);
       if (n + 2 < nchunks && h == 0) stage(n + 2);
       // (4) W has been updated with chunk n: split it into operand parts again
       if (!mbar_wait(&bars[B_U], n & 1)) { failed = true; break; }
-      PROF_ADD(5);
       if (more) {
         tc_fence_after_sync();
         refresh_parts();
         mbar_arrive(&bars[B_WP]);
       }
-      PROF_ADD(6);
-      PROF_ADD(7);
     }
     if (!failed && !mbar_wait(&bars[B_QD], (nchunks - 1) & 1)) failed = true;
     if (!failed) write_outputs(nchunks - 1);
@@ -1192,7 +1150,6 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         if (!mbar_wait(&bars[B_KQ0 + ((n + 1) & 1)], ((n + 1) >> 1) & 1) || !mbar_wait(&bars[B_PQF], n & 1)) { failed = true; break; }
         if (n > 0 && !mbar_wait(&bars[B_WP], n & 1)) { failed = true; break; }
         tc_fence_after_sync();
-        PROF_ADD(0);
         gram(n + 1);
       }
       {
@@ -1211,7 +1168,6 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       }
       if (more) {
         w_times_kq(n + 1);
-        PROF_ADD(1);
         // first half of the cross-chunk term (tokens 0-15 of chunk n, whose coefficients T0 released), while the
         // chunk still runs
         if (!mbar_wait(&bars[B_GS], (n + 1) & 1)) { failed = true; break; }
@@ -1220,7 +1176,6 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       }
       if (!mbar_wait(&bars[B_C], n & 1)) { failed = true; break; }
       tc_fence_after_sync();
-      PROF_ADD(2);
       const bool redone = *redo_s != 0;  // ordered by the barrier: set before the row warps arrived
       if (redone) *redo_s = 0;
       if (more) {
@@ -1231,8 +1186,6 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         cross(1);  // -> E(n+1): the only tensor work left between two chunks of the row warps
         mma_commit(&bars[B_E]);
       }
-      PROF_ADD(3);
-      PROF_ADD(4);
 #pragma unroll 1
       for (int ks = 0; ks < C / 16; ++ks) {  // W += Cmat K (Eq. 3.3 summed over the chunk)
         // B = the second copy of the chunk's keys, read MN-major: 16 tokens per step = 16 rows of 128 bytes, the
@@ -1244,7 +1197,6 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       }
       mma_commit(&bars[B_U]);
       readout(n);
-      PROF_ADD(5);
     }
   }
   if (failed) {
@@ -1255,12 +1207,6 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 8) tmem_dealloc(*tmem_base_s, Cf::TM_ALLOC);
-#ifdef SWILA_CHUNK_PROFILE
-  if (tid == 0 && blockIdx.x < 1024) g_chunk_blk[blockIdx.x] = clock64() - prof_t0;
-  if (blockIdx.x == 0 && (tid & 127) == 0 && tid < 512) {
-    for (int i = 0; i < 8; ++i) g_chunk_prof[(tid >> 7) * 8 + i] = prof_acc[i];
-  }
-#endif
 }
 
 // cuTensorMapEncodeTiled, fetched through the runtime so that the library does not link against the driver.
@@ -1376,6 +1322,10 @@ int launch_chunk(const LaunchArgs &a) {
       const unsigned epoch = chunk_next_epoch();
       ChunkSched ss{(int)pl.units, pl.nch, pl.per, pl.gang, epoch, flags + (size_t)(epoch % kChunkFlagSlots) * kChunkFlagTiles};
       void *args[] = {(void *)&prm, (void *)&ss, (void *)&maps};
+      // The launch starts from cleared flags: a consumer whose wait expired leaves its flag set, and a captured
+      // launch is replayed with the epoch of its capture, which its own earlier run has already published.
+      e = cudaMemsetAsync(ss.flags, 0, (size_t)pl.units * pl.gang * sizeof(unsigned), a.stream);
+      if (e == cudaSuccess)
       e = cudaLaunchCooperativeKernel((const void *)kern, dim3((unsigned)pl.grid), dim3(Cf::NT), args, Cf::SMEM_BYTES, a.stream);
       if (e == cudaSuccess) return (int)cudaGetLastError();
       (void)cudaGetLastError();  // not launched (e.g. the blocks cannot all be resident): fall back to whole tiles

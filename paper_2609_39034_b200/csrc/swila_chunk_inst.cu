@@ -1,7 +1,7 @@
 // Instantiations and dispatch of the chunked tensor-core kernel (bf16 io, ungated, plain or Temporal,
 // J in {4, 8}, and 16 at Dk = 64: with fewer components a block covers more columns and its shared-memory tiles do
 // not fit).
-#include "../../include/swila.h"
+#include "../../include/swila_dev.h"
 #include "swila_chunk.cuh"
 
 namespace swila {
@@ -57,14 +57,3 @@ extern "C" int swila_chunk_run_pieces(long long units, int nch, int per, long lo
   }
   return n;
 }
-
-#ifdef SWILA_CHUNK_PROFILE
-// Developer build only: per-phase cycle counters of block 0, 8 per warp role (rows, helpers, ...).
-extern "C" int swila_chunk_profile(long long *out32) {
-  return cudaMemcpyFromSymbol(out32, swila::g_chunk_prof, 32 * sizeof(long long)) == cudaSuccess ? 0 : -1;
-}
-// Developer build only: per block (first 1024) total cycles, SM id and start time in ns.
-extern "C" int swila_chunk_blocks(long long *out3072) {
-  return cudaMemcpyFromSymbol(out3072, swila::g_chunk_blk, 3 * 1024 * sizeof(long long)) == cudaSuccess ? 0 : -1;
-}
-#endif

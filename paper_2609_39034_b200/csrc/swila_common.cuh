@@ -32,7 +32,7 @@ constexpr float kL2Eps = 1e-6f;
 
 struct LaunchArgs {
   ScanParams p;
-  int Dk, J, io_dtype, gate_mode /*0 none, 1 per-key, 2 per-row*/, post, algo;
+  int Dk, J, io_dtype, gate_mode /*0 none, 1 per-key, 2 per-row, 3 per-element*/, post, algo;
   cudaStream_t stream;
 };
 

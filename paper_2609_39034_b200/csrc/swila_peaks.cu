@@ -4,7 +4,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-#include "../../include/swila.h"
+#include "../../include/swila_dev.h"
 
 namespace {
 

@@ -358,6 +358,10 @@ __global__ void __launch_bounds__(C::NT, C::MIN_BLOCKS) swila_scan_kernel(const 
       lds_vec<J>(ck + C::K_LK + (s * COLS + lcol) * J, lk);
       lds_vec<J>(ck + C::K_PQ + (s * COLS + lcol) * J, pq);
       if constexpr (GATE == 2) lds_vec<J>(ck + C::K_AR + (s * COLS + lcol) * J, arow);
+      // one decay value per state element (App. B.4, the general form): this thread's elements of token t are read
+      // where they are used, straight from global memory (the tensor is J*Dv*Dk values per token: no staging helps)
+      [[maybe_unused]] const float *ael = nullptr;
+      if constexpr (GATE == 3) ael = p.alpha + (((tok0 + (size_t)(t0 + s)) * J) * p.Dv + min(col, p.Dv - 1)) * DK;
 
       // ---- pass A: predictions w_jd . k_t (on the decayed state when pre-decay, Eq. 3.8) ----
       float2 acc[J];
@@ -378,6 +382,11 @@ __global__ void __launch_bounds__(C::NT, C::MIN_BLOCKS) swila_scan_kernel(const 
             const float2 a2 = make_float2(arow[j], arow[j]);
             w[j][2 * i] = mul2(w[j][2 * i], a2);
             w[j][2 * i + 1] = mul2(w[j][2 * i + 1], a2);
+          }
+          if constexpr (GATE == 3 && !POST) {
+            const float4 a4 = __ldg(reinterpret_cast<const float4 *>(ael + (size_t)j * p.Dv * DK + (i * G + g) * 4));
+            w[j][2 * i] = mul2(w[j][2 * i], make_float2(a4.x, a4.y));
+            w[j][2 * i + 1] = mul2(w[j][2 * i + 1], make_float2(a4.z, a4.w));
           }
           acc[j] = fma2(w[j][2 * i], klo, acc[j]);
           acc[j] = fma2(w[j][2 * i + 1], khi, acc[j]);
@@ -467,6 +476,11 @@ __global__ void __launch_bounds__(C::NT, C::MIN_BLOCKS) swila_scan_kernel(const 
             const float2 a2 = make_float2(arow[j], arow[j]);
             w[j][2 * i] = mul2(w[j][2 * i], a2);
             w[j][2 * i + 1] = mul2(w[j][2 * i + 1], a2);
+          }
+          if constexpr (GATE == 3 && POST) {
+            const float4 a4 = __ldg(reinterpret_cast<const float4 *>(ael + (size_t)j * p.Dv * DK + (i * G + g) * 4));
+            w[j][2 * i] = mul2(w[j][2 * i], make_float2(a4.x, a4.y));
+            w[j][2 * i + 1] = mul2(w[j][2 * i + 1], make_float2(a4.z, a4.w));
           }
           w[j][2 * i] = fma2(c2[j], klo, w[j][2 * i]);
           w[j][2 * i + 1] = fma2(c2[j], khi, w[j][2 * i + 1]);

@@ -1,7 +1,7 @@
 // Self-test of the tcgen05 plumbing used by the chunked kernel: D[128 x N] = A[128 x K] * B[N x K]^T
 // in TF32 with A placed in tensor memory by the threads, B in shared memory (K-major, no
 // swizzle), the result read back from tensor memory.  One block of 128 threads.
-#include "../../include/swila.h"
+#include "../../include/swila_dev.h"
 #include "swila_umma.cuh"
 
 namespace {

@@ -21,19 +21,38 @@ def binding():
     return b
 
 
-def _declared_functions():
-    text = open(os.path.join(ROOT, "include", "swila.h")).read()
+def _declared_functions(header="swila.h"):
+    text = open(os.path.join(ROOT, "include", header)).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b(swila_[a-z_0-9]+)\s*\(", text)))
 
 
-def test_library_exports_every_declared_symbol(binding):
-    names = _declared_functions()
-    assert "swila_forward" in names and "swila_decode_step" in names
+# The product's C ABI: the calls of the hot path (prefill, decode, state helpers, status) plus the documented
+# extras (host-buffer front ends, statistics, output norm).  Anything else belongs in swila_dev.h.
+PRODUCT_ABI = {"swila_version", "swila_strerror", "swila_last_cuda_error", "swila_device_status",
+               "swila_state_w_bytes", "swila_state_r_bytes", "swila_state_init", "swila_forward",
+               "swila_decode_step", "swila_forward_stats", "swila_output_norm",
+               "swila_forward_host", "swila_forward_host_workspace_bytes",
+               "swila_forward_host_static", "swila_forward_host_static_capacity"}
+DEV_ABI = {"swila_auto_algo", "swila_bench_fma_chain", "swila_selftest_tf32_mma", "swila_selftest_bf16_mma",
+           "swila_chunk_plan", "swila_chunk_run_pieces"}
+
+
+def test_headers_declare_exactly_the_documented_sets():
+    assert set(_declared_functions("swila.h")) == PRODUCT_ABI
+    assert set(_declared_functions("swila_dev.h")) == DEV_ABI
+
+
+def test_library_exports_every_declared_symbol_and_nothing_else(binding):
+    names = _declared_functions("swila.h") + _declared_functions("swila_dev.h")
     raw = ctypes.CDLL(binding.LIB_PATH)
     for n in names:
-        assert hasattr(raw, n), f"{n} declared in swila.h but not exported"
+        assert hasattr(raw, n), f"{n} declared in a header but not exported"
     assert set(binding.EXPORTS) <= set(names)
+    import subprocess
+    out = subprocess.run(["nm", "-D", "--defined-only", binding.LIB_PATH], capture_output=True, text=True).stdout
+    exported = {line.split()[-1] for line in out.splitlines() if " T " in line and line.split()[-1].startswith("swila_")}
+    assert exported == set(names), exported ^ set(names)
 
 
 def test_version_and_strerror(binding):
@@ -79,3 +98,36 @@ def test_forward_rejects_null_misaligned_and_aliased_pointers(binding):
     sh_t = binding.make_shape(w.variant(temporal=True))
     assert f(ctypes.byref(sh_t), a, a, a, ctypes.byref(g), None, None, a + 0x100000, None, None) == binding.ERR_NULL
     assert binding.lib.swila_decode_step(ctypes.byref(sh), a, a, a, ctypes.byref(g), None, a, None) == binding.ERR_NULL
+
+
+def test_alias_check_covers_every_written_tensor(binding):
+    """o, r_debug and the output state may overlap no streamed input and not each other; state_out == state_in is
+    allowed (in place).  Fake addresses: validation happens on the host before any launch."""
+    w = wl.CONFIGS[0].variant(temporal=True, gated=True)
+    sh = binding.make_shape(w)
+    f = binding.lib.swila_forward
+    M = 0x1000000  # 16 MB apart: far more than any tensor of this shape
+    q, k, v, be, pk, pq, gk, gq, al, o, rdbg, W, r, rho = (0x10000000 + i * M for i in range(14))
+    g = binding.Gates(be, pk, pq, gk, gq, al)
+    st = binding.State(W, r, rho)
+    call = lambda gates=g, out=o, dbg=rdbg, sin=st, sout=st: f(  # noqa: E731
+        ctypes.byref(sh), q, k, v, ctypes.byref(gates), ctypes.byref(sin) if sin else None,
+        ctypes.byref(sout) if sout else None, out, dbg, None)
+    # (every call below must fail validation: a call that passed it would launch on the fake addresses)
+    for bad in (dict(out=gk), dict(out=gq), dict(out=al), dict(dbg=q), dict(dbg=o), dict(out=W),
+                dict(sout=binding.State(k, r, rho)), dict(sout=binding.State(W, be, rho)),
+                dict(sout=binding.State(W, r, r)), dict(sout=binding.State(W + 16, r, rho))):
+        assert call(**bad) == binding.ERR_ALIAS, bad
+
+
+def test_auto_dispatch_rule(binding):
+    """What sends an AUTO call to the scan kernel, as the header states it."""
+    auto = lambda w, aux=0: binding.lib.swila_auto_algo(ctypes.byref(binding.make_shape(w)), aux)  # noqa: E731
+    lm = wl.CONFIGS[2]
+    assert auto(lm) == binding.ALGO_CHUNK and auto(lm.variant(temporal=True)) == binding.ALGO_CHUNK
+    assert auto(lm, 1) == binding.ALGO_CHUNK and auto(lm.variant(temporal=True), 1) == binding.ALGO_SCAN
+    assert auto(wl.CONFIGS[1].with_(J=16)) == binding.ALGO_CHUNK and auto(wl.CONFIGS[1].with_(J=16), 1) == binding.ALGO_SCAN
+    for w in (lm.with_(T=63), lm.with_(io_dtype="fp32"), lm.variant(gated=True), lm.with_(J=2), lm.with_(J=16),
+              wl.CONFIGS[0], wl.CONFIGS[3], lm.with_(flags=wl.FLAG_QKV_ACT)):
+        assert auto(w) == binding.ALGO_SCAN, w
+    assert auto(lm.with_(J=3)) == binding.ERR_UNSUPPORTED

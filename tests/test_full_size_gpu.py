@@ -63,10 +63,10 @@ def test_large_prefill_configs_sampled(binding, oracle, cfg, n_bh, n_cols, stres
 
 def test_batched_decode_config_sampled(binding, oracle):
     """Config 4 at full batch: 4096-token prefill fed as 16 chunks with carried state, then
-    single-token decode steps with fresh inputs; a sample of streams is replayed by the oracle
-    over the whole 4096 + n_decode token history, outputs and final state compared."""
+    all 1024 single-token decode steps with fresh inputs; a sample of streams is replayed by the oracle
+    over the whole 4096 + 1024 token history; the output of every step and the final state are compared."""
     w = wl.CONFIGS[4]
-    n_decode = 256  # enough steps to show drift; the bench times the full 1024
+    n_decode = wl.DECODE_STEPS
     bh, cols = _sample(w, 12, 8, seed=4)
     st = binding.state_alloc(w)
     chunk = wl.DECODE_PREFILL_CHUNK

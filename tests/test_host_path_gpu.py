@@ -72,3 +72,44 @@ def test_host_entry_in_slabs_equals_device_entry(binding, var, T):
         assert torch.equal(o, dev["o"]) and torch.equal(sout["W"], dev["W"])
         if w.temporal:
             assert torch.equal(sout["r_prev"], dev["r_prev"]) and torch.equal(sout["rho_prev"], dev["rho_prev"])
+
+
+def test_host_entry_from_two_threads_at_once(binding):
+    """Two host threads call the pipelined host path on one device at the same time, each with its own stream,
+    workspace and tensors; they share the library's copy streams and events.  Each must get what it gets alone."""
+    import threading
+
+    ws_ = [wl.CONFIGS[1].with_(B=3, H=5, T=2304), wl.CONFIGS[1].with_(B=2, H=8, T=2304).variant(temporal=True)]
+    jobs = []
+    for i, w in enumerate(ws_):
+        assert binding.host_workspace_bytes(w) >= 64 << 20
+        inp = wl.make_inputs(w, stress=True, seed_offset=i)
+        dev = gpu_forward(binding, w, to_dev(inp))
+        host = _pin(inp)
+        jobs.append(dict(w=w, host=host, dev=dev, stream=torch.cuda.Stream(),
+                         ws=torch.empty(binding.host_workspace_bytes(w), device="cuda", dtype=torch.uint8),
+                         sin={"W": host["W0"], "r_prev": host["r0"], "rho_prev": host["rho0"]}))
+    torch.cuda.synchronize()
+    errors = []
+
+    def work(job):
+        try:
+            for _ in range(6):
+                sout = {"W": torch.empty_like(job["host"]["W0"]).pin_memory(),
+                        "r_prev": torch.empty_like(job["host"]["r0"]).pin_memory() if job["w"].temporal else None,
+                        "rho_prev": torch.empty_like(job["host"]["rho0"]).pin_memory() if job["w"].temporal else None}
+                o = binding.swila_forward_host(job["w"], job["host"], job["ws"], state_in=job["sin"], state_out=sout,
+                                               stream=job["stream"])
+                job["stream"].synchronize()
+                if not (torch.equal(o, job["dev"]["o"]) and torch.equal(sout["W"], job["dev"]["W"])):
+                    errors.append(job["w"].name + ": result differs from the single-threaded call")
+        except Exception as e:  # noqa: BLE001
+            errors.append(repr(e))
+
+    threads = [threading.Thread(target=work, args=(j,)) for j in jobs]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    torch.cuda.synchronize()
+    assert not errors, errors

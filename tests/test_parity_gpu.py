@@ -63,6 +63,8 @@ VARIANTS = [
     dict(gated=True, granularity=wl.GRAN_PER_OUT),
     dict(gated=True, granularity=wl.GRAN_SCALAR, post_decay=True),
     dict(temporal=True, gated=True, granularity=wl.GRAN_SCALAR),
+    dict(gated=True, granularity=wl.GRAN_ELEMENTWISE),                    # one gate per state element (App. B.4)
+    dict(temporal=True, gated=True, post_decay=True, granularity=wl.GRAN_ELEMENTWISE),
 ]
 VAR_SHAPES = [SMALL[0], SMALL[2], SMALL[3], SMALL[4], SMALL[6], SMALL[10], SMALL[15]]
 
@@ -162,15 +164,19 @@ def test_chunked_kernel_extreme_prediction_errors(binding, oracle, temporal):
     got = gpu_forward(binding, w, to_dev(inp), algo=binding.ALGO_CHUNK)
     binding.device_status()
     scan = gpu_forward(binding, w, to_dev(inp), algo=binding.ALGO_SCAN)
-    # With |delta| ~ 50 the exponent delta^2/2 ~ 1e3 carries an fp32 rounding error of ~1e-4, which is the
-    # relative error of the responsibilities whatever the kernel: the state bar is relaxed to 2e-3 here.
-    # The chunked kernel's predictions also carry its 16-bit operand split (4e-6 of |w.k| ~ 50), which the
-    # same amplification by |delta| turns into a few 1e-4 of the state: the two kernels agree to 1e-3.
+    # The fp32 floor here: with |delta| up to 55 the exponent delta^2/2 is ~1.5e3, whose fp32 spacing is 2^-13 = 1.2e-4,
+    # so any fp32 evaluation of exp(-delta^2/2) -- and with it the responsibilities and the update coefficients of
+    # those tokens -- is off by ~1e-4 relative, and the coefficients are themselves ~50 times the usual size.  The
+    # chunked kernel's predictions also carry its 16-bit operand split (4e-6 of |w.k| ~ 50), amplified by |delta| the
+    # same way.  Measured state errors against the oracle on this input (B200): plain 9.8e-4 (chunk), 9.5e-4 (scan),
+    # the two kernels 7.3e-4 apart; Temporal 6.8e-4 (chunk), 1.2e-4 (scan), 6.9e-4 apart; o 3.8e-3 for all four.
+    # Each bound below is twice the measured value (the 1e-4 bar of the calm inputs is out of reach of fp32 here).
+    bound = {"chunk": 1.4e-3 if temporal else 2e-3, "scan": 2.4e-4 if temporal else 1.9e-3}
     for name, g in (("chunk", got), ("scan", scan)):
-        assert wl.rel_err(g["o"], torch.from_numpy(ref["o"])) < 2e-2, name
-        assert wl.rel_err(g["W"], torch.from_numpy(ref["W"])) < 2e-3, name
+        assert wl.rel_err(g["o"], torch.from_numpy(ref["o"])) < 8e-3, name
+        assert wl.rel_err(g["W"], torch.from_numpy(ref["W"])) < bound[name], name
         assert bool(torch.isfinite(g["W"]).all())
-    assert wl.rel_err(got["W"], scan["W"]) < 1e-3
+    assert wl.rel_err(got["W"], scan["W"]) < 1.5e-3
 
 
 def test_chunked_kernel_state_carry(binding, oracle):
@@ -245,28 +251,99 @@ def test_zero_tokens_passes_the_state_through(binding):
         assert torch.equal(sout[n], sin[n])
 
 
-def test_outputs_stay_inside_their_buffers(binding):
-    """Canary words around o and the output state must survive a call with ragged tails."""
-    w = SMALL[3]  # T=61, Dv=72: ragged token block and ragged last column slice
+def _canary(n, dtype, pad=64):
+    big = torch.full((n + 2 * pad,), 7.0, device="cuda", dtype=dtype)
+    return big, big[pad:pad + n]
+
+
+def _canaries_intact(big, n, pad=64):
+    return bool((big[:pad] == 7.0).all()) and bool((big[pad + n:] == 7.0).all())
+
+
+@pytest.mark.parametrize("algo", ["scan", "chunk"])
+@pytest.mark.parametrize("temporal", [False, True], ids=["plain", "temporal"])
+@pytest.mark.parametrize("T", [61, 99])
+def test_outputs_stay_inside_their_buffers(binding, algo, temporal, T):
+    """Canary words around everything a call writes -- o, the output state (W, r_prev, rho_prev) and the four
+    statistics buffers -- must survive a call with a ragged last token block / chunk and a ragged last column slice
+    (Dv = 72).  Both kernels; the chunked one fills tails with zeros in its tensor copies and adds its statistics
+    with atomics, and compute-sanitizer cannot be run on it here, so this is its bounds check."""
+    w = SMALL[3].with_(T=T).variant(temporal=temporal)  # Dv = 72
     inp = to_dev(wl.make_inputs(w, stress=True))
-    pad = 64
-    n_o = w.B * w.H * w.T * w.Dv
-    big_o = torch.full((n_o + 2 * pad,), 7.0, device="cuda", dtype=w.torch_io_dtype)
-    o = big_o[pad:pad + n_o].view(w.B, w.H, w.T, w.Dv)
-    n_w = w.B * w.H * w.J * w.Dv * w.Dk
-    big_w = torch.full((n_w + 2 * pad,), 7.0, device="cuda", dtype=torch.float32)
-    st = {"W": big_w[pad:pad + n_w].view(w.B, w.H, w.J, w.Dv, w.Dk), "r_prev": None, "rho_prev": None}
-    binding.swila_forward(w, inp, state_in={"W": inp["W0"]}, state_out=st, o=o)
+    with_stats = not (temporal and algo == "chunk")  # the chunked kernel forms no statistics for the Temporal variant
+    n_o, n_w, n_r = w.B * w.H * w.T * w.Dv, w.B * w.H * w.J * w.Dv * w.Dk, w.B * w.H * w.J * w.Dv
+    n_e = w.B * w.H * w.Dv
+    bufs = {"o": _canary(n_o, w.torch_io_dtype), "W": _canary(n_w, torch.float32)}
+    if temporal:
+        bufs["r_prev"], bufs["rho_prev"] = _canary(n_r, torch.float32), _canary(n_r, torch.float32)
+    if with_stats:
+        for n, cnt in (("r_sum", n_r), ("rho_sum", n_r), ("r_ent", n_e), ("rho_ent", n_e)):
+            bufs[n] = _canary(cnt, torch.float32)
+            bufs[n][1].zero_()
+    o = bufs["o"][1].view(w.B, w.H, w.T, w.Dv)
+    st = {"W": bufs["W"][1].view(w.B, w.H, w.J, w.Dv, w.Dk),
+          "r_prev": bufs["r_prev"][1].view(w.B, w.H, w.J, w.Dv) if temporal else None,
+          "rho_prev": bufs["rho_prev"][1].view(w.B, w.H, w.J, w.Dv) if temporal else None}
+    sin = {"W": inp["W0"], "r_prev": inp.get("r0"), "rho_prev": inp.get("rho0")}
+    a = getattr(binding, "ALGO_" + algo.upper())
+    if with_stats:
+        stats = {"r_sum": bufs["r_sum"][1].view(w.B, w.H, w.J, w.Dv), "rho_sum": bufs["rho_sum"][1].view(w.B, w.H, w.J, w.Dv),
+                 "r_ent": bufs["r_ent"][1].view(w.B, w.H, w.Dv), "rho_ent": bufs["rho_ent"][1].view(w.B, w.H, w.Dv)}
+        binding.swila_forward_stats(w, inp, stats, state_in=sin, state_out=st, o=o, algo=a)
+    else:
+        binding.swila_forward(w, inp, state_in=sin, state_out=st, o=o, algo=a)
     torch.cuda.synchronize()
-    for big, n in ((big_o, n_o), (big_w, n_w)):
-        assert bool((big[:pad] == 7.0).all()) and bool((big[pad + n:] == 7.0).all())
-    assert not bool((o == 7.0).all())
+    binding.device_status()
+    for name, (big, view) in bufs.items():
+        assert _canaries_intact(big, view.numel()), name
+        assert not bool((view == 7.0).all()), name
+    if with_stats:  # the responsibilities of every token sum to one over the components: the sums add up to T
+        assert torch.allclose(stats["r_sum"].sum(2), torch.full((w.B, w.H, w.Dv), float(w.T), device="cuda"), rtol=1e-3)
 
 
-def test_inputs_are_not_written(binding):
-    w = SMALL[2].variant(temporal=True, gated=True)
+@pytest.mark.parametrize("temporal", [False, True], ids=["plain", "temporal"])
+def test_state_handed_over_between_blocks_stays_inside_its_buffers(binding, temporal):
+    """More tiles than SMs: the chunked kernel cuts the chunk sequence into equal runs and a tile that falls into two
+    runs travels through the state output.  Canaries around the output state and o."""
+    w = wl.CONFIGS[2].with_(B=2, H=20, T=1024, recipe="gauss").variant(temporal=temporal)
+    inp = wl.make_inputs(w, device="cuda", stress=True)
+    n_o, n_w, n_r = w.B * w.H * w.T * w.Dv, w.B * w.H * w.J * w.Dv * w.Dk, w.B * w.H * w.J * w.Dv
+    bufs = {"o": _canary(n_o, w.torch_io_dtype), "W": _canary(n_w, torch.float32)}
+    if temporal:
+        bufs["r_prev"], bufs["rho_prev"] = _canary(n_r, torch.float32), _canary(n_r, torch.float32)
+    st = {"W": bufs["W"][1].view(w.B, w.H, w.J, w.Dv, w.Dk),
+          "r_prev": bufs["r_prev"][1].view(w.B, w.H, w.J, w.Dv) if temporal else None,
+          "rho_prev": bufs["rho_prev"][1].view(w.B, w.H, w.J, w.Dv) if temporal else None}
+    sin = {"W": inp["W0"], "r_prev": inp.get("r0"), "rho_prev": inp.get("rho0")}
+    binding.swila_forward(w, inp, state_in=sin, state_out=st, o=bufs["o"][1].view(w.B, w.H, w.T, w.Dv), algo=binding.ALGO_CHUNK)
+    torch.cuda.synchronize()
+    binding.device_status()
+    for name, (big, view) in bufs.items():
+        assert _canaries_intact(big, view.numel()), name
+        assert bool(torch.isfinite(view.float()).all()), name
+
+
+@pytest.mark.parametrize("case", ["scan_gated_temporal", "chunk_plain", "chunk_temporal"])
+def test_inputs_are_not_written(binding, case):
+    if case == "scan_gated_temporal":
+        w, algo = SMALL[2].variant(temporal=True, gated=True), binding.ALGO_AUTO
+    else:
+        w, algo = SMALL[3].with_(T=99).variant(temporal=case == "chunk_temporal"), binding.ALGO_CHUNK
     inp = to_dev(wl.make_inputs(w, stress=True))
     before = {n: x.clone() for n, x in inp.items() if x is not None}
-    gpu_forward(binding, w, inp)
+    gpu_forward(binding, w, inp, algo=algo)
     for n, x in before.items():
         assert torch.equal(x, inp[n]), n
+
+
+def test_decode_step_ignores_a_request_for_the_chunked_kernel(binding):
+    """A decode step always runs the scan kernel: with algo = CHUNK in the shape it gives the bits of the default."""
+    w = SMALL[4].with_(T=1)
+    inp = to_dev(wl.make_inputs(w, stress=True))
+    outs = []
+    for algo in (binding.ALGO_AUTO, binding.ALGO_CHUNK):
+        st = {"W": inp["W0"].clone(), "r_prev": None, "rho_prev": None}
+        o = binding.swila_decode_step(w, inp, st, algo=algo)
+        torch.cuda.synchronize()
+        outs.append((o.clone(), st["W"].clone()))
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])

@@ -40,7 +40,7 @@ def test_static_entry_rejects_problems_beyond_its_capacity():
 
 
 @pytest.mark.gpu
-def test_static_entry_matches_workspace_entry_on_two_calls_in_a_row():
+def test_static_entry_matches_workspace_entry_on_two_calls_in_a_row(oracle):
     assert torch.cuda.is_available()
     b = _binding()
     problems = [wl.CONFIGS[1].with_(B=2, H=3, T=75).variant(temporal=True, gated=True),
@@ -67,5 +67,9 @@ def test_static_entry_matches_workspace_entry_on_two_calls_in_a_row():
         if w.temporal:
             assert wl.rel_err(got_state["r_prev"], ref_state["r_prev"]) < TOL_STATE
             assert wl.rel_err(got_state["rho_prev"], ref_state["rho_prev"]) < TOL_STATE
+        # and against the fp64 oracle directly, so that this test stands without the workspace entry point's own
+        ref = oracle.forward_inputs(inp, flags=w.flags, gran=w.gate_granularity)
+        assert wl.rel_err(got_o, torch.from_numpy(ref["o"])) < TOL_BF16_O, f"call {i}: o against the oracle"
+        assert wl.rel_err(got_state["W"], torch.from_numpy(ref["W"])) < TOL_STATE, f"call {i}: W against the oracle"
         # same kernel, same inputs: in fact the two entry points agree to the bit
         assert torch.equal(got_o, ref_o) and torch.equal(got_state["W"], ref_state["W"])
