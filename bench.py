@@ -34,9 +34,21 @@ METRIC = "swila_fwd_tokens_per_s"
 UNIT = "tokens/s"
 HEADLINE = 2  # config index of the workload the metric is quoted on
 
-# DRAM traffic of one launch on the headline workload, from the ncu captures summarised under
-# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum: 2.172 GB chunked kernel, 2.188 GB scan kernel).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 2.172e9
+# DRAM traffic per launch comes from profiles/traffic.json (ncu: dram__bytes_read.sum + dram__bytes_write.sum of one
+# captured launch), keyed by kernel and workload; an entry counts only while the kernel source it was captured from
+# is unchanged (sha256 of the file), else the bench line reports null.
+def ncu_traffic(kernel: str, workload: str):
+    import hashlib
+
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    if not os.path.exists(path):
+        return None
+    for e in json.load(open(path)).get("entries", []):
+        if e.get("kernel") == kernel and e.get("workload") == workload:
+            src = os.path.join(ROOT, e.get("source", ""))
+            if os.path.exists(src) and hashlib.sha256(open(src, "rb").read()).hexdigest()[:16] == e.get("source_sha16"):
+                return e.get("dram_bytes_per_launch")
+    return None
 
 
 # ----------------------------------------------------------------------------------------------
@@ -48,7 +60,8 @@ def algorithmic_bytes(w: wl.Workload) -> float:
     if w.temporal:
         per_tok_head += 2 * w.Dv * es
     if w.gated:
-        per = {wl.GRAN_PER_KEY: w.Dk, wl.GRAN_PER_OUT: w.Dv, wl.GRAN_SCALAR: 1}[w.gate_granularity]
+        per = {wl.GRAN_PER_KEY: w.Dk, wl.GRAN_PER_OUT: w.Dv, wl.GRAN_SCALAR: 1,
+               wl.GRAN_ELEMENTWISE: w.Dk * w.Dv}[w.gate_granularity]
         per_tok_head += w.J * per * 4
     state = 2 * w.J * w.Dk * w.Dv * 4
     return float(w.B * w.H * (w.T * per_tok_head + state))
@@ -126,6 +139,17 @@ def max_over_ranks(ms: float, world: int, device="cpu") -> float:
 def whole_job_tokens_per_s(world: int, B: int, T: int, ms_per_step: float) -> float:
     """Independent replicas (weak scaling): every rank processes its own B x T tokens per step."""
     return world * B * T / (ms_per_step * 1e-3)
+
+
+def time_blocks(fn, steps: int, stream, min_seconds: float = 2.0, max_blocks: int = 400):
+    """Blocks of `steps` back-to-back calls, each block timed with its own CUDA event pair, repeated until
+    `min_seconds` of device time have been covered: the per-step times of the blocks (ms)."""
+    out, total = [], 0.0
+    while not out or (total < min_seconds * 1e3 and len(out) < max_blocks):
+        ms = time_steps(fn, steps, stream)
+        out.append(ms / steps)
+        total += ms
+    return out
 
 
 def time_steps(fn, steps: int, stream) -> float:
@@ -277,7 +301,7 @@ def paper_shapes_leg(binding, stream):
                                        "tokens_per_s": lm16.B * lm16.T / (ms * 1e-3)}
     del inp, o, st
     gen_out = []
-    for B in (1, 8, 128):
+    for B in (1, 2, 4, 8, 16, 32, 64, 128):
         g = wl.CONFIGS[1].with_(name="generation", B=B, H=8, T=2048)
         prompt = wl.make_inputs(g, device="cuda")
         steps = [wl.decode_step_inputs(g, s, device="cuda") for s in range(128)]
@@ -300,14 +324,29 @@ def paper_shapes_leg(binding, stream):
 
 
 def variants_leg(binding, stream, fma_peak_tflops: float):
-    """The Temporal and Gated variants (App. B.3, Eqs. 3.7-3.8) on all five configurations: prefill time per
-    variant for configs 0-3, decode time per step for config 4 (after a 256-token prefill).  Every variant runs in
-    the scan kernel; the vanilla line is there for comparison (AUTO: the chunked kernel where it applies)."""
+    """The Temporal and Gated variants (App. B.3, Eqs. 3.7-3.8, App. B.4) on all five configurations: prefill time per
+    variant for configs 0-3, decode time per step for config 4 (after a 256-token prefill).  Every line is ALGO_AUTO;
+    `kernel` says which kernel that resolved to, and `roofline` is taken against the slower bound of that kernel's
+    pipes: the FP32 ALUs (3 FMAs per state element and token, one more multiply when gated) or HBM for the scan, HBM
+    or the bf16 tensor peak for the chunked kernel."""
     names = [("vanilla", {}), ("temporal", dict(temporal=True)), ("gated_pre_per_key", dict(gated=True)),
              ("gated_post_per_key", dict(gated=True, post_decay=True)),
              ("gated_pre_per_out", dict(gated=True, granularity=wl.GRAN_PER_OUT)),
+             ("gated_pre_scalar", dict(gated=True, granularity=wl.GRAN_SCALAR)),
              ("gated_temporal", dict(temporal=True, gated=True))]
     peaks = _peaks()
+
+    def roofline(w, ms, chunk):
+        sec = ms * 1e-3
+        t_hbm = algorithmic_bytes(w) / (peaks["hbm_gbs"] * 1e9)
+        if chunk:
+            t_pipe, pipe = algorithmic_flops(w) / (peaks["bf16_tflops"] * 1e12), "tensor"
+        else:  # FP32 instruction slots: 3 FMAs (+ 1 multiply when gated) per state element and token, 2 flop each slot
+            slots = (4.0 if w.gated else 3.0) / 3.0 * algorithmic_flops(w)
+            t_pipe, pipe = slots / (fma_peak_tflops * 1e12), "alu"
+        bound = "hbm" if t_hbm >= t_pipe else pipe
+        return {"bound": bound, "frac": max(t_hbm, t_pipe) / sec, "t_hbm_ms": t_hbm * 1e3, "t_pipe_ms": t_pipe * 1e3}
+
     out = {}
     for cfg in (0, 1, 2, 3):
         rows = {}
@@ -321,9 +360,9 @@ def variants_leg(binding, stream, fma_peak_tflops: float):
                 f()
             torch.cuda.synchronize()
             ms = time_steps(f, 10, stream) / 10
-            tfl = algorithmic_flops(w) / (ms * 1e-3) / 1e12
-            rows[name] = {"ms": ms, "tokens_per_s": w.B * w.T / (ms * 1e-3), "alu_frac": tfl / fma_peak_tflops,
-                          "hbm_frac": algorithmic_bytes(w) / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+            chunk = binding.auto_algo(w) == binding.ALGO_CHUNK
+            rows[name] = {"ms": ms, "tokens_per_s": w.B * w.T / (ms * 1e-3), "kernel": "chunk" if chunk else "scan",
+                          "roofline": roofline(w, ms, chunk)}
             del inp, st, o
         out[wl.CONFIGS[cfg].name] = rows
     rows = {}
@@ -345,8 +384,9 @@ def variants_leg(binding, stream, fma_peak_tflops: float):
             step()
         torch.cuda.synchronize()
         ms = time_steps(step, 64, stream) / 64
-        rows[name] = {"ms_per_step": ms, "steps_per_s": 1e3 / ms,
-                      "hbm_frac": algorithmic_bytes(w.with_(T=1)) / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}
+        rows[name] = {"ms_per_step": ms, "steps_per_s": 1e3 / ms, "kernel": "scan",
+                      "roofline": {"bound": "hbm",
+                                   "frac": algorithmic_bytes(w.with_(T=1)) / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}}
         del st, steps, o1
     out[wl.CONFIGS[4].name + "_decode"] = rows
     return out
@@ -409,15 +449,24 @@ def main():
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     ap.add_argument("--no-scan", action="store_true", help="skip the scan-kernel comparison leg")
-    ap.add_argument("--paper-shapes", action="store_true", help="also time the shapes the paper itself quotes")
-    ap.add_argument("--variants", action="store_true", help="also time the Temporal / Gated variants on all five configs")
-    ap.add_argument("--fusions", action="store_true", help="also time the q/k/v activation, the statistics and the output norm")
+    ap.add_argument("--no-paper-shapes", action="store_true", help="skip the shapes the paper itself quotes")
+    ap.add_argument("--no-variants", action="store_true", help="skip the Temporal / Gated variants on all five configs")
+    ap.add_argument("--no-fusions", action="store_true", help="skip the q/k/v activation, the statistics and the output norm")
+    ap.add_argument("--only-headline", action="store_true", help="time the headline step only (profiling runs)")
+    ap.add_argument("--min-seconds", type=float, default=2.0, help="repeat the block of --steps until this much is timed")
+    # accepted for older command lines; these legs now run by default
+    ap.add_argument("--paper-shapes", action="store_true", help=argparse.SUPPRESS)
+    ap.add_argument("--variants", action="store_true", help=argparse.SUPPRESS)
+    ap.add_argument("--fusions", action="store_true", help=argparse.SUPPRESS)
     ap.add_argument("--decode-steps", type=int, default=wl.DECODE_STEPS)
     ap.add_argument("--decode-prefill", type=int, default=4096)
     ap.add_argument("--decode-batch", type=int, default=0, help="override B of the decode leg (0 = 256)")
     ap.add_argument("--batch", type=int, default=0, help="override B of the prefill workload (profiling only)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.only_headline:
+        args.no_decode = args.no_e2e = args.no_cpu = args.no_scan = True
+        args.no_paper_shapes = args.no_variants = args.no_fusions = True
 
     if args.impl == "reference":
         run_reference(args)
@@ -460,14 +509,20 @@ def main():
     for _ in range(args.warmup):
         step()
     barrier()
+    # Timed region: blocks of exactly --steps launches, each with its own event pair, repeated until --min-seconds
+    # have been covered, so that the clock samples below see the load.  ms_per_step is the median block; the minimum
+    # and the block count are reported beside it.
     sampler = ClockSampler(local)
     sampler.start()
-    ms = time_steps(step, args.steps, stream)
+    blocks = time_blocks(step, args.steps, stream, args.min_seconds)
     barrier()
     clocks = sampler.stop()
-    ms = max_over_ranks(ms, world, "cuda")
-    ms_per_step = ms / args.steps
+    ms_per_step = max_over_ranks(statistics.median(blocks), world, "cuda")
+    ms_min = max_over_ranks(min(blocks), world, "cuda")
     value = whole_job_tokens_per_s(world, w.B, w.T, ms_per_step)
+    timing = {"blocks": len(blocks), "steps_per_block": args.steps, "ms_per_step_median": ms_per_step,
+              "ms_per_step_min": ms_min, "timed_seconds": sum(blocks) * args.steps * 1e-3,
+              "ms_x_sm_mhz": ms_per_step * clocks["sm_mhz"] if clocks.get("sm_mhz") else None}
 
     # ---- roofline of the kernel the step launches (one launch per step) ----
     props = torch.cuda.get_device_properties(local)
@@ -487,7 +542,7 @@ def main():
         roofline = {
             "bound": "hbm", "achieved": abytes / sec / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
             "frac": abytes / sec / 1e9 / peaks["hbm_gbs"], "peak_source": peaks["source"],
-            "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if not args.batch else None,
+            "traffic": ncu_traffic("swila_chunk_kernel", w.name) if not args.batch else None,
             "algorithmic_bytes_per_launch": abytes, "algorithmic_flops_per_launch": flops,
             "kernel": "swila_chunk_kernel",
             "tensor_bound": {"achieved_tflops": flops / sec / 1e12, "peak_tflops": bf16_peak,
@@ -502,7 +557,7 @@ def main():
             "bound": "alu", "achieved": ach_tflops, "peak": fma_peak_nominal, "unit": "TFLOP/s",
             "frac": ach_tflops / fma_peak_nominal, "peak_source": "derived: SMs x 128 FP32 lanes x 2 x 1.965 GHz",
             "peak_measured_fma_chain": fma_peak_measured, "frac_of_measured_fma_chain": ach_tflops / fma_peak_measured,
-            "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH if not args.batch else None,
+            "traffic": ncu_traffic("swila_scan_kernel", w.name) if not args.batch else None,
             "algorithmic_bytes_per_launch": abytes, "algorithmic_flops_per_launch": flops,
             "hbm_achieved_gbs": abytes / sec / 1e9, "hbm_peak_gbs": peaks["hbm_gbs"], "kernel": "swila_scan_kernel",
         }
@@ -559,13 +614,14 @@ def main():
         decode = decode_leg(binding, args, stream, local)
         torch.cuda.empty_cache()
 
-    paper = paper_shapes_leg(binding, stream) if args.paper_shapes else None
-    variants = variants_leg(binding, stream, fma_peak_nominal) if args.variants else None
-    fusions = fusions_leg(binding, stream) if args.fusions else None
+    extras = world == 1  # the further legs describe one GPU; a scaling run times the headline step only
+    paper = paper_shapes_leg(binding, stream) if extras and not args.no_paper_shapes else None
+    variants = variants_leg(binding, stream, fma_peak_nominal) if extras and not args.no_variants else None
+    fusions = fusions_leg(binding, stream) if extras and not args.no_fusions else None
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
-        n_bh = 32
+        n_bh = wl.CONFIGS[HEADLINE].B * wl.CONFIGS[HEADLINE].H  # the whole workload: a few seconds on 16 cores
         val, sec, cores = cpu_baseline(wl.CONFIGS[HEADLINE], n_bh)
         cpu = {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "seconds": sec,
                "sample": f"{n_bh} of {wl.CONFIGS[HEADLINE].B * wl.CONFIGS[HEADLINE].H} (batch, head) rows, all tokens "
@@ -578,10 +634,14 @@ def main():
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "B": w.B, "H": w.H, "T": w.T, "Dk": w.Dk, "Dv": w.Dv, "J": w.J,
                        "io_dtype": w.io_dtype, "state_dtype": "fp32", "algo": args.algo,
+                       "arithmetic": "E-step, corrections inside a chunk and every accumulation in fp32",
+                       "mma_operands": ("bf16 hi+lo (16 bit) for the state and Gram operands, update coefficients 24 bit, "
+                                        "k and q exact bf16, fp32 accumulate") if chunked else None,
+                       "error_measure": "max |x - y| / max(|y|, rms(y)) per tensor against the fp64 oracle",
                        "l2": "inputs (2.1 GB) larger than L2; no flush needed",
                        "multi_gpu": "independent replicas, no collective"},
-            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": args.steps,
-            "clocks": clocks, "decode": decode, "scan": scan, "paper_shapes": paper, "variants": variants, "fusions": fusions,
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": args.steps * len(blocks),
+            "timing": timing, "clocks": clocks, "decode": decode, "scan": scan, "paper_shapes": paper, "variants": variants, "fusions": fusions,
         }
         print(json.dumps(line))
     if world > 1:

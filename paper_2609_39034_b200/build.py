@@ -23,16 +23,27 @@ DKS = (16, 64, 128)
 GATE_MODES = ((0, 0), (1, 0), (1, 1), (2, 0), (2, 1), (3, 0), (3, 1))  # (decay mode, post-decay)
 
 
-def _sources():
-    return sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC)) + sorted(os.path.join(INC, f) for f in os.listdir(INC))
+def _deps(path, seen=None):
+    """The file and every file it includes with #include "..." (recursively), as absolute paths."""
+    seen = set() if seen is None else seen
+    path = os.path.normpath(path)
+    if path in seen or not os.path.exists(path):
+        return seen
+    seen.add(path)
+    for line in open(path, errors="replace"):
+        line = line.strip()
+        if line.startswith("#include \""):
+            _deps(os.path.join(os.path.dirname(path), line.split('"')[1]), seen)
+    return seen
 
 
-def _stamp() -> str:
+def _unit_stamp(unit) -> str:
+    name, src, defs = unit
     h = hashlib.sha256()
-    for f in _sources():
+    for f in sorted(_deps(src)):
         h.update(f.encode())
         h.update(open(f, "rb").read())
-    h.update(" ".join(NVCC_FLAGS).encode())
+    h.update(" ".join(NVCC_FLAGS + defs).encode())
     return h.hexdigest()
 
 
@@ -61,25 +72,35 @@ def _compile(unit, verbose):
 
 
 def build(force: bool = False, verbose: bool = False, jobs: int | None = None) -> str:
+    """Compile what changed (an object is rebuilt when its source, a file it includes or the flags change) and link."""
     os.makedirs(OBJ, exist_ok=True)
-    stamp_file = os.path.join(OBJ, "stamp")
-    stamp = _stamp()
-    if not force and os.path.exists(LIB) and os.path.exists(stamp_file) and open(stamp_file).read() == stamp:
-        return LIB
     units = _units()
-    jobs = jobs or min(len(units), os.cpu_count() or 4)
-    objs, logs = [], []
-    with cf.ThreadPoolExecutor(max_workers=jobs) as ex:
-        for out, log in ex.map(lambda u: _compile(u, verbose), units):
-            objs.append(out)
-            logs.append(log)
+    stamps = {u[0]: _unit_stamp(u) for u in units}
+    stale = []
+    for u in units:
+        sf = os.path.join(OBJ, u[0] + ".stamp")
+        if force or not os.path.exists(os.path.join(OBJ, u[0])) or not os.path.exists(sf) or open(sf).read() != stamps[u[0]]:
+            stale.append(u)
+    link_stamp = hashlib.sha256("".join(sorted(stamps.values())).encode()).hexdigest()
+    link_file = os.path.join(OBJ, "stamp")
+    if not stale and os.path.exists(LIB) and os.path.exists(link_file) and open(link_file).read() == link_stamp:
+        return LIB
+    logs = []
+    if stale:
+        jobs = jobs or min(len(stale), os.cpu_count() or 4)
+        with cf.ThreadPoolExecutor(max_workers=jobs) as ex:
+            for (name, _, _), (out, log) in zip(stale, ex.map(lambda u: _compile(u, verbose), stale)):
+                logs.append(log)
+                with open(os.path.join(OBJ, name + ".stamp"), "w") as f:
+                    f.write(stamps[name])
+    objs = [os.path.join(OBJ, u[0]) for u in units]
     tmp = LIB + f".tmp{os.getpid()}"
     r = subprocess.run(["nvcc", "-shared", "-o", tmp, *objs, "-lcudart"], capture_output=True, text=True)
     if r.returncode != 0:
         raise RuntimeError(f"link failed:\n{r.stdout}\n{r.stderr}")
     os.replace(tmp, LIB)
-    with open(stamp_file, "w") as f:
-        f.write(stamp)
+    with open(link_file, "w") as f:
+        f.write(link_stamp)
     if verbose:
         sys.stderr.write("\n".join(logs))
     return LIB

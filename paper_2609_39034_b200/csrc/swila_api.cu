@@ -3,6 +3,7 @@
 // their events) that the host-buffer front end creates per device on first use for problems of 64 MB and more.  (The
 // library image itself carries three device arrays: the staging array of the allocation-free entry point, and the
 // hand-over flags and the error word of the chunked kernel.)
+#include <stdio.h>
 #include <string.h>
 
 #include <mutex>
@@ -20,7 +21,9 @@ SWILA_DECL_DK(64)
 SWILA_DECL_DK(128)
 
 int chunk_dispatch(const LaunchArgs &a);
+int chunk_gated_dispatch(LaunchArgs &a);
 int chunk_error_fetch(int *flag);
+int chunk_gated_error_fetch(int *flag);
 
 static thread_local char g_cuda_err[256] = "";
 
@@ -76,7 +79,12 @@ static bool overlaps(const void *a, size_t na, const void *b, size_t nb) {
 // {64, 128}, J in {4, 8} or J = 16 at Dk = 64, plain or Temporal; auxiliary outputs (r_debug, statistics) only for
 // plain shapes with J <= 8.
 static bool chunk_covers(const swila_shape_t *s, bool aux) {
-  if (s->io_dtype != SWILA_IO_BF16 || (s->flags & ~SWILA_TEMPORAL) != 0 || (s->Dk != 64 && s->Dk != 128)) return false;
+  if (s->io_dtype != SWILA_IO_BF16 || (s->Dk != 64 && s->Dk != 128)) return false;
+  if (s->flags & SWILA_QKV_ACT) return false;
+  if (s->flags & SWILA_GATED) {  // one decay per state row (per output dimension, or per component), pre- or post-decay
+    if (s->gate_granularity != SWILA_GATE_PER_OUT && s->gate_granularity != SWILA_GATE_SCALAR) return false;
+    return !(s->flags & SWILA_TEMPORAL) && (s->J == 4 || (s->J == 8 && s->Dk == 64)) && !aux;
+  }
   if (!(s->J == 4 || s->J == 8 || (s->J == 16 && s->Dk == 64))) return false;
   if (aux && ((s->flags & SWILA_TEMPORAL) || s->J == 16)) return false;
   return true;
@@ -151,6 +159,7 @@ static int run(const swila_shape_t *s, int T, const void *q, const void *k, cons
   a.p.o = o;
   a.p.r_debug = r_debug;
   a.p.qkv_act = (s->flags & SWILA_QKV_ACT) ? 1 : 0;
+  a.p.post = (s->flags & SWILA_POST_DECAY) ? 1 : 0;
   if (stats) {
     a.p.r_sum = stats->r_sum; a.p.r_ent = stats->r_ent;
     a.p.rho_sum = stats->rho_sum; a.p.rho_ent = stats->rho_ent;
@@ -165,11 +174,16 @@ static int run(const swila_shape_t *s, int T, const void *q, const void *k, cons
   const bool aux = r_debug || a.p.r_sum || a.p.r_ent || a.p.rho_sum || a.p.rho_ent;
   const bool chunk_ok = chunk_covers(s, aux);
   if (s->algo == SWILA_ALGO_CHUNK || (s->algo == SWILA_ALGO_AUTO && chunk_ok && T >= 64)) {
-    rc = chunk_dispatch(a);
+    const bool gated_rows = gated && a.gate_mode == 2;
+    rc = gated_rows ? chunk_gated_dispatch(a) : chunk_dispatch(a);
     if (rc == -1000 && s->algo == SWILA_ALGO_CHUNK) return SWILA_ERR_UNSUPPORTED;
     if (rc != -1000) {
       if (rc != 0) return cuda_fail((cudaError_t)rc);
-      return SWILA_OK;
+      if (!gated_rows) return SWILA_OK;
+      // Gated rows: the scan kernel is launched behind the chunked one; exactly one of the two does the work,
+      // as the guard pass over the decays has decided (chunk_gated_dispatch)
+      a.p.guard_runs_scan = 1;
+      a.algo = SWILA_ALGO_SCAN;
     }
   }
 #define SWILA_CASE(DK)                                                                          \
@@ -226,10 +240,14 @@ const char *swila_last_cuda_error(void) { return g_cuda_err; }
 
 int swila_device_status(void) {
   int flag = 0;
-  cudaError_t e = (cudaError_t)chunk_error_fetch(&flag);
+  cudaError_t e = (cudaError_t)chunk_error_fetch(&flag);  // (the error word exists once per translation unit)
   if (e != cudaSuccess) return cuda_fail(e);
-  if (flag) {
-    strncpy(g_cuda_err, "a tensor-core completion wait expired inside the chunked kernel", sizeof(g_cuda_err) - 1);
+  if (!flag) {
+    e = (cudaError_t)chunk_gated_error_fetch(&flag);
+    if (e != cudaSuccess) return cuda_fail(e);
+  }
+  if (flag) {  // (warp + 1) * 256 + barrier slot of the first wait that gave up; 1 if only the hand-over flag did
+    snprintf(g_cuda_err, sizeof(g_cuda_err), "a bounded wait expired inside the chunked kernel (code 0x%x)", flag);
     return SWILA_ERR_CUDA;
   }
   return SWILA_OK;

@@ -89,16 +89,20 @@ static __device__ unsigned g_chunk_flags[kChunkFlagSlots][kChunkFlagTiles];
 
 // TEMPORAL_: Temporal SwiLA (App. B.3): two more streamed inputs (the temporal gate logits), the key-side prior
 // normalised by the helpers (it enters a convex combination), and two carried distributions per row.
-template <int J_, int DK_, bool TEMPORAL_ = false>
+// GATED_: Gated SwiLA (Sec. 3.4) with one decay value per state ROW and token: alpha_tjd (Eq. 3.7 / 3.8 as printed,
+// "Diag(alpha_tj) W" of App. B.4) or one per component.  A row's state is then a scalar multiple of an undecayed
+// one, w_t = A_t (w_0 + sum_{s<=t} (c_s / A_s) k_s) with A_t the product of the row's decays since the chunk began,
+// so the Gram matrices stay shared by all rows and the decay enters as per-row scalars on the FP32 ALUs.
+template <int J_, int DK_, bool TEMPORAL_ = false, bool GATED_ = false>
 struct ChunkCfg {
   static constexpr int J = J_, DK = DK_;
-  static constexpr bool TEMPORAL = TEMPORAL_;
+  static constexpr bool TEMPORAL = TEMPORAL_, GATED = GATED_;
   static constexpr int C = 32;            // tokens per chunk
   static constexpr int WIN = 24;          // tokens ahead (incl. its own trip) that a token's pushes reach on the ALUs;
                                           // the pushes of tokens 0-7 into tokens 24-31 go through the tensor cores
   static constexpr int GT = 8;            // tokens per trip of the rolled loops (keeps the hot code inside the instruction cache)
   static constexpr int NROW = 128;        // row threads = rows of the tile
-  static constexpr int NT = 288;          // 4 row warps + 4 helper warps + 1 MMA warp
+  static constexpr int NT = GATED_ ? 320 : 288;  // 4 row warps + 4 helper warps + 1 MMA warp (+ 1 decay warp when Gated)
   static constexpr int COLS = NROW / J;   // output columns per block
   static constexpr int ES = 2;            // bf16 io
   // tensor-memory columns.  W: the state (FP32 accumulator); WHI / WLO: its bf16 operand parts, two key
@@ -128,7 +132,7 @@ struct ChunkCfg {
   // A fourth slot mirrors slot 0 (a chunk that goes to slot 0 is copied there too), so that the pair is adjacent
   // also when the ring wraps: (slot 2, slot 3).  Not in the Temporal kernel at Dk = 128, which is not bound by its
   // MMA count and measured 1 % slower with the extra copies (two MMAs per K step on those chunks there).
-  static constexpr bool KU_MIRROR = !(TEMPORAL && DK == 128);
+  static constexpr bool KU_MIRROR = !((TEMPORAL || GATED) && DK == 128);
   static constexpr int KU_HALF = C * 128;        // one slot of one half
   static constexpr int KU_HSTRIDE = (KU_MIRROR ? 4 : 3) * KU_HALF;  // distance between the halves
   static constexpr int KU_BYTES = (DK / 64) * KU_HALF;
@@ -174,8 +178,12 @@ struct ChunkCfg {
   static constexpr int OFF_P0 = OFF_FAR + 2 * 2 * FAR_TILE;  // [C/4][NROW] float4: a chunk's P0 rows, kept for the rare redo
   static constexpr int OFF_RP = OFF_P0 + C * NROW * 4;  // Temporal: [NROW] fp32, a piece's initial r_prev, helpers -> row warps
   static constexpr int OFF_OS = OFF_RP + (TEMPORAL ? NROW * 4 : 0);  // J = 16: [C][COLS][J] fp32, a chunk's readouts regrouped by output
-  static constexpr int OFF_BAR = OFF_OS + (J > 8 ? C * NROW * 4 : 0);
-  static constexpr int SMEM_BYTES = OFF_BAR + 128 + 1024;  // + 1024: the kernel aligns its window to 1024 bytes
+  // Gated: 2 x [C + 1][NROW] fp32, the running products of a chunk's decays per row: entry t + 1 holds A_t, entry 0
+  // is 1 (the pre-decay form of Eq. 3.8 predicts with A_t, the post-decay form of Eq. 3.7 with A_{t-1})
+  static constexpr int OFF_A = OFF_OS + (J > 8 ? C * NROW * 4 : 0);
+  static constexpr int A_STAGE = (C + 1) * NROW * 4;
+  static constexpr int OFF_BAR = OFF_A + (GATED ? 2 * A_STAGE : 0);
+  static constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;  // barriers and three words; + 1024: the kernel aligns its window to 1024 bytes
   static_assert(R_GK % 128 == 0 && RQ_GQ % 128 == 0, "temporal gate rows start 128-byte aligned");
   static_assert(RAW_BYTES % 128 == 0 && RPQ_BYTES % 128 == 0 && R_B % 128 == 0 && R_PK % 128 == 0 && OFF_RAW % 128 == 0 &&
                     OFF_RPQ % 128 == 0 && OFF_TILE % 1024 == 0 && OFF_KU % 1024 == 0 && KU_BYTES % 1024 == 0 && DK % 64 == 0 && (COLS * ES) % 16 == 0 && (GROW * ES) % 16 == 0,
@@ -189,7 +197,8 @@ struct ChunkCfg {
 // (Gram batch spilled, 2 helper warps), C (chunk finished, 128 rows), PQF ([P0|Q0] taken out of tensor memory, 128
 // rows), BE (gates of a chunk ready, 128 helpers), OD (outputs of a chunk formed, 128 helpers), T0 (update
 // coefficients of a chunk's first 8 tokens stored, 128 rows).
-enum { B_E = 0, B_G, B_U, B_QD, B_KQ0, B_KQ1, B_WP, B_GS, B_C, B_PQF, B_BE, B_OD, B_T0, B_FAR, B_COUNT };
+// Gated only: A (running decay products of a chunk in place, 32 lanes of the decay warp).
+enum { B_E = 0, B_G, B_U, B_QD, B_KQ0, B_KQ1, B_WP, B_GS, B_C, B_PQF, B_BE, B_OD, B_T0, B_FAR, B_A, B_COUNT };
 
 // bf16 split of FP32 values: hi = bf16(x) (nearest), lo = bf16(x - hi); pairs packed with the first
 // value in the low half, which is where the tensor cores expect the even K index.
@@ -258,6 +267,13 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   constexpr int J = Cf::J, DK = Cf::DK, C = Cf::C, NROW = Cf::NROW, COLS = Cf::COLS;
   static_assert(!(RDEBUG && Cf::TEMPORAL), "the auxiliary outputs of the Temporal variant come from the scan kernel");
   static_assert(!(RDEBUG && J > 8), "the auxiliary outputs for J = 16 come from the scan kernel");
+  static_assert(!(RDEBUG && Cf::GATED), "the auxiliary outputs of the Gated variant come from the scan kernel");
+  static_assert(!(Cf::GATED && (Cf::TEMPORAL || J > 8)), "gated rows: plain kernel, J <= 8");
+  // Gated: a guard pass has looked at the decays first; if the product over some chunk is so small that quantities
+  // taken relative to the chunk's start would overflow, the scan kernel runs this call instead
+  if constexpr (Cf::GATED) {
+    if (p.guard && *p.guard != 0u) return;
+  }
   constexpr bool kOdWaitAtTop = DK == 128;  // where the row warps wait for the helpers' outputs of an earlier chunk
   extern __shared__ __align__(128) unsigned char smem_raw[];
   // the swizzled operand tile needs a 1024-byte aligned shared-memory address
@@ -304,6 +320,25 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     const int col = col0 + dl;
     const bool col_ok = col < p.Dv;
     bool failed = false;
+    // a wait on barrier slot b that gave up: remembered as (warp + 1) * 256 + b for swila_device_status
+    int fail_where = 0;
+    // the same for a warp that is in nobody's way as long as it does not compete for issue slots: it sleeps between polls
+    auto bwait_idle = [&](int b, uint32_t parity) -> bool {
+      const unsigned long long t_begin = global_timer_ns();
+      while (!mbar_try_wait(&bars[b], parity)) {
+        if (global_timer_ns() - t_begin > 2000000000ull) {
+          if (fail_where == 0) fail_where = (warp + 1) * 256 + b;
+          return false;
+        }
+        __nanosleep(200);
+      }
+      return true;
+    };
+    auto bwait = [&](int b, uint32_t parity) -> bool {
+      if (mbar_wait(&bars[b], parity)) return true;
+      if (fail_where == 0) fail_where = (warp + 1) * 256 + b;
+      return false;
+    };
   if (pi > 0) {  // every barrier of the previous piece is quiescent: all its phases were waited for
     __syncthreads();
     if (tid == 0) {
@@ -325,6 +360,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     mbar_init(&bars[B_OD], 128);
     mbar_init(&bars[B_T0], 128);
     mbar_init(&bars[B_FAR], 1);
+    mbar_init(&bars[B_A], 32);
     mbar_fence_init();
   }
   tc_fence_before_sync();
@@ -355,6 +391,12 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       float hq[8];
       tmem_ld8(tb + Cf::TM_QD + (n & 1) * C + tg, hq);
       tmem_ld_wait();
+      if constexpr (Cf::GATED) {
+        // the readouts were accumulated in units of the chunk's start: w_t.q_t = A_t (w_0.q_t + sum_{s<=t} (c_s / A_s) k_s.q_t)
+        const float *As = reinterpret_cast<const float *>(smem + Cf::OFF_A + (n & 1) * Cf::A_STAGE);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) hq[i] *= As[(tg + i + 1) * NROW + r];
+      }
       if constexpr (Cf::TEMPORAL) {
         // readout weight of this lane's own component: rho_t = (1 - g) rho_{t-1} + g pi^q_t, g = sigmoid(gq logit),
         // a running average along the tokens, so it is applied before the transposition
@@ -507,8 +549,12 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     // =============================== row warps ===============================================
     const int jbase = lane - j;
     [[maybe_unused]] float st_r = 0.f, st_h = 0.f;  // auxiliary instantiation: this piece's sums over time
-    if (!mbar_wait(&bars[B_BE], 0) || !mbar_wait(&bars[B_GS], 0)) failed = true;
+    if (!bwait(B_BE, 0) || !bwait(B_GS, 0)) failed = true;
     [[maybe_unused]] float rprev = 1.0f / J;  // Temporal: this row's previous responsibility r_{t-1} (App. B.3)
+    // Gated: the product of this row's decays over the previous chunk of the piece.  What the tensor cores hand over
+    // for a chunk, W_n [K;Q]^T + Cmat'_{n-1} (K_{n-1} [K;Q]^T), is in units of the state at the START of chunk n-1.
+    [[maybe_unused]] float acarry = 1.0f;
+    [[maybe_unused]] const int a_off = p.post ? 0 : 1;  // entry of the running products that a token's prediction uses
     if constexpr (Cf::TEMPORAL) rprev = reinterpret_cast<const float *>(smem + Cf::OFF_RP)[r];
 #pragma unroll 1
     for (int n = 0; n < nchunks && !failed; ++n) {
@@ -521,14 +567,15 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       [[maybe_unused]] const float *pks = reinterpret_cast<const float *>(raw + Cf::R_PK);            // Temporal: normalised prior
       [[maybe_unused]] const __nv_bfloat16 *rgk = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_GK);  // Temporal: gate logits
       const float *Gkk = G_all + (n & 1) * C * C;
+      [[maybe_unused]] const float *As = reinterpret_cast<const float *>(smem + Cf::OFF_A + (n & 1) * Cf::A_STAGE);
 
-      if (!mbar_wait(&bars[B_E], n & 1)) { failed = true; break; }
+      if (!bwait(B_E, n & 1)) { failed = true; break; }
       tc_fence_after_sync();
       // the readout buffer this chunk seeds below was last read by the helpers for the outputs of chunk n-2.  At
       // Dk = 128 they finish those about when chunk n-1 ends, so the wait sits here, where it has long been met; at
       // Dk = 64 they are early and the wait is cheaper at the hand-over below (both placements measured)
       if constexpr (kOdWaitAtTop) {
-        if (n >= 2 && !mbar_wait(&bars[B_OD], n & 1)) { failed = true; break; }
+        if (n >= 2 && !bwait(B_OD, n & 1)) { failed = true; break; }
       }
       // [P0 | Q0] out of tensor memory: P0 to registers, Q0 seeds the readout accumulator of this chunk;
       // then the tensor cores may overwrite the region with the next chunk's products
@@ -539,6 +586,10 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         tmem_ld16(tb + Cf::TM_PQ + cc * 16, a);
         tmem_ld16(tb + Cf::TM_PQ + C + cc * 16, b);
         tmem_ld_wait();
+        if constexpr (Cf::GATED) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) { a[i] *= acarry; b[i] *= acarry; }
+        }
         tmem_st16(tb + Cf::TM_QD + (n & 1) * C + cc * 16, b);
 #pragma unroll
         for (int i = 0; i < 16; ++i) pred0[cc * 16 + i] = a[i];
@@ -573,18 +624,25 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         constexpr int WINS = EXACT ? C : Cf::WIN;
         float pred[WINS];
 #pragma unroll
-        for (int t = 0; t < WINS; ++t) pred[t] = __bfloat162float(rv[t * COLS + dl]) - pred0[t];
+        for (int t = 0; t < WINS; ++t) {
+          // Gated: the window holds minus the prediction in units of the chunk's start; the decay and v enter per token
+          if constexpr (Cf::GATED) pred[t] = -pred0[t];
+          else pred[t] = __bfloat162float(rv[t * COLS + dl]) - pred0[t];
+        }
         [[maybe_unused]] float p0late[C - Cf::WIN];
         if constexpr (!EXACT) {
 #pragma unroll
-          for (int t = 0; t < C - Cf::WIN; ++t) p0late[t] = __bfloat162float(rv[(Cf::WIN + t) * COLS + dl]) - pred0[Cf::WIN + t];
+          for (int t = 0; t < C - Cf::WIN; ++t) {
+            if constexpr (Cf::GATED) p0late[t] = -pred0[Cf::WIN + t];
+            else p0late[t] = __bfloat162float(rv[(Cf::WIN + t) * COLS + dl]) - pred0[Cf::WIN + t];
+          }
         }
         float c_prev = 0.f;
 #pragma unroll 1
         for (int tg = 0; tg < C; tg += GT) {
           if constexpr (!EXACT) {
             if (tg == Cf::WIN) {  // far pushes of tokens 0-6 into tokens 24-31
-              if (!mbar_wait(&bars[B_FAR], n & 1)) failed = true;
+              if (!bwait(B_FAR, n & 1)) failed = true;
               tc_fence_after_sync();
               float far[8];
               tmem_ld8(tb + Cf::TM_FAR + Cf::WIN - C / 2, far);
@@ -599,7 +657,12 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
             const int t = tg + i;
             const float be = bes[t * NROW + r];
             // serial chain: prediction error -> responsibilities (Eq. 3.4) -> update coefficient (Eq. 3.3)
-            const float delta = pred[i];
+            // Gated: delta = v - A (w_0.k + sum_s (c_s / A_s) k_s.k), A = the row's decay product up to this token
+            // (pre-decay, Eq. 3.8) or up to the previous one (post-decay, Eq. 3.7); beta arrives divided by A_t, so
+            // that the coefficient below is already c_t / A_t
+            float delta;
+            if constexpr (Cf::GATED) delta = fmaf(As[(t + a_off) * NROW + r], pred[i], __bfloat162float(rv[t * COLS + dl]));
+            else delta = pred[i];
             float a;
             if constexpr (Cf::TEMPORAL) {
               // key-side prior (1 - g) r_{t-1} + g pi^k with g = sigmoid(gk logit) (App. B.3): a convex combination of
@@ -674,7 +737,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
           // the coefficient columns are still operands of the previous chunk's update and readout MMAs until
           // those complete (normally long before the first trip ends)
           if (tg == 0 && n > 0) {
-            if (!mbar_wait(&bars[B_QD], (n - 1) & 1)) failed = true;
+            if (!bwait(B_QD, (n - 1) & 1)) failed = true;
           }
           {  // GT update coefficients complete: park their bf16 parts in tensor memory, two tokens per column
             uint32_t hi[GT / 2], lo[GT / 2], l3[GT / 2];
@@ -721,19 +784,20 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         sequential(std::true_type{}, rprev);
       }
       if constexpr (Cf::TEMPORAL) rprev = chunk_rp;
+      if constexpr (Cf::GATED) acarry = As[C * NROW + r];
       if constexpr (RDEBUG) { st_r += chunk_r; st_h += chunk_h; }
       tmem_st_wait();
       tc_fence_before_sync();
       // what the next steps rely on must be in place before this chunk is handed over (this also keeps every
       // barrier at most one phase ahead of its waiters): gates and Gram rows of chunk n+1
-      if (n + 1 < nchunks && (!mbar_wait(&bars[B_BE], (n + 1) & 1) || !mbar_wait(&bars[B_GS], (n + 1) & 1))) failed = true;
+      if (n + 1 < nchunks && (!bwait(B_BE, (n + 1) & 1) || !bwait(B_GS, (n + 1) & 1))) failed = true;
       if constexpr (!kOdWaitAtTop) {
-        if (n > 0 && !mbar_wait(&bars[B_OD], (n - 1) & 1)) failed = true;
+        if (n > 0 && !bwait(B_OD, (n - 1) & 1)) failed = true;
       }
       mbar_arrive(&bars[B_C]);
     }
     // ---- final state row -> global ----
-    if (!failed && !mbar_wait(&bars[B_U], (nchunks - 1) & 1)) failed = true;
+    if (!failed && !bwait(B_U, (nchunks - 1) & 1)) failed = true;
     if (!failed && p.W_out && col_ok) {
       tc_fence_after_sync();
       float *dst = p.W_out + (((size_t)bh * J + j) * p.Dv + col) * DK;
@@ -742,6 +806,10 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         float w[16];
         tmem_ld16(tb + Cf::TM_W + cc * 16, w);
         tmem_ld_wait();
+        if constexpr (Cf::GATED) {  // the last update left the state in units of the last chunk's start
+#pragma unroll
+          for (int i = 0; i < 16; ++i) w[i] *= acarry;
+        }
 #pragma unroll
         for (int i = 0; i < 4; ++i)
           __stcs(reinterpret_cast<float4 *>(dst + cc * 16 + i * 4), make_float4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]));
@@ -772,7 +840,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     // logits of its own tokens -- which every helper has read by the barrier -- and of later, finished ones
     // Tokens past the end of the sequence (the last chunk's padding) get beta = 0: their update coefficient is then
     // zero by itself and the row warps need no test on their serial chain.
-    auto cook_be = [&](unsigned char *raw, const int nvalid) {
+    auto cook_be = [&](unsigned char *raw, const int nvalid, [[maybe_unused]] const float *As) {
       const __nv_bfloat16 *rb = reinterpret_cast<const __nv_bfloat16 *>(raw + Cf::R_B);
       float *bes = reinterpret_cast<float *>(raw + Cf::R_B);
       static_assert(J * Cf::GROW * Cf::ES <= NROW * 4, "a token's logits end before its FP32 row does");
@@ -782,6 +850,8 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           be[i] = sigmoid_approx(__bfloat162float(rb[((t8 + i) * J + j) * Cf::GROW + dl]));
+          // Gated: beta / A_t, so that the row warps' coefficient is c_t / A_t without a further operation
+          if constexpr (Cf::GATED) be[i] *= rcp_approx(As[(t8 + i + 1) * NROW + h]);
           if (t8 + i >= nvalid) be[i] = 0.f;
         }
         named_bar_sync(3, 128);
@@ -833,13 +903,18 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       }
     };
     // operand parts of W after an update, this helper's tensor-memory lane
-    auto refresh_parts = [&]() {
+    auto refresh_parts = [&]([[maybe_unused]] const float decay) {
 #pragma unroll 2
       for (int cc = 0; cc < DK / 16; ++cc) {
         float w[16];
         uint32_t hi[8], lo[8];
         tmem_ld16(tb + Cf::TM_W + cc * 16, w);
         tmem_ld_wait();
+        if constexpr (Cf::GATED) {  // the update was taken in units of the chunk's start: now the chunk's decay
+#pragma unroll
+          for (int i = 0; i < 16; ++i) w[i] *= decay;
+          tmem_st16(tb + Cf::TM_W + cc * 16, w);
+        }
 #pragma unroll
         for (int i = 0; i < 8; ++i) bf16_split2(w[2 * i], w[2 * i + 1], hi[i], lo[i]);
         tmem_st8(tb + Cf::TM_WHI + cc * 8, reinterpret_cast<const float(&)[8]>(hi));
@@ -917,7 +992,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
                       (Cf::KU_MIRROR && m > 0 && m % 3 == 0) ? smem + Cf::OFF_KU + 3 * Cf::KU_HALF : nullptr);
     };
     // everything staged for chunk m has landed (the barrier of m's parity completes once per chunk of that parity)
-    auto staged = [&](int m) { return mbar_wait(&bars[B_KQ0 + (m & 1)], (m >> 1) & 1); };
+    auto staged = [&](int m) { return bwait(B_KQ0 + (m & 1), (m >> 1) & 1); };
     if (h == 0) {
       stage(0);
       if (nchunks > 1) stage(1);
@@ -994,11 +1069,18 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         *reinterpret_cast<uint4 *>(tile + (e / (2 * C * 8)) * Cf::TILE_HALF + 2 * C * 128 + (e % (2 * C * 8)) * 16) = make_uint4(0, 0, 0, 0);
     }
     if (!staged(0)) failed = true;
-    cook_be(smem + Cf::OFF_RAW, min(C, Tseg));
+    {
+      const float *As0 = nullptr;
+      if constexpr (Cf::GATED) {  // the decay warp has the running products of chunk 0 in place
+        if (!bwait(B_A, 0)) failed = true;
+        As0 = reinterpret_cast<const float *>(smem + Cf::OFF_A);
+      }
+      cook_be(smem + Cf::OFF_RAW, min(C, Tseg), As0);
+    }
     if constexpr (Cf::TEMPORAL) cook_pk(smem + Cf::OFF_RAW);
     mbar_arrive(&bars[B_BE]);
     if (spill_mine[0]) {
-      if (!mbar_wait(&bars[B_G], 0)) failed = true;
+      if (!bwait(B_G, 0)) failed = true;
       tc_fence_after_sync();
       if (!failed) spill_gram(0);
       mbar_arrive(&bars[B_GS]);
@@ -1008,41 +1090,58 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
 #pragma unroll 1
     for (int n = 0; n < nchunks && !failed; ++n) {
       const bool more = n + 1 < nchunks;
+      // (2) outputs of chunk n-1, whose readouts completed shortly after chunk n started.  The row warps wait for
+      // OD(n-2) at the top of chunk n, and OD must not complete another phase before they have: in every iteration
+      // but the last the Gram batch spilled in (1) was issued after the row warps passed that point (PQF(n)); in the
+      // last one, and in the Gated kernel, the same barrier is waited for here.
+      auto outputs_of_previous = [&]() -> bool {
+        if (n == 0) return true;
+        if ((!more || Cf::GATED) && !bwait(B_PQF, n & 1)) return false;
+        if (!bwait(B_QD, (n - 1) & 1)) return false;
+        write_outputs(n - 1);
+        mbar_arrive(&bars[B_OD]);
+        return true;
+      };
+      if constexpr (Cf::GATED) {
+        // the outputs of chunk n-1 take the running products of its decays from the stage that the decay warp fills
+        // for chunk n+1 once these outputs are formed (it waits for OD): outputs first here
+        if (!outputs_of_previous()) { failed = true; break; }
+      }
       if (more) {
         // (1) gates of chunk n+1 for the row warps, then its Gram batch
         if (!staged(n + 1)) { failed = true; break; }
-        cook_be(smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES, min(C, Tseg - (n + 1) * C));
+        const float *As1 = nullptr;
+        if constexpr (Cf::GATED) {
+          if (!bwait(B_A, (n + 1) & 1)) { failed = true; break; }
+          As1 = reinterpret_cast<const float *>(smem + Cf::OFF_A + ((n + 1) & 1) * Cf::A_STAGE);
+        }
+        cook_be(smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES, min(C, Tseg - (n + 1) * C), As1);
         if constexpr (Cf::TEMPORAL) cook_pk(smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES);
         mbar_arrive(&bars[B_BE]);
         if (spill_mine[(n + 1) & 1]) {
-          if (!mbar_wait(&bars[B_G], (n + 1) & 1)) failed = true;
+          if (!bwait(B_G, (n + 1) & 1)) failed = true;
           tc_fence_after_sync();
           if (!failed) spill_gram(n + 1);
           mbar_arrive(&bars[B_GS]);
         }
       }
-      // (2) outputs of chunk n-1, whose readouts completed shortly after chunk n started.  The row warps wait for
-      // OD(n-2) at the top of chunk n, and OD must not complete another phase before they have: in every iteration
-      // but the last the Gram batch spilled above was issued after the row warps passed that point (PQF(n)); in the
-      // last one the same barrier is waited for here.
-      if (n > 0) {
-        if (!more && !mbar_wait(&bars[B_PQF], n & 1)) { failed = true; break; }
-        if (!mbar_wait(&bars[B_QD], (n - 1) & 1)) { failed = true; break; }
-        write_outputs(n - 1);
-        mbar_arrive(&bars[B_OD]);
+      if constexpr (!Cf::GATED) {
+        if (!outputs_of_previous()) { failed = true; break; }
       }
       // (3) chunk n is finished by the row warps: stage chunk n+2 into the buffers chunk n used
-      if (!mbar_wait(&bars[B_C], n & 1)) { failed = true; break; }
+      if (!bwait(B_C, n & 1)) { failed = true; break; }
       if (n + 2 < nchunks && h == 0) stage(n + 2);
       // (4) W has been updated with chunk n: split it into operand parts again
-      if (!mbar_wait(&bars[B_U], n & 1)) { failed = true; break; }
+      if (!bwait(B_U, n & 1)) { failed = true; break; }
       if (more) {
         tc_fence_after_sync();
-        refresh_parts();
+        float decay = 1.0f;
+        if constexpr (Cf::GATED) decay = reinterpret_cast<const float *>(smem + Cf::OFF_A + (n & 1) * Cf::A_STAGE)[C * NROW + h];
+        refresh_parts(decay);
         mbar_arrive(&bars[B_WP]);
       }
     }
-    if (!failed && !mbar_wait(&bars[B_QD], (nchunks - 1) & 1)) failed = true;
+    if (!failed && !bwait(B_QD, (nchunks - 1) & 1)) failed = true;
     if (!failed) write_outputs(nchunks - 1);
     if constexpr (Cf::TEMPORAL) {
       if (!failed && p.rho_out && col_ok) p.rho_out[((size_t)bh * J + j) * p.Dv + col] = rho_run;
@@ -1067,7 +1166,62 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         if (p.rho_ent) atomicAdd(p.rho_ent + (size_t)bh * p.Dv + col, sq_ent * kLn2);
       }
     }
-  } else if (lane == 0) {
+  } else if (warp == 9) {
+    // =============================== decay warp (Gated only) =================================
+    // Lane L serves rows 4L .. 4L+3 of the tile.  Per chunk: the rows' decays straight from global memory (one value
+    // per row and token; a warp of its own, so that the load latency stalls nobody else), their running products
+    // A_t since the chunk began into the stage of the chunk's parity: entry t + 1 = A_t, entry 0 = 1.  Tokens past
+    // the end of the sequence decay by 1.  A stage is refilled once the outputs of the chunk two back are formed.
+    if constexpr (Cf::GATED) {
+      const float *src[4];
+      size_t tstride;  // elements between consecutive tokens
+      bool ok[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int rr = 4 * lane + i, jj = rr % J, cc = col0 + rr / J;
+        ok[i] = cc < p.Dv;
+        src[i] = p.gran == SWILA_GATE_PER_OUT ? p.alpha + (tok0 * J + jj) * (size_t)p.Dv + cc : p.alpha + tok0 * J + jj;
+      }
+      tstride = p.gran == SWILA_GATE_PER_OUT ? (size_t)J * p.Dv : (size_t)J;
+#pragma unroll 1
+      for (int m = 0; m < nchunks && !failed; ++m) {
+        const int nv = min(C, Tseg - m * C);
+        float4 *As = reinterpret_cast<float4 *>(smem + Cf::OFF_A + (m & 1) * Cf::A_STAGE);
+        // the chunk's decays and their running products into registers, 8 tokens (32 loads per lane) at a time: more
+        // loads in flight crowd the load/store path that the row warps' shared-memory reads also go through
+        float prod[C][4];
+        float run[4] = {1.f, 1.f, 1.f, 1.f};
+#pragma unroll
+        for (int t8 = 0; t8 < C; t8 += 8) {
+          float al[8][4];
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              al[u][i] = (t8 + u < nv && ok[i]) ? __ldg(src[i] + (size_t)(m * C + t8 + u) * tstride) : 1.0f;
+          }
+#pragma unroll
+          for (int u = 0; u < 8; ++u) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              run[i] *= al[u][i];
+              prod[t8 + u][i] = run[i];
+            }
+          }
+        }
+        // ... then the stage must be free: the outputs of the chunk two back are formed
+        if (m >= 2 && !bwait_idle(B_OD, (m - 2) & 1)) { failed = true; break; }
+        As[lane] = make_float4(1.f, 1.f, 1.f, 1.f);
+#pragma unroll
+        for (int t = 0; t < C; ++t) As[(t + 1) * (NROW / 4) + lane] = make_float4(prod[t][0], prod[t][1], prod[t][2], prod[t][3]);
+        // A must never run two phases ahead of its waiters (the helpers): for m >= 2 the wait above implies that they
+        // have taken chunk m-1's products; chunk 1's must not be announced before they have taken chunk 0's, which
+        // the first gates (BE) tell -- a piece that waits for its state to be handed over gets there late
+        if (m == 1 && !bwait_idle(B_BE, 0)) failed = true;
+        mbar_arrive(&bars[B_A]);
+      }
+    }
+  } else if (warp == 8 && lane == 0) {
     // =============================== MMA issuer ==============================================
     constexpr uint32_t idE = idesc_bf16(128, 2 * C);  // N = 2C: [P0 | Q0], Gram batch, cross-chunk term
     constexpr uint32_t idU = idesc_bf16_bmn(128, DK);  // B (the keys) is read MN-major
@@ -1134,7 +1288,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       }
       mma_commit(&bars[B_QD]);
     };
-    if (!mbar_wait(&bars[B_KQ0], 0) || !mbar_wait(&bars[B_WP], 0)) failed = true;
+    if (!bwait(B_KQ0, 0) || !bwait(B_WP, 0)) failed = true;
     tc_fence_after_sync();
     if (!failed) {
       gram(0);
@@ -1147,8 +1301,8 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       if (more) {
         // ahead of the serial path: Gram batch and state x [K;Q] of chunk n+1 with the state before chunk n's
         // update (W is final up to chunk n-1 and split into parts; [P0|Q0] of chunk n has been taken out)
-        if (!mbar_wait(&bars[B_KQ0 + ((n + 1) & 1)], ((n + 1) >> 1) & 1) || !mbar_wait(&bars[B_PQF], n & 1)) { failed = true; break; }
-        if (n > 0 && !mbar_wait(&bars[B_WP], n & 1)) { failed = true; break; }
+        if (!bwait(B_KQ0 + ((n + 1) & 1), ((n + 1) >> 1) & 1) || !bwait(B_PQF, n & 1)) { failed = true; break; }
+        if (n > 0 && !bwait(B_WP, n & 1)) { failed = true; break; }
         tc_fence_after_sync();
         gram(n + 1);
       }
@@ -1156,7 +1310,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         // far pushes of chunk n: what its first 8 tokens add to the predictions of its last 8, needed when the row
         // warps reach token 24.  A = the coefficient columns of tokens 0..15 (8..15 are stale but finite and meet
         // zero rows of the operand), B = rows 16..31 of K K^T against tokens 0..7.
-        if (!mbar_wait(&bars[B_T0], n & 1)) { failed = true; break; }
+        if (!bwait(B_T0, n & 1)) { failed = true; break; }
         tc_fence_after_sync();
         const uint32_t fa = smem_u32(smem + Cf::OFF_FAR + (n & 1) * 2 * Cf::FAR_TILE);
         const uint64_t f_hi = smem_desc_kmajor(fa, Cf::FAR_LBO, 128), f_lo = smem_desc_kmajor(fa + Cf::FAR_TILE, Cf::FAR_LBO, 128);
@@ -1170,11 +1324,11 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         w_times_kq(n + 1);
         // first half of the cross-chunk term (tokens 0-15 of chunk n, whose coefficients T0 released), while the
         // chunk still runs
-        if (!mbar_wait(&bars[B_GS], (n + 1) & 1)) { failed = true; break; }
+        if (!bwait(B_GS, (n + 1) & 1)) { failed = true; break; }
         tc_fence_after_sync();
         cross(0);
       }
-      if (!mbar_wait(&bars[B_C], n & 1)) { failed = true; break; }
+      if (!bwait(B_C, n & 1)) { failed = true; break; }
       tc_fence_after_sync();
       const bool redone = *redo_s != 0;  // ordered by the barrier: set before the row warps arrived
       if (redone) *redo_s = 0;
@@ -1185,6 +1339,12 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         }
         cross(1);  // -> E(n+1): the only tensor work left between two chunks of the row warps
         mma_commit(&bars[B_E]);
+      }
+      if constexpr (Cf::GATED) {
+        // the helpers wrote the decayed state back over W after the previous update: that must be complete (in
+        // every iteration but the last it has been waited for above already)
+        if (n > 0 && !bwait(B_WP, n & 1)) { failed = true; break; }
+        tc_fence_after_sync();
       }
 #pragma unroll 1
       for (int ks = 0; ks < C / 16; ++ks) {  // W += Cmat K (Eq. 3.3 summed over the chunk)
@@ -1200,7 +1360,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     }
   }
   if (failed) {
-    atomicExch(&g_chunk_error, 1);
+    atomicCAS(&g_chunk_error, 0, fail_where ? fail_where : 1);  // the first failure of the launch is kept
     *fail_s = 1;
   }
   }  // pieces
@@ -1289,14 +1449,15 @@ inline unsigned chunk_next_epoch() {
   return e;
 }
 
-template <int J, int DK, bool TEMPORAL = false>
+template <int J, int DK, bool TEMPORAL = false, bool GATED = false>
 int launch_chunk(const LaunchArgs &a) {
-  using Cf = ChunkCfg<J, DK, TEMPORAL>;
+  using Cf = ChunkCfg<J, DK, TEMPORAL, GATED>;
   const bool aux = a.p.r_debug || a.p.r_sum || a.p.r_ent || a.p.rho_sum || a.p.rho_ent;
   if (TEMPORAL && aux) return -1000;  // the Temporal variant's auxiliary outputs come from the scan kernel
   if (J > 8 && aux) return -1000;     // likewise for J = 16
+  if (GATED && aux) return -1000;     // and for the Gated variant
   auto kern = swila_chunk_kernel<Cf, false>;
-  if constexpr (!TEMPORAL && J <= 8) {
+  if constexpr (!TEMPORAL && !GATED && J <= 8) {
     if (aux) kern = swila_chunk_kernel<Cf, true>;
   }
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cf::SMEM_BYTES);

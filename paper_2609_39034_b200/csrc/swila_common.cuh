@@ -24,6 +24,11 @@ struct ScanParams {
   void *o;
   float *r_debug;                     // may be null
   int qkv_act;                        // 0/1: SiLU on q, k, v and L2 normalisation of q, k inside the kernel
+  int post;                           // 0/1: post-decay form (Eq. 3.7) of the gated variants
+  // Gated rows in the chunked kernel: a word written by the guard pass that looks at the decays first.  The chunked
+  // kernel returns at once when it is non-zero, the scan kernel launched behind it when it is zero (null: no guard).
+  const unsigned *guard;
+  int guard_runs_scan;                // scan kernel: 1 = run only if *guard != 0
   float *r_sum, *r_ent, *rho_sum, *rho_ent;  // sums over time of the mixture weights; each may be null
 };
 

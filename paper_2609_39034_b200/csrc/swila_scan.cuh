@@ -284,6 +284,7 @@ __global__ void __launch_bounds__(C::NT, C::MIN_BLOCKS) swila_scan_kernel(const 
   constexpr int J = C::J, DK = C::DK, NT = C::NT, TB = C::TB, GATE = C::GATE;
   (void)J; (void)DK; (void)NT; (void)TB; (void)GATE;
   constexpr int L = C::L, G = C::G, COLS = C::COLS, S = C::S;
+  if (p.guard && p.guard_runs_scan && *p.guard == 0u) return;  // the chunked kernel took this call
   extern __shared__ __align__(16) unsigned char smem[];
   float *cooked = reinterpret_cast<float *>(smem + C::OFF_COOKED);
   unsigned char *obuf = smem + C::OFF_O;

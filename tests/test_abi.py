@@ -127,7 +127,12 @@ def test_auto_dispatch_rule(binding):
     assert auto(lm) == binding.ALGO_CHUNK and auto(lm.variant(temporal=True)) == binding.ALGO_CHUNK
     assert auto(lm, 1) == binding.ALGO_CHUNK and auto(lm.variant(temporal=True), 1) == binding.ALGO_SCAN
     assert auto(wl.CONFIGS[1].with_(J=16)) == binding.ALGO_CHUNK and auto(wl.CONFIGS[1].with_(J=16), 1) == binding.ALGO_SCAN
+    rows = dict(gated=True, granularity=wl.GRAN_PER_OUT)
+    assert auto(lm.variant(**rows)) == binding.ALGO_CHUNK and auto(lm.variant(gated=True, granularity=wl.GRAN_SCALAR, post_decay=True)) == binding.ALGO_CHUNK
+    assert auto(lm.variant(**rows), 1) == binding.ALGO_SCAN and auto(lm.variant(temporal=True, **rows)) == binding.ALGO_SCAN
+    assert auto(lm.with_(J=8).variant(**rows)) == binding.ALGO_SCAN and auto(wl.CONFIGS[1].with_(J=8).variant(**rows)) == binding.ALGO_CHUNK
     for w in (lm.with_(T=63), lm.with_(io_dtype="fp32"), lm.variant(gated=True), lm.with_(J=2), lm.with_(J=16),
+              lm.variant(gated=True, granularity=wl.GRAN_ELEMENTWISE),
               wl.CONFIGS[0], wl.CONFIGS[3], lm.with_(flags=wl.FLAG_QKV_ACT)):
         assert auto(w) == binding.ALGO_SCAN, w
     assert auto(lm.with_(J=3)) == binding.ERR_UNSUPPORTED

@@ -252,3 +252,33 @@ def test_temporal_prefill_sampled(binding, oracle, shape):
     assert wl.rel_err(pick(st["W"])[:, :, cols.cuda()].unsqueeze(1).cpu(), torch.from_numpy(ref["W"])) < TOL_STATE
     for name in ("r_prev", "rho_prev"):
         assert wl.rel_err(pick(st[name])[..., cols.cuda()].unsqueeze(1).cpu(), torch.from_numpy(ref[name])) < TOL_STATE, name
+
+
+@pytest.mark.parametrize("shape,gran,post", [("headline", wl.GRAN_PER_OUT, False), ("more_tiles_than_sms", wl.GRAN_SCALAR, True),
+                                             ("more_tiles_than_sms", wl.GRAN_PER_OUT, False)],
+                         ids=["headline_out_pre", "split_scalar_post", "split_out_pre"])
+def test_gated_rows_prefill_sampled(binding, oracle, shape, gran, post):
+    """Gated SwiLA with one decay per state row (Eqs. 3.7 / 3.8 as printed) at full size through the default dispatch
+    (guard pass, chunked kernel, scan kernel standing by): the LM-shaped configuration, and a shape whose tiles are
+    split between blocks (tail pieces wait for their state, which is where the decay warp once ran ahead of the
+    helpers).  Sampled rows are replayed by the oracle; the whole state is compared with the scan kernel's."""
+    base = wl.CONFIGS[2] if shape == "headline" else wl.CONFIGS[2].with_(B=2, H=20, T=1024)
+    w = base.variant(gated=True, granularity=gran, post_decay=post)
+    assert binding.auto_algo(w) == binding.ALGO_CHUNK
+    inp = wl.make_inputs(w, device="cuda", stress=True)
+    sin = {"W": inp["W0"]}
+    st = binding.state_alloc(w, init=False)
+    o = binding.swila_forward(w, inp, state_in=sin, state_out=st)
+    st_scan = binding.state_alloc(w, init=False)
+    o_scan = binding.swila_forward(w, inp, state_in=sin, state_out=st_scan, algo=binding.ALGO_SCAN)
+    torch.cuda.synchronize()
+    binding.device_status()
+    assert not torch.equal(st["W"], st_scan["W"])  # two kernels
+    assert wl.rel_err(o.float().cpu(), o_scan.float().cpu()) < TOL_BF16_O
+    assert wl.rel_err(st["W"].cpu(), st_scan["W"].cpu()) < 2 * TOL_STATE
+    bh, cols = _sample(w, 4, 8, seed=31)
+    sub = wl.slice_rows(inp, bh.cuda(), cols.cuda(), gran=gran)
+    ref = oracle.forward_inputs({n: (x.cpu() if x is not None else None) for n, x in sub.items()}, flags=w.flags, gran=gran)
+    pick = lambda x: x.reshape((w.B * w.H,) + tuple(x.shape[2:]))[bh.cuda()]  # noqa: E731
+    assert wl.rel_err(pick(o)[..., cols.cuda()].unsqueeze(1).cpu(), torch.from_numpy(ref["o"])) < TOL_BF16_O
+    assert wl.rel_err(pick(st["W"])[:, :, cols.cuda()].unsqueeze(1).cpu(), torch.from_numpy(ref["W"])) < TOL_STATE

@@ -122,6 +122,54 @@ def test_chunked_kernel_temporal_matches_oracle(binding, oracle, w, stress):
     assert_close(wt, got, ref, wt.name)
 
 
+GATED_ROW_SHAPES = [w for w in CHUNK_SHAPES if (w.J == 4 or (w.J == 8 and w.Dk == 64))]
+
+
+@pytest.mark.parametrize("w", GATED_ROW_SHAPES, ids=lambda w: w.name)
+@pytest.mark.parametrize("gran,post", [(wl.GRAN_PER_OUT, False), (wl.GRAN_PER_OUT, True), (wl.GRAN_SCALAR, False),
+                                       (wl.GRAN_SCALAR, True)], ids=["out_pre", "out_post", "scalar_pre", "scalar_post"])
+@pytest.mark.parametrize("alpha", ["near_one", "down_to_half"])
+def test_chunked_kernel_gated_rows_match_oracle(binding, oracle, w, gran, post, alpha):
+    """Gated SwiLA with one decay per state row (Eqs. 3.7 / 3.8 as printed; per component: the scalar gate of
+    App. B.4) in the chunked kernel: the decay enters as a running product per row, the Gram matrices stay shared.
+    Decays near one as a trained gate gives them (sigmoid(3 + .)), and uniform in [0.5, 1], where the product over a
+    32-token chunk falls to 2^-32."""
+    wg = w.variant(gated=True, granularity=gran, post_decay=post)
+    inp = wl.make_inputs(wg, stress=True)
+    if alpha == "down_to_half":
+        g = torch.Generator().manual_seed(77)
+        inp["alpha"] = (0.5 + 0.5 * torch.rand(inp["alpha"].shape, generator=g)).contiguous()
+    ref = oracle.forward_inputs(inp, flags=wg.flags, gran=gran)
+    dev = to_dev(inp)
+    got = gpu_forward(binding, wg, dev, algo=binding.ALGO_CHUNK)
+    binding.device_status()
+    assert_close(wg, got, ref, wg.name)
+    if wg.T >= 32:  # it was the chunked kernel that ran: the scan kernel's bits differ
+        scan = gpu_forward(binding, wg, dev, algo=binding.ALGO_SCAN)
+        assert not torch.equal(scan["W"], got["W"])
+
+
+def test_chunked_kernel_gated_rows_hand_over_to_the_scan_when_a_chunk_decays_to_nothing(binding, oracle):
+    """Decays whose product over one chunk drops below 2^-40 would overflow the chunked kernel's quotients: the guard
+    pass sees them and the scan kernel evaluates the call (same bits as asking for the scan), in place on the state."""
+    w = SMALL[4].with_(T=130).variant(gated=True, granularity=wl.GRAN_PER_OUT)
+    inp = wl.make_inputs(w, stress=True)
+    a = inp["alpha"].clone()
+    a[:, :, 70:80, 1, 5] = 0.01          # one row, ten tokens: 1e-20 within one chunk
+    a[:, :, 100, 2, 7] = 0.0             # and an exact zero
+    inp["alpha"] = a
+    ref = oracle.forward_inputs(inp, flags=w.flags, gran=w.gate_granularity)
+    dev = to_dev(inp)
+    scan = gpu_forward(binding, w, dev, algo=binding.ALGO_SCAN)
+    st = {"W": dev["W0"].clone(), "r_prev": None, "rho_prev": None}
+    o = binding.swila_forward(w, dev, state_in=st, state_out=st, algo=binding.ALGO_CHUNK)  # in place
+    torch.cuda.synchronize()
+    binding.device_status()
+    got = {"o": o.cpu(), "W": st["W"].cpu()}
+    assert_close(w, got, ref, "guarded")
+    assert torch.equal(got["W"], scan["W"]) and torch.equal(got["o"], scan["o"])
+
+
 def test_chunked_kernel_temporal_in_pieces_and_decode(binding, oracle):
     """A Temporal sequence fed to the chunked kernel in two calls with the state carried (W, r_prev, rho_prev), then
     decode steps (scan kernel) on that state: the whole must equal one oracle pass over all tokens."""
