@@ -182,6 +182,10 @@ struct ChunkCfg {
   // is 1 (the pre-decay form of Eq. 3.8 predicts with A_t, the post-decay form of Eq. 3.7 with A_{t-1})
   static constexpr int OFF_A = OFF_OS + (J > 8 ? C * NROW * 4 : 0);
   static constexpr int A_STAGE = (C + 1) * NROW * 4;
+  // entry of row (column dl, component j) inside a token's NROW products: component-major, the column index XORed
+  // with 8 j so that the J lanes of a column (adjacent row threads) fall into different banks; four consecutive
+  // columns of one component stay four consecutive words, which is what the decay warp stores
+  __host__ __device__ static constexpr int a_slot(int dl, int j) { return j * COLS + (dl ^ ((8 * j) & (COLS - 1))); }
   static constexpr int OFF_BAR = OFF_A + (GATED ? 2 * A_STAGE : 0);
   static constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;  // barriers and three words; + 1024: the kernel aligns its window to 1024 bytes
   static_assert(R_GK % 128 == 0 && RQ_GQ % 128 == 0, "temporal gate rows start 128-byte aligned");
@@ -303,6 +307,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
   // row served by this thread in either 128-thread role
   const int r = tid & 127;
   const int dl = r / J, j = r % J;
+  [[maybe_unused]] const int a_slot = Cf::a_slot(dl, j);  // Gated: this row's entry in a token's decay products
 
 #pragma unroll 1
   for (int pi = 0; pi < npieces; ++pi) {
@@ -395,7 +400,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         // the readouts were accumulated in units of the chunk's start: w_t.q_t = A_t (w_0.q_t + sum_{s<=t} (c_s / A_s) k_s.q_t)
         const float *As = reinterpret_cast<const float *>(smem + Cf::OFF_A + (n & 1) * Cf::A_STAGE);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) hq[i] *= As[(tg + i + 1) * NROW + r];
+        for (int i = 0; i < 8; ++i) hq[i] *= As[(tg + i + 1) * NROW + a_slot];
       }
       if constexpr (Cf::TEMPORAL) {
         // readout weight of this lane's own component: rho_t = (1 - g) rho_{t-1} + g pi^q_t, g = sigmoid(gq logit),
@@ -661,7 +666,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
             // (pre-decay, Eq. 3.8) or up to the previous one (post-decay, Eq. 3.7); beta arrives divided by A_t, so
             // that the coefficient below is already c_t / A_t
             float delta;
-            if constexpr (Cf::GATED) delta = fmaf(As[(t + a_off) * NROW + r], pred[i], __bfloat162float(rv[t * COLS + dl]));
+            if constexpr (Cf::GATED) delta = fmaf(As[(t + a_off) * NROW + a_slot], pred[i], __bfloat162float(rv[t * COLS + dl]));
             else delta = pred[i];
             float a;
             if constexpr (Cf::TEMPORAL) {
@@ -784,7 +789,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         sequential(std::true_type{}, rprev);
       }
       if constexpr (Cf::TEMPORAL) rprev = chunk_rp;
-      if constexpr (Cf::GATED) acarry = As[C * NROW + r];
+      if constexpr (Cf::GATED) acarry = As[C * NROW + a_slot];
       if constexpr (RDEBUG) { st_r += chunk_r; st_h += chunk_h; }
       tmem_st_wait();
       tc_fence_before_sync();
@@ -851,7 +856,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         for (int i = 0; i < 8; ++i) {
           be[i] = sigmoid_approx(__bfloat162float(rb[((t8 + i) * J + j) * Cf::GROW + dl]));
           // Gated: beta / A_t, so that the row warps' coefficient is c_t / A_t without a further operation
-          if constexpr (Cf::GATED) be[i] *= rcp_approx(As[(t8 + i + 1) * NROW + h]);
+          if constexpr (Cf::GATED) be[i] *= rcp_approx(As[(t8 + i + 1) * NROW + a_slot]);
           if (t8 + i >= nvalid) be[i] = 0.f;
         }
         named_bar_sync(3, 128);
@@ -1136,7 +1141,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       if (more) {
         tc_fence_after_sync();
         float decay = 1.0f;
-        if constexpr (Cf::GATED) decay = reinterpret_cast<const float *>(smem + Cf::OFF_A + (n & 1) * Cf::A_STAGE)[C * NROW + h];
+        if constexpr (Cf::GATED) decay = reinterpret_cast<const float *>(smem + Cf::OFF_A + (n & 1) * Cf::A_STAGE)[C * NROW + a_slot];
         refresh_parts(decay);
         mbar_arrive(&bars[B_WP]);
       }
@@ -1168,52 +1173,46 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     }
   } else if (warp == 9) {
     // =============================== decay warp (Gated only) =================================
-    // Lane L serves rows 4L .. 4L+3 of the tile.  Per chunk: the rows' decays straight from global memory (one value
-    // per row and token; a warp of its own, so that the load latency stalls nobody else), their running products
-    // A_t since the chunk began into the stage of the chunk's parity: entry t + 1 = A_t, entry 0 = 1.  Tokens past
-    // the end of the sequence decay by 1.  A stage is refilled once the outputs of the chunk two back are formed.
+    // Lane L serves component L / (COLS / 4) and four consecutive columns of the tile.  Per chunk: their decays straight
+    // from global memory (one 16-byte load per token, or one value when there is one decay per component; a warp of
+    // its own, so that the load latency stalls nobody else, and few instructions, because every issue slot it takes
+    // on its scheduler is taken from a row warp), their running products A_t since the chunk began into the stage of
+    // the chunk's parity: entry t + 1 = A_t, entry 0 = 1.  Tokens past the end of the sequence and columns past Dv
+    // decay by 1.  A stage is refilled once the outputs of the chunk two back are formed.
     if constexpr (Cf::GATED) {
-      const float *src[4];
-      size_t tstride;  // elements between consecutive tokens
-      bool ok[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int rr = 4 * lane + i, jj = rr % J, cc = col0 + rr / J;
-        ok[i] = cc < p.Dv;
-        src[i] = p.gran == SWILA_GATE_PER_OUT ? p.alpha + (tok0 * J + jj) * (size_t)p.Dv + cc : p.alpha + tok0 * J + jj;
-      }
-      tstride = p.gran == SWILA_GATE_PER_OUT ? (size_t)J * p.Dv : (size_t)J;
+      const int gj = lane / (COLS / 4), gc = 4 * (lane % (COLS / 4));
+      const bool per_out = p.gran == SWILA_GATE_PER_OUT;
+      const bool cols_ok = col0 + gc < p.Dv;  // Dv is a multiple of 8: four columns are inside or outside together
+      const float *src = per_out ? p.alpha + (tok0 * J + gj) * (size_t)p.Dv + col0 + gc : p.alpha + tok0 * J + gj;
+      const size_t tstride = per_out ? (size_t)J * p.Dv : (size_t)J;
+      const int slot4 = Cf::a_slot(gc, gj) / 4;
 #pragma unroll 1
       for (int m = 0; m < nchunks && !failed; ++m) {
         const int nv = min(C, Tseg - m * C);
         float4 *As = reinterpret_cast<float4 *>(smem + Cf::OFF_A + (m & 1) * Cf::A_STAGE);
-        // the chunk's decays and their running products into registers, 8 tokens (32 loads per lane) at a time: more
-        // loads in flight crowd the load/store path that the row warps' shared-memory reads also go through
-        float prod[C][4];
-        float run[4] = {1.f, 1.f, 1.f, 1.f};
+        // the chunk's decays and their running products into registers, a whole chunk ahead of their use
+        float4 prod[C];
+        if (per_out) {
 #pragma unroll
-        for (int t8 = 0; t8 < C; t8 += 8) {
-          float al[8][4];
+          for (int t = 0; t < C; ++t)
+            prod[t] = (t < nv && cols_ok) ? __ldg(reinterpret_cast<const float4 *>(src + t * tstride)) : make_float4(1.f, 1.f, 1.f, 1.f);
+        } else {
 #pragma unroll
-          for (int u = 0; u < 8; ++u) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-              al[u][i] = (t8 + u < nv && ok[i]) ? __ldg(src[i] + (size_t)(m * C + t8 + u) * tstride) : 1.0f;
+          for (int t = 0; t < C; ++t) {
+            const float a1 = (t < nv && cols_ok) ? __ldg(src + t * tstride) : 1.0f;
+            prod[t] = make_float4(a1, a1, a1, a1);
           }
+        }
+        src += C * tstride;
 #pragma unroll
-          for (int u = 0; u < 8; ++u) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              run[i] *= al[u][i];
-              prod[t8 + u][i] = run[i];
-            }
-          }
+        for (int t = 1; t < C; ++t) {
+          prod[t].x *= prod[t - 1].x; prod[t].y *= prod[t - 1].y; prod[t].z *= prod[t - 1].z; prod[t].w *= prod[t - 1].w;
         }
         // ... then the stage must be free: the outputs of the chunk two back are formed
         if (m >= 2 && !bwait_idle(B_OD, (m - 2) & 1)) { failed = true; break; }
-        As[lane] = make_float4(1.f, 1.f, 1.f, 1.f);
+        As[slot4] = make_float4(1.f, 1.f, 1.f, 1.f);
 #pragma unroll
-        for (int t = 0; t < C; ++t) As[(t + 1) * (NROW / 4) + lane] = make_float4(prod[t][0], prod[t][1], prod[t][2], prod[t][3]);
+        for (int t = 0; t < C; ++t) As[(t + 1) * (NROW / 4) + slot4] = prod[t];
         // A must never run two phases ahead of its waiters (the helpers): for m >= 2 the wait above implies that they
         // have taken chunk m-1's products; chunk 1's must not be announced before they have taken chunk 0's, which
         // the first gates (BE) tell -- a piece that waits for its state to be handed over gets there late

@@ -17,29 +17,47 @@ namespace swila {
 constexpr int kGuardSlots = 8;
 static __device__ unsigned g_gate_guard[kGuardSlots];
 
-// One thread per (batch-head, chunk, component, column) -- or per (batch-head, chunk, component) for scalar decays --
-// multiplies the decays of the chunk's tokens.  per = Dv (one decay per output dimension) or 1.
+// One thread per (batch-head, chunk, component, group of V columns) -- V = 4 with one decay per output dimension (Dv
+// is a multiple of 8, rows are 16-byte aligned), V = 1 with one per component -- multiplies the decays of the chunk's
+// tokens.  per = decays per (token, component): Dv or 1.
+template <int V>
 __global__ void __launch_bounds__(256) swila_gate_guard_kernel(const float *__restrict__ alpha, long long nbh, int T, int J,
                                                               int per, int C, unsigned *flag) {
   const long long nch = (T + C - 1) / C;
-  const long long total = nbh * nch * J * per;
+  const int groups = per / V;
+  const long long total = nbh * nch * J * groups;
   bool bad = false;
   for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
-    const int d = (int)(i % per);
-    const int j = (int)((i / per) % J);
-    const long long c = (i / ((long long)per * J)) % nch;
-    const long long bh = i / ((long long)per * J * nch);
-    const float *a0 = alpha + ((bh * T + c * C) * J + j) * (size_t)per + d;
+    const int g = (int)(i % groups);
+    const int j = (int)((i / groups) % J);
+    const long long c = (i / ((long long)groups * J)) % nch;
+    const long long bh = i / ((long long)groups * J * nch);
+    const float *a0 = alpha + ((bh * T + c * C) * J + j) * (size_t)per + (size_t)g * V;
+    const size_t tstride = (size_t)J * per;
     const int nt = min(C, T - (int)c * C);
-    float prod[4] = {1.0f, 1.0f, 1.0f, 1.0f};  // four independent chains: the loads of a trip are all in flight together
-#pragma unroll 1
-    for (int t = 0; t < nt; t += 16) {
+    float prod[V];
 #pragma unroll
-      for (int u = 0; u < 16; ++u)
-        prod[u & 3] *= (t + u < nt) ? __ldg(a0 + (size_t)(t + u) * J * per) : 1.0f;
+    for (int v = 0; v < V; ++v) prod[v] = 1.0f;
+#pragma unroll 1
+    for (int t = 0; t < nt; t += 8) {
+      float x[8][V];  // the loads of a trip are all in flight together
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        if constexpr (V == 4) {
+          const float4 q = (t + u < nt) ? __ldg(reinterpret_cast<const float4 *>(a0 + (size_t)(t + u) * tstride)) : make_float4(1.f, 1.f, 1.f, 1.f);
+          x[u][0] = q.x; x[u][1] = q.y; x[u][2] = q.z; x[u][3] = q.w;
+        } else {
+          x[u][0] = (t + u < nt) ? __ldg(a0 + (size_t)(t + u) * tstride) : 1.0f;
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+#pragma unroll
+        for (int v = 0; v < V; ++v) prod[v] *= x[u][v];
+      }
     }
-    const float all = (prod[0] * prod[1]) * (prod[2] * prod[3]);
-    bad = bad || !(all >= 9.094947e-13f && all <= 1.0000001f);  // 2^-40; also catches NaN and decays above 1
+#pragma unroll
+    for (int v = 0; v < V; ++v) bad = bad || !(prod[v] >= 9.094947e-13f && prod[v] <= 1.0000001f);  // 2^-40; NaN and decays above 1 too
   }
   if (__any_sync(0xffffffffu, bad) && (threadIdx.x & 31) == 0) atomicOr(flag, 1u);
 }
@@ -61,9 +79,10 @@ int chunk_gated_dispatch(LaunchArgs &a) {
   if (e != cudaSuccess) return (int)e;
   const int per = a.p.gran == SWILA_GATE_PER_OUT ? a.p.Dv : 1;
   const long long nbh = (long long)a.p.B * a.p.H, nch = (a.p.T + 31) / 32;
-  const long long total = nbh * nch * a.J * per;
+  const long long total = nbh * nch * a.J * (per == 1 ? 1 : per / 4);
   const unsigned grid = (unsigned)((total + 255) / 256 < 148 * 32 ? (total + 255) / 256 : 148 * 32);
-  swila_gate_guard_kernel<<<grid, 256, 0, a.stream>>>(a.p.alpha, nbh, a.p.T, a.J, per, 32, flag);
+  if (per == 1) swila_gate_guard_kernel<1><<<grid, 256, 0, a.stream>>>(a.p.alpha, nbh, a.p.T, a.J, per, 32, flag);
+  else swila_gate_guard_kernel<4><<<grid, 256, 0, a.stream>>>(a.p.alpha, nbh, a.p.T, a.J, per, 32, flag);
   e = cudaGetLastError();
   if (e != cudaSuccess) return (int)e;
   a.p.guard = flag;
