@@ -33,6 +33,11 @@ from paper_2609_39034_b200 import workloads as wl  # noqa: E402
 METRIC = "swila_fwd_tokens_per_s"
 UNIT = "tokens/s"
 HEADLINE = 2  # config index of the workload the metric is quoted on
+VARIANTS = {"vanilla": {}, "temporal": dict(temporal=True), "gated_pre_per_key": dict(gated=True),
+            "gated_post_per_key": dict(gated=True, post_decay=True),
+            "gated_pre_per_out": dict(gated=True, granularity=wl.GRAN_PER_OUT),
+            "gated_pre_scalar": dict(gated=True, granularity=wl.GRAN_SCALAR),
+            "gated_temporal": dict(temporal=True, gated=True)}
 
 # DRAM traffic per launch comes from profiles/traffic.json (ncu: dram__bytes_read.sum + dram__bytes_write.sum of one
 # captured launch), keyed by kernel and workload; an entry counts only while the kernel source it was captured from
@@ -329,11 +334,7 @@ def variants_leg(binding, stream, fma_peak_tflops: float):
     `kernel` says which kernel that resolved to, and `roofline` is taken against the slower bound of that kernel's
     pipes: the FP32 ALUs (3 FMAs per state element and token, one more multiply when gated) or HBM for the scan, HBM
     or the bf16 tensor peak for the chunked kernel."""
-    names = [("vanilla", {}), ("temporal", dict(temporal=True)), ("gated_pre_per_key", dict(gated=True)),
-             ("gated_post_per_key", dict(gated=True, post_decay=True)),
-             ("gated_pre_per_out", dict(gated=True, granularity=wl.GRAN_PER_OUT)),
-             ("gated_pre_scalar", dict(gated=True, granularity=wl.GRAN_SCALAR)),
-             ("gated_temporal", dict(temporal=True, gated=True))]
+    names = list(VARIANTS.items())
     peaks = _peaks()
 
     def roofline(w, ms, chunk):
@@ -462,6 +463,7 @@ def main():
     ap.add_argument("--decode-prefill", type=int, default=4096)
     ap.add_argument("--decode-batch", type=int, default=0, help="override B of the decode leg (0 = 256)")
     ap.add_argument("--batch", type=int, default=0, help="override B of the prefill workload (profiling only)")
+    ap.add_argument("--variant", default="vanilla", choices=sorted(VARIANTS), help="variant of the timed step (profiling only; the metric is quoted on vanilla)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.only_headline:
@@ -495,7 +497,9 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    w = wl.CONFIGS[HEADLINE]
+    w = wl.CONFIGS[HEADLINE].variant(**VARIANTS[args.variant])
+    if args.variant != "vanilla":
+        w = w.with_(name=w.name + "+" + args.variant)
     if args.batch:
         w = w.with_(B=args.batch)
     stream = torch.cuda.current_stream()
@@ -532,7 +536,7 @@ def main():
     flops = algorithmic_flops(w)
     abytes = algorithmic_bytes(w)
     sec = ms_per_step * 1e-3
-    chunked = args.algo in (0, binding.ALGO_CHUNK)
+    chunked = args.algo == binding.ALGO_CHUNK or (args.algo == 0 and binding.auto_algo(w) == binding.ALGO_CHUNK)
     if chunked:
         # The chunked kernel runs the state contractions on the tensor cores (bf16 operands, fp32
         # accumulation), so of the two bounds -- HBM bytes at the measured copy bandwidth, flops at the
@@ -585,9 +589,10 @@ def main():
     # ---- end to end from pinned host buffers through the C ABI ----
     e2e = None
     if not args.no_e2e:
-        names = ("q", "k", "v", "beta_logit", "pik_logit", "piq_logit")
-        host = {n: inp[n].cpu().pin_memory() for n in names}
-        host.update(gk_logit=None, gq_logit=None, alpha=None)
+        names = tuple(n for n in ("q", "k", "v", "beta_logit", "pik_logit", "piq_logit", "gk_logit", "gq_logit", "alpha")
+                      if inp.get(n) is not None)
+        host = {n: None for n in ("gk_logit", "gq_logit", "alpha")}
+        host.update({n: inp[n].cpu().pin_memory() for n in names})
         o_host = torch.empty(o.shape, dtype=o.dtype).pin_memory()
         ws = torch.empty(binding.host_workspace_bytes(w), device="cuda", dtype=torch.uint8)
 

@@ -317,3 +317,17 @@ def rel_err(x: torch.Tensor, y: torch.Tensor) -> float:
     rms = float(torch.sqrt(torch.mean(y * y)))
     den = torch.clamp(y.abs(), min=max(rms, 1e-300))
     return float(((x - y).abs() / den).max())
+
+
+def rel_err_unfloored(x: torch.Tensor, y: torch.Tensor, min_frac: float = 1e-2) -> float:
+    """Plain elementwise relative error max_i |x_i - y_i| / |y_i| over the elements with |y_i| >= min_frac * rms(y):
+    the measure of ``rel_err`` without its floor, reported beside it so that the gap between the two is visible."""
+    x = x.detach().double().cpu().reshape(-1)
+    y = y.detach().double().cpu().reshape(-1)
+    if y.numel() == 0:
+        return 0.0
+    rms = float(torch.sqrt(torch.mean(y * y)))
+    keep = y.abs() >= min_frac * rms
+    if not bool(keep.any()):
+        return 0.0
+    return float(((x - y).abs()[keep] / y.abs()[keep]).max())
