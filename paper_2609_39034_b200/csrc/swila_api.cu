@@ -246,8 +246,9 @@ int swila_device_status(void) {
     e = (cudaError_t)chunk_gated_error_fetch(&flag);
     if (e != cudaSuccess) return cuda_fail(e);
   }
-  if (flag) {  // (warp + 1) * 256 + barrier slot of the first wait that gave up; 1 if only the hand-over flag did
-    snprintf(g_cuda_err, sizeof(g_cuda_err), "a bounded wait expired inside the chunked kernel (code 0x%x)", flag);
+  if (flag) {  // (warp + 1) << 16 | low half of the barrier's shared-memory address; 1 if only a hand-over flag gave up
+    snprintf(g_cuda_err, sizeof(g_cuda_err), "a bounded wait expired inside the chunked kernel (warp %d, barrier at 0x%x)",
+             (flag >> 16) - 1, flag & 0xffff);
     return SWILA_ERR_CUDA;
   }
   return SWILA_OK;

@@ -66,8 +66,6 @@
 
 namespace swila {
 
-// Set when a bounded wait on a completion barrier expires (never expected).
-static __device__ int g_chunk_error = 0;
 
 // How the (tile, chunk) work items are spread over the blocks of a launch.  The ntiles * nch chunks, tile
 // after tile, are cut into equal runs of `per` chunks, one run per block; within a run the piece that
@@ -325,24 +323,17 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     const int col = col0 + dl;
     const bool col_ok = col < p.Dv;
     bool failed = false;
-    // a wait on barrier slot b that gave up: remembered as (warp + 1) * 256 + b for swila_device_status
-    int fail_where = 0;
     // the same for a warp that is in nobody's way as long as it does not compete for issue slots: it sleeps between polls
-    auto bwait_idle = [&](int b, uint32_t parity) -> bool {
+    [[maybe_unused]] auto bwait_idle = [&](int b, uint32_t parity) -> bool {
       const unsigned long long t_begin = global_timer_ns();
       while (!mbar_try_wait(&bars[b], parity)) {
         if (global_timer_ns() - t_begin > 2000000000ull) {
-          if (fail_where == 0) fail_where = (warp + 1) * 256 + b;
+          atomicCAS(&g_chunk_error, 0, (int)((warp + 1) * 65536 + (smem_u32(&bars[b]) & 0xffffu)));
           return false;
         }
         __nanosleep(200);
       }
       return true;
-    };
-    auto bwait = [&](int b, uint32_t parity) -> bool {
-      if (mbar_wait(&bars[b], parity)) return true;
-      if (fail_where == 0) fail_where = (warp + 1) * 256 + b;
-      return false;
     };
   if (pi > 0) {  // every barrier of the previous piece is quiescent: all its phases were waited for
     __syncthreads();
@@ -554,7 +545,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     // =============================== row warps ===============================================
     const int jbase = lane - j;
     [[maybe_unused]] float st_r = 0.f, st_h = 0.f;  // auxiliary instantiation: this piece's sums over time
-    if (!bwait(B_BE, 0) || !bwait(B_GS, 0)) failed = true;
+    if (!mbar_wait(&bars[B_BE], 0) || !mbar_wait(&bars[B_GS], 0)) failed = true;
     [[maybe_unused]] float rprev = 1.0f / J;  // Temporal: this row's previous responsibility r_{t-1} (App. B.3)
     // Gated: the product of this row's decays over the previous chunk of the piece.  What the tensor cores hand over
     // for a chunk, W_n [K;Q]^T + Cmat'_{n-1} (K_{n-1} [K;Q]^T), is in units of the state at the START of chunk n-1.
@@ -574,13 +565,13 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       const float *Gkk = G_all + (n & 1) * C * C;
       [[maybe_unused]] const float *As = reinterpret_cast<const float *>(smem + Cf::OFF_A + (n & 1) * Cf::A_STAGE);
 
-      if (!bwait(B_E, n & 1)) { failed = true; break; }
+      if (!mbar_wait(&bars[B_E], n & 1)) { failed = true; break; }
       tc_fence_after_sync();
       // the readout buffer this chunk seeds below was last read by the helpers for the outputs of chunk n-2.  At
       // Dk = 128 they finish those about when chunk n-1 ends, so the wait sits here, where it has long been met; at
       // Dk = 64 they are early and the wait is cheaper at the hand-over below (both placements measured)
       if constexpr (kOdWaitAtTop) {
-        if (n >= 2 && !bwait(B_OD, n & 1)) { failed = true; break; }
+        if (n >= 2 && !mbar_wait(&bars[B_OD], n & 1)) { failed = true; break; }
       }
       // [P0 | Q0] out of tensor memory: P0 to registers, Q0 seeds the readout accumulator of this chunk;
       // then the tensor cores may overwrite the region with the next chunk's products
@@ -647,7 +638,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         for (int tg = 0; tg < C; tg += GT) {
           if constexpr (!EXACT) {
             if (tg == Cf::WIN) {  // far pushes of tokens 0-6 into tokens 24-31
-              if (!bwait(B_FAR, n & 1)) failed = true;
+              if (!mbar_wait(&bars[B_FAR], n & 1)) failed = true;
               tc_fence_after_sync();
               float far[8];
               tmem_ld8(tb + Cf::TM_FAR + Cf::WIN - C / 2, far);
@@ -742,7 +733,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
           // the coefficient columns are still operands of the previous chunk's update and readout MMAs until
           // those complete (normally long before the first trip ends)
           if (tg == 0 && n > 0) {
-            if (!bwait(B_QD, (n - 1) & 1)) failed = true;
+            if (!mbar_wait(&bars[B_QD], (n - 1) & 1)) failed = true;
           }
           {  // GT update coefficients complete: park their bf16 parts in tensor memory, two tokens per column
             uint32_t hi[GT / 2], lo[GT / 2], l3[GT / 2];
@@ -795,14 +786,14 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       tc_fence_before_sync();
       // what the next steps rely on must be in place before this chunk is handed over (this also keeps every
       // barrier at most one phase ahead of its waiters): gates and Gram rows of chunk n+1
-      if (n + 1 < nchunks && (!bwait(B_BE, (n + 1) & 1) || !bwait(B_GS, (n + 1) & 1))) failed = true;
+      if (n + 1 < nchunks && (!mbar_wait(&bars[B_BE], (n + 1) & 1) || !mbar_wait(&bars[B_GS], (n + 1) & 1))) failed = true;
       if constexpr (!kOdWaitAtTop) {
-        if (n > 0 && !bwait(B_OD, (n - 1) & 1)) failed = true;
+        if (n > 0 && !mbar_wait(&bars[B_OD], (n - 1) & 1)) failed = true;
       }
       mbar_arrive(&bars[B_C]);
     }
     // ---- final state row -> global ----
-    if (!failed && !bwait(B_U, (nchunks - 1) & 1)) failed = true;
+    if (!failed && !mbar_wait(&bars[B_U], (nchunks - 1) & 1)) failed = true;
     if (!failed && p.W_out && col_ok) {
       tc_fence_after_sync();
       float *dst = p.W_out + (((size_t)bh * J + j) * p.Dv + col) * DK;
@@ -997,7 +988,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
                       (Cf::KU_MIRROR && m > 0 && m % 3 == 0) ? smem + Cf::OFF_KU + 3 * Cf::KU_HALF : nullptr);
     };
     // everything staged for chunk m has landed (the barrier of m's parity completes once per chunk of that parity)
-    auto staged = [&](int m) { return bwait(B_KQ0 + (m & 1), (m >> 1) & 1); };
+    auto staged = [&](int m) { return mbar_wait(&bars[B_KQ0 + (m & 1)], (m >> 1) & 1); };
     if (h == 0) {
       stage(0);
       if (nchunks > 1) stage(1);
@@ -1077,7 +1068,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     {
       const float *As0 = nullptr;
       if constexpr (Cf::GATED) {  // the decay warp has the running products of chunk 0 in place
-        if (!bwait(B_A, 0)) failed = true;
+        if (!mbar_wait(&bars[B_A], 0)) failed = true;
         As0 = reinterpret_cast<const float *>(smem + Cf::OFF_A);
       }
       cook_be(smem + Cf::OFF_RAW, min(C, Tseg), As0);
@@ -1085,7 +1076,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     if constexpr (Cf::TEMPORAL) cook_pk(smem + Cf::OFF_RAW);
     mbar_arrive(&bars[B_BE]);
     if (spill_mine[0]) {
-      if (!bwait(B_G, 0)) failed = true;
+      if (!mbar_wait(&bars[B_G], 0)) failed = true;
       tc_fence_after_sync();
       if (!failed) spill_gram(0);
       mbar_arrive(&bars[B_GS]);
@@ -1101,8 +1092,8 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       // last one, and in the Gated kernel, the same barrier is waited for here.
       auto outputs_of_previous = [&]() -> bool {
         if (n == 0) return true;
-        if ((!more || Cf::GATED) && !bwait(B_PQF, n & 1)) return false;
-        if (!bwait(B_QD, (n - 1) & 1)) return false;
+        if ((!more || Cf::GATED) && !mbar_wait(&bars[B_PQF], n & 1)) return false;
+        if (!mbar_wait(&bars[B_QD], (n - 1) & 1)) return false;
         write_outputs(n - 1);
         mbar_arrive(&bars[B_OD]);
         return true;
@@ -1117,14 +1108,14 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         if (!staged(n + 1)) { failed = true; break; }
         const float *As1 = nullptr;
         if constexpr (Cf::GATED) {
-          if (!bwait(B_A, (n + 1) & 1)) { failed = true; break; }
+          if (!mbar_wait(&bars[B_A], (n + 1) & 1)) { failed = true; break; }
           As1 = reinterpret_cast<const float *>(smem + Cf::OFF_A + ((n + 1) & 1) * Cf::A_STAGE);
         }
         cook_be(smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES, min(C, Tseg - (n + 1) * C), As1);
         if constexpr (Cf::TEMPORAL) cook_pk(smem + Cf::OFF_RAW + ((n + 1) & 1) * Cf::RAW_BYTES);
         mbar_arrive(&bars[B_BE]);
         if (spill_mine[(n + 1) & 1]) {
-          if (!bwait(B_G, (n + 1) & 1)) failed = true;
+          if (!mbar_wait(&bars[B_G], (n + 1) & 1)) failed = true;
           tc_fence_after_sync();
           if (!failed) spill_gram(n + 1);
           mbar_arrive(&bars[B_GS]);
@@ -1134,10 +1125,10 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         if (!outputs_of_previous()) { failed = true; break; }
       }
       // (3) chunk n is finished by the row warps: stage chunk n+2 into the buffers chunk n used
-      if (!bwait(B_C, n & 1)) { failed = true; break; }
+      if (!mbar_wait(&bars[B_C], n & 1)) { failed = true; break; }
       if (n + 2 < nchunks && h == 0) stage(n + 2);
       // (4) W has been updated with chunk n: split it into operand parts again
-      if (!bwait(B_U, n & 1)) { failed = true; break; }
+      if (!mbar_wait(&bars[B_U], n & 1)) { failed = true; break; }
       if (more) {
         tc_fence_after_sync();
         float decay = 1.0f;
@@ -1146,7 +1137,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         mbar_arrive(&bars[B_WP]);
       }
     }
-    if (!failed && !bwait(B_QD, (nchunks - 1) & 1)) failed = true;
+    if (!failed && !mbar_wait(&bars[B_QD], (nchunks - 1) & 1)) failed = true;
     if (!failed) write_outputs(nchunks - 1);
     if constexpr (Cf::TEMPORAL) {
       if (!failed && p.rho_out && col_ok) p.rho_out[((size_t)bh * J + j) * p.Dv + col] = rho_run;
@@ -1287,7 +1278,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       }
       mma_commit(&bars[B_QD]);
     };
-    if (!bwait(B_KQ0, 0) || !bwait(B_WP, 0)) failed = true;
+    if (!mbar_wait(&bars[B_KQ0], 0) || !mbar_wait(&bars[B_WP], 0)) failed = true;
     tc_fence_after_sync();
     if (!failed) {
       gram(0);
@@ -1300,8 +1291,8 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       if (more) {
         // ahead of the serial path: Gram batch and state x [K;Q] of chunk n+1 with the state before chunk n's
         // update (W is final up to chunk n-1 and split into parts; [P0|Q0] of chunk n has been taken out)
-        if (!bwait(B_KQ0 + ((n + 1) & 1), ((n + 1) >> 1) & 1) || !bwait(B_PQF, n & 1)) { failed = true; break; }
-        if (n > 0 && !bwait(B_WP, n & 1)) { failed = true; break; }
+        if (!mbar_wait(&bars[B_KQ0 + ((n + 1) & 1)], ((n + 1) >> 1) & 1) || !mbar_wait(&bars[B_PQF], n & 1)) { failed = true; break; }
+        if (n > 0 && !mbar_wait(&bars[B_WP], n & 1)) { failed = true; break; }
         tc_fence_after_sync();
         gram(n + 1);
       }
@@ -1309,7 +1300,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         // far pushes of chunk n: what its first 8 tokens add to the predictions of its last 8, needed when the row
         // warps reach token 24.  A = the coefficient columns of tokens 0..15 (8..15 are stale but finite and meet
         // zero rows of the operand), B = rows 16..31 of K K^T against tokens 0..7.
-        if (!bwait(B_T0, n & 1)) { failed = true; break; }
+        if (!mbar_wait(&bars[B_T0], n & 1)) { failed = true; break; }
         tc_fence_after_sync();
         const uint32_t fa = smem_u32(smem + Cf::OFF_FAR + (n & 1) * 2 * Cf::FAR_TILE);
         const uint64_t f_hi = smem_desc_kmajor(fa, Cf::FAR_LBO, 128), f_lo = smem_desc_kmajor(fa + Cf::FAR_TILE, Cf::FAR_LBO, 128);
@@ -1323,11 +1314,11 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         w_times_kq(n + 1);
         // first half of the cross-chunk term (tokens 0-15 of chunk n, whose coefficients T0 released), while the
         // chunk still runs
-        if (!bwait(B_GS, (n + 1) & 1)) { failed = true; break; }
+        if (!mbar_wait(&bars[B_GS], (n + 1) & 1)) { failed = true; break; }
         tc_fence_after_sync();
         cross(0);
       }
-      if (!bwait(B_C, n & 1)) { failed = true; break; }
+      if (!mbar_wait(&bars[B_C], n & 1)) { failed = true; break; }
       tc_fence_after_sync();
       const bool redone = *redo_s != 0;  // ordered by the barrier: set before the row warps arrived
       if (redone) *redo_s = 0;
@@ -1342,7 +1333,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
       if constexpr (Cf::GATED) {
         // the helpers wrote the decayed state back over W after the previous update: that must be complete (in
         // every iteration but the last it has been waited for above already)
-        if (n > 0 && !bwait(B_WP, n & 1)) { failed = true; break; }
+        if (n > 0 && !mbar_wait(&bars[B_WP], n & 1)) { failed = true; break; }
         tc_fence_after_sync();
       }
 #pragma unroll 1
@@ -1359,7 +1350,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     }
   }
   if (failed) {
-    atomicCAS(&g_chunk_error, 0, fail_where ? fail_where : 1);  // the first failure of the launch is kept
+    atomicCAS(&g_chunk_error, 0, 1);  // (a wait that gave up has left its own code already)
     *fail_s = 1;
   }
   }  // pieces

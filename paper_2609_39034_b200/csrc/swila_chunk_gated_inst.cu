@@ -94,8 +94,8 @@ int chunk_gated_dispatch(LaunchArgs &a) {
 // Reads (and clears) this translation unit's copy of the device-side error word; synchronises.
 int chunk_gated_error_fetch(int *flag) {
   int zero = 0;
-  cudaError_t e = cudaMemcpyFromSymbol(flag, g_chunk_error, sizeof(int));
-  if (e == cudaSuccess && *flag) e = cudaMemcpyToSymbol(g_chunk_error, &zero, sizeof(int));
+  cudaError_t e = cudaMemcpyFromSymbol(flag, umma::g_chunk_error, sizeof(int));
+  if (e == cudaSuccess && *flag) e = cudaMemcpyToSymbol(umma::g_chunk_error, &zero, sizeof(int));
   return (int)e;
 }
 

@@ -27,8 +27,8 @@ int chunk_dispatch(const LaunchArgs &a) {
 // Reads (and clears) the device-side error flag of the current device; synchronises.
 int chunk_error_fetch(int *flag) {
   int zero = 0;
-  cudaError_t e = cudaMemcpyFromSymbol(flag, g_chunk_error, sizeof(int));
-  if (e == cudaSuccess && *flag) e = cudaMemcpyToSymbol(g_chunk_error, &zero, sizeof(int));
+  cudaError_t e = cudaMemcpyFromSymbol(flag, umma::g_chunk_error, sizeof(int));
+  if (e == cudaSuccess && *flag) e = cudaMemcpyToSymbol(umma::g_chunk_error, &zero, sizeof(int));
   return (int)e;
 }
 

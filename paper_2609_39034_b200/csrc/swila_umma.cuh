@@ -39,6 +39,12 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
+// Set when a bounded wait expires (never expected): (warp + 1) * 65536 + the low 16 bits of the shared-memory address of
+// the barrier that the first such wait of the launch was on (barriers are 8 bytes apart, in the order of the kernel's
+// barrier enum), or 1 when only a hand-over flag gave up.  One copy per translation unit.  The wait sites themselves
+// carry no bookkeeping: the kernel's pace reacts to every instruction added there.
+static __device__ int g_chunk_error = 0;
+
 // The polling loop is kept out of line (one copy per translation unit) so that the many wait sites of a kernel
 // cost the instruction cache one test and one call each.
 static __device__ __noinline__ bool mbar_wait_poll(uint32_t bar_addr, uint32_t parity) {
@@ -54,7 +60,10 @@ static __device__ __noinline__ bool mbar_wait_poll(uint32_t bar_addr, uint32_t p
         : "r"(bar_addr), "r"(parity)
         : "memory");
     if (ok) return true;
-    if ((i & 255u) == 0 && global_timer_ns() - t0 > 2000000000ull) return false;
+    if ((i & 255u) == 0 && global_timer_ns() - t0 > 2000000000ull) {
+      atomicCAS(&g_chunk_error, 0, (int)(((threadIdx.x >> 5) + 1) * 65536 + (bar_addr & 0xffffu)));
+      return false;
+    }
   }
 }
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
