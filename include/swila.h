@@ -154,9 +154,10 @@ int swila_state_init(const swila_shape_t *shape, swila_state_t *state, void *str
  *          inside a chunk on the FP32 ALUs; several times faster.  It covers: bf16 io; Dk in {64, 128};
  *          not SWILA_QKV_ACT; and
  *            - ungated: J in {4, 8}, and J = 16 at Dk = 64; plain or SWILA_TEMPORAL; r_debug and the sums of
- *              swila_forward_stats only for plain (non-Temporal) shapes with J <= 8;
+ *              swila_forward_stats for J <= 8;
  *            - SWILA_GATED with one decay per state row, SWILA_GATE_PER_OUT or SWILA_GATE_SCALAR, pre- or
- *              post-decay: J = 4, or J = 8 at Dk = 64; not SWILA_TEMPORAL, no r_debug / statistics.  Such a
+ *              post-decay: J = 4, or J = 8 at Dk = 64; with SWILA_TEMPORAL at Dk = 64 only; no r_debug /
+ *              statistics.  Such a
  *              call launches a guard pass over alpha, the chunked kernel and the scan kernel; exactly one of
  *              the two does the work: the scan if the product of some row's decays over a 32-token chunk is
  *              below 2^-40 (the chunked form divides by that product), which costs the scan's time.
@@ -164,8 +165,8 @@ int swila_state_init(const swila_shape_t *shape, swila_state_t *state, void *str
  *          differs per key dimension, so the rows of a tile share no operand): SWILA_ERR_UNSUPPORTED.
  *   AUTO   CHUNK when the call is inside that coverage and T >= 64, else SCAN.  So the following send an
  *          AUTO call to the scan kernel, at 3-6 times the cost per token: fp32 io, SWILA_QKV_ACT, Dk = 16,
- *          J in {1, 2}, T < 64, SWILA_GATED with per-key or elementwise decays or together with SWILA_TEMPORAL,
- *          and r_debug or statistics together with SWILA_TEMPORAL, SWILA_GATED or J = 16.
+ *          J in {1, 2}, T < 64, SWILA_GATED with per-key or elementwise decays or, at Dk = 128, with SWILA_TEMPORAL,
+ *          and r_debug or statistics together with SWILA_GATED or J = 16.
  * Inside CHUNK the work distribution depends on state_out: with a state output, when the 128-row tiles
  * of the launch do not fill a whole number of waves of SMs, the chunk sequence is cut into equal runs
  * per SM and a tile that falls into two runs hands its state over through state_out (a cooperative

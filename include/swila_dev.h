@@ -52,6 +52,14 @@ int swila_selftest_bf16_mma(const float *A, const float *B, float *D, int N, int
                             void *stream);
 
 /*
+ * Self-test of the failure path of the chunked kernel's waits (no counterpart in the paper): launches one small block
+ * that waits, with the library's bounded wait (about two seconds), on a barrier nothing arrives at.  The wait must
+ * give up and the kernel end normally; *gave_up (DEVICE int) receives 1, and the next swila_device_status() reports
+ * SWILA_ERR_CUDA once (then SWILA_OK again).  Nothing traps or faults: the context stays usable.
+ */
+int swila_selftest_wait_timeout(int *gave_up, void *stream);
+
+/*
  * Which kernel SWILA_ALGO_AUTO resolves to for `shape` (no counterpart in the paper; host arithmetic only):
  * returns SWILA_ALGO_CHUNK or SWILA_ALGO_SCAN, or a negative status for an invalid shape.  aux_outputs != 0: the
  * call also asks for r_debug or for the sums of swila_forward_stats.  The rule is the one stated with swila_forward.

@@ -25,7 +25,7 @@ EXPORTS = ("swila_version", "swila_strerror", "swila_last_cuda_error", "swila_st
            "swila_state_r_bytes", "swila_state_init", "swila_forward", "swila_decode_step",
            "swila_bench_fma_chain", "swila_forward_host", "swila_forward_host_workspace_bytes",
            "swila_forward_host_static", "swila_forward_host_static_capacity", "swila_selftest_tf32_mma", "swila_selftest_bf16_mma", "swila_device_status", "swila_chunk_plan", "swila_chunk_run_pieces",
-           "swila_forward_stats", "swila_output_norm", "swila_auto_algo")
+           "swila_forward_stats", "swila_output_norm", "swila_auto_algo", "swila_selftest_wait_timeout")
 
 
 class Shape(ctypes.Structure):
@@ -108,6 +108,8 @@ def _load() -> ctypes.CDLL:
     L.swila_chunk_run_pieces.argtypes = [ctypes.c_longlong, ctypes.c_int, ctypes.c_int, ctypes.c_longlong,
                                          ctypes.POINTER(ctypes.c_int), ctypes.c_int]
     L.swila_device_status.restype = ctypes.c_int
+    L.swila_selftest_wait_timeout.restype = ctypes.c_int
+    L.swila_selftest_wait_timeout.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
     L.swila_auto_algo.restype = ctypes.c_int
     L.swila_auto_algo.argtypes = [ctypes.POINTER(Shape), ctypes.c_int]
     L.swila_bench_fma_chain.restype = ctypes.c_int

@@ -76,17 +76,18 @@ static bool overlaps(const void *a, size_t na, const void *b, size_t nb) {
 }
 
 // What the chunked tensor-core kernel covers (the AUTO rule of swila_forward is this and T >= 64): bf16 io, Dk in
-// {64, 128}, J in {4, 8} or J = 16 at Dk = 64, plain or Temporal; auxiliary outputs (r_debug, statistics) only for
-// plain shapes with J <= 8.
+// {64, 128}, J in {4, 8} or J = 16 at Dk = 64, plain or Temporal, or Gated with one decay per state row; auxiliary
+// outputs (r_debug, statistics) for the ungated shapes with J <= 8.
 static bool chunk_covers(const swila_shape_t *s, bool aux) {
   if (s->io_dtype != SWILA_IO_BF16 || (s->Dk != 64 && s->Dk != 128)) return false;
   if (s->flags & SWILA_QKV_ACT) return false;
   if (s->flags & SWILA_GATED) {  // one decay per state row (per output dimension, or per component), pre- or post-decay
     if (s->gate_granularity != SWILA_GATE_PER_OUT && s->gate_granularity != SWILA_GATE_SCALAR) return false;
-    return !(s->flags & SWILA_TEMPORAL) && (s->J == 4 || (s->J == 8 && s->Dk == 64)) && !aux;
+    if ((s->flags & SWILA_TEMPORAL) && s->Dk != 64) return false;
+    return (s->J == 4 || (s->J == 8 && s->Dk == 64)) && !aux;
   }
   if (!(s->J == 4 || s->J == 8 || (s->J == 16 && s->Dk == 64))) return false;
-  if (aux && ((s->flags & SWILA_TEMPORAL) || s->J == 16)) return false;
+  if (aux && s->J == 16) return false;
   return true;
 }
 

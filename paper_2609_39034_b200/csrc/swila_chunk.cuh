@@ -267,10 +267,9 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
                                                                      const __grid_constant__ ChunkMaps maps) {
   using namespace umma;
   constexpr int J = Cf::J, DK = Cf::DK, C = Cf::C, NROW = Cf::NROW, COLS = Cf::COLS;
-  static_assert(!(RDEBUG && Cf::TEMPORAL), "the auxiliary outputs of the Temporal variant come from the scan kernel");
   static_assert(!(RDEBUG && J > 8), "the auxiliary outputs for J = 16 come from the scan kernel");
   static_assert(!(RDEBUG && Cf::GATED), "the auxiliary outputs of the Gated variant come from the scan kernel");
-  static_assert(!(Cf::GATED && (Cf::TEMPORAL || J > 8)), "gated rows: plain kernel, J <= 8");
+  static_assert(!(Cf::GATED && J > 8), "gated rows: J <= 8");
   // Gated: a guard pass has looked at the decays first; if the product over some chunk is so small that quantities
   // taken relative to the chunk's start would overflow, the scan kernel runs this call instead
   if constexpr (Cf::GATED) {
@@ -415,6 +414,17 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
           const float gq = sigmoid_approx(__bfloat162float(rgq[t * COLS + dl]));
           if (t < nvalid) rho_run = fmaf(gq, pq - rho_run, rho_run);
           hq[i] *= rho_run;
+          if constexpr (RDEBUG) {
+            // sums over time of the readout weights (this lane: its own component) and of their entropy over the
+            // components (bits; summed over the J lanes of the column, kept by every lane, added once at the end)
+            float hb = rho_run > 0.f ? rho_run * lg2_approx(rho_run) : 0.f;
+#pragma unroll
+            for (int off = 1; off < J; off <<= 1) hb += __shfl_xor_sync(0xffffffffu, hb, off);
+            if (t < nvalid) {
+              sq_sum[0] += rho_run;
+              sq_ent -= hb;
+            }
+          }
         }
       }
       if constexpr (J > 8) {
@@ -1149,9 +1159,14 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
     if constexpr (RDEBUG) {
       // this piece's sums of the readout weights: the J lanes of a column hold disjoint tokens, and other pieces of
       // the tile may run in other blocks, hence atomic additions
-      if (!failed && col_ok) {
+      constexpr float kLn2 = 0.6931471805599453f;
+      if constexpr (Cf::TEMPORAL) {
+        if (!failed && col_ok) {
+          if (p.rho_sum) atomicAdd(p.rho_sum + ((size_t)bh * J + j) * p.Dv + col, sq_sum[0]);
+          if (p.rho_ent && j == 0) atomicAdd(p.rho_ent + (size_t)bh * p.Dv + col, sq_ent * kLn2);
+        }
+      } else if (!failed && col_ok) {
         constexpr int LJ = (J == 4) ? 2 : 3;
-        constexpr float kLn2 = 0.6931471805599453f;
 #pragma unroll
         for (int c = 0; c < J; ++c) {
           int pat = 0;
@@ -1443,11 +1458,10 @@ template <int J, int DK, bool TEMPORAL = false, bool GATED = false>
 int launch_chunk(const LaunchArgs &a) {
   using Cf = ChunkCfg<J, DK, TEMPORAL, GATED>;
   const bool aux = a.p.r_debug || a.p.r_sum || a.p.r_ent || a.p.rho_sum || a.p.rho_ent;
-  if (TEMPORAL && aux) return -1000;  // the Temporal variant's auxiliary outputs come from the scan kernel
   if (J > 8 && aux) return -1000;     // likewise for J = 16
   if (GATED && aux) return -1000;     // and for the Gated variant
   auto kern = swila_chunk_kernel<Cf, false>;
-  if constexpr (!TEMPORAL && !GATED && J <= 8) {
+  if constexpr (!GATED && J <= 8) {
     if (aux) kern = swila_chunk_kernel<Cf, true>;
   }
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cf::SMEM_BYTES);

@@ -65,7 +65,8 @@ __global__ void __launch_bounds__(256) swila_gate_guard_kernel(const float *__re
 // Returns a cudaError_t value (>= 0), or -1000 when the combination is not compiled.  On success a.p.guard points at
 // the flag the caller must hand to the scan kernel it launches behind this one.
 int chunk_gated_dispatch(LaunchArgs &a) {
-  if (a.io_dtype != SWILA_IO_BF16 || a.gate_mode != 2 || a.p.qkv_act || a.p.temporal) return -1000;
+  if (a.io_dtype != SWILA_IO_BF16 || a.gate_mode != 2 || a.p.qkv_act) return -1000;
+  if (a.p.temporal && a.Dk != 64) return -1000;  // Temporal with row gates fits shared memory at Dk = 64 only
   if (a.p.gran != SWILA_GATE_PER_OUT && a.p.gran != SWILA_GATE_SCALAR) return -1000;
   // (J = 8 at Dk = 128 does not fit shared memory with the decay products beside the wider gate stages)
   if (!((a.J == 4 && (a.Dk == 64 || a.Dk == 128)) || (a.J == 8 && a.Dk == 64))) return -1000;
@@ -87,6 +88,7 @@ int chunk_gated_dispatch(LaunchArgs &a) {
   if (e != cudaSuccess) return (int)e;
   a.p.guard = flag;
   a.p.guard_runs_scan = 0;
+  if (a.p.temporal) return a.J == 4 ? launch_chunk<4, 64, true, true>(a) : launch_chunk<8, 64, true, true>(a);
   if (a.J == 4) return a.Dk == 128 ? launch_chunk<4, 128, false, true>(a) : launch_chunk<4, 64, false, true>(a);
   return launch_chunk<8, 64, false, true>(a);
 }

@@ -34,6 +34,27 @@ int chunk_error_fetch(int *flag) {
 
 }  // namespace swila
 
+namespace swila {
+// One block, one barrier that nothing ever arrives at: the bounded wait must give up, leave its code in the error word
+// and let the kernel end normally (no trap, no fault: the context stays usable).
+__global__ void swila_wait_timeout_kernel(int *gave_up) {
+  __shared__ __align__(8) uint64_t bar;
+  if (threadIdx.x == 0) {
+    umma::mbar_init(&bar, 1);
+    umma::mbar_fence_init();
+  }
+  __syncthreads();
+  const bool ok = umma::mbar_wait(&bar, 0);
+  if (threadIdx.x == 0) *gave_up = ok ? 0 : 1;
+}
+}  // namespace swila
+
+extern "C" int swila_selftest_wait_timeout(int *gave_up, void *stream) {
+  if (!gave_up) return SWILA_ERR_NULL;
+  swila::swila_wait_timeout_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(gave_up);
+  return cudaGetLastError() == cudaSuccess ? SWILA_OK : SWILA_ERR_CUDA;
+}
+
 // Host-only probes of the chunked kernel's work distribution (no GPU call): what the CPU tests check.
 extern "C" int swila_chunk_plan(int B, int H, int T, int Dv, int J, int sm_count, int has_state_out, long long out[6]) {
   if (!out) return SWILA_ERR_NULL;

@@ -34,7 +34,7 @@ PRODUCT_ABI = {"swila_version", "swila_strerror", "swila_last_cuda_error", "swil
                "swila_decode_step", "swila_forward_stats", "swila_output_norm",
                "swila_forward_host", "swila_forward_host_workspace_bytes",
                "swila_forward_host_static", "swila_forward_host_static_capacity"}
-DEV_ABI = {"swila_auto_algo", "swila_bench_fma_chain", "swila_selftest_tf32_mma", "swila_selftest_bf16_mma",
+DEV_ABI = {"swila_auto_algo", "swila_selftest_wait_timeout", "swila_bench_fma_chain", "swila_selftest_tf32_mma", "swila_selftest_bf16_mma",
            "swila_chunk_plan", "swila_chunk_run_pieces"}
 
 
@@ -125,11 +125,11 @@ def test_auto_dispatch_rule(binding):
     auto = lambda w, aux=0: binding.lib.swila_auto_algo(ctypes.byref(binding.make_shape(w)), aux)  # noqa: E731
     lm = wl.CONFIGS[2]
     assert auto(lm) == binding.ALGO_CHUNK and auto(lm.variant(temporal=True)) == binding.ALGO_CHUNK
-    assert auto(lm, 1) == binding.ALGO_CHUNK and auto(lm.variant(temporal=True), 1) == binding.ALGO_SCAN
+    assert auto(lm, 1) == binding.ALGO_CHUNK and auto(lm.variant(temporal=True), 1) == binding.ALGO_CHUNK
     assert auto(wl.CONFIGS[1].with_(J=16)) == binding.ALGO_CHUNK and auto(wl.CONFIGS[1].with_(J=16), 1) == binding.ALGO_SCAN
     rows = dict(gated=True, granularity=wl.GRAN_PER_OUT)
     assert auto(lm.variant(**rows)) == binding.ALGO_CHUNK and auto(lm.variant(gated=True, granularity=wl.GRAN_SCALAR, post_decay=True)) == binding.ALGO_CHUNK
-    assert auto(lm.variant(**rows), 1) == binding.ALGO_SCAN and auto(lm.variant(temporal=True, **rows)) == binding.ALGO_SCAN
+    assert auto(lm.variant(**rows), 1) == binding.ALGO_SCAN and auto(lm.variant(temporal=True, **rows)) == binding.ALGO_SCAN and auto(wl.CONFIGS[1].variant(temporal=True, **rows)) == binding.ALGO_CHUNK
     assert auto(lm.with_(J=8).variant(**rows)) == binding.ALGO_SCAN and auto(wl.CONFIGS[1].with_(J=8).variant(**rows)) == binding.ALGO_CHUNK
     for w in (lm.with_(T=63), lm.with_(io_dtype="fp32"), lm.variant(gated=True), lm.with_(J=2), lm.with_(J=16),
               lm.variant(gated=True, granularity=wl.GRAN_ELEMENTWISE),

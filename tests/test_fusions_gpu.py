@@ -84,8 +84,8 @@ def test_qkv_activation_is_refused_by_the_chunked_kernel(binding):
 
 
 @pytest.mark.parametrize("w", SHAPES)
-@pytest.mark.parametrize("temporal,algo", [(False, "scan"), (True, "scan"), (False, "auto")],
-                         ids=["vanilla_scan", "temporal_scan", "vanilla_auto"])
+@pytest.mark.parametrize("temporal,algo", [(False, "scan"), (True, "scan"), (False, "auto"), (True, "auto")],
+                         ids=["vanilla_scan", "temporal_scan", "vanilla_auto", "temporal_auto"])
 def test_statistics_match_the_oracle(binding, oracle, fus, w, temporal, algo):
     """`auto` takes the chunked tensor-core kernel for the bf16 shapes of 64 tokens and more."""
     algo = getattr(binding, "ALGO_" + algo.upper())
@@ -138,13 +138,14 @@ def test_statistics_members_are_optional(binding, algo):
     assert torch.equal(only["r_sum"], full["r_sum"])  # one piece per tile here: a single addition per element
 
 
-def test_statistics_on_the_balanced_schedule(binding, oracle, fus):
+@pytest.mark.parametrize("temporal", [False, True], ids=["plain", "temporal"])
+def test_statistics_on_the_balanced_schedule(binding, oracle, fus, temporal):
     """More tiles than SMs: the chunked kernel cuts sequences into pieces that run in different blocks, whose sums
     meet in the caller's buffers through atomic additions.  Checked against the scan kernel's sums and, on sampled
     rows, against the oracle."""
-    w = wl.CONFIGS[2].with_(B=2, H=20, T=1024)
+    w = wl.CONFIGS[2].with_(B=2, H=20, T=1024).variant(temporal=temporal)
     inp = wl.make_inputs(w, device="cuda", stress=True)
-    sin = {"W": inp["W0"]}
+    sin = {"W": inp["W0"], "r_prev": inp.get("r0"), "rho_prev": inp.get("rho0")}
     got, ref = binding.stats_alloc(w), binding.stats_alloc(w)
     st = binding.state_alloc(w, init=False)
     binding.swila_forward_stats(w, inp, got, state_in=sin, state_out=st, algo=binding.ALGO_CHUNK)
@@ -155,9 +156,10 @@ def test_statistics_on_the_balanced_schedule(binding, oracle, fus):
         assert wl.rel_err(got[name].cpu(), ref[name].cpu()) < 1e-4, name
     bh = torch.tensor([3, 17, 38])
     cols = torch.tensor([0, 31, 32, 77, 127])
-    rows = wl.slice_rows(inp, bh.cuda(), cols.cuda())
-    o_ref = oracle.forward_inputs({k: (v.cpu() if v is not None else None) for k, v in rows.items()}, want_r=True)
-    want = fus.responsibility_stats(o_ref["r"], fus.readout_weights(rows["piq_logit"].cpu()))
+    rows = {k: (v.cpu() if v is not None else None) for k, v in wl.slice_rows(inp, bh.cuda(), cols.cuda()).items()}
+    o_ref = oracle.forward_inputs(rows, flags=w.flags, want_r=True)
+    want = fus.responsibility_stats(o_ref["r"], fus.readout_weights(rows["piq_logit"], rows.get("gq_logit") if temporal else None,
+                                                                    rows.get("rho0") if temporal else None))
     for name in ("r_sum", "rho_sum"):
         g = got[name].reshape(w.B * w.H, w.J, w.Dv)[bh.cuda()][:, :, cols.cuda()].unsqueeze(1).cpu()
         assert wl.rel_err(g, torch.from_numpy(want[name])) < 1e-4, name

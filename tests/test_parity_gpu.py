@@ -116,8 +116,9 @@ def test_chunked_kernel_temporal_matches_oracle(binding, oracle, w, stress):
     both carried distributions enter and leave with the state."""
     wt = w.variant(temporal=True)
     inp = wl.make_inputs(wt, stress=stress)
-    ref = oracle.forward_inputs(inp, flags=wt.flags)
-    got = gpu_forward(binding, wt, to_dev(inp), algo=binding.ALGO_CHUNK)
+    want_r = wt.J <= 8  # the responsibilities of J = 16 come from the scan kernel only
+    ref = oracle.forward_inputs(inp, flags=wt.flags, want_r=want_r)
+    got = gpu_forward(binding, wt, to_dev(inp), want_r=want_r, algo=binding.ALGO_CHUNK)
     binding.device_status()
     assert_close(wt, got, ref, wt.name)
 
@@ -147,6 +148,18 @@ def test_chunked_kernel_gated_rows_match_oracle(binding, oracle, w, gran, post, 
     if wg.T >= 32:  # it was the chunked kernel that ran: the scan kernel's bits differ
         scan = gpu_forward(binding, wg, dev, algo=binding.ALGO_SCAN)
         assert not torch.equal(scan["W"], got["W"])
+
+
+@pytest.mark.parametrize("w", [w for w in GATED_ROW_SHAPES if w.Dk == 64], ids=lambda w: w.name)
+@pytest.mark.parametrize("gran,post", [(wl.GRAN_PER_OUT, False), (wl.GRAN_SCALAR, True)], ids=["out_pre", "scalar_post"])
+def test_chunked_kernel_gated_rows_with_temporal_priors(binding, oracle, w, gran, post):
+    """Gated Temporal SwiLA with row gates in the chunked kernel (it fits shared memory at Dk = 64)."""
+    wg = w.variant(temporal=True, gated=True, granularity=gran, post_decay=post)
+    inp = wl.make_inputs(wg, stress=True)
+    ref = oracle.forward_inputs(inp, flags=wg.flags, gran=gran)
+    got = gpu_forward(binding, wg, to_dev(inp), algo=binding.ALGO_CHUNK)
+    binding.device_status()
+    assert_close(wg, got, ref, wg.name)
 
 
 def test_chunked_kernel_gated_rows_hand_over_to_the_scan_when_a_chunk_decays_to_nothing(binding, oracle):
@@ -318,7 +331,7 @@ def test_outputs_stay_inside_their_buffers(binding, algo, temporal, T):
     with atomics, and compute-sanitizer cannot be run on it here, so this is its bounds check."""
     w = SMALL[3].with_(T=T).variant(temporal=temporal)  # Dv = 72
     inp = to_dev(wl.make_inputs(w, stress=True))
-    with_stats = not (temporal and algo == "chunk")  # the chunked kernel forms no statistics for the Temporal variant
+    with_stats = True
     n_o, n_w, n_r = w.B * w.H * w.T * w.Dv, w.B * w.H * w.J * w.Dv * w.Dk, w.B * w.H * w.J * w.Dv
     n_e = w.B * w.H * w.Dv
     bufs = {"o": _canary(n_o, w.torch_io_dtype), "W": _canary(n_w, torch.float32)}

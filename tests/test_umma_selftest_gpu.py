@@ -38,3 +38,31 @@ def test_bf16_mma_matches_matmul(N, K, a_in_smem):
     ref = A.bfloat16().double() @ B.bfloat16().double().T  # the kernel rounds to bf16 the same way
     err = float((D.double() - ref).abs().max() / ref.abs().max())
     assert err < 1e-5, err
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_context_survives():
+    """Failure detection without a fault: a bounded wait on a barrier that nothing arrives at gives up after about two
+    seconds, the kernel ends normally, swila_device_status reports it once, and the next launch works."""
+    import ctypes
+    import time
+
+    from paper_2609_39034_b200 import binding, workloads as wl
+
+    binding.device_status()  # clean before
+    gave_up = torch.zeros(1, device="cuda", dtype=torch.int32)
+    t0 = time.time()
+    binding.check(binding.lib.swila_selftest_wait_timeout(ctypes.c_void_p(gave_up.data_ptr()),
+                                                          ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)))
+    torch.cuda.synchronize()
+    assert 1.5 < time.time() - t0 < 10.0
+    assert int(gave_up.item()) == 1
+    with pytest.raises(binding.SwilaError) as e:
+        binding.device_status()
+    assert e.value.status == binding.ERR_CUDA and "bounded wait" in str(e.value)
+    binding.device_status()  # reported once, then clean again
+    w = wl.CONFIGS[1].with_(B=1, H=1, T=64)  # and the context still runs kernels
+    inp = wl.make_inputs(w, device="cuda")
+    o = binding.swila_forward(w, inp, state_in=None, state_out=None, algo=binding.ALGO_CHUNK)
+    torch.cuda.synchronize()
+    binding.device_status()
+    assert bool(torch.isfinite(o.float()).all())
