@@ -51,8 +51,9 @@ def test_host_entry_rejects_a_small_workspace(binding):
     assert e.value.status == binding.ERR_SIZE
 
 
-@pytest.mark.parametrize("var,T", [(dict(), 2304), (dict(temporal=True), 2304), (dict(temporal=True, gated=True), 1400)],
-                         ids=["vanilla", "temporal", "gated_temporal"])
+@pytest.mark.parametrize("var,T", [(dict(), 2304), (dict(temporal=True), 2304), (dict(temporal=True, gated=True), 1400),
+                                   (dict(gated=True, granularity=wl.GRAN_PER_OUT), 2048)],
+                         ids=["vanilla", "temporal", "gated_temporal", "gated_rows"])
 def test_host_entry_in_slabs_equals_device_entry(binding, var, T):
     """Problems of 64 MB and more go through in slabs of (batch, head) pairs over internal copy streams; with 15
     pairs the 8 slabs are uneven.  The results must be those of one call on device tensors."""

@@ -162,6 +162,27 @@ def test_chunked_kernel_gated_rows_with_temporal_priors(binding, oracle, w, gran
     assert_close(wg, got, ref, wg.name)
 
 
+@pytest.mark.parametrize("gran,post", [(wl.GRAN_PER_OUT, False), (wl.GRAN_SCALAR, True)], ids=["out_pre", "scalar_post"])
+def test_chunked_kernel_gated_rows_state_carry(binding, oracle, gran, post):
+    """Gated rows: chunked prefill -> scan decode steps -> chunked prefill on one carried state equals one oracle pass;
+    and a call that discards the state (one tile per block, no hand-over) gives the same outputs."""
+    w = SMALL[4].with_(T=120).variant(gated=True, granularity=gran, post_decay=post)
+    inp = wl.make_inputs(w, stress=True)
+    ref = oracle.forward_inputs(inp, flags=w.flags, gran=gran)
+    dev = to_dev(inp)
+    st = {"W": dev["W0"].clone(), "r_prev": None, "rho_prev": None}
+    outs = [binding.swila_forward(w, wl.slice_time(dev, 0, 70), state_in=st, state_out=st, algo=binding.ALGO_CHUNK)]
+    outs += [binding.swila_decode_step(w, wl.slice_time(dev, t, t + 1), st) for t in range(70, 75)]
+    outs.append(binding.swila_forward(w, wl.slice_time(dev, 75, 120), state_in=st, state_out=st, algo=binding.ALGO_CHUNK))
+    torch.cuda.synchronize()
+    binding.device_status()
+    got = {"o": torch.cat(outs, dim=2).cpu(), "W": st["W"].cpu()}
+    assert_close(w, got, ref, "gated carry")
+    o_nostate = binding.swila_forward(w, dev, state_in={"W": dev["W0"]}, state_out=None, algo=binding.ALGO_CHUNK)
+    torch.cuda.synchronize()
+    assert wl.rel_err(o_nostate.float().cpu(), torch.from_numpy(ref["o"])) < TOL_BF16_O
+
+
 def test_chunked_kernel_gated_rows_hand_over_to_the_scan_when_a_chunk_decays_to_nothing(binding, oracle):
     """Decays whose product over one chunk drops below 2^-40 would overflow the chunked kernel's quotients: the guard
     pass sees them and the scan kernel evaluates the call (same bits as asking for the scan), in place on the state."""
