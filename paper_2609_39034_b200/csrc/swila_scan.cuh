@@ -53,11 +53,13 @@ struct ScanCfg {
   static constexpr int R_GK = R_PQ + TB * J * COLS * ES;
   static constexpr int R_GQ = R_GK + TB * COLS * ES;
   static constexpr int R_A = R_GQ + TB * COLS * ES;
-  static constexpr int RAW_BYTES = R_A + (GATE == 1 ? TB * J * DK * 4 : 0);
+  // decays staged with the block: one per key dimension [TB][J][DK], or (GATE == 2) one per output dimension, the
+  // block's column slice [TB][J][COLS]; one per component is read in place (J values per token)
+  static constexpr int RAW_BYTES = R_A + (GATE == 1 ? TB * J * DK * 4 : (GATE == 2 ? TB * J * COLS * 4 : 0));
   // 16-byte chunks per token of each segment
   static constexpr int C_K = DK * ES / 16;
   static constexpr int C_V = COLS * ES / 16;
-  static constexpr int C_A = (GATE == 1) ? J * DK * 4 / 16 : 0;
+  static constexpr int C_A = (GATE == 1) ? J * DK * 4 / 16 : ((GATE == 2) ? J * COLS * 4 / 16 : 0);
   static constexpr int CH_BASE = 2 * C_K + C_V + 3 * J * C_V;  // k q v beta pik piq
   static constexpr int CH_TEMP = 2 * C_V;
   // ---- cooked stage (floats) ----
@@ -133,6 +135,13 @@ __device__ __forceinline__ void issue_block(const ScanParams &p, unsigned char *
             valid = valid && col < p.Dv;
             src = (const char *)(isq ? p.gq_logit : p.gk_logit) + (tok * p.Dv + col) * ES;
             dst = raw + (isq ? C::R_GQ : C::R_GK) + s * COLS * ES + cc * 16;
+          } else if constexpr (GATE == 2) {  // decay per output dimension: this block's columns, fp32 [J][COLS] per token
+            if (p.temporal) cc -= C::CH_TEMP;
+            const int j = cc / (COLS / 4), c4 = cc - j * (COLS / 4);
+            const int col = col0 + c4 * 4;
+            valid = valid && col < p.Dv && p.gran == SWILA_GATE_PER_OUT;
+            src = (const char *)p.alpha + ((tok * J + j) * (size_t)p.Dv + col) * 4;
+            dst = raw + C::R_A + ((s * J + j) * COLS + c4 * 4) * 4;
           } else {  // per-key decay, fp32 [J][DK] per token
             if (p.temporal) cc -= C::CH_TEMP;
             src = (const char *)p.alpha + (tok * J * DK) * 4 + cc * 16;
@@ -242,14 +251,14 @@ __device__ __forceinline__ void cook_block(const ScanParams &p, const unsigned c
       ck[C::K_PQ + i * J + j] = pq[j];
     }
     if constexpr (GATE == 2) {
-      // one decay value per (component, output column) -- or per component -- read in place
+      // one decay value per (component, output column), staged with the block -- or per component, read in place
       const size_t tok = tok0 + (size_t)(t0 + s);
       const int col = col0 + c;
 #pragma unroll
       for (int j = 0; j < J; ++j) {
         float a = 1.f;
         if (col < p.Dv)
-          a = (p.gran == SWILA_GATE_PER_OUT) ? __ldg(p.alpha + (tok * J + j) * (size_t)p.Dv + col)
+          a = (p.gran == SWILA_GATE_PER_OUT) ? reinterpret_cast<const float *>(raw + C::R_A)[(s * J + j) * COLS + c]
                                              : __ldg(p.alpha + tok * J + j);
         ck[C::K_AR + i * J + j] = a;
       }
