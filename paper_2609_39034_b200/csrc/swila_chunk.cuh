@@ -621,19 +621,21 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
         constexpr int GT = Cf::GT;
         bool bad = false;
         [[maybe_unused]] float cr = 0.f, ch = 0.f;  // auxiliary instantiation: this chunk's sums of r and of r log2 r
-        // pred[i]: v - prediction (the prediction error so far) of token tg + i of the current trip, for the WINS
+        // P(i): v - prediction (the prediction error so far) of token tg + i of the current trip, for the WINS
         // tokens that the pushes of a token reach on the ALUs (slots past the chunk end are dead weight that keeps the
         // trip's code independent of tg); the Gram rows are stored negated, so a push is one FMA and the error of
         // the next token is ready without a subtraction on the serial chain.  The fast pass reaches WIN = 24 tokens:
         // the pushes of tokens 0-7 into tokens 24-31 come from the tensor cores (FAR) when token 24 is reached.
         // The redo pass does everything itself.
         constexpr int WINS = EXACT ? C : Cf::WIN;
-        float pred[WINS];
+        // (held as pairs: the deferred pushes below are packed two-wide FMAs, half the instructions)
+        float2 pred2[WINS / 2];
+        auto P = [&](int k) -> float & { return (k & 1) ? pred2[k >> 1].y : pred2[k >> 1].x; };
 #pragma unroll
         for (int t = 0; t < WINS; ++t) {
           // Gated: the window holds minus the prediction in units of the chunk's start; the decay and v enter per token
-          if constexpr (Cf::GATED) pred[t] = -pred0[t];
-          else pred[t] = __bfloat162float(rv[t * COLS + dl]) - pred0[t];
+          if constexpr (Cf::GATED) P(t) = -pred0[t];
+          else P(t) = __bfloat162float(rv[t * COLS + dl]) - pred0[t];
         }
         [[maybe_unused]] float p0late[C - Cf::WIN];
         if constexpr (!EXACT) {
@@ -654,7 +656,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
               tmem_ld8(tb + Cf::TM_FAR + Cf::WIN - C / 2, far);
               tmem_ld_wait();
 #pragma unroll
-              for (int i = 0; i < 8; ++i) pred[i] -= far[i];
+              for (int i = 0; i < 8; ++i) P(i) -= far[i];
             }
           }
           float cs[GT];
@@ -667,8 +669,8 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
             // (pre-decay, Eq. 3.8) or up to the previous one (post-decay, Eq. 3.7); beta arrives divided by A_t, so
             // that the coefficient below is already c_t / A_t
             float delta;
-            if constexpr (Cf::GATED) delta = fmaf(As[(t + a_off) * NROW + a_slot], pred[i], __bfloat162float(rv[t * COLS + dl]));
-            else delta = pred[i];
+            if constexpr (Cf::GATED) delta = fmaf(As[(t + a_off) * NROW + a_slot], P(i), __bfloat162float(rv[t * COLS + dl]));
+            else delta = P(i);
             float a;
             if constexpr (Cf::TEMPORAL) {
               // key-side prior (1 - g) r_{t-1} + g pi^k with g = sigmoid(gk logit) (App. B.3): a convex combination of
@@ -716,10 +718,11 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
 #pragma unroll
               for (int u4 = (i + 1) / 4; u4 < WINS / 4; ++u4) {
                 const float4 g = gp[u4];
-                if (4 * u4 + 0 > i) pred[4 * u4 + 0] = fmaf(c_prev, g.x, pred[4 * u4 + 0]);
-                if (4 * u4 + 1 > i) pred[4 * u4 + 1] = fmaf(c_prev, g.y, pred[4 * u4 + 1]);
-                if (4 * u4 + 2 > i) pred[4 * u4 + 2] = fmaf(c_prev, g.z, pred[4 * u4 + 2]);
-                if (4 * u4 + 3 > i) pred[4 * u4 + 3] = fmaf(c_prev, g.w, pred[4 * u4 + 3]);
+                const float2 cc = make_float2(c_prev, c_prev);
+                if (4 * u4 + 0 > i) pred2[2 * u4] = __ffma2_rn(cc, make_float2(g.x, g.y), pred2[2 * u4]);
+                else if (4 * u4 + 1 > i) pred2[2 * u4].y = fmaf(c_prev, g.y, pred2[2 * u4].y);
+                if (4 * u4 + 2 > i) pred2[2 * u4 + 1] = __ffma2_rn(cc, make_float2(g.z, g.w), pred2[2 * u4 + 1]);
+                else if (4 * u4 + 3 > i) pred2[2 * u4 + 1].y = fmaf(c_prev, g.w, pred2[2 * u4 + 1].y);
               }
             }
             const float rs = rcp_approx(sum);
@@ -737,7 +740,7 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
                 if (rr > 0.f) ch = fmaf(rr, lg2_approx(e) - lg2_approx(sum), ch);
               }
             }
-            pred[i + 1] = fmaf(c, Gkk[t * C + t + 1], pred[i + 1]);  // the push the next token waits for
+            P(i + 1) = fmaf(c, Gkk[t * C + t + 1], P(i + 1));  // the push the next token waits for
             c_prev = c;
           }
           // the coefficient columns are still operands of the previous chunk's update and readout MMAs until
@@ -763,13 +766,13 @@ __global__ void __launch_bounds__(Cf::NT, 1) swila_chunk_kernel(const __grid_con
             }
           }
 #pragma unroll
-          for (int i = 0; i + GT < WINS; ++i) pred[i] = pred[i + GT];
+          for (int i = 0; i + GT < WINS; i += 2) pred2[i / 2] = pred2[(i + GT) / 2];
 #pragma unroll
           for (int i = 0; i < GT; ++i) {  // the slots that enter the window: tokens 24-31 after the first trip, dead later
             if constexpr (EXACT) {
-              pred[WINS - GT + i] = 0.f;
+              P(WINS - GT + i) = 0.f;
             } else {
-              pred[WINS - GT + i] = p0late[i];
+              P(WINS - GT + i) = p0late[i];
               p0late[i] = 0.f;
             }
           }
