@@ -175,13 +175,13 @@ def test_long_sequence_from_zero_state(binding, oracle, algo):
     assert wl.rel_err(got["W"], torch.from_numpy(ref["W"])) < TOL_STATE
 
 
-@pytest.mark.parametrize("temporal", [False, True], ids=["vanilla", "temporal"])
-def test_calls_replay_from_a_cuda_graph(binding, temporal):
+@pytest.mark.parametrize("temporal,gated", [(False, False), (True, False), (False, True)], ids=["vanilla", "temporal", "gated_rows"])
+def test_calls_replay_from_a_cuda_graph(binding, temporal, gated):
     """A prefill on the balanced schedule (cooperative launch, state handed over between blocks through flags that
     carry the launch's epoch) and a decode step, captured once in a CUDA graph and replayed on fresh inputs: every
     replay must equal the eager call on the same inputs.  A replay reuses the captured epoch, so the hand-over flags
     must not keep last replay's value."""
-    w = wl.CONFIGS[2].with_(B=2, H=20, T=1024).variant(temporal=temporal)
+    w = wl.CONFIGS[2].with_(B=2, H=20, T=1024).variant(temporal=temporal, gated=gated, granularity=wl.GRAN_PER_OUT)
     inp = wl.make_inputs(w, device="cuda", stress=True)
     st = binding.state_alloc(w, init=False)
     o = torch.empty((w.B, w.H, w.T, w.Dv), device="cuda", dtype=w.torch_io_dtype)
@@ -202,7 +202,8 @@ def test_calls_replay_from_a_cuda_graph(binding, temporal):
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph):
         call()
-    names = ("q", "k", "v", "beta_logit", "pik_logit", "piq_logit") + (("gk_logit", "gq_logit") if temporal else ())
+    names = ("q", "k", "v", "beta_logit", "pik_logit", "piq_logit") + (("gk_logit", "gq_logit") if temporal else ()) + (
+        ("alpha",) if gated else ())
     for rep in range(3):
         fresh = wl.make_inputs(w, device="cuda", seed_offset=rep + 1, stress=True)
         fresh_step = wl.decode_step_inputs(w, rep + 1, device="cuda")
