@@ -148,6 +148,13 @@ def test_chunked_kernel_gated_rows_match_oracle(binding, oracle, w, gran, post, 
     if wg.T >= 32:  # it was the chunked kernel that ran: the scan kernel's bits differ
         scan = gpu_forward(binding, wg, dev, algo=binding.ALGO_SCAN)
         assert not torch.equal(scan["W"], got["W"])
+    if alpha == "down_to_half" and wg.T >= 45:
+        # test power: a kernel that ignored the decay, or took the other form's decay (Eq. 3.7 against Eq. 3.8),
+        # would be far outside the tolerance on these inputs
+        no_decay = oracle.forward_inputs(dict(inp, alpha=torch.ones_like(inp["alpha"])), flags=wg.flags, gran=gran)
+        other = oracle.forward_inputs(inp, flags=wg.flags ^ wl.FLAG_POST_DECAY, gran=gran)
+        for wrong in (no_decay, other):
+            assert wl.rel_err(torch.from_numpy(wrong["W"]), torch.from_numpy(ref["W"])) > 100 * TOL_STATE
 
 
 @pytest.mark.parametrize("w", [w for w in GATED_ROW_SHAPES if w.Dk == 64], ids=lambda w: w.name)
